@@ -1,0 +1,180 @@
+/*
+ * libscissorhands — budgeted KV-cache decode attention for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the data-parallel hot path of Scissorhands (arXiv 2305.17118):
+ * per-step decode attention over a per-(sequence, head) KV cache held under a
+ * fixed token budget B, fused with the importance-record update over the
+ * history window w, and the compression step that evicts m tokens per
+ * (sequence, head) once the cache fills while keeping the r most recent.
+ *
+ * Conventions
+ *   - A "unit" is one independent (sequence, head) pair; a handle serves
+ *     `heads` units (batch x heads of one layer).  Units never interact
+ *     (Section 4.1 drops the layer and batch indices).
+ *   - Every unit receives the same stream of calls, so the number of live
+ *     tokens n and the step counter t are the same for all units and are kept
+ *     on the host: no call below synchronises the device except sh_state,
+ *     sh_export_unit and the *_host variants.
+ *   - All device memory is owned by the caller.  The library allocates only a
+ *     small host struct per handle.  Pointers named *_dev are device pointers,
+ *     *_host are host pointers.  `stream` is a cudaStream_t passed as void*
+ *     (NULL = the legacy default stream).  Calls enqueue work and return.
+ *   - Every function returns an sh_status (0 = SH_OK, negative = error) and
+ *     never aborts, throws or prints.  On error nothing has been enqueued
+ *     unless stated otherwise.
+ *   - Slots [0, n) of a unit's cache are live and sorted by stream position;
+ *     compaction is stable, so "the r newest" are slots [n-r, n).
+ */
+#ifndef SCISSORHANDS_H_
+#define SCISSORHANDS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sh_context *sh_handle;
+
+typedef enum {
+    SH_OK = 0,
+    SH_EINVAL = -1, /* bad argument (NULL pointer, size out of range, bad dtype) */
+    SH_EFULL = -2,  /* decode step on a full cache: call sh_compress first */
+    SH_ESTATE = -3, /* call out of order (e.g. no workspace bound) */
+    SH_ECUDA = -4,  /* a CUDA runtime call or launch failed; see sh_last_cuda_error */
+    SH_ENOMEM = -5  /* host allocation failed or workspace too small */
+} sh_status;
+
+typedef enum {
+    SH_F32 = 0,         /* K/V rows stored as fp32 */
+    SH_F16 = 1,         /* fp16 */
+    SH_BF16 = 2,        /* bf16 */
+    SH_INT4_G64_F16 = 3 /* symmetric int4, groups of 64 along head_dim, fp16 scale per group;
+                           q/k/v arrive as fp16 and rows are quantised when appended */
+} sh_dtype;
+
+typedef enum {
+    SH_OPT_SOFTMAX_SCALE = 0, /* multiplier of the logits; default 1/sqrt(head_dim) */
+    SH_OPT_SPLIT = 1,         /* CTAs cooperating on one unit (1, 2, 4 or 8); default chosen from `heads` */
+    SH_OPT_AUTO_COMPRESS = 2  /* 1 (default): sh_decode_step compresses by itself when the cache fills;
+                                 0: the caller calls sh_compress */
+} sh_option;
+
+/*
+ * Create a handle.  Definition 4.1 and the inputs of Algorithms 1 and 2:
+ * B = token budget per unit, r = recent window (never evicted), w = history
+ * window of the importance record in steps, m = tokens dropped per
+ * compression, heads = number of units, head_dim = d.
+ * Requires B >= 1, r >= 0, 1 <= w <= 16384, 1 <= m <= B - r, B <= 65535,
+ * head_dim in {64, 128} (int4: 128 or 64), dtype an sh_dtype.
+ * Errors: SH_EINVAL, SH_ENOMEM.
+ */
+int sh_create(int B, int r, int w, int m, int heads, int head_dim, int dtype, sh_handle *out);
+
+/* Free the host struct.  Device memory stays with the caller. */
+void sh_destroy(sh_handle h);
+
+/* Bytes of device workspace the handle needs (K, V, scales, record bit-planes,
+ * positions, selection scratch, staging for the *_host calls). */
+size_t sh_workspace_bytes(sh_handle h);
+
+/*
+ * Give the handle its workspace: `bytes` >= sh_workspace_bytes(h) of device
+ * memory aligned to 256 bytes, owned by the caller and kept alive until
+ * sh_destroy.  The library zero-fills it on `stream` and resets n = t = 0.
+ * Errors: SH_EINVAL (NULL, misaligned), SH_ENOMEM (too small), SH_ECUDA.
+ */
+int sh_bind(sh_handle h, void *slab_dev, size_t bytes, void *stream);
+
+/* Set an option before the first step.  Errors: SH_EINVAL, SH_ESTATE. */
+int sh_set_option(sh_handle h, int key, double value);
+
+/*
+ * One generation step of Algorithm 1 for every unit: append (k_new, v_new) as
+ * the token at stream position t+1 (n <- n+1), attend with q over the n
+ * cached tokens including the new one (estimator of Section 4.1:
+ * alpha_j = softmax_j(scale*<q,K[j]>), out = sum_j alpha_j V[j]), and record
+ * for every cached token whether alpha_j < 1/(t+1) as this step's entry of
+ * the importance record (Algorithm 2's loop body, maintained online as the
+ * "Overhead Tradeoff" paragraph describes).  With SH_OPT_AUTO_COMPRESS the
+ * compression of Algorithm 2 follows when n == B.
+ * q_dev, k_new_dev, v_new_dev: [heads][head_dim] in the handle's dtype (fp16
+ * for the int4 store), 16-byte aligned.  attn_out_dev: [heads][head_dim] fp32.
+ * Errors: SH_EFULL when n == B on entry, SH_EINVAL, SH_ESTATE, SH_ECUDA.
+ */
+int sh_decode_step(sh_handle h, const void *q_dev, const void *k_new_dev, const void *v_new_dev,
+                   float *attn_out_dev, void *stream);
+
+/*
+ * Same step with HOST buffers (pinned memory recommended): copies q, k_new,
+ * v_new to the device, runs the step, copies attn_out back, all on `stream`,
+ * and returns after the stream has been synchronised.
+ */
+int sh_decode_step_host(sh_handle h, const void *q_host, const void *k_new_host, const void *v_new_host,
+                        float *attn_out_host, void *stream);
+
+/*
+ * Prompt phase, stream semantics of Definition 4.1: equivalent to p calls of
+ * sh_decode_step (each followed by a compression when the cache fills),
+ * whatever SH_OPT_AUTO_COMPRESS says.  q_dev, k_dev, v_dev: time-major
+ * [p][heads][head_dim].  out_dev: [p][heads][head_dim] fp32 or NULL to discard.
+ */
+int sh_prefill(sh_handle h, const void *q_dev, const void *k_dev, const void *v_dev, int p,
+               float *out_dev, void *stream);
+
+/*
+ * Algorithm 2 for every unit, if the cache is full (n == B): importance
+ * record I_j = number of the last w steps at which token j was below the
+ * threshold; the r newest tokens are not candidates; the m candidates with
+ * the largest I are dropped, the oldest first among equal I; survivors keep
+ * their order (K, V, record and positions are compacted in place); n <- n-m.
+ * A no-op when n < B.  *evicted_per_unit (may be NULL) receives m or 0.
+ */
+int sh_compress(sh_handle h, void *stream, int *evicted_per_unit);
+
+/*
+ * Selection of Algorithm 2 on caller-supplied records, for testing the
+ * selection kernel on its own: counters_dev [units][n] uint16 (tokens in
+ * position order); evicted_dev [units][m] int32 receives the indices of the
+ * dropped tokens in ascending order.  Needs 0 <= r, 1 <= m <= n - r,
+ * n <= 65535, every counter <= 16384.  Uses no handle and no workspace.
+ */
+int sh_select(const uint16_t *counters_dev, int units, int n, int r, int m, int32_t *evicted_dev,
+              void *stream);
+
+/*
+ * Snapshot for checking and checkpointing; synchronises `stream`.  Any output
+ * pointer may be NULL.  n_out: live tokens per unit.  t_out: tokens streamed.
+ * pos_host [heads][B] int32: stream positions (1-based) of slots [0,n), 0 beyond.
+ * counters_host [heads][B] uint16: importance record I of Algorithm 2 at the
+ * current step, 0 beyond n.  low_host [heads][ceil(B/32)] uint32: bit j%32 of
+ * word j/32 = the last step's comparison alpha_j < 1/t for the token now in slot j
+ * (a compression that followed the step has already moved the bits with their tokens).
+ */
+int sh_state(sh_handle h, void *stream, int *n_out, long long *t_out, int32_t *pos_host,
+             uint16_t *counters_host, uint32_t *low_host);
+
+/* Stored K and V rows of one unit as fp32 (int4: dequantised), [B][head_dim]
+ * each on the host; rows beyond n are whatever the slots hold.  Synchronises. */
+int sh_export_unit(sh_handle h, int unit, float *K_host, float *V_host, void *stream);
+
+/*
+ * Resume from a workspace image: after the caller has copied back a saved
+ * copy of the whole workspace, set the host counters that went with it.
+ */
+int sh_restore(sh_handle h, int n, long long t);
+
+/* Number of kernels this handle has launched since creation. */
+long long sh_launch_count(sh_handle h);
+
+/* Text for a status code; never NULL. */
+const char *sh_strerror(int status);
+
+/* cudaGetErrorString of the last CUDA failure seen by this handle ("" if none). */
+const char *sh_last_cuda_error(sh_handle h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SCISSORHANDS_H_ */

@@ -1,0 +1,228 @@
+"""ctypes binding of libscissorhands.so: argument marshalling only.
+
+Every function mirrors one entry point of ``include/scissorhands.h``.  Device
+buffers are torch CUDA tensors (PyTorch is used for device memory and streams
+only); the kernels do all of the method's work.  There is no CPU fallback: if
+the library cannot be loaded this module raises at import.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Tuple
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+SH_OK, SH_EINVAL, SH_EFULL, SH_ESTATE, SH_ECUDA, SH_ENOMEM = 0, -1, -2, -3, -4, -5
+SH_F32, SH_F16, SH_BF16, SH_INT4_G64_F16 = 0, 1, 2, 3
+SH_OPT_SOFTMAX_SCALE, SH_OPT_SPLIT, SH_OPT_AUTO_COMPRESS = 0, 1, 2
+
+DTYPE_CODE = {"f32": SH_F32, "f16": SH_F16, "bf16": SH_BF16, "int4": SH_INT4_G64_F16}
+INPUT_TORCH_DTYPE = {SH_F32: torch.float32, SH_F16: torch.float16, SH_BF16: torch.bfloat16,
+                     SH_INT4_G64_F16: torch.float16}
+
+EXPORTS = ["sh_create", "sh_destroy", "sh_workspace_bytes", "sh_bind", "sh_set_option", "sh_decode_step",
+           "sh_decode_step_host", "sh_prefill", "sh_compress", "sh_select", "sh_state", "sh_export_unit",
+           "sh_restore", "sh_launch_count", "sh_strerror", "sh_last_cuda_error"]
+
+
+def _load() -> C.CDLL:
+    path = _build.LIB
+    if _build.stale():
+        try:
+            path = _build.build()
+        except Exception as e:  # no nvcc here: use what was shipped, if anything
+            if not os.path.exists(_build.LIB):
+                raise ImportError(f"libscissorhands.so is not built and cannot be built: {e}") from e
+    lib = C.CDLL(path)
+    vp, ip, llp = C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_longlong)
+    lib.sh_create.argtypes = [C.c_int] * 7 + [C.POINTER(vp)]
+    lib.sh_destroy.argtypes = [vp]
+    lib.sh_destroy.restype = None
+    lib.sh_workspace_bytes.argtypes = [vp]
+    lib.sh_workspace_bytes.restype = C.c_size_t
+    lib.sh_bind.argtypes = [vp, vp, C.c_size_t, vp]
+    lib.sh_set_option.argtypes = [vp, C.c_int, C.c_double]
+    lib.sh_decode_step.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.sh_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.sh_prefill.argtypes = [vp, vp, vp, vp, C.c_int, vp, vp]
+    lib.sh_compress.argtypes = [vp, vp, ip]
+    lib.sh_select.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
+    lib.sh_state.argtypes = [vp, vp, ip, llp, vp, vp, vp]
+    lib.sh_export_unit.argtypes = [vp, C.c_int, vp, vp, vp]
+    lib.sh_restore.argtypes = [vp, C.c_int, C.c_longlong]
+    lib.sh_launch_count.argtypes = [vp]
+    lib.sh_launch_count.restype = C.c_longlong
+    lib.sh_strerror.argtypes = [C.c_int]
+    lib.sh_strerror.restype = C.c_char_p
+    lib.sh_last_cuda_error.argtypes = [vp]
+    lib.sh_last_cuda_error.restype = C.c_char_p
+    return lib
+
+
+lib = _load()
+
+
+class ShError(RuntimeError):
+    def __init__(self, status: int, detail: str = ""):
+        self.status = status
+        msg = lib.sh_strerror(status).decode()
+        super().__init__(f"libscissorhands: {msg} ({status})" + (f": {detail}" if detail else ""))
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+def _dev(t: torch.Tensor, dtype: torch.dtype, numel: int, what: str) -> int:
+    if not (t.is_cuda and t.is_contiguous() and t.dtype == dtype and t.numel() == numel):
+        raise ValueError(f"{what}: need a contiguous CUDA tensor of {numel} x {dtype}, got "
+                         f"{tuple(t.shape)} {t.dtype} on {t.device}")
+    return t.data_ptr()
+
+
+class Handle:
+    """One budgeted KV cache: ``heads`` independent units of one layer.
+
+    Mirrors ``sh_create`` + ``sh_bind``; the workspace is a torch uint8 tensor
+    owned by this object.
+    """
+
+    def __init__(self, B: int, r: int, w: int, m: int, heads: int, head_dim: int, dtype, device="cuda:0",
+                 split: Optional[int] = None, scale: Optional[float] = None, auto_compress: bool = True):
+        self.dtype = DTYPE_CODE[dtype] if isinstance(dtype, str) else int(dtype)
+        self.B, self.r, self.w, self.m, self.U, self.D = B, r, w, m, heads, head_dim
+        self.Bw = (B + 31) // 32
+        self.device = torch.device(device)
+        self.in_dtype = INPUT_TORCH_DTYPE.get(self.dtype, torch.float16)
+        h = C.c_void_p()
+        rc = lib.sh_create(B, r, w, m, heads, head_dim, self.dtype, C.byref(h))
+        if rc:
+            raise ShError(rc)
+        self._h = h
+        if scale is not None:
+            self.set_option(SH_OPT_SOFTMAX_SCALE, scale)
+        if split is not None:
+            self.set_option(SH_OPT_SPLIT, split)
+        self.set_option(SH_OPT_AUTO_COMPRESS, 1.0 if auto_compress else 0.0)
+        self.workspace_bytes = int(lib.sh_workspace_bytes(h))
+        with torch.cuda.device(self.device):
+            self.slab = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device=self.device)
+            off = (-self.slab.data_ptr()) % 256
+            self._slab_ptr = self.slab.data_ptr() + off
+            self._slab_off = off
+            self._check(lib.sh_bind(h, self._slab_ptr, self.workspace_bytes, _stream_ptr(None)))
+
+    def __del__(self):
+        h, self._h = getattr(self, "_h", None), None
+        if h:
+            lib.sh_destroy(h)
+
+    def _check(self, rc: int):
+        if rc:
+            raise ShError(rc, lib.sh_last_cuda_error(self._h).decode() if rc == SH_ECUDA else "")
+
+    # -- sh_set_option -------------------------------------------------------
+    def set_option(self, key: int, value: float):
+        self._check(lib.sh_set_option(self._h, key, float(value)))
+
+    # -- sh_decode_step ------------------------------------------------------
+    def decode_step(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
+                    out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        n = self.U * self.D
+        if out is None:
+            out = torch.empty(self.U, self.D, dtype=torch.float32, device=self.device)
+        self._check(lib.sh_decode_step(self._h, _dev(q, self.in_dtype, n, "q"), _dev(k_new, self.in_dtype, n, "k_new"),
+                                       _dev(v_new, self.in_dtype, n, "v_new"), _dev(out, torch.float32, n, "out"),
+                                       _stream_ptr(stream)))
+        return out
+
+    # -- sh_decode_step_host ---------------------------------------------------
+    def decode_step_host(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, out: torch.Tensor,
+                         stream=None) -> torch.Tensor:
+        n = self.U * self.D
+        for t, dt, what in ((q, self.in_dtype, "q"), (k_new, self.in_dtype, "k_new"), (v_new, self.in_dtype, "v_new"),
+                            (out, torch.float32, "out")):
+            if t.is_cuda or not t.is_contiguous() or t.dtype != dt or t.numel() != n:
+                raise ValueError(f"{what}: need a contiguous host tensor of {n} x {dt}")
+        self._check(lib.sh_decode_step_host(self._h, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(),
+                                            _stream_ptr(stream)))
+        return out
+
+    # -- sh_prefill ------------------------------------------------------------
+    def prefill(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: Optional[torch.Tensor] = None,
+                stream=None):
+        p = q.shape[0]
+        n = p * self.U * self.D
+        optr = _dev(out, torch.float32, n, "out") if out is not None else None
+        self._check(lib.sh_prefill(self._h, _dev(q, self.in_dtype, n, "q"), _dev(k, self.in_dtype, n, "k"),
+                                   _dev(v, self.in_dtype, n, "v"), p, optr, _stream_ptr(stream)))
+        return out
+
+    # -- sh_compress -------------------------------------------------------------
+    def compress(self, stream=None) -> int:
+        ev = C.c_int(0)
+        self._check(lib.sh_compress(self._h, _stream_ptr(stream), C.byref(ev)))
+        return ev.value
+
+    # -- sh_state ------------------------------------------------------------------
+    def state(self, pos: bool = True, counters: bool = True, low: bool = True, stream=None):
+        """Returns ``(n, t, pos [U,n] int32 | None, counters [U,n] uint16 | None,
+        low [U,n] bool | None)`` on the host."""
+        n, t = C.c_int(0), C.c_longlong(0)
+        pos_a = np.zeros((self.U, self.B), dtype=np.int32) if pos else None
+        cnt_a = np.zeros((self.U, self.B), dtype=np.uint16) if counters else None
+        low_a = np.zeros((self.U, self.Bw), dtype=np.uint32) if low else None
+        ptr = lambda a: a.ctypes.data if a is not None else None
+        self._check(lib.sh_state(self._h, _stream_ptr(stream), C.byref(n), C.byref(t), ptr(pos_a), ptr(cnt_a),
+                                 ptr(low_a)))
+        nn = n.value
+        low_b = None
+        if low:
+            bits = np.unpackbits(low_a.view(np.uint8), axis=1, bitorder="little")
+            low_b = bits[:, :nn].astype(bool)
+            assert not bits[:, nn:].any(), "record bits set beyond the live slots"
+        return (nn, t.value, pos_a[:, :nn] if pos else None, cnt_a[:, :nn] if counters else None, low_b)
+
+    @property
+    def n(self) -> int:
+        n = C.c_int(0)
+        self._check(lib.sh_state(self._h, _stream_ptr(None), C.byref(n), None, None, None, None))
+        return n.value
+
+    # -- sh_export_unit ---------------------------------------------------------------
+    def export_unit(self, unit: int, stream=None) -> Tuple[np.ndarray, np.ndarray]:
+        K = np.zeros((self.B, self.D), dtype=np.float32)
+        V = np.zeros((self.B, self.D), dtype=np.float32)
+        self._check(lib.sh_export_unit(self._h, unit, K.ctypes.data, V.ctypes.data, _stream_ptr(stream)))
+        return K, V
+
+    # -- checkpoint / sh_restore -------------------------------------------------------
+    def snapshot(self):
+        """Copy of the whole workspace plus the host counters that go with it."""
+        n, t, *_ = self.state(pos=False, counters=False, low=False)
+        return self.slab.clone(), n, t
+
+    def restore(self, snap):
+        slab, n, t = snap
+        self.slab.copy_(slab)
+        self._check(lib.sh_restore(self._h, n, t))
+
+    @property
+    def launch_count(self) -> int:
+        return int(lib.sh_launch_count(self._h))
+
+
+def select(counters: torch.Tensor, r: int, m: int, stream=None) -> torch.Tensor:
+    """``sh_select``: counters ``[units, n]`` (CUDA, any integer dtype, values
+    <= 16384) -> dropped indices ``[units, m]`` int32, ascending."""
+    units, n = counters.shape
+    c16 = counters.to(torch.int16).contiguous()   # values <= 16384: same bits as uint16
+    out = torch.empty(units, m, dtype=torch.int32, device=counters.device)
+    rc = lib.sh_select(c16.data_ptr(), units, n, r, m, out.data_ptr(), _stream_ptr(stream))
+    if rc:
+        raise ShError(rc)
+    return out

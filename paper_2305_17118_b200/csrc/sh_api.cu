@@ -1,0 +1,358 @@
+// C ABI and host state machine of libscissorhands.  The number of live tokens
+// n and the step counter t are the same for every unit (each unit appends one
+// token per step and drops exactly m when full), so they live on the host and
+// no call needs to read anything back from the device to schedule its work.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "sh_internal.h"
+
+namespace {
+
+constexpr double LOG2E = 1.4426950408889634;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+void make_layout(sh_context *c) {
+    ShLayout &L = c->L;
+    const size_t U = c->U, B = c->B, D = c->D;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        size_t at = off;
+        off = align_up(off + bytes, 256);
+        return at;
+    };
+    L.K = take(U * B * c->row_bytes);
+    L.V = take(U * B * c->row_bytes);
+    const size_t sc = c->dtype == SH_INT4_G64_F16 ? U * B * (D / 64) * 2 : 0;
+    L.Ks = take(sc);
+    L.Vs = take(sc);
+    L.hist = take(U * (size_t)c->w * c->Bw * 4);
+    L.pos = take(U * B * 4);
+    L.src_idx = take(U * B * 4);
+    L.counters = take(U * B * 2);
+    L.xport = take(2 * B * D * 4);
+    L.stage_q = take(U * (size_t)c->in_bytes);
+    L.stage_k = take(U * (size_t)c->in_bytes);
+    L.stage_v = take(U * (size_t)c->in_bytes);
+    L.stage_out = take(U * D * 4);
+    L.total = off;
+}
+
+int cuda_fail(sh_context *c, cudaError_t e) {
+    if (c) c->last_err = e;
+    return SH_ECUDA;
+}
+
+int default_split(int U, int B) {
+    // Aim for at least two CTAs per SM's worth of work items, while every
+    // CTA still owns a few dozen rows.
+    int s = 1;
+    while (s < 8 && (long long)U * s < 2 * 148 && B / (2 * s) >= 32) s *= 2;
+    return s;
+}
+
+// Stored rows -> fp32, for sh_export_unit.
+__global__ void sh_export_kernel(const char *K, const char *V, const __half *Ks, const __half *Vs, float *dst,
+                                 int B, int D, int dtype, int row_bytes) {
+    const int total = B * D;
+    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < 2 * total; idx += gridDim.x * blockDim.x) {
+        const int which = idx / total, rem = idx % total, j = rem / D, i = rem % D;
+        const char *row = (which ? V : K) + (size_t)j * row_bytes;
+        float val;
+        if (dtype == SH_F32) val = reinterpret_cast<const float *>(row)[i];
+        else if (dtype == SH_F16) val = __half2float(reinterpret_cast<const __half *>(row)[i]);
+        else if (dtype == SH_BF16) val = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(row)[i]);
+        else {
+            const uint32_t word = reinterpret_cast<const uint32_t *>(row)[i >> 3];
+            const int e = i & 7, nib = (e >> 1) + 4 * (e & 1);
+            const int code = (int)((word >> (4 * nib)) & 0xFu) - 8;
+            const __half *sc = (which ? Vs : Ks) + (size_t)j * (D / 64);
+            val = (float)code * __half2float(sc[i >> 6]);
+        }
+        dst[idx] = val;
+    }
+}
+
+int do_compress(sh_context *c, cudaStream_t s) {
+    SelectParams sp = {};
+    sp.hist = reinterpret_cast<const uint32_t *>(c->slab + c->L.hist);
+    sp.counters = nullptr;
+    sp.src_idx = reinterpret_cast<int32_t *>(c->slab + c->L.src_idx);
+    sp.evicted = nullptr;
+    sp.U = c->U; sp.B = c->B; sp.Bw = c->Bw; sp.w = c->w; sp.n = c->n; sp.r = c->r; sp.m = c->m;
+    sp.cmax = c->w;
+    cudaError_t e = sh_launch_select(sp, true, s, &c->launches);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    CompactParams cp = {};
+    cp.K = c->slab + c->L.K; cp.V = c->slab + c->L.V;
+    cp.Ks = c->slab + c->L.Ks; cp.Vs = c->slab + c->L.Vs;
+    cp.hist = reinterpret_cast<uint32_t *>(c->slab + c->L.hist);
+    cp.pos = reinterpret_cast<int32_t *>(c->slab + c->L.pos);
+    cp.src_idx = sp.src_idx;
+    cp.U = c->U; cp.B = c->B; cp.Bw = c->Bw; cp.w = c->w; cp.n = c->n; cp.m = c->m;
+    cp.row_bytes = c->row_bytes;
+    cp.scale_bytes = c->dtype == SH_INT4_G64_F16 ? (c->D / 64) * 2 : 0;
+    e = sh_launch_compact(cp, s, &c->launches);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->n -= c->m;
+    return SH_OK;
+}
+
+int do_step(sh_context *c, const void *q, const void *k, const void *v, float *out, cudaStream_t s,
+            bool compress_after) {
+    DecodeParams p = {};
+    p.q = q; p.k_new = k; p.v_new = v; p.out = out;
+    p.K = c->slab + c->L.K; p.V = c->slab + c->L.V;
+    p.Ks = c->slab + c->L.Ks; p.Vs = c->slab + c->L.Vs;
+    p.hist = reinterpret_cast<uint32_t *>(c->slab + c->L.hist);
+    p.pos = reinterpret_cast<int32_t *>(c->slab + c->L.pos);
+    p.U = c->U; p.B = c->B; p.Bw = c->Bw; p.w = c->w;
+    p.n = c->n + 1;
+    p.t = (int)(c->t + 1);
+    p.hist_row = (int)((c->t + 1) % c->w);
+    p.scale_log2e = (float)((double)c->scale * LOG2E);
+    cudaError_t e = sh_launch_decode(c, p, s, &c->launches);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->started = true;
+    c->n += 1;
+    c->t += 1;
+    if (compress_after && c->n == c->B) return do_compress(c, s);
+    return SH_OK;
+}
+
+bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+}  // namespace
+
+extern "C" {
+
+int sh_create(int B, int r, int w, int m, int heads, int head_dim, int dtype, sh_handle *out) {
+    if (!out) return SH_EINVAL;
+    *out = nullptr;
+    if (B < 1 || B > 65535 || r < 0 || w < 1 || w > 16384 || m < 1 || m > B - r || heads < 1) return SH_EINVAL;
+    if (head_dim != 64 && head_dim != 128) return SH_EINVAL;
+    if (dtype < SH_F32 || dtype > SH_INT4_G64_F16) return SH_EINVAL;
+    sh_context *c = new (std::nothrow) sh_context();
+    if (!c) return SH_ENOMEM;
+    c->B = B; c->r = r; c->w = w; c->m = m; c->U = heads; c->D = head_dim; c->dtype = dtype;
+    c->Bw = (B + 31) / 32;
+    c->row_bytes = dtype == SH_F32 ? head_dim * 4 : (dtype == SH_INT4_G64_F16 ? head_dim / 2 : head_dim * 2);
+    c->in_bytes = dtype == SH_F32 ? head_dim * 4 : head_dim * 2;
+    c->n = 0; c->t = 0;
+    c->scale = (float)(1.0 / std::sqrt((double)head_dim));
+    c->split = default_split(heads, B);
+    c->auto_compress = 1;
+    c->started = false;
+    c->slab = nullptr; c->slab_bytes = 0;
+    c->launches = 0;
+    c->last_err = cudaSuccess;
+    make_layout(c);
+    *out = c;
+    return SH_OK;
+}
+
+void sh_destroy(sh_handle h) { delete h; }
+
+size_t sh_workspace_bytes(sh_handle h) { return h ? h->L.total : 0; }
+
+int sh_bind(sh_handle h, void *slab_dev, size_t bytes, void *stream) {
+    if (!h || !slab_dev) return SH_EINVAL;
+    if (reinterpret_cast<uintptr_t>(slab_dev) & 255u) return SH_EINVAL;
+    if (bytes < h->L.total) return SH_ENOMEM;
+    cudaError_t e = cudaMemsetAsync(slab_dev, 0, h->L.total, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->slab = static_cast<char *>(slab_dev);
+    h->slab_bytes = bytes;
+    h->n = 0; h->t = 0;
+    h->started = false;
+    return SH_OK;
+}
+
+int sh_set_option(sh_handle h, int key, double value) {
+    if (!h) return SH_EINVAL;
+    if (h->started) return SH_ESTATE;
+    switch (key) {
+        case SH_OPT_SOFTMAX_SCALE:
+            if (!(value > 0.0) || !std::isfinite(value)) return SH_EINVAL;
+            h->scale = (float)value;
+            return SH_OK;
+        case SH_OPT_SPLIT: {
+            const int s = (int)value;
+            if (s != 1 && s != 2 && s != 4 && s != 8) return SH_EINVAL;
+            h->split = s;
+            return SH_OK;
+        }
+        case SH_OPT_AUTO_COMPRESS:
+            h->auto_compress = value != 0.0;
+            return SH_OK;
+        default: return SH_EINVAL;
+    }
+}
+
+int sh_decode_step(sh_handle h, const void *q_dev, const void *k_new_dev, const void *v_new_dev,
+                   float *attn_out_dev, void *stream) {
+    if (!h || !q_dev || !k_new_dev || !v_new_dev || !attn_out_dev) return SH_EINVAL;
+    if (misaligned(q_dev) || misaligned(k_new_dev) || misaligned(v_new_dev)) return SH_EINVAL;
+    if (!h->slab) return SH_ESTATE;
+    if (h->n >= h->B) return SH_EFULL;
+    return do_step(h, q_dev, k_new_dev, v_new_dev, attn_out_dev, (cudaStream_t)stream, h->auto_compress != 0);
+}
+
+int sh_decode_step_host(sh_handle h, const void *q_host, const void *k_new_host, const void *v_new_host,
+                        float *attn_out_host, void *stream) {
+    if (!h || !q_host || !k_new_host || !v_new_host || !attn_out_host) return SH_EINVAL;
+    if (!h->slab) return SH_ESTATE;
+    if (h->n >= h->B) return SH_EFULL;
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t inb = (size_t)h->U * h->in_bytes, outb = (size_t)h->U * h->D * 4;
+    char *sq = h->slab + h->L.stage_q, *sk = h->slab + h->L.stage_k, *sv = h->slab + h->L.stage_v;
+    float *so = reinterpret_cast<float *>(h->slab + h->L.stage_out);
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(sq, q_host, inb, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(h, e);
+    if ((e = cudaMemcpyAsync(sk, k_new_host, inb, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(h, e);
+    if ((e = cudaMemcpyAsync(sv, v_new_host, inb, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(h, e);
+    // The result leaves before any compression that follows, so the copy
+    // overlaps nothing it depends on and the caller sees the step's output.
+    int rc = do_step(h, sq, sk, sv, so, s, false);
+    if (rc != SH_OK) return rc;
+    if ((e = cudaMemcpyAsync(attn_out_host, so, outb, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(h, e);
+    if (h->auto_compress && h->n == h->B) {
+        rc = do_compress(h, s);
+        if (rc != SH_OK) return rc;
+    }
+    if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(h, e);
+    return SH_OK;
+}
+
+int sh_prefill(sh_handle h, const void *q_dev, const void *k_dev, const void *v_dev, int p, float *out_dev,
+               void *stream) {
+    if (!h || !q_dev || !k_dev || !v_dev || p < 0) return SH_EINVAL;
+    if (misaligned(q_dev) || misaligned(k_dev) || misaligned(v_dev)) return SH_EINVAL;
+    if (!h->slab) return SH_ESTATE;
+    if (h->n >= h->B) return SH_EFULL;
+    const size_t in_stride = (size_t)h->U * h->in_bytes, out_stride = (size_t)h->U * h->D;
+    float *sink = reinterpret_cast<float *>(h->slab + h->L.stage_out);
+    for (int i = 0; i < p; ++i) {
+        const char *q = static_cast<const char *>(q_dev) + i * in_stride;
+        const char *k = static_cast<const char *>(k_dev) + i * in_stride;
+        const char *v = static_cast<const char *>(v_dev) + i * in_stride;
+        float *o = out_dev ? out_dev + i * out_stride : sink;
+        int rc = do_step(h, q, k, v, o, (cudaStream_t)stream, true);
+        if (rc != SH_OK) return rc;
+    }
+    return SH_OK;
+}
+
+int sh_compress(sh_handle h, void *stream, int *evicted_per_unit) {
+    if (!h) return SH_EINVAL;
+    if (!h->slab) return SH_ESTATE;
+    if (evicted_per_unit) *evicted_per_unit = 0;
+    if (h->n < h->B) return SH_OK;
+    int rc = do_compress(h, (cudaStream_t)stream);
+    if (rc == SH_OK && evicted_per_unit) *evicted_per_unit = h->m;
+    return rc;
+}
+
+int sh_select(const uint16_t *counters_dev, int units, int n, int r, int m, int32_t *evicted_dev, void *stream) {
+    if (!counters_dev || !evicted_dev || units < 1 || n < 1 || n > 65535 || r < 0 || m < 1 || m > n - r)
+        return SH_EINVAL;
+    SelectParams sp = {};
+    sp.hist = nullptr;
+    sp.counters = counters_dev;
+    sp.src_idx = nullptr;
+    sp.evicted = evicted_dev;
+    sp.U = units; sp.B = n; sp.Bw = (n + 31) / 32; sp.w = 0; sp.n = n; sp.r = r; sp.m = m;
+    sp.cmax = 16384;
+    cudaError_t e = sh_launch_select(sp, false, (cudaStream_t)stream, nullptr);
+    return e == cudaSuccess ? SH_OK : SH_ECUDA;
+}
+
+int sh_state(sh_handle h, void *stream, int *n_out, long long *t_out, int32_t *pos_host, uint16_t *counters_host,
+             uint32_t *low_host) {
+    if (!h) return SH_EINVAL;
+    if (!h->slab) return SH_ESTATE;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e;
+    if (n_out) *n_out = h->n;
+    if (t_out) *t_out = h->t;
+    const size_t U = h->U, B = h->B;
+    if (pos_host) {
+        e = cudaMemcpyAsync(pos_host, h->slab + h->L.pos, U * B * 4, cudaMemcpyDeviceToHost, s);
+        if (e != cudaSuccess) return cuda_fail(h, e);
+    }
+    if (counters_host) {
+        uint16_t *cd = reinterpret_cast<uint16_t *>(h->slab + h->L.counters);
+        e = sh_launch_counters(reinterpret_cast<const uint32_t *>(h->slab + h->L.hist), cd, h->U, h->B, h->Bw, h->w,
+                               h->n, s, &h->launches);
+        if (e != cudaSuccess) return cuda_fail(h, e);
+        e = cudaMemcpyAsync(counters_host, cd, U * B * 2, cudaMemcpyDeviceToHost, s);
+        if (e != cudaSuccess) return cuda_fail(h, e);
+    }
+    if (low_host) {
+        const int row = (int)(h->t % h->w);
+        const char *src = h->slab + h->L.hist + (size_t)row * h->Bw * 4;
+        e = cudaMemcpy2DAsync(low_host, (size_t)h->Bw * 4, src, (size_t)h->w * h->Bw * 4, (size_t)h->Bw * 4, U,
+                              cudaMemcpyDeviceToHost, s);
+        if (e != cudaSuccess) return cuda_fail(h, e);
+    }
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    return SH_OK;
+}
+
+int sh_export_unit(sh_handle h, int unit, float *K_host, float *V_host, void *stream) {
+    if (!h || unit < 0 || unit >= h->U || !K_host || !V_host) return SH_EINVAL;
+    if (!h->slab) return SH_ESTATE;
+    cudaStream_t s = (cudaStream_t)stream;
+    float *dst = reinterpret_cast<float *>(h->slab + h->L.xport);
+    const size_t B = h->B, D = h->D;
+    const char *K = h->slab + h->L.K + (size_t)unit * B * h->row_bytes;
+    const char *V = h->slab + h->L.V + (size_t)unit * B * h->row_bytes;
+    const __half *Ks = reinterpret_cast<const __half *>(h->slab + h->L.Ks) + (size_t)unit * B * (D / 64);
+    const __half *Vs = reinterpret_cast<const __half *>(h->slab + h->L.Vs) + (size_t)unit * B * (D / 64);
+    sh_export_kernel<<<64, 256, 0, s>>>(K, V, Ks, Vs, dst, h->B, h->D, h->dtype, h->row_bytes);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->launches += 1;
+    if ((e = cudaMemcpyAsync(K_host, dst, B * D * 4, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(h, e);
+    if ((e = cudaMemcpyAsync(V_host, dst + B * D, B * D * 4, cudaMemcpyDeviceToHost, s)) != cudaSuccess)
+        return cuda_fail(h, e);
+    if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(h, e);
+    return SH_OK;
+}
+
+int sh_restore(sh_handle h, int n, long long t) {
+    if (!h || n < 0 || n >= h->B || t < n) return SH_EINVAL;
+    if (!h->slab) return SH_ESTATE;
+    h->n = n;
+    h->t = t;
+    h->started = true;
+    return SH_OK;
+}
+
+long long sh_launch_count(sh_handle h) { return h ? h->launches : 0; }
+
+const char *sh_strerror(int status) {
+    switch (status) {
+        case SH_OK: return "ok";
+        case SH_EINVAL: return "invalid argument";
+        case SH_EFULL: return "cache is full: compress before the next step";
+        case SH_ESTATE: return "call out of order (no workspace bound, or option set after the first step)";
+        case SH_ECUDA: return "CUDA runtime error";
+        case SH_ENOMEM: return "allocation failed or workspace too small";
+        default: return "unknown status";
+    }
+}
+
+const char *sh_last_cuda_error(sh_handle h) {
+    if (!h || h->last_err == cudaSuccess) return "";
+    return cudaGetErrorString(h->last_err);
+}
+
+}  // extern "C"

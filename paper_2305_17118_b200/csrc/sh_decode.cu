@@ -1,0 +1,483 @@
+// Fused decode step: append + logits + stable softmax + P.V + importance-record
+// bits, one CTA (or one cluster of S CTAs) per (sequence, head) unit.
+//
+// The work is a GEMV per unit (one query against n cached rows), so it is bound
+// by HBM bandwidth and runs on CUDA cores.  Layout of the work inside a CTA:
+// a K (or V) row of D elements is D*es bytes = LPR lanes x 16 bytes, so a warp
+// reads RPW = 32/LPR whole rows per 128-bit load instruction, fully coalesced,
+// and every lane keeps R such loads in flight before it touches the data.
+// Logits stay in shared memory until the softmax denominator is known, so K and
+// V are each read from HBM exactly once per step and the record bits
+// (alpha_j < 1/t  <=>  e_j * t < L) cost one ballot word per 32 slots.
+#include <cooperative_groups.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "sh_internal.h"
+
+namespace cg = cooperative_groups;
+
+namespace {
+
+// ---------------------------------------------------------------- loads / stores
+__device__ __forceinline__ uint4 ld_stream(const void *p) {
+    // read-only, read-once data: keep it out of L1
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint4 ld_plain(const void *p) { return *reinterpret_cast<const uint4 *>(p); }
+__device__ __forceinline__ void st_plain(void *p, const uint4 &v) { *reinterpret_cast<uint4 *>(p) = v; }
+
+// ---------------------------------------------------------------- element traits
+// A "chunk" is the 16 bytes one lane loads from a stored row; EPL elements.
+template <int DT> struct Elem;
+
+template <> struct Elem<SH_F32> {
+    static constexpr int EPL = 4;        // elements per 16-byte chunk of a stored row
+    static __device__ __forceinline__ void cvt(const uint4 &r, float *f) {
+        f[0] = __uint_as_float(r.x); f[1] = __uint_as_float(r.y);
+        f[2] = __uint_as_float(r.z); f[3] = __uint_as_float(r.w);
+    }
+};
+template <> struct Elem<SH_F16> {
+    static constexpr int EPL = 8;
+    static __device__ __forceinline__ void cvt(const uint4 &r, float *f) {
+        const __half2 *h = reinterpret_cast<const __half2 *>(&r);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float2 t = __half22float2(h[i]);
+            f[2 * i] = t.x; f[2 * i + 1] = t.y;
+        }
+    }
+};
+template <> struct Elem<SH_BF16> {
+    static constexpr int EPL = 8;
+    static __device__ __forceinline__ void cvt(const uint4 &r, float *f) {
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            f[2 * i] = __uint_as_float(w[i] << 16);
+            f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    }
+};
+// int4 store: a chunk is 32 codes.  Word k of the chunk holds elements 8k..8k+7;
+// element e of a word sits in nibble (e>>1) + 4*(e&1), biased by +8, so that
+// ((word >> 4i) & 0x000F000F) | 0x64006400 is the half2 (1024+e_{2i}, 1024+e_{2i+1}).
+template <> struct Elem<SH_INT4_G64_F16> {
+    static constexpr int EPL = 32;
+    static __device__ __forceinline__ void cvt(const uint4 &r, float *f) {
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+        const __half2 bias = __floats2half2_rn(1032.f, 1032.f);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint32_t bits = ((w[k] >> (4 * i)) & 0x000F000Fu) | 0x64006400u;
+                __half2 h = __hsub2(*reinterpret_cast<__half2 *>(&bits), bias);
+                float2 t = __half22float2(h);
+                f[8 * k + 2 * i] = t.x; f[8 * k + 2 * i + 1] = t.y;
+            }
+        }
+    }
+};
+
+template <int DT> __device__ __forceinline__ int stored_row_bytes(int D) {
+    return DT == SH_F32 ? D * 4 : (DT == SH_INT4_G64_F16 ? D / 2 : D * 2);
+}
+
+// Load this lane's EPL elements of a q / k_new / v_new row as fp32.
+template <int DT> __device__ __forceinline__ void load_input(const void *row, int c, float *f) {
+    using E = Elem<DT>;
+    if constexpr (DT == SH_INT4_G64_F16) {
+        const char *p = reinterpret_cast<const char *>(row) + c * 64;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) Elem<SH_F16>::cvt(ld_plain(p + 16 * k), f + 8 * k);
+    } else {
+        E::cvt(ld_plain(reinterpret_cast<const char *>(row) + c * 16), f);
+    }
+}
+
+// Quantise this lane's 32 elements (half a group of 64; the partner lane c^1
+// holds the other half): a = max|x| over the group, sc = fp16(a / 7),
+// code = clamp(rint(x / sc), -7, 7), all in IEEE fp32.  On return f holds the
+// dequantised values code*sc; the packed codes and the scale are returned.
+__device__ __forceinline__ uint4 quantize32(float *f, float &sc_out) {
+    float a = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) a = fmaxf(a, fabsf(f[i]));
+    a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
+    const float sc = __half2float(__float2half_rn(__fdiv_rn(a, 7.0f)));
+    uint32_t w[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        w[k] = 0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            float code = 0.f;
+            if (sc != 0.f) code = fminf(fmaxf(rintf(__fdiv_rn(f[8 * k + e], sc)), -7.f), 7.f);
+            f[8 * k + e] = code * sc;
+            w[k] |= (uint32_t)((int)code + 8) << (4 * ((e >> 1) + 4 * (e & 1)));
+        }
+    }
+    sc_out = sc;
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// ---------------------------------------------------------------- reductions
+// Reduce CNT per-lane values across the LPR lanes of a row group so that the
+// lanes end up owning different rows: at each halving a lane keeps the upper or
+// lower half of its values according to one bit of its chunk index and adds
+// what its partner sends.  Costs CNT-1 shuffles instead of CNT*log2(LPR).
+template <int CNT, int HALF> struct TransposeReduce {
+    static __device__ __forceinline__ void run(float *v, int c, int &rowi) {
+        if constexpr (HALF >= 1) {
+            if constexpr (CNT > 1) {
+                const bool up = (c & HALF) != 0;
+#pragma unroll
+                for (int k = 0; k < CNT / 2; ++k) {
+                    const float send = up ? v[k] : v[k + CNT / 2];
+                    const float keep = up ? v[k + CNT / 2] : v[k];
+                    v[k] = keep + __shfl_xor_sync(0xffffffffu, send, HALF);
+                }
+                rowi += up ? CNT / 2 : 0;
+                TransposeReduce<CNT / 2, HALF / 2>::run(v, c, rowi);
+            } else {
+                v[0] += __shfl_xor_sync(0xffffffffu, v[0], HALF);
+                TransposeReduce<1, HALF / 2>::run(v, c, rowi);
+            }
+        }
+    }
+};
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// ---------------------------------------------------------------- the kernel
+// DT dtype, D head_dim, NW warps per CTA, R rows in flight per lane,
+// S CTAs per unit (a thread-block cluster when S > 1).
+template <int DT, int D, int NW, int R, int S>
+__global__ void __launch_bounds__(NW * 32) sh_decode_kernel(const DecodeParams p) {
+    using E = Elem<DT>;
+    constexpr int EPL = E::EPL;
+    constexpr int LPR = D / EPL;     // lanes per row
+    constexpr int RPW = 32 / LPR;    // rows per warp-wide load
+    constexpr int PASS = NW * RPW;   // rows per CTA-wide load
+    constexpr bool Q4 = (DT == SH_INT4_G64_F16);
+    static_assert(LPR >= 1 && LPR <= 32 && (LPR & (LPR - 1)) == 0, "row must be 1..32 chunks");
+    static_assert(D <= NW * 32, "output reduction needs one thread per column");
+    const int ROWB = stored_row_bytes<DT>(D);
+    const int INB = (DT == SH_F32) ? D * 4 : D * 2;
+
+    extern __shared__ __align__(16) float smem[];
+    // s_sh[cap] | red[NW*D] | wred[NW] | xM[8] | xL[8] | xo[D]
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int sub = lane / LPR, c = lane % LPR;
+    const int u = blockIdx.x / S;
+    const int cr = (S > 1) ? (int)(blockIdx.x % S) : 0;
+    const int n = p.n, n_old = p.n - 1, B = p.B;
+
+    int chunk, lo;
+    if constexpr (S > 1) {
+        chunk = (((n + S - 1) / S) + 31) & ~31;
+        lo = cr * chunk;
+    } else {
+        chunk = (B + 31) & ~31;
+        lo = 0;
+    }
+    const int cap = (S > 1) ? ((((B + S - 1) / S) + 31) & ~31) : ((B + 31) & ~31);
+    float *s_sh = smem;
+    float *red = s_sh + cap;
+    float *wred = red + NW * D;
+    float *xM = wred + NW;
+    float *xL = xM + 8;
+    float *xo = xL + 8;
+
+    if constexpr (S > 1) cg::this_cluster().sync();   // every CTA of the cluster is running: its shared memory may be written
+
+    const int hi_all = min(n, lo + chunk);   // this CTA owns slots [lo, hi_all)
+    const int hi = min(n_old, hi_all);       // ... of which [lo, hi) are already cached
+    const bool has_new = (n_old >= lo) && (n_old < lo + chunk);
+    const int cnt = max(hi_all - lo, 0);
+
+    // ---- q chunk of this lane, fp32
+    float qf[EPL];
+    load_input<DT>(reinterpret_cast<const char *>(p.q) + (size_t)u * INB, c, qf);
+
+    const char *Kb = p.K + (size_t)u * B * ROWB;
+    const char *Vb = p.V + (size_t)u * B * ROWB;
+    const __half *Ksb = Q4 ? reinterpret_cast<const __half *>(p.Ks) + (size_t)u * B * (D / 64) : nullptr;
+    const __half *Vsb = Q4 ? reinterpret_cast<const __half *>(p.Vs) + (size_t)u * B * (D / 64) : nullptr;
+
+    // ---- logits of the cached rows
+    float lmax = -INFINITY;
+    for (int b0 = lo; b0 < hi; b0 += PASS * R) {
+        uint4 raw[R];
+        float rs[R];
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            const int j = b0 + i * PASS + warp * RPW + sub;
+            raw[i] = make_uint4(0, 0, 0, 0);
+            rs[i] = 1.f;
+            if (j < hi) {
+                raw[i] = ld_stream(Kb + (size_t)j * ROWB + c * 16);
+                if constexpr (Q4) rs[i] = __half2float(Ksb[(size_t)j * (D / 64) + (c >> 1)]);
+            }
+        }
+        float part[R];
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            float f[EPL];
+            E::cvt(raw[i], f);
+            float a = 0.f;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) a = fmaf(qf[e], f[e], a);
+            part[i] = Q4 ? a * rs[i] : a;
+        }
+        int rowi = 0;
+        TransposeReduce<R, LPR / 2>::run(part, c, rowi);
+        constexpr int NV = (LPR >= R) ? 1 : R / LPR;   // complete sums per lane
+        constexpr int WF = (LPR > R) ? LPR / R : 1;    // lanes holding the same sum
+        if ((c & (WF - 1)) == 0) {
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int j = b0 + (rowi + k) * PASS + warp * RPW + sub;
+                if (j < hi) {
+                    const float s = part[k] * p.scale_log2e;
+                    s_sh[j - lo] = s;
+                    lmax = fmaxf(lmax, s);
+                }
+            }
+        }
+    }
+
+    // ---- the token of this step: append it and score it (warp 0 of the owning CTA)
+    float fv_new[EPL];
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) fv_new[e] = 0.f;
+    if (has_new && warp == 0) {
+        float fk[EPL];
+        load_input<DT>(reinterpret_cast<const char *>(p.k_new) + (size_t)u * INB, c, fk);
+        load_input<DT>(reinterpret_cast<const char *>(p.v_new) + (size_t)u * INB, c, fv_new);
+        char *kdst = p.K + ((size_t)u * B + n_old) * ROWB + c * 16;
+        char *vdst = p.V + ((size_t)u * B + n_old) * ROWB + c * 16;
+        if constexpr (Q4) {
+            float sck, scv;
+            const uint4 ck = quantize32(fk, sck);
+            const uint4 cv = quantize32(fv_new, scv);
+            if (sub == 0) {
+                st_plain(kdst, ck);
+                st_plain(vdst, cv);
+                if ((c & 1) == 0) {
+                    reinterpret_cast<__half *>(p.Ks)[((size_t)u * B + n_old) * (D / 64) + (c >> 1)] = __float2half_rn(sck);
+                    reinterpret_cast<__half *>(p.Vs)[((size_t)u * B + n_old) * (D / 64) + (c >> 1)] = __float2half_rn(scv);
+                }
+            }
+        } else if (sub == 0) {
+            st_plain(kdst, ld_plain(reinterpret_cast<const char *>(p.k_new) + (size_t)u * INB + c * 16));
+            st_plain(vdst, ld_plain(reinterpret_cast<const char *>(p.v_new) + (size_t)u * INB + c * 16));
+        }
+        float a = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) a = fmaf(qf[e], fk[e], a);
+#pragma unroll
+        for (int o = LPR / 2; o; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        const float s = a * p.scale_log2e;
+        if (lane == 0) s_sh[n_old - lo] = s;
+        lmax = fmaxf(lmax, s);
+        if (lane == 0) p.pos[(size_t)u * B + n_old] = p.t;
+    }
+
+    // ---- max over the unit
+    lmax = warp_max(lmax);
+    if (lane == 0) wred[warp] = lmax;
+    __syncthreads();
+    float M = wred[0];
+#pragma unroll
+    for (int i = 1; i < NW; ++i) M = fmaxf(M, wred[i]);
+    if constexpr (S > 1) {
+        cg::cluster_group cluster = cg::this_cluster();
+        if (tid < S) cluster.map_shared_rank(xM, tid)[cr] = M;
+        cluster.sync();
+        M = xM[0];
+#pragma unroll
+        for (int i = 1; i < S; ++i) M = fmaxf(M, xM[i]);
+    }
+
+    // ---- exponentials and the denominator
+    float lsum = 0.f;
+    for (int j = tid; j < cnt; j += NW * 32) {
+        const float e = exp2f(s_sh[j] - M);
+        s_sh[j] = e;
+        lsum += e;
+    }
+    lsum = warp_sum(lsum);
+    __syncthreads();   // every thread has read wred (max) before it is reused
+    if (lane == 0) wred[warp] = lsum;
+    __syncthreads();
+    float L = 0.f;
+#pragma unroll
+    for (int i = 0; i < NW; ++i) L += wred[i];
+
+    // ---- P.V
+    float acc[EPL];
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+    for (int b0 = lo; b0 < hi; b0 += PASS * R) {
+        uint4 raw[R];
+        float pe[R];
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            const int j = b0 + i * PASS + warp * RPW + sub;
+            raw[i] = make_uint4(0, 0, 0, 0);
+            pe[i] = 0.f;
+            if (j < hi) {
+                raw[i] = ld_stream(Vb + (size_t)j * ROWB + c * 16);
+                pe[i] = s_sh[j - lo];
+                if constexpr (Q4) pe[i] *= __half2float(Vsb[(size_t)j * (D / 64) + (c >> 1)]);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            float f[EPL];
+            E::cvt(raw[i], f);
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) acc[e] = fmaf(pe[i], f[e], acc[e]);
+        }
+    }
+    if (has_new && warp == 0 && sub == 0) {
+        const float e_new = s_sh[n_old - lo];
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) acc[e] = fmaf(e_new, fv_new[e], acc[e]);
+    }
+#pragma unroll
+    for (int o = LPR; o < 32; o <<= 1) {
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], o);
+    }
+    if (sub == 0) {
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) red[warp * D + c * EPL + e] = acc[e];
+    }
+    __syncthreads();
+    float o = 0.f;
+    if (tid < D) {
+#pragma unroll
+        for (int i = 0; i < NW; ++i) o += red[i * D + tid];
+    }
+
+    if constexpr (S > 1) {
+        cg::cluster_group cluster = cg::this_cluster();
+        if (tid < D) xo[tid] = o;
+        if (tid < S) cluster.map_shared_rank(xL, tid)[cr] = L;
+        cluster.sync();
+        float Lt = 0.f;
+#pragma unroll
+        for (int i = 0; i < S; ++i) Lt += xL[i];
+        L = Lt;
+        if (cr == 0 && tid < D) {
+            float ot = 0.f;
+#pragma unroll
+            for (int i = 0; i < S; ++i) ot += cluster.map_shared_rank(xo, i)[tid];
+            p.out[(size_t)u * D + tid] = ot / L;
+        }
+    } else {
+        if (tid < D) p.out[(size_t)u * D + tid] = o / L;
+    }
+
+    // ---- record: low_j = [alpha_j < 1/t] = [e_j * t < L], one bit-plane row per step
+    {
+        const float tf = (float)p.t;
+        uint32_t *hrow = p.hist + ((size_t)u * p.w + p.hist_row) * p.Bw;
+        const int w_lo = lo >> 5;
+        const int w_hi = (S > 1 && cr != S - 1) ? min(p.Bw, (lo + chunk) >> 5) : p.Bw;
+        for (int wd = w_lo + warp; wd < w_hi; wd += NW) {
+            const int j = (wd << 5) + lane;   // slot
+            bool low = false;
+            if (j < hi_all) low = s_sh[j - lo] * tf < L;
+            const uint32_t word = __ballot_sync(0xffffffffu, low);
+            if (lane == 0) hrow[wd] = word;
+        }
+    }
+    if constexpr (S > 1) {
+        // peers may still be reading this CTA's shared memory
+        cg::this_cluster().sync();
+    }
+}
+
+template <int DT, int D, int NW, int R, int S>
+cudaError_t launch_one(const sh_context *c, const DecodeParams &p, cudaStream_t s) {
+    const int B = c->B;
+    const int cap = (S > 1) ? ((((B + S - 1) / S) + 31) & ~31) : ((B + 31) & ~31);
+    const size_t smem = sizeof(float) * ((size_t)cap + (size_t)NW * D + NW + 8 + 8 + D);
+    auto kern = sh_decode_kernel<DT, D, NW, R, S>;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(c->U * S), 1, 1);
+    cfg.blockDim = dim3(NW * 32, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    if (S > 1) {
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = S;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    return cudaLaunchKernelEx(&cfg, kern, p);
+}
+
+template <int DT, int D, int NW, int R>
+cudaError_t launch_split(const sh_context *c, const DecodeParams &p, cudaStream_t s) {
+    switch (c->split) {
+        case 1: return launch_one<DT, D, NW, R, 1>(c, p, s);
+        case 2: return launch_one<DT, D, NW, R, 2>(c, p, s);
+        case 4: return launch_one<DT, D, NW, R, 4>(c, p, s);
+        case 8: return launch_one<DT, D, NW, R, 8>(c, p, s);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace
+
+cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches) {
+    cudaError_t e = cudaErrorInvalidValue;
+    constexpr int NW = 8;
+    switch (c->dtype) {
+        case SH_F32:
+            if (c->D == 64) e = launch_split<SH_F32, 64, NW, 8>(c, p, s);
+            else if (c->D == 128) e = launch_split<SH_F32, 128, NW, 8>(c, p, s);
+            break;
+        case SH_F16:
+            if (c->D == 64) e = launch_split<SH_F16, 64, NW, 8>(c, p, s);
+            else if (c->D == 128) e = launch_split<SH_F16, 128, NW, 8>(c, p, s);
+            break;
+        case SH_BF16:
+            if (c->D == 64) e = launch_split<SH_BF16, 64, NW, 8>(c, p, s);
+            else if (c->D == 128) e = launch_split<SH_BF16, 128, NW, 8>(c, p, s);
+            break;
+        case SH_INT4_G64_F16:
+            if (c->D == 64) e = launch_split<SH_INT4_G64_F16, 64, NW, 4>(c, p, s);
+            else if (c->D == 128) e = launch_split<SH_INT4_G64_F16, 128, NW, 4>(c, p, s);
+            break;
+        default: break;
+    }
+    if (e == cudaSuccess) *launches += 1;
+    return e;
+}

@@ -1,0 +1,77 @@
+// Internal declarations shared by the translation units of libscissorhands.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "scissorhands.h"
+
+// Byte offsets of the regions inside the caller's workspace slab.
+struct ShLayout {
+    size_t K, V;            // [U][B][row_bytes]
+    size_t Ks, Vs;          // int4 only: [U][B][D/64] fp16 group scales
+    size_t hist;            // [U][w][Bw] u32 bit-planes: row (step mod w), bit j = "slot j was low at that step"
+    size_t pos;             // [U][B] int32 stream positions
+    size_t src_idx;         // [U][B] int32 selection result: source slot of each surviving destination slot
+    size_t counters;        // [U][B] u16 scratch for sh_state
+    size_t xport;           // [2][B][D] fp32 scratch for sh_export_unit
+    size_t stage_q, stage_k, stage_v, stage_out;  // staging for the *_host calls
+    size_t total;
+};
+
+struct sh_context {
+    int B, r, w, m, U, D, dtype;
+    int Bw;          // ceil(B / 32)
+    int row_bytes;   // bytes of one stored K (or V) row, without int4 scales
+    int in_bytes;    // bytes of one q / k_new / v_new row
+    int n;           // live tokens per unit
+    long long t;     // tokens streamed per unit
+    float scale;
+    int split;
+    int auto_compress;
+    bool started;    // a step has run: options are frozen
+    char *slab;
+    size_t slab_bytes;
+    ShLayout L;
+    long long launches;
+    cudaError_t last_err;
+};
+
+struct DecodeParams {
+    const void *q, *k_new, *v_new;
+    float *out;
+    char *K, *V;
+    char *Ks, *Vs;
+    uint32_t *hist;
+    int32_t *pos;
+    int U, B, Bw, w;
+    int n;          // live rows per unit including the token appended by this step
+    int hist_row;   // t mod w
+    int t;          // 1-based stream position of this step's token
+    float scale_log2e;
+};
+
+struct SelectParams {
+    const uint32_t *hist;       // bit-planes, or
+    const uint16_t *counters;   // [U][n] caller-supplied records
+    int32_t *src_idx;           // [U][B] or NULL
+    int32_t *evicted;           // [U][m] or NULL
+    int U, B, Bw, w, n, r, m;
+    int cmax;                   // largest possible counter value
+};
+
+struct CompactParams {
+    char *K, *V, *Ks, *Vs;
+    uint32_t *hist;
+    int32_t *pos;
+    const int32_t *src_idx;
+    int U, B, Bw, w, n, m;
+    int row_bytes, scale_bytes;
+};
+
+// Launchers (each returns the cudaError_t of its launch and adds to *launches).
+cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches);
+cudaError_t sh_launch_select(const SelectParams &p, bool from_hist, cudaStream_t s, long long *launches);
+cudaError_t sh_launch_compact(const CompactParams &p, cudaStream_t s, long long *launches);
+cudaError_t sh_launch_counters(const uint32_t *hist, uint16_t *counters, int U, int B, int Bw, int w, int n,
+                               cudaStream_t s, long long *launches);

@@ -1,0 +1,84 @@
+"""Lockstep parity harness: drives the CUDA library and the CPU oracle through
+the same stream, step by step.
+
+The library decides ``alpha_j < 1/t`` in fp32, the oracle in fp64; they can
+differ only where alpha_j is within rounding of the threshold.  Because the
+record feeds back into which tokens survive, one such flip would make every
+later kept set incomparable, so at each step the oracle takes over the
+library's bit wherever its own alpha_j lies within 1e-6 of 1/t (an "adoption",
+counted and reported) and any other disagreement is a failure.  With that,
+positions, counters and kept sets must agree bit for bit at every step, and
+attention outputs within the stated tolerance.
+"""
+from __future__ import annotations
+
+import dataclasses
+
+import numpy as np
+import torch
+
+import oracle as oracle_mod
+
+
+@dataclasses.dataclass
+class LockstepResult:
+    steps: int = 0
+    compressions: int = 0
+    adoptions: int = 0
+    slot_steps: int = 0
+    max_abs_err: float = 0.0
+
+
+def to_oracle(x: torch.Tensor, units) -> np.ndarray:
+    """Rows ``units`` of a [U, d] storage-dtype tensor as exact fp64."""
+    return x[units].to(torch.float64).cpu().numpy()
+
+
+def run_lockstep(handle, cfg_dtype: str, inputs, steps: int, units, tol: float, state_every: int = 1,
+                 res: LockstepResult = None, orc=None):
+    """``inputs(t)`` -> (q, k, v) CUDA tensors [U, d] for 1-based step t.
+    ``units``: LongTensor of unit indices checked against the oracle.
+    The handle must have been created with auto_compress=False.
+    Returns (LockstepResult, oracle)."""
+    units = torch.as_tensor(units, dtype=torch.long)
+    un = units.numpy()
+    if orc is None:
+        orc = oracle_mod.Oracle(len(un), handle.B, handle.r, handle.w, handle.m, handle.D,
+                                quant=(cfg_dtype == "int4"))
+    res = res or LockstepResult()
+    dev_units = units.to(handle.device)
+    for _ in range(steps):
+        t = orc.t + 1
+        q, k, v = inputs(t)
+        out = handle.decode_step(q, k, v)
+        want_state = (t % state_every == 0) or (orc.n + 1 == handle.B)
+        n, tt, pos, cnt, low = handle.state(pos=want_state, counters=want_state, low=True)
+        o_out, alpha, o_low, amb = orc.attend(to_oracle(q, dev_units), to_oracle(k, dev_units),
+                                              to_oracle(v, dev_units))
+        assert n == orc.n and tt == orc.t == t
+        err = float(np.abs(out[dev_units].double().cpu().numpy() - o_out).max())
+        res.max_abs_err = max(res.max_abs_err, err)
+        assert err <= tol, f"step {t}: attention output off by {err:.3e} > {tol}"
+        g_low = low[un]
+        diff = g_low != o_low
+        bad = diff & ~amb
+        assert not bad.any(), (f"step {t}: {int(bad.sum())} record bits differ where the oracle's score is not "
+                               f"within 1e-6 of 1/t; first at (unit, slot) {np.argwhere(bad)[0].tolist()}")
+        res.adoptions += int(diff.sum())
+        res.slot_steps += g_low.size
+        orc.record(g_low)
+        if want_state:
+            assert (pos[un] == orc.positions()).all(), f"step {t}: positions differ"
+            assert (cnt[un].astype(np.int32) == orc.counters()).all(), f"step {t}: importance records differ"
+        if orc.full:
+            dropped = orc.compress()
+            got = handle.compress()
+            assert dropped is not None and got == handle.m
+            n2, _, pos2, cnt2, _ = handle.state(low=False)
+            assert n2 == orc.n == handle.B - handle.m
+            o_pos = orc.positions()
+            assert (pos2[un] == o_pos).all(), f"step {t}: kept sets differ after compression"
+            assert (cnt2[un].astype(np.int32) == orc.counters()).all(), f"step {t}: records differ after compaction"
+            res.compressions += 1
+        res.steps += 1
+    return res, orc
