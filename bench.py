@@ -1,0 +1,358 @@
+#!/usr/bin/env python
+"""Benchmark of the compressed decode-attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl reference]
+
+One "step" is one pass of the whole hot path over every unit of the workload:
+sh_decode_step (append + attention + importance-record update) for each layer's
+handle, plus the compression (select-m + compaction) whenever the cache fills.
+The default workload is the OPT-66B-shaped one the headline metric is quoted on
+(batch 128 x 72 heads, head_dim 128, fp16 K/V, B=410, prompt 2048); the prompt is
+streamed through the same path, untimed, before the timed decode steps.
+
+Prints ONE JSON line.  `value` = steps/s with inputs resident in HBM; `e2e` =
+the same through sh_decode_step_host with pinned host buffers (copies inside the
+timed region); `roofline` = algorithmic K+V bytes of the fused decode kernel per
+launch / its mean CUDA-event duration, against the measured HBM copy peak;
+`cpu_baseline` = the CPU oracle timed on this machine's host cores on a bounded
+sample.  `--impl reference` times only that oracle.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2305_17118_b200 import workloads as wl  # noqa: E402
+
+METRIC = "compressed_decode_attn_steps_per_s"
+UNIT = "steps/s"
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0
+ES = {"f32": 4.0, "f16": 2.0, "bf16": 2.0, "int4": 0.5 + 2.0 / 64.0}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """SM clock and throttle reasons sampled through NVML (read-only) while the
+    timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        self.period = period_s
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _reasons(self):
+        nv = self.nv
+        get = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or nv.nvmlDeviceGetCurrentClocksThrottleReasons
+        bits = int(get(self.h))
+        names = {
+            "sw_power_cap": 0x4, "hw_slowdown": 0x8, "sync_boost": 0x10, "sw_thermal_slowdown": 0x20,
+            "hw_thermal_slowdown": 0x40, "hw_power_brake_slowdown": 0x80, "applications_clocks_setting": 0x2,
+        }
+        return {k for k, b in names.items() if bits & b}
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)))
+                self.reasons |= self._reasons()
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv:
+            self._thr = threading.Thread(target=self._run, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thr:
+            self._thr.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"], "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def live_rows_schedule(cfg, first_step: int, count: int):
+    """n (rows attended, new token included) at stream steps first_step.. ; the
+    schedule is data-independent: n grows by one per step and drops by m when it reaches B."""
+    n, out = 0, []
+    for t in range(1, first_step + count):
+        n += 1
+        if t >= first_step:
+            out.append(n)
+        if n == cfg.B:
+            n -= cfg.m
+    return out
+
+
+# --------------------------------------------------------------------------- CPU oracle arm
+def oracle_run(cfg, steps: int, warmup: int, sample_units: int, budget_s: float = 60.0):
+    """Times the CPU oracle (as it stands) on `sample_units` units: an untimed
+    run-in of B + warmup tokens to reach the steady-state saw-tooth, then up to
+    `steps` timed steps.  Returns (steps/s scaled to all units, info)."""
+    import numpy as np
+    import oracle
+    U = min(sample_units, cfg.units)
+    st = wl.Stream(cfg.scaled(units=U), device="cpu")
+    orc = oracle.Oracle(U, cfg.B, cfg.r, cfg.w, cfg.m, cfg.head_dim, quant=(cfg.dtype == "int4"))
+    f64 = lambda x: x.to(torch.float64).numpy()
+    run_in = cfg.B + warmup
+    for t in range(1, run_in + 1):
+        q, k, v = st.step(t)
+        orc.step(f64(q), f64(k), f64(v))
+    pre = [tuple(f64(x) for x in st.step(run_in + 1 + i)) for i in range(steps)]
+    done, t0 = 0, time.perf_counter()
+    for q, k, v in pre:
+        orc.step(q, k, v)
+        done += 1
+        if time.perf_counter() - t0 > budget_s:
+            break
+    dt = time.perf_counter() - t0
+    unit_steps_per_s = done * U / dt
+    value = unit_steps_per_s / (cfg.units * cfg.layers)
+    info = {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": (f"{U} of {cfg.units * cfg.layers} units, {done} timed steps after an untimed run-in of "
+                       f"{run_in} tokens (steady-state saw-tooth n in [{cfg.B - cfg.m + 1}, {cfg.B}]); "
+                       f"{dt:.1f} s of CPU work; unit-steps/s scaled to all units"),
+            "unit_steps_per_s": unit_steps_per_s}
+    return value, info, dt / max(done, 1)
+
+
+def reference_arm(args, cfg, rank):
+    if rank != 0:
+        return
+    value, info, s_per_step = oracle_run(cfg, args.steps, args.warmup, args.oracle_units, budget_s=150.0)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / value if value else None,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "units": cfg.units, "layers": cfg.layers, "head_dim": cfg.head_dim,
+                   "kv_dtype": cfg.dtype, "B": cfg.B, "r": cfg.r, "w": cfg.w, "m": cfg.m},
+        "cpu_baseline": info,
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- CUDA arm
+def cuda_arm(args, cfg, rank, world):
+    from paper_2305_17118_b200 import binding as sh
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    K, W = args.steps, args.warmup
+    U, d, Ly = cfg.units, cfg.head_dim, cfg.layers
+    streams = [wl.Stream(cfg, device=dev, layer=l + 1000 * rank) for l in range(Ly)]
+    handles = [sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, U, d, cfg.dtype, device=dev, auto_compress=False)
+               for _ in range(Ly)]
+
+    # ---- prompt: streamed through the same path, untimed
+    blk = max(1, min(64, (1 << 28) // (U * d * 2 * 3)))
+    for l, (h, st) in enumerate(zip(handles, streams)):
+        for t0 in range(1, cfg.prompt + 1, blk):
+            q, k, v = st.block(t0, min(t0 + blk, cfg.prompt + 1))
+            h.prefill(q, k, v)
+        torch.cuda.synchronize()
+    # ---- decode inputs resident in HBM; cycle if the run is longer than the buffer
+    n_in = min(W + K, max(1, int(6e9 // (Ly * U * d * 2 * 3))))
+    dec = [st.block(cfg.prompt + 1, cfg.prompt + 1 + n_in) for st in streams]
+    torch.cuda.synchronize()
+    snaps = [h.snapshot() for h in handles]
+    kv_bytes = 2 * Ly * U * cfg.B * d * ES[cfg.dtype]
+    flush = kv_bytes < 2 * L2_BYTES
+    flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev) if flush else None
+    out = torch.empty(U, d, device=dev)
+
+    def one_step(i, timed_pairs=None):
+        for l, h in enumerate(handles):
+            q, k, v = dec[l][0][i % n_in], dec[l][1][i % n_in], dec[l][2][i % n_in]
+            if timed_pairs is not None:
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                h.decode_step(q, k, v, out)
+                b.record()
+                timed_pairs.append((a, b))
+            else:
+                h.decode_step(q, k, v, out)
+            h.compress()           # no-op unless the cache just filled
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing
+    for i in range(W):
+        one_step(i)
+    launches0 = sum(h.launch_count for h in handles)
+    pairs, step_pairs = [], []
+    sampler = ClockSampler(local)
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with sampler:
+        ev0.record()
+        for i in range(W, W + K):
+            if flush:
+                flush_buf.fill_(i & 0xFF)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                one_step(i, pairs)
+                b.record()
+                step_pairs.append((a, b))
+            else:
+                one_step(i, pairs)
+        ev1.record()
+        barrier()
+    launches = sum(h.launch_count for h in handles) - launches0
+    if flush:
+        total_ms = sum(a.elapsed_time(b) for a, b in step_pairs)
+    else:
+        total_ms = ev0.elapsed_time(ev1)
+    kern_ms = [a.elapsed_time(b) for a, b in pairs]
+    if dist:
+        tt = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / K
+    value = world * 1e3 / ms_per_step
+
+    # ---- roofline of the fused decode kernel (one launch = one layer's units)
+    n_sched = live_rows_schedule(cfg, cfg.prompt + W + 1, K)
+    alg_bytes_launch = statistics.fmean(n_sched) * U * d * ES[cfg.dtype] * 2
+    kern_avg_ms = statistics.fmean(kern_ms)
+    achieved = alg_bytes_launch / (kern_avg_ms * 1e-3) / 1e9
+    peak, peak_src = measured_peak()
+    traffic = None
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            tr = json.load(f).get(cfg.name)
+            if tr:
+                traffic = tr["dram_bytes_per_unit_row"] * statistics.fmean(n_sched) * U
+    except Exception:
+        pass
+    roofline = {"bound": "hbm", "kernel": "sh_decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                "frac_of_8TBs_nominal": achieved / 8000.0, "alg_bytes_per_launch": alg_bytes_launch,
+                "avg_launch_us": kern_avg_ms * 1e3, "launches_timed": len(kern_ms),
+                "decode_kernel_share_of_step": kern_avg_ms * Ly / ms_per_step}
+
+    # ---- end to end: host buffers through sh_decode_step_host
+    e2e = None
+    if rank == 0 or dist:
+        for h, s in zip(handles, snaps):
+            h.restore(s)
+        Ke = min(K, n_in)
+        host = [[x[:Ke].cpu().pin_memory() for x in dec[l]] for l in range(Ly)]
+        oh = torch.empty(U, d).pin_memory()
+        for i in range(min(W, Ke)):
+            for l, h in enumerate(handles):
+                h.decode_step_host(host[l][0][i], host[l][1][i], host[l][2][i], oh)
+                h.compress()
+        for h, s in zip(handles, snaps):
+            h.restore(s)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(Ke):
+            for l, h in enumerate(handles):
+                h.decode_step_host(host[l][0][i], host[l][1][i], host[l][2][i], oh)
+                h.compress()
+        e1.record()
+        barrier()
+        e_ms = e0.elapsed_time(e1)
+        if dist:
+            tt = torch.tensor([e_ms], device=dev)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e_ms = float(tt.item())
+        in_b = Ly * U * d * (4 if cfg.dtype == "f32" else 2) * 3
+        e2e = {"value": world * Ke * 1e3 / e_ms, "unit": UNIT, "h2d_bytes_per_step": in_b,
+               "d2h_bytes_per_step": Ly * U * d * 4, "steps": Ke}
+
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+    cpu = None
+    if world == 1 or rank == 0:
+        _, cpu, _ = oracle_run(cfg, min(K, 256), 0, args.oracle_units, budget_s=20.0)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": {"f32": "f32", "f16": "f16", "bf16": "bf16", "int4": "int4"}[cfg.dtype] + " KV, f32 accumulate",
+        "data": "synthetic",
+        "config": {"workload": cfg.name, "batch": cfg.batch, "heads": cfg.heads, "layers": Ly, "units": U * Ly,
+                   "head_dim": d, "kv_dtype": cfg.dtype, "B": cfg.B, "r": cfg.r, "w": cfg.w, "m": cfg.m,
+                   "prompt": cfg.prompt, "l2": "flushed between steps" if flush else "inputs larger than L2",
+                   "kv_bytes": kv_bytes, "parallelism": f"units replicated x{world}" if world > 1 else "1 GPU"},
+        "attn_GBps": statistics.fmean(n_sched) * U * Ly * d * ES[cfg.dtype] * 2 / (ms_per_step * 1e-3) / 1e9,
+        "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": launches,
+        "roofline": roofline, "cpu_baseline": cpu,
+    }
+    print(json.dumps(line), flush=True)
+    if dist:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--config", default="opt66b", choices=wl.CONFIG_ORDER)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--oracle-units", type=int, default=2048)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
+    cfg = wl.CONFIGS[args.config]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        reference_arm(args, cfg, rank)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA path has no CPU fallback "
+                         "(use --impl reference for the CPU oracle)")
+    cuda_arm(args, cfg, rank, world)
+
+
+if __name__ == "__main__":
+    main()
