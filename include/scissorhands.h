@@ -43,7 +43,8 @@ typedef enum {
     SH_EFULL = -2,  /* decode step on a full cache: call sh_compress first */
     SH_ESTATE = -3, /* call out of order (e.g. no workspace bound) */
     SH_ECUDA = -4,  /* a CUDA runtime call or launch failed; see sh_last_cuda_error */
-    SH_ENOMEM = -5  /* host allocation failed or workspace too small */
+    SH_ENOMEM = -5, /* host allocation failed or workspace too small */
+    SH_ETOOBIG = -6 /* problem larger than a fixed-capacity entry point can take */
 } sh_status;
 
 typedef enum {
@@ -132,6 +133,33 @@ int sh_prefill(sh_handle h, const void *q_dev, const void *k_dev, const void *v_
  * A no-op when n < B.  *evicted_per_unit (may be NULL) receives m or 0.
  */
 int sh_compress(sh_handle h, void *stream, int *evicted_per_unit);
+
+/*
+ * sh_compress for callers that cannot allocate device memory.  (The paper has
+ * no counterpart: this is a deployment variant of sh_compress, same result.)
+ *
+ * Some users of this library never get to call cudaMalloc after start-up: a
+ * serving engine that gives all of HBM to its own KV-block pool has nothing
+ * left to ask for, and code inside a latency-critical decode loop must avoid
+ * the device-wide synchronisation an allocation implies.  For them this entry
+ * point keeps the selection scratch (one int32 per unit and slot, written by
+ * the select-m kernel and read by the compaction kernel) in a static device
+ * array inside the library instead of the workspace's scratch region, and
+ * calls no allocator of any kind.
+ *
+ * Limit: heads * B <= SH_STATIC_SCRATCH_MAX_ENTRIES (4 MiB of device memory,
+ * held by every GPU that loads the library until the process exits); beyond it
+ * the call returns SH_ETOOBIG and does nothing.  Inputs and outputs are the
+ * handle's bound workspace, exactly as for sh_compress.
+ * The first call on each device looks up the array's device address (with that
+ * device current); make that first call before any stream capture.
+ * All calls on a device share the one array and it keeps the previous call's
+ * contents.  Nothing in it needs to start at zero: the selection writes every
+ * entry the compaction reads.  Two calls whose kernels overlap on the GPU
+ * (different streams, different handles) race on it: serialise them.
+ */
+#define SH_STATIC_SCRATCH_MAX_ENTRIES (1u << 20)
+int sh_compress_static(sh_handle h, void *stream, int *evicted_per_unit);
 
 /*
  * Selection of Algorithm 2 on caller-supplied records, for testing the

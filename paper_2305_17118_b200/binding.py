@@ -16,7 +16,8 @@ import torch
 
 from . import build as _build
 
-SH_OK, SH_EINVAL, SH_EFULL, SH_ESTATE, SH_ECUDA, SH_ENOMEM = 0, -1, -2, -3, -4, -5
+SH_OK, SH_EINVAL, SH_EFULL, SH_ESTATE, SH_ECUDA, SH_ENOMEM, SH_ETOOBIG = 0, -1, -2, -3, -4, -5, -6
+SH_STATIC_SCRATCH_MAX_ENTRIES = 1 << 20
 SH_F32, SH_F16, SH_BF16, SH_INT4_G64_F16 = 0, 1, 2, 3
 SH_OPT_SOFTMAX_SCALE, SH_OPT_SPLIT, SH_OPT_AUTO_COMPRESS = 0, 1, 2
 
@@ -25,7 +26,7 @@ INPUT_TORCH_DTYPE = {SH_F32: torch.float32, SH_F16: torch.float16, SH_BF16: torc
                      SH_INT4_G64_F16: torch.float16}
 
 EXPORTS = ["sh_create", "sh_destroy", "sh_workspace_bytes", "sh_bind", "sh_set_option", "sh_decode_step",
-           "sh_decode_step_host", "sh_prefill", "sh_compress", "sh_select", "sh_state", "sh_export_unit",
+           "sh_decode_step_host", "sh_prefill", "sh_compress", "sh_compress_static", "sh_select", "sh_state", "sh_export_unit",
            "sh_restore", "sh_launch_count", "sh_strerror", "sh_last_cuda_error"]
 
 
@@ -50,6 +51,7 @@ def _load() -> C.CDLL:
     lib.sh_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.sh_prefill.argtypes = [vp, vp, vp, vp, C.c_int, vp, vp]
     lib.sh_compress.argtypes = [vp, vp, ip]
+    lib.sh_compress_static.argtypes = [vp, vp, ip]
     lib.sh_select.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
     lib.sh_state.argtypes = [vp, vp, ip, llp, vp, vp, vp]
     lib.sh_export_unit.argtypes = [vp, C.c_int, vp, vp, vp]
@@ -166,6 +168,16 @@ class Handle:
     def compress(self, stream=None) -> int:
         ev = C.c_int(0)
         self._check(lib.sh_compress(self._h, _stream_ptr(stream), C.byref(ev)))
+        return ev.value
+
+    # -- sh_compress_static ----------------------------------------------------------
+    def compress_static(self, stream=None) -> int:
+        """sh_compress without any device allocation or workspace scratch: for
+        callers that cannot cudaMalloc (all HBM already pooled, or inside a
+        latency-critical loop).  Needs heads * B <= SH_STATIC_SCRATCH_MAX_ENTRIES;
+        calls on one device must not overlap."""
+        ev = C.c_int(0)
+        self._check(lib.sh_compress_static(self._h, _stream_ptr(stream), C.byref(ev)))
         return ev.value
 
     # -- sh_state ------------------------------------------------------------------

@@ -346,6 +346,7 @@ const char *sh_strerror(int status) {
         case SH_ESTATE: return "call out of order (no workspace bound, or option set after the first step)";
         case SH_ECUDA: return "CUDA runtime error";
         case SH_ENOMEM: return "allocation failed or workspace too small";
+        case SH_ETOOBIG: return "problem exceeds the fixed capacity of this entry point";
         default: return "unknown status";
     }
 }

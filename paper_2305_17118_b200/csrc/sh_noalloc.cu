@@ -1,0 +1,82 @@
+// sh_compress_static: the compression step with its selection scratch held in
+// a static device array instead of the caller's workspace.
+//
+// Who needs this: an inference server that hands all of HBM to its own KV-block
+// pool at start-up has nothing left for cudaMalloc afterwards, and a caller
+// inside a latency-critical decode loop cannot afford cudaMalloc's implicit
+// device synchronisation.  Such a caller may have carved the handle's workspace
+// out of memory it already owned; this entry point lets the compression run
+// without touching any allocator, and without depending on the workspace's
+// scratch region.
+#include <mutex>
+
+#include "sh_internal.h"
+
+namespace {
+
+// One int32 per (unit, slot): source slot of every surviving destination slot.
+// Held by every device that loads the library, until the process exits.
+constexpr size_t SH_STATIC_SCRATCH_ENTRIES = SH_STATIC_SCRATCH_MAX_ENTRIES;
+static __device__ __align__(256) int32_t g_static_src_idx[SH_STATIC_SCRATCH_ENTRIES];
+
+constexpr int MAX_DEVICES = 64;
+std::mutex g_mu;
+int32_t *g_scratch_ptr[MAX_DEVICES] = {};   // device address of g_static_src_idx, per device
+
+// The array's name is only a host-side stand-in in host code; the device
+// address comes from cudaGetSymbolAddress, asked once per device while that
+// device is current.
+cudaError_t scratch_address(int32_t **out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!g_scratch_ptr[dev]) {
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_src_idx);
+        if (e != cudaSuccess) return e;
+        g_scratch_ptr[dev] = static_cast<int32_t *>(p);
+    }
+    *out = g_scratch_ptr[dev];
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int sh_compress_static(sh_handle h, void *stream, int *evicted_per_unit) {
+    if (!h) return SH_EINVAL;
+    if (!h->slab) return SH_ESTATE;
+    if (evicted_per_unit) *evicted_per_unit = 0;
+    if ((size_t)h->U * (size_t)h->B > SH_STATIC_SCRATCH_ENTRIES) return SH_ETOOBIG;
+    if (h->n < h->B) return SH_OK;
+    int32_t *src_idx = nullptr;
+    cudaError_t e = scratch_address(&src_idx);
+    if (e != cudaSuccess) { h->last_err = e; return SH_ECUDA; }
+    cudaStream_t s = (cudaStream_t)stream;
+
+    SelectParams sp = {};
+    sp.hist = reinterpret_cast<const uint32_t *>(h->slab + h->L.hist);
+    sp.counters = nullptr;
+    sp.src_idx = src_idx;
+    sp.evicted = nullptr;
+    sp.U = h->U; sp.B = h->B; sp.Bw = h->Bw; sp.w = h->w; sp.n = h->n; sp.r = h->r; sp.m = h->m;
+    sp.cmax = h->w;
+    e = sh_launch_select(sp, true, s, &h->launches);
+    if (e != cudaSuccess) { h->last_err = e; return SH_ECUDA; }
+
+    CompactParams cp = {};
+    cp.K = h->slab + h->L.K; cp.V = h->slab + h->L.V;
+    cp.Ks = h->slab + h->L.Ks; cp.Vs = h->slab + h->L.Vs;
+    cp.hist = reinterpret_cast<uint32_t *>(h->slab + h->L.hist);
+    cp.pos = reinterpret_cast<int32_t *>(h->slab + h->L.pos);
+    cp.src_idx = src_idx;
+    cp.U = h->U; cp.B = h->B; cp.Bw = h->Bw; cp.w = h->w; cp.n = h->n; cp.m = h->m;
+    cp.row_bytes = h->row_bytes;
+    cp.scale_bytes = h->dtype == SH_INT4_G64_F16 ? (h->D / 64) * 2 : 0;
+    e = sh_launch_compact(cp, s, &h->launches);
+    if (e != cudaSuccess) { h->last_err = e; return SH_ECUDA; }
+    h->n -= h->m;
+    if (evicted_per_unit) *evicted_per_unit = h->m;
+    return SH_OK;
+}
