@@ -181,7 +181,8 @@ def cuda_arm(args, cfg, rank, world):
     K, W = args.steps, args.warmup
     U, d, Ly = cfg.units, cfg.head_dim, cfg.layers
     streams = [wl.Stream(cfg, device=dev, layer=l + 1000 * rank) for l in range(Ly)]
-    handles = [sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, U, d, cfg.dtype, device=dev, auto_compress=False)
+    handles = [sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, U, d, cfg.dtype, device=dev, auto_compress=False,
+                         split=args.split)
                for _ in range(Ly)]
 
     # ---- prompt: streamed through the same path, untimed
@@ -312,7 +313,7 @@ def cuda_arm(args, cfg, rank, world):
             dist.destroy_process_group()
         return
     cpu = None
-    if world == 1 or rank == 0:
+    if (world == 1 or rank == 0) and not args.no_cpu_baseline:
         _, cpu, _ = oracle_run(cfg, min(K, 256), 0, args.oracle_units, budget_s=20.0)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
@@ -340,6 +341,8 @@ def main():
     ap.add_argument("--config", default="opt66b", choices=wl.CONFIG_ORDER)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--oracle-units", type=int, default=2048)
+    ap.add_argument("--split", type=int, default=None, help="CTAs per unit (default: chosen by the library)")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (tuning runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     cfg = wl.CONFIGS[args.config]

@@ -108,9 +108,11 @@ int sh_decode_step(sh_handle h, const void *q_dev, const void *k_new_dev, const 
                    float *attn_out_dev, void *stream);
 
 /*
- * Same step with HOST buffers (pinned memory recommended): copies q, k_new,
- * v_new to the device, runs the step, copies attn_out back, all on `stream`,
- * and returns after the stream has been synchronised.
+ * Same step with HOST buffers; returns after `stream` has been synchronised,
+ * with attn_out_host filled.  Page-locked (pinned), 16-byte aligned buffers are
+ * read and written by the kernel directly over PCIe, overlapped with the
+ * streaming of K and V; pageable buffers are staged through the workspace with
+ * cudaMemcpyAsync before and after the kernel.
  */
 int sh_decode_step_host(sh_handle h, const void *q_host, const void *k_new_host, const void *v_new_host,
                         float *attn_out_host, void *stream);

@@ -204,6 +204,20 @@ int sh_decode_step(sh_handle h, const void *q_dev, const void *k_new_dev, const 
     return do_step(h, q_dev, k_new_dev, v_new_dev, attn_out_dev, (cudaStream_t)stream, h->auto_compress != 0);
 }
 
+// Device-visible alias of a pinned host buffer (unified addressing maps pinned
+// host memory into the device's address space), or NULL if the buffer is
+// pageable or misaligned and has to be staged through the workspace.
+static void *pinned_alias(const void *host_ptr) {
+    if (misaligned(host_ptr)) return nullptr;
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, host_ptr) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return nullptr;
+    }
+    if (a.type != cudaMemoryTypeHost || !a.devicePointer) return nullptr;
+    return a.devicePointer;
+}
+
 int sh_decode_step_host(sh_handle h, const void *q_host, const void *k_new_host, const void *v_new_host,
                         float *attn_out_host, void *stream) {
     if (!h || !q_host || !k_new_host || !v_new_host || !attn_out_host) return SH_EINVAL;
@@ -211,17 +225,30 @@ int sh_decode_step_host(sh_handle h, const void *q_host, const void *k_new_host,
     if (h->n >= h->B) return SH_EFULL;
     cudaStream_t s = (cudaStream_t)stream;
     const size_t inb = (size_t)h->U * h->in_bytes, outb = (size_t)h->U * h->D * 4;
-    char *sq = h->slab + h->L.stage_q, *sk = h->slab + h->L.stage_k, *sv = h->slab + h->L.stage_v;
-    float *so = reinterpret_cast<float *>(h->slab + h->L.stage_out);
     cudaError_t e;
-    if ((e = cudaMemcpyAsync(sq, q_host, inb, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(h, e);
-    if ((e = cudaMemcpyAsync(sk, k_new_host, inb, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(h, e);
-    if ((e = cudaMemcpyAsync(sv, v_new_host, inb, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(h, e);
-    // The result leaves before any compression that follows, so the copy
-    // overlaps nothing it depends on and the caller sees the step's output.
-    int rc = do_step(h, sq, sk, sv, so, s, false);
+    // Pinned buffers are read and written by the kernel itself over PCIe, so
+    // the transfers overlap the streaming of K and V instead of preceding and
+    // following it; pageable ones go through staging copies.
+    const void *src[3] = {q_host, k_new_host, v_new_host};
+    const size_t stage_off[3] = {h->L.stage_q, h->L.stage_k, h->L.stage_v};
+    const void *in[3];
+    for (int i = 0; i < 3; ++i) {
+        in[i] = pinned_alias(src[i]);
+        if (!in[i]) {
+            char *st = h->slab + stage_off[i];
+            if ((e = cudaMemcpyAsync(st, src[i], inb, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(h, e);
+            in[i] = st;
+        }
+    }
+    float *out = static_cast<float *>(pinned_alias(attn_out_host));
+    const bool stage_out = out == nullptr;
+    if (stage_out) out = reinterpret_cast<float *>(h->slab + h->L.stage_out);
+    int rc = do_step(h, in[0], in[1], in[2], out, s, false);
     if (rc != SH_OK) return rc;
-    if ((e = cudaMemcpyAsync(attn_out_host, so, outb, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(h, e);
+    // The result leaves before any compression that follows.
+    if (stage_out &&
+        (e = cudaMemcpyAsync(attn_out_host, out, outb, cudaMemcpyDeviceToHost, s)) != cudaSuccess)
+        return cuda_fail(h, e);
     if (h->auto_compress && h->n == h->B) {
         rc = do_compress(h, s);
         if (rc != SH_OK) return rc;

@@ -160,13 +160,15 @@ def test_prefill_equals_token_by_token_steps(sh):
     assert torch.equal(a.slab[a._slab_off:a._slab_off + 2 * U * B * d * 2], b.slab[b._slab_off:b._slab_off + 2 * U * B * d * 2])
 
 
-def test_host_buffer_step_matches_device_step(sh):
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_buffer_step_matches_device_step(sh, pinned):
     U, d, B, r, w, m, T, dtype = 7, 128, 64, 4, 16, 20, 100, "bf16"
     q, k, v = wl.random_stream(U, d, T, seed=6, dtype=dtype, peaked=2.0, device="cuda")
     a = sh.Handle(B, r, w, m, U, d, dtype)
     b = sh.Handle(B, r, w, m, U, d, dtype)
-    qh, kh, vh = (x.cpu().pin_memory() for x in (q, k, v))
-    oh = torch.empty(U, d).pin_memory()
+    pin = (lambda x: x.pin_memory()) if pinned else (lambda x: x)
+    qh, kh, vh = (pin(x.cpu()) for x in (q, k, v))
+    oh = pin(torch.empty(U, d))
     for t in range(T):
         oa = a.decode_step(q[t], k[t], v[t])
         b.decode_step_host(qh[t], kh[t], vh[t], oh)
