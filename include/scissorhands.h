@@ -44,7 +44,9 @@ typedef enum {
     SH_ESTATE = -3, /* call out of order (e.g. no workspace bound) */
     SH_ECUDA = -4,  /* a CUDA runtime call or launch failed; see sh_last_cuda_error */
     SH_ENOMEM = -5, /* host allocation failed or workspace too small */
-    SH_ETOOBIG = -6 /* problem larger than a fixed-capacity entry point can take */
+    SH_ETOOBIG = -6, /* problem larger than a fixed-capacity entry point can take */
+    SH_EDEVICE = -7  /* reported by sh_state: a kernel gave up one of its bounded waits on an
+                        asynchronous copy and left its work undone */
 } sh_status;
 
 typedef enum {

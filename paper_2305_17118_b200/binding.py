@@ -16,7 +16,7 @@ import torch
 
 from . import build as _build
 
-SH_OK, SH_EINVAL, SH_EFULL, SH_ESTATE, SH_ECUDA, SH_ENOMEM, SH_ETOOBIG = 0, -1, -2, -3, -4, -5, -6
+SH_OK, SH_EINVAL, SH_EFULL, SH_ESTATE, SH_ECUDA, SH_ENOMEM, SH_ETOOBIG, SH_EDEVICE = 0, -1, -2, -3, -4, -5, -6, -7
 SH_STATIC_SCRATCH_MAX_ENTRIES = 1 << 20
 SH_F32, SH_F16, SH_BF16, SH_INT4_G64_F16 = 0, 1, 2, 3
 SH_OPT_SOFTMAX_SCALE, SH_OPT_SPLIT, SH_OPT_AUTO_COMPRESS = 0, 1, 2

@@ -41,6 +41,7 @@ void make_layout(sh_context *c) {
     L.stage_k = take(U * (size_t)c->in_bytes);
     L.stage_v = take(U * (size_t)c->in_bytes);
     L.stage_out = take(U * D * 4);
+    L.err = take(256);
     L.total = off;
 }
 
@@ -98,6 +99,7 @@ int do_compress(sh_context *c, cudaStream_t s) {
     cp.U = c->U; cp.B = c->B; cp.Bw = c->Bw; cp.w = c->w; cp.n = c->n; cp.m = c->m;
     cp.row_bytes = c->row_bytes;
     cp.scale_bytes = c->dtype == SH_INT4_G64_F16 ? (c->D / 64) * 2 : 0;
+    cp.err = reinterpret_cast<int *>(c->slab + c->L.err);
     e = sh_launch_compact(cp, s, &c->launches);
     if (e != cudaSuccess) return cuda_fail(c, e);
     c->n -= c->m;
@@ -328,9 +330,12 @@ int sh_state(sh_handle h, void *stream, int *n_out, long long *t_out, int32_t *p
                               cudaMemcpyDeviceToHost, s);
         if (e != cudaSuccess) return cuda_fail(h, e);
     }
+    int dev_err = 0;
+    e = cudaMemcpyAsync(&dev_err, h->slab + h->L.err, sizeof(int), cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail(h, e);
     e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return cuda_fail(h, e);
-    return SH_OK;
+    return dev_err ? SH_EDEVICE : SH_OK;
 }
 
 int sh_export_unit(sh_handle h, int unit, float *K_host, float *V_host, void *stream) {
@@ -374,6 +379,7 @@ const char *sh_strerror(int status) {
         case SH_ECUDA: return "CUDA runtime error";
         case SH_ENOMEM: return "allocation failed or workspace too small";
         case SH_ETOOBIG: return "problem exceeds the fixed capacity of this entry point";
+        case SH_EDEVICE: return "a kernel gave up a bounded wait (device error word set); state is unreliable";
         default: return "unknown status";
     }
 }

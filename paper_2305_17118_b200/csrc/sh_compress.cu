@@ -1,7 +1,9 @@
 // Compression step (Algorithm 2): importance record from the bit-planes,
 // select-m with a deterministic tie-break, and stable in-place compaction of
-// K, V, scales, bit-planes and positions.  One CTA per unit for the selection,
-// three CTAs per unit (K, V, record+positions) for the compaction.
+// K, V, scales, bit-planes and positions.  One CTA per unit for the selection;
+// the compaction is two kernels: K/V rows through bulk asynchronous copies
+// (two CTAs per unit), and record bit-planes + positions (one CTA per unit).
+#include "sh_async.cuh"
 #include "sh_internal.h"
 
 namespace {
@@ -33,7 +35,8 @@ __device__ __forceinline__ int slot_counter(const uint32_t *hist_u, int w, int B
     const uint32_t *col = hist_u + (j >> 5);
     const int sh = j & 31;
     int cnt = 0;
-    for (int s = 0; s < w; ++s) cnt += (col[(size_t)s * Bw] >> sh) & 1u;
+#pragma unroll 8
+    for (int s = 0; s < w; ++s) cnt += (col[s * Bw] >> sh) & 1u;
     return cnt;
 }
 
@@ -48,15 +51,52 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
     int *bins = cnt_sh + p.n;              // [cmax + 1]
     int *wsum = bins + (p.cmax + 1);       // [32]
     int *cut = wsum + 32;                  // [2] = {cstar, need}
+    uint32_t *planes = reinterpret_cast<uint32_t *>(cut + 2);   // [w * Bw] when staged, then [G][5][Bw] partial sums
     const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
     const int n = p.n, ncand = p.n - p.r, m = p.m;
 
     for (int i = tid; i <= p.cmax; i += SEL_THREADS) bins[i] = 0;
-    for (int j = tid; j < n; j += SEL_THREADS) {
-        int I;
-        if (FROM_HIST) I = slot_counter(p.hist + (size_t)u * p.w * p.Bw, p.w, p.Bw, j);
-        else I = min((int)p.counters[(size_t)u * n + j], p.cmax);
-        cnt_sh[j] = I;
+    if (FROM_HIST) {
+        const uint32_t *hist_u = p.hist + (size_t)u * p.w * p.Bw;
+        if (p.stage_planes) {
+            // One coalesced pass brings the unit's bit-planes to shared memory.  Then the
+            // rows are summed 32 slots at a time: thread (g, k) adds rows g, g+G, ... of
+            // word column k into a 5-plane bit-sliced counter (at most 31 rows each), and
+            // every slot finally picks its bits out of the G partial counters.
+            const int Bw = p.Bw, w = p.w, G = (w + 30) / 31;
+            for (int i = tid; i < w * Bw; i += SEL_THREADS) planes[i] = hist_u[i];
+            __syncthreads();
+            uint32_t *part = planes + w * Bw;
+            for (int item = tid; item < G * Bw; item += SEL_THREADS) {
+                const int g = item / Bw, k = item % Bw;
+                uint32_t c0 = 0, c1 = 0, c2 = 0, c3 = 0, c4 = 0;
+                for (int s = g; s < w; s += G) {
+                    uint32_t x = planes[s * Bw + k], t;
+                    t = c0 & x; c0 ^= x; x = t;
+                    t = c1 & x; c1 ^= x; x = t;
+                    t = c2 & x; c2 ^= x; x = t;
+                    t = c3 & x; c3 ^= x; x = t;
+                    c4 ^= x;
+                }
+                uint32_t *o = part + (size_t)g * 5 * Bw + k;
+                o[0] = c0; o[Bw] = c1; o[2 * Bw] = c2; o[3 * Bw] = c3; o[4 * Bw] = c4;
+            }
+            __syncthreads();
+            for (int j = tid; j < n; j += SEL_THREADS) {
+                const uint32_t *col = part + (j >> 5);
+                const int sh = j & 31;
+                int cnt = 0;
+                for (int g = 0; g < G; ++g) {
+#pragma unroll
+                    for (int pl = 0; pl < 5; ++pl) cnt += ((col[(g * 5 + pl) * Bw] >> sh) & 1u) << pl;
+                }
+                cnt_sh[j] = cnt;
+            }
+        } else {
+            for (int j = tid; j < n; j += SEL_THREADS) cnt_sh[j] = slot_counter(hist_u, p.w, p.Bw, j);
+        }
+    } else {
+        for (int j = tid; j < n; j += SEL_THREADS) cnt_sh[j] = min((int)p.counters[(size_t)u * n + j], p.cmax);
     }
     __syncthreads();
     for (int j = tid; j < ncand; j += SEL_THREADS) atomicAdd(&bins[cnt_sh[j]], 1);
@@ -109,94 +149,170 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
     }
 }
 
-// Rows of `row_bytes` (a multiple of 16) moved dst <- src_idx[dst] for dst in
-// [0, n_keep).  Destinations never exceed their sources and sources increase
-// with the destination, so batches in ascending order with all reads of a batch
-// before its writes never overwrite a row that is still needed.
-__device__ void compact_rows(char *base, const int32_t *src, int n_keep, int row_bytes) {
-    constexpr int RR = 4;
-    const int lpr = row_bytes >> 4;                 // 16-byte chunks per row
-    const int rpp = CMP_THREADS / lpr;              // rows per pass
-    const int row_in_pass = threadIdx.x / lpr, ch = threadIdx.x % lpr;
-    const bool active = row_in_pass < rpp;
-    for (int b = 0; b < n_keep; b += rpp * RR) {
-        uint4 v[RR];
-        int sj[RR];
-#pragma unroll
-        for (int i = 0; i < RR; ++i) {
-            const int dst = b + i * rpp + row_in_pass;
-            sj[i] = -1;
-            if (active && dst < n_keep) {
-                const int s = src[dst];
-                if (s != dst) {
-                    sj[i] = s;
-                    v[i] = *reinterpret_cast<const uint4 *>(base + (size_t)s * row_bytes + ch * 16);
-                }
-            }
-        }
-        __syncthreads();
-#pragma unroll
-        for (int i = 0; i < RR; ++i) {
-            const int dst = b + i * rpp + row_in_pass;
-            if (sj[i] >= 0) *reinterpret_cast<uint4 *>(base + (size_t)dst * row_bytes + ch * 16) = v[i];
-        }
-    }
-}
+// K or V rows of one unit, moved dst <- src_idx[dst] for dst in [0, n_keep).
+// Destinations never exceed their sources and sources increase with the
+// destination, so everything from the first moved row on can be handled in
+// ascending chunks, each read completely before it is written.  A chunk is
+// gathered into shared memory by bulk asynchronous copies (one per run of
+// consecutive source rows, all counted on one mbarrier) and written back to its
+// contiguous destination by a single bulk store.
+constexpr int ROWS_THREADS = 128;
 
-// Same for small per-slot items (positions, int4 scales); slots [n_keep, n) get `fill`.
-template <typename T>
-__device__ void compact_items(T *base, const int32_t *src, int n_keep, int n, T fill) {
-    for (int b = 0; b < n; b += CMP_THREADS) {
-        const int dst = b + threadIdx.x;
-        T val = fill;
-        if (dst < n_keep) val = base[src[dst]];
-        __syncthreads();
-        if (dst < n) base[dst] = val;
-    }
-}
-
-// Bit-planes: every row (one past step) is gathered through src_idx.  A warp
-// owns a row: it stages the row's words in shared memory, then writes the
-// gathered words; bits of the freed slots become 0.
-__device__ void compact_hist(uint32_t *hist_u, const int32_t *src, int n_keep, int w, int Bw, uint32_t *stage) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = CMP_THREADS / 32;
-    uint32_t *st = stage + warp * Bw;
-    for (int s = warp; s < w; s += nw) {
-        uint32_t *row = hist_u + (size_t)s * Bw;
-        for (int k = lane; k < Bw; k += 32) st[k] = row[k];
-        __syncwarp();
-        for (int k = 0; k < Bw; ++k) {
-            const int dst = (k << 5) + lane;
-            bool bit = false;
-            if (dst < n_keep) {
-                const int sj = src[dst];
-                bit = (st[sj >> 5] >> (sj & 31)) & 1u;
-            }
-            const uint32_t word = __ballot_sync(0xffffffffu, bit);
-            if (lane == 0) row[k] = word;
-        }
-        __syncwarp();
-    }
-}
-
-__global__ void __launch_bounds__(CMP_THREADS) sh_compact_kernel(const CompactParams p) {
-    extern __shared__ uint32_t stage[];
-    const int u = blockIdx.x, what = blockIdx.y;
-    const int n_keep = p.n - p.m;
+__global__ void __launch_bounds__(ROWS_THREADS) sh_compact_rows_kernel(const CompactParams p) {
+    extern __shared__ __align__(128) unsigned char buf[];
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int first_moved;
+    const int u = blockIdx.x, what = blockIdx.y, tid = threadIdx.x;
+    const int n_keep = p.n - p.m, rb = p.row_bytes;
     const int32_t *src = p.src_idx + (size_t)u * p.B;
-    if (what == 0 || what == 1) {
-        char *rows = (what == 0 ? p.K : p.V) + (size_t)u * p.B * p.row_bytes;
-        compact_rows(rows, src, n_keep, p.row_bytes);
+    char *rows = (what == 0 ? p.K : p.V) + (size_t)u * p.B * rb;
+
+    if (tid == 0) {
+        first_moved = n_keep;
+        shasync::mbar_init(&bar, 1);
+        shasync::fence_barrier_init();
+    }
+    __syncthreads();
+    {
+        int mine = n_keep;
+        for (int d = tid; d < n_keep; d += ROWS_THREADS)
+            if (src[d] != d) { mine = d; break; }
+        if (mine < n_keep) atomicMin(&first_moved, mine);
+    }
+    __syncthreads();
+    const int d0 = first_moved;
+    const int chunk_rows = p.chunk_bytes / rb;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int a = d0; a < n_keep && ok; a += chunk_rows) {
+        const int b = min(n_keep, a + chunk_rows);
+        if (tid == 0) shasync::mbar_arrive_expect_tx(&bar, (uint32_t)(b - a) * rb);
+        __syncthreads();   // the expectation is posted before any copy can complete
+        for (int d = a + tid; d < b; d += ROWS_THREADS) {
+            const int s0 = src[d];
+            if (d != a && src[d - 1] + 1 == s0) continue;        // inside someone else's run
+            int len = 1;
+            while (d + len < b && src[d + len] == s0 + len) ++len;
+            shasync::bulk_g2s(buf + (size_t)(d - a) * rb, rows + (size_t)s0 * rb, (uint32_t)len * rb, &bar);
+        }
+        ok = __syncthreads_and(shasync::mbar_wait(&bar, phase, p.err, 1));   // uniform across the CTA
+        phase ^= 1;
+        if (tid == 0 && ok) {
+            shasync::fence_async_shared();
+            shasync::bulk_s2g(rows + (size_t)a * rb, buf, (uint32_t)(b - a) * rb);
+            shasync::bulk_commit();
+            shasync::bulk_wait_read_all();    // the buffer may be refilled
+        }
+        __syncthreads();
+    }
+    if (tid == 0) shasync::bulk_wait_all();
+
+    // int4 group scales travel with their rows
+    if (p.scale_bytes) {
+        __syncthreads();
         if (p.scale_bytes == 4) {
             uint32_t *sc = reinterpret_cast<uint32_t *>(what == 0 ? p.Ks : p.Vs) + (size_t)u * p.B;
-            compact_items<uint32_t>(sc, src, n_keep, p.n, 0u);
-        } else if (p.scale_bytes == 2) {
+            for (int base = 0; base < p.n; base += ROWS_THREADS) {
+                const int d = base + tid;
+                uint32_t val = 0;
+                if (d < n_keep) val = sc[src[d]];
+                __syncthreads();
+                if (d < p.n) sc[d] = val;
+            }
+        } else {
             uint16_t *sc = reinterpret_cast<uint16_t *>(what == 0 ? p.Ks : p.Vs) + (size_t)u * p.B;
-            compact_items<uint16_t>(sc, src, n_keep, p.n, (uint16_t)0);
+            for (int base = 0; base < p.n; base += ROWS_THREADS) {
+                const int d = base + tid;
+                uint16_t val = 0;
+                if (d < n_keep) val = sc[src[d]];
+                __syncthreads();
+                if (d < p.n) sc[d] = val;
+            }
         }
-    } else {
-        compact_hist(p.hist + (size_t)u * p.w * p.Bw, src, n_keep, p.w, p.Bw, stage);
-        compact_items<int32_t>(p.pos + (size_t)u * p.B, src, n_keep, p.n, 0);
+    }
+}
+
+// Record bit-planes and positions of one unit.  Removing the dropped slots
+// from a bit-plane row is a bit compress (keep the bits under a mask, squeezed
+// to the right).  The mask is the same for all w rows, so the five butterfly
+// masks of the classic compress network are computed once per 32-slot word and
+// every row is then handled by one thread: 20 logic operations per source word
+// plus a funnel shift into the output stream.  Bits of the freed slots become 0.
+__device__ __forceinline__ uint32_t compress_bits(uint32_t x, uint32_t m, const uint32_t *mv) {
+    x &= m;
+#pragma unroll
+    for (int i = 0; i < 5; ++i) {
+        const uint32_t t = x & mv[i];
+        x = (x ^ t) | (t >> (1 << i));
+    }
+    return x;
+}
+
+__global__ void __launch_bounds__(CMP_THREADS) sh_compact_record_kernel(const CompactParams p) {
+    extern __shared__ uint32_t rec_sm[];
+    const int u = blockIdx.x, tid = threadIdx.x;
+    const int n_keep = p.n - p.m, Bw = p.Bw, w = p.w;
+    const int stride = Bw | 1;                       // odd row stride: no bank conflicts
+    const int32_t *src = p.src_idx + (size_t)u * p.B;
+    uint32_t *hist_u = p.hist + (size_t)u * w * Bw;
+    uint32_t *keep = rec_sm;                         // [Bw] keep mask per source word
+    uint32_t *mvs = keep + Bw;                       // [Bw][5] butterfly masks
+    uint32_t *rows = mvs + 5 * Bw;                   // [p.rec_rows][stride] staged bit-plane rows
+
+    for (int k = tid; k < Bw; k += CMP_THREADS) keep[k] = 0;
+    __syncthreads();
+    for (int d = tid; d < n_keep; d += CMP_THREADS) {
+        const int sj = src[d];
+        atomicOr(&keep[sj >> 5], 1u << (sj & 31));
+    }
+    __syncthreads();
+    for (int k = tid; k < Bw; k += CMP_THREADS) {
+        uint32_t m = keep[k], mk = ~m << 1;
+#pragma unroll
+        for (int i = 0; i < 5; ++i) {
+            uint32_t mp = mk ^ (mk << 1);
+            mp ^= mp << 2; mp ^= mp << 4; mp ^= mp << 8; mp ^= mp << 16;
+            const uint32_t mv = mp & m;
+            mvs[k * 5 + i] = mv;
+            m = (m ^ mv) | (mv >> (1 << i));
+            mk &= ~mp;
+        }
+    }
+    __syncthreads();
+    for (int s0 = 0; s0 < w; s0 += p.rec_rows) {
+        const int nr = min(p.rec_rows, w - s0);
+        for (int i = tid; i < nr * Bw; i += CMP_THREADS) rows[(i / Bw) * stride + (i % Bw)] = hist_u[(size_t)s0 * Bw + i];
+        __syncthreads();
+        for (int r = tid; r < nr; r += CMP_THREADS) {
+            uint32_t *row = rows + r * stride;
+            unsigned long long acc = 0;
+            int fill = 0, o = 0;
+            for (int k = 0; k < Bw; ++k) {
+                const uint32_t m = keep[k];
+                const uint32_t c = compress_bits(row[k], m, mvs + k * 5);
+                acc |= (unsigned long long)c << fill;
+                fill += __popc(m);
+                if (fill >= 32) {
+                    row[o++] = (uint32_t)acc;     // o <= k: the word was already consumed
+                    acc >>= 32;
+                    fill -= 32;
+                }
+            }
+            if (o < Bw) row[o++] = (uint32_t)acc;
+            for (; o < Bw; ++o) row[o] = 0;
+        }
+        __syncthreads();
+        for (int i = tid; i < nr * Bw; i += CMP_THREADS) hist_u[(size_t)s0 * Bw + i] = rows[(i / Bw) * stride + (i % Bw)];
+        __syncthreads();
+    }
+    // positions: read a batch, barrier, write it (destinations never pass sources)
+    int32_t *pos = p.pos + (size_t)u * p.B;
+    for (int base = 0; base < p.n; base += CMP_THREADS) {
+        const int d = base + threadIdx.x;
+        int32_t val = 0;
+        if (d < n_keep) val = pos[src[d]];
+        __syncthreads();
+        if (d < p.n) pos[d] = val;
     }
 }
 
@@ -212,8 +328,12 @@ __global__ void __launch_bounds__(256) sh_counters_kernel(const uint32_t *hist, 
 
 }  // namespace
 
-cudaError_t sh_launch_select(const SelectParams &p, bool from_hist, cudaStream_t s, long long *launches) {
-    const size_t smem = sizeof(int) * ((size_t)p.n + p.cmax + 1 + 32 + 2);
+cudaError_t sh_launch_select(const SelectParams &p_in, bool from_hist, cudaStream_t s, long long *launches) {
+    SelectParams p = p_in;
+    size_t smem = sizeof(int) * ((size_t)p.n + p.cmax + 1 + 32 + 2);
+    const size_t planes = from_hist ? sizeof(uint32_t) * ((size_t)p.w * p.Bw + (size_t)((p.w + 30) / 31) * 5 * p.Bw) : 0;
+    p.stage_planes = from_hist && smem + planes <= 96 * 1024;
+    if (p.stage_planes) smem += planes;
     cudaError_t e;
     if (from_hist) {
         if (smem > 48 * 1024) {
@@ -233,10 +353,40 @@ cudaError_t sh_launch_select(const SelectParams &p, bool from_hist, cudaStream_t
     return e;
 }
 
-cudaError_t sh_launch_compact(const CompactParams &p, cudaStream_t s, long long *launches) {
-    const size_t smem = sizeof(uint32_t) * (size_t)(CMP_THREADS / 32) * p.Bw;
-    sh_compact_kernel<<<dim3(p.U, 3, 1), CMP_THREADS, smem, s>>>(p);
-    cudaError_t e = cudaGetLastError();
+cudaError_t sh_launch_compact(const CompactParams &p_in, cudaStream_t s, long long *launches) {
+    CompactParams p = p_in;
+    // K/V rows: chunks of ~32 KB keep several CTAs per SM, so the reads of one
+    // overlap the writes of another (measured best on B200 among 16..100 KB)
+    const int max_chunk = p.row_bytes > 32 * 1024 ? p.row_bytes : 32 * 1024;
+    int chunk_rows = max_chunk / p.row_bytes;
+    if (chunk_rows > p.n - p.m) chunk_rows = p.n - p.m;
+    if (chunk_rows < 1) chunk_rows = 1;
+    p.chunk_bytes = chunk_rows * p.row_bytes;
+    cudaError_t e;
+    if (p.n - p.m > 0) {
+        if (p.chunk_bytes > 40 * 1024) {
+            e = cudaFuncSetAttribute(sh_compact_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, p.chunk_bytes);
+            if (e != cudaSuccess) return e;
+        }
+        sh_compact_rows_kernel<<<dim3(p.U, 2, 1), ROWS_THREADS, p.chunk_bytes, s>>>(p);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        if (launches) *launches += 1;
+    }
+    // bit-plane rows staged per pass: up to one per thread, within ~64 KB
+    const int stride = p.Bw | 1;
+    int rec_rows = (64 * 1024) / (stride * 4);
+    if (rec_rows > CMP_THREADS) rec_rows = CMP_THREADS;
+    if (rec_rows > p.w) rec_rows = p.w;
+    if (rec_rows < 1) rec_rows = 1;
+    p.rec_rows = rec_rows;
+    const size_t smem = sizeof(uint32_t) * ((size_t)6 * p.Bw + (size_t)rec_rows * stride);
+    if (smem > 48 * 1024) {
+        e = cudaFuncSetAttribute(sh_compact_record_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    sh_compact_record_kernel<<<p.U, CMP_THREADS, smem, s>>>(p);
+    e = cudaGetLastError();
     if (e == cudaSuccess && launches) *launches += 1;
     return e;
 }

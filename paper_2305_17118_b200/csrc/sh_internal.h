@@ -16,6 +16,7 @@ struct ShLayout {
     size_t counters;        // [U][B] u16 scratch for sh_state
     size_t xport;           // [2][B][D] fp32 scratch for sh_export_unit
     size_t stage_q, stage_k, stage_v, stage_out;  // staging for the *_host calls
+    size_t err;             // one int: set by a kernel whose bounded wait gave up
     size_t total;
 };
 
@@ -58,6 +59,7 @@ struct SelectParams {
     int32_t *evicted;           // [U][m] or NULL
     int U, B, Bw, w, n, r, m;
     int cmax;                   // largest possible counter value
+    int stage_planes;           // set by the launcher: copy the unit's bit-planes to shared memory first
 };
 
 struct CompactParams {
@@ -67,6 +69,9 @@ struct CompactParams {
     const int32_t *src_idx;
     int U, B, Bw, w, n, m;
     int row_bytes, scale_bytes;
+    int chunk_bytes;            // set by the launcher: shared-memory gather buffer of the row kernel
+    int rec_rows;               // set by the launcher: bit-plane rows staged per pass of the record kernel
+    int *err;                   // device error word (a bounded wait gave up)
 };
 
 // Launchers (each returns the cudaError_t of its launch and adds to *launches).
