@@ -182,7 +182,7 @@ def cuda_arm(args, cfg, rank, world):
     U, d, Ly = cfg.units, cfg.head_dim, cfg.layers
     streams = [wl.Stream(cfg, device=dev, layer=l + 1000 * rank) for l in range(Ly)]
     handles = [sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, U, d, cfg.dtype, device=dev, auto_compress=False,
-                         split=args.split)
+                         split=args.split, kernel=args.kernel)
                for _ in range(Ly)]
 
     # ---- prompt: streamed through the same path, untimed
@@ -342,6 +342,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--oracle-units", type=int, default=2048)
     ap.add_argument("--split", type=int, default=None, help="CTAs per unit (default: chosen by the library)")
+    ap.add_argument("--kernel", type=int, default=None, help="decode kernel: 1 direct loads, 2 pipelined bulk copies")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (tuning runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup

@@ -60,8 +60,11 @@ typedef enum {
 typedef enum {
     SH_OPT_SOFTMAX_SCALE = 0, /* multiplier of the logits; default 1/sqrt(head_dim) */
     SH_OPT_SPLIT = 1,         /* CTAs cooperating on one unit (1, 2, 4 or 8); default chosen from `heads` */
-    SH_OPT_AUTO_COMPRESS = 2  /* 1 (default): sh_decode_step compresses by itself when the cache fills;
+    SH_OPT_AUTO_COMPRESS = 2, /* 1 (default): sh_decode_step compresses by itself when the cache fills;
                                  0: the caller calls sh_compress */
+    SH_OPT_DECODE_KERNEL = 3  /* 0 (default): chosen from the shape; 1: one CTA (or cluster) per unit with
+                                 direct loads; 2: persistent CTAs fed by bulk asynchronous copies
+                                 (fp16/bf16, head_dim 128, split 1 only; otherwise 1 is used) */
 } sh_option;
 
 /*

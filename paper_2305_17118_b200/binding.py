@@ -19,7 +19,7 @@ from . import build as _build
 SH_OK, SH_EINVAL, SH_EFULL, SH_ESTATE, SH_ECUDA, SH_ENOMEM, SH_ETOOBIG, SH_EDEVICE = 0, -1, -2, -3, -4, -5, -6, -7
 SH_STATIC_SCRATCH_MAX_ENTRIES = 1 << 20
 SH_F32, SH_F16, SH_BF16, SH_INT4_G64_F16 = 0, 1, 2, 3
-SH_OPT_SOFTMAX_SCALE, SH_OPT_SPLIT, SH_OPT_AUTO_COMPRESS = 0, 1, 2
+SH_OPT_SOFTMAX_SCALE, SH_OPT_SPLIT, SH_OPT_AUTO_COMPRESS, SH_OPT_DECODE_KERNEL = 0, 1, 2, 3
 
 DTYPE_CODE = {"f32": SH_F32, "f16": SH_F16, "bf16": SH_BF16, "int4": SH_INT4_G64_F16}
 INPUT_TORCH_DTYPE = {SH_F32: torch.float32, SH_F16: torch.float16, SH_BF16: torch.bfloat16,
@@ -32,7 +32,12 @@ EXPORTS = ["sh_create", "sh_destroy", "sh_workspace_bytes", "sh_bind", "sh_set_o
 
 def _load() -> C.CDLL:
     path = _build.LIB
-    if _build.stale():
+    override = os.environ.get("SH_LIBRARY")      # an alternative build of the same library
+    if override:
+        if not os.path.exists(override):
+            raise ImportError(f"SH_LIBRARY={override} does not exist")
+        path = override
+    elif _build.stale():
         try:
             path = _build.build()
         except Exception as e:  # no nvcc here: use what was shipped, if anything
@@ -94,7 +99,8 @@ class Handle:
     """
 
     def __init__(self, B: int, r: int, w: int, m: int, heads: int, head_dim: int, dtype, device="cuda:0",
-                 split: Optional[int] = None, scale: Optional[float] = None, auto_compress: bool = True):
+                 split: Optional[int] = None, scale: Optional[float] = None, auto_compress: bool = True,
+                 kernel: Optional[int] = None):
         self.dtype = DTYPE_CODE[dtype] if isinstance(dtype, str) else int(dtype)
         self.B, self.r, self.w, self.m, self.U, self.D = B, r, w, m, heads, head_dim
         self.Bw = (B + 31) // 32
@@ -109,6 +115,8 @@ class Handle:
             self.set_option(SH_OPT_SOFTMAX_SCALE, scale)
         if split is not None:
             self.set_option(SH_OPT_SPLIT, split)
+        if kernel is not None:
+            self.set_option(SH_OPT_DECODE_KERNEL, kernel)
         self.set_option(SH_OPT_AUTO_COMPRESS, 1.0 if auto_compress else 0.0)
         self.workspace_bytes = int(lib.sh_workspace_bytes(h))
         with torch.cuda.device(self.device):

@@ -35,24 +35,25 @@ def stale() -> bool:
     return any(os.path.getmtime(f) > mt for f in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, out: str = LIB) -> str:
     """Compile every .cu under csrc/ into one shared library.  Returns its path."""
-    if not force and not stale():
+    if out == LIB and not force and not stale():
         return LIB
-    os.makedirs(LIB_DIR, exist_ok=True)
-    tmp = LIB + f".{os.getpid()}.tmp"
+    os.makedirs(os.path.dirname(out), exist_ok=True)
+    tmp = out + f".{os.getpid()}.tmp"
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC, "-o", tmp]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += os.environ.get("SH_NVCC_FLAGS", "").split()
     cmd += sources()
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
     if verbose:
         print(res.stderr)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, out)
+    return out
 
 
 if __name__ == "__main__":

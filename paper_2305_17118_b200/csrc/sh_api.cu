@@ -150,6 +150,7 @@ int sh_create(int B, int r, int w, int m, int heads, int head_dim, int dtype, sh
     c->scale = (float)(1.0 / std::sqrt((double)head_dim));
     c->split = default_split(heads, B);
     c->auto_compress = 1;
+    c->kernel = 0;
     c->started = false;
     c->slab = nullptr; c->slab_bytes = 0;
     c->launches = 0;
@@ -193,6 +194,12 @@ int sh_set_option(sh_handle h, int key, double value) {
         case SH_OPT_AUTO_COMPRESS:
             h->auto_compress = value != 0.0;
             return SH_OK;
+        case SH_OPT_DECODE_KERNEL: {
+            const int k = (int)value;
+            if (k < 0 || k > 2) return SH_EINVAL;
+            h->kernel = k;
+            return SH_OK;
+        }
         default: return SH_EINVAL;
     }
 }

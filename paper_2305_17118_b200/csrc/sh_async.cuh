@@ -2,14 +2,18 @@
 // helpers.  Only CTA-local forms are used: no cluster-wide delivery of a load
 // to several CTAs and no remote memory.
 //
-// Every wait is bounded: after SH_WAIT_LIMIT unsuccessful polls the waiter
-// records a code in a device error word and gives up, so a kernel can never
-// spin forever; the host reports the word through sh_state.
+// Every wait is bounded, by a poll count and by wall time (about a second on
+// the global timer): the waiter then records a code in a device error word and
+// gives up, so a kernel can never spin forever; the host reports the word
+// through sh_state.
 #pragma once
 #include <stdint.h>
 
 #ifndef SH_WAIT_LIMIT
-#define SH_WAIT_LIMIT (1u << 24)
+#define SH_WAIT_LIMIT (1u << 26)
+#endif
+#ifndef SH_WAIT_NS
+#define SH_WAIT_NS 1000000000ull
 #endif
 
 namespace shasync {
@@ -44,9 +48,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     return ok != 0;
 }
 // Wait for the phase with the given parity to complete; false (and *err = code) on giving up.
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *err, int code) {
-    for (uint32_t i = 0; i < SH_WAIT_LIMIT; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t i = 1; i < SH_WAIT_LIMIT; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 255u) == 0 && global_ns() - t0 > SH_WAIT_NS) break;
+    }
     if (err) atomicCAS(err, 0, code);
     return false;
 }

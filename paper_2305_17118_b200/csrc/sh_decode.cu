@@ -457,20 +457,30 @@ cudaError_t launch_split(const sh_context *c, const DecodeParams &p, cudaStream_
 }  // namespace
 
 cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches) {
+    // Large unit counts stream through the persistent pipelined kernel; small ones
+    // (where a cluster split is needed to fill the GPU) and the other dtypes use this file's.
+    if (c->kernel != 1 && sh_decode_tma_supported(c) && (c->kernel == 2 || c->U >= 2 * 148))
+        return sh_launch_decode_tma(c, p, s, launches);
     cudaError_t e = cudaErrorInvalidValue;
-    constexpr int NW = 8;
+#ifndef SH_DECODE_NW
+#define SH_DECODE_NW 8
+#endif
+#ifndef SH_DECODE_R
+#define SH_DECODE_R 8
+#endif
+    constexpr int NW = SH_DECODE_NW;
     switch (c->dtype) {
         case SH_F32:
-            if (c->D == 64) e = launch_split<SH_F32, 64, NW, 8>(c, p, s);
-            else if (c->D == 128) e = launch_split<SH_F32, 128, NW, 8>(c, p, s);
+            if (c->D == 64) e = launch_split<SH_F32, 64, NW, SH_DECODE_R>(c, p, s);
+            else if (c->D == 128) e = launch_split<SH_F32, 128, NW, SH_DECODE_R>(c, p, s);
             break;
         case SH_F16:
-            if (c->D == 64) e = launch_split<SH_F16, 64, NW, 8>(c, p, s);
-            else if (c->D == 128) e = launch_split<SH_F16, 128, NW, 8>(c, p, s);
+            if (c->D == 64) e = launch_split<SH_F16, 64, NW, SH_DECODE_R>(c, p, s);
+            else if (c->D == 128) e = launch_split<SH_F16, 128, NW, SH_DECODE_R>(c, p, s);
             break;
         case SH_BF16:
-            if (c->D == 64) e = launch_split<SH_BF16, 64, NW, 8>(c, p, s);
-            else if (c->D == 128) e = launch_split<SH_BF16, 128, NW, 8>(c, p, s);
+            if (c->D == 64) e = launch_split<SH_BF16, 64, NW, SH_DECODE_R>(c, p, s);
+            else if (c->D == 128) e = launch_split<SH_BF16, 128, NW, SH_DECODE_R>(c, p, s);
             break;
         case SH_INT4_G64_F16:
             if (c->D == 64) e = launch_split<SH_INT4_G64_F16, 64, NW, 4>(c, p, s);

@@ -30,6 +30,7 @@ struct sh_context {
     float scale;
     int split;
     int auto_compress;
+    int kernel;      // SH_OPT_DECODE_KERNEL: 0 automatic, 1 direct loads, 2 pipelined bulk copies
     bool started;    // a step has run: options are frozen
     char *slab;
     size_t slab_bytes;
@@ -76,6 +77,9 @@ struct CompactParams {
 
 // Launchers (each returns the cudaError_t of its launch and adds to *launches).
 cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches);
+// Pipelined (bulk-copy ring) variant of the decode kernel and its applicability test.
+bool sh_decode_tma_supported(const sh_context *c);
+cudaError_t sh_launch_decode_tma(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches);
 cudaError_t sh_launch_select(const SelectParams &p, bool from_hist, cudaStream_t s, long long *launches);
 cudaError_t sh_launch_compact(const CompactParams &p, cudaStream_t s, long long *launches);
 cudaError_t sh_launch_counters(const uint32_t *hist, uint16_t *counters, int U, int B, int Bw, int w, int n,

@@ -28,11 +28,12 @@ def main():
     ap.add_argument("--rows", type=int, default=None, help="live rows before the first step")
     ap.add_argument("--compress", action="store_true")
     ap.add_argument("--split", type=int, default=None)
+    ap.add_argument("--kernel", type=int, default=None, help="1 direct loads, 2 pipelined bulk copies")
     args = ap.parse_args()
     cfg = wl.CONFIGS[args.config]
     U, d = args.units, cfg.head_dim
     torch.cuda.set_device(0)
-    h = sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, U, d, cfg.dtype, split=args.split, auto_compress=True)
+    h = sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, U, d, cfg.dtype, split=args.split, kernel=args.kernel, auto_compress=True)
     rows = args.rows if args.rows is not None else (cfg.B - 1 if args.compress else cfg.B - cfg.m // 2)
     # K then V sit at the start of the workspace, [U][B][row_bytes] each.
     row_bytes = {"f32": 4 * d, "f16": 2 * d, "bf16": 2 * d, "int4": d // 2}[cfg.dtype]

@@ -48,6 +48,19 @@ def test_lockstep_edge_parameters(sh, B, r, w, m):
     assert res.compressions >= 1
 
 
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("U,B,r,w,m", [(5, 150, 9, 37, 41), (301, 130, 16, 33, 50), (3, 700, 5, 64, 300), (2, 40, 3, 9, 20)])
+def test_lockstep_pipelined_kernel(sh, dtype, U, B, r, w, m):
+    """The persistent bulk-copy variant of the decode kernel, forced on shapes that
+    cover fewer units than CTAs, more units than SMs, ragged last tiles and tiny caches."""
+    d, T = 128, 2 * B + 2 * m + 7
+    q, k, v = wl.random_stream(U, d, T, seed=11 + U, dtype=dtype, peaked=3.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, split=1, kernel=2, auto_compress=False)
+    res, _ = run_lockstep(h, dtype, _stream_fn(q, k, v), T, torch.arange(U), TOL[dtype])
+    assert res.compressions >= 3
+    assert res.adoptions <= 1e-4 * res.slot_steps + 2
+
+
 # ---- the benchmark's own configurations ----------------------------------------------------
 def test_config_tiny_every_step(sh):
     cfg = wl.CONFIGS["tiny"]
