@@ -368,7 +368,7 @@ cudaError_t launch_tma(const sh_context *c, const DecodeParams &p, cudaStream_t 
 }  // namespace
 
 #ifndef SH_TMA_NWC
-#define SH_TMA_NWC 16
+#define SH_TMA_NWC 8
 #endif
 #ifndef SH_TMA_SR
 #define SH_TMA_SR 128
