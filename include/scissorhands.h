@@ -64,7 +64,7 @@ typedef enum {
                                  0: the caller calls sh_compress */
     SH_OPT_DECODE_KERNEL = 3  /* 0 (default): chosen from the shape; 1: one CTA (or cluster) per unit with
                                  direct loads; 2: persistent CTAs fed by bulk asynchronous copies
-                                 (fp16/bf16, head_dim 128, split 1 only; otherwise 1 is used) */
+                                 (fp16/bf16 with head_dim 128 only, SH_OPT_SPLIT ignored; other shapes use 1) */
 } sh_option;
 
 /*

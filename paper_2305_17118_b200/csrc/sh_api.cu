@@ -149,6 +149,7 @@ int sh_create(int B, int r, int w, int m, int heads, int head_dim, int dtype, sh
     c->n = 0; c->t = 0;
     c->scale = (float)(1.0 / std::sqrt((double)head_dim));
     c->split = default_split(heads, B);
+    c->split_explicit = false;
     c->auto_compress = 1;
     c->kernel = 0;
     c->started = false;
@@ -189,6 +190,7 @@ int sh_set_option(sh_handle h, int key, double value) {
             const int s = (int)value;
             if (s != 1 && s != 2 && s != 4 && s != 8) return SH_EINVAL;
             h->split = s;
+            h->split_explicit = true;
             return SH_OK;
         }
         case SH_OPT_AUTO_COMPRESS:

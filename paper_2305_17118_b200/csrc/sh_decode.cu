@@ -31,8 +31,30 @@ __device__ __forceinline__ uint4 ld_stream(const void *p) {
 __device__ __forceinline__ uint4 ld_plain(const void *p) { return *reinterpret_cast<const uint4 *>(p); }
 __device__ __forceinline__ void st_plain(void *p, const uint4 &v) { *reinterpret_cast<uint4 *>(p) = v; }
 
+// d0 += a0*b, d1 += a1*b in one packed fp32 instruction (sm_100 FFMA2).
+__device__ __forceinline__ void ffma2(float &d0, float &d1, float a0, float a1, float b) {
+    asm("{.reg .b64 ra, rb, rc;\n\t"
+        "mov.b64 ra, {%2, %3}; mov.b64 rb, {%4, %4}; mov.b64 rc, {%0, %1};\n\t"
+        "fma.rn.f32x2 rc, ra, rb, rc;\n\t"
+        "mov.b64 {%0, %1}, rc;}"
+        : "+f"(d0), "+f"(d1)
+        : "f"(a0), "f"(a1), "f"(b));
+}
+// a0 += q.lo*k.lo, a1 += q.hi*k.hi for one packed pair: mixed-precision FMA (16-bit inputs,
+// exact fp32 product and sum), so no separate conversion instructions are needed.
+__device__ __forceinline__ void fma_pair_f16(float &a0, float &a1, uint32_t q2, uint32_t k2) {
+    asm("{.reg .b16 kl, kh, ql, qh;\n\t"
+        "mov.b32 {kl, kh}, %2; mov.b32 {ql, qh}, %3;\n\t"
+        "fma.rn.f32.f16 %0, ql, kl, %0; fma.rn.f32.f16 %1, qh, kh, %1;}"
+        : "+f"(a0), "+f"(a1)
+        : "r"(k2), "r"(q2));
+}
+
 // ---------------------------------------------------------------- element traits
 // A "chunk" is the 16 bytes one lane loads from a stored row; EPL elements.
+//   Q:    this lane's EPL elements of the query, in the form `dot` wants them
+//   dot:  sum over the chunk of q*k (fp32 accumulation; int4: of q*code, scale applied by the caller)
+//   axpy: acc[0..EPL) += p * v (int4: p * code)
 template <int DT> struct Elem;
 
 template <> struct Elem<SH_F32> {
@@ -40,6 +62,22 @@ template <> struct Elem<SH_F32> {
     static __device__ __forceinline__ void cvt(const uint4 &r, float *f) {
         f[0] = __uint_as_float(r.x); f[1] = __uint_as_float(r.y);
         f[2] = __uint_as_float(r.z); f[3] = __uint_as_float(r.w);
+    }
+    struct Q { float f[4]; };
+    static __device__ __forceinline__ void load_q(const void *row, int c, Q &q) { cvt(ld_plain(reinterpret_cast<const char *>(row) + c * 16), q.f); }
+    static __device__ __forceinline__ void q_floats(const Q &q, float *f) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) f[e] = q.f[e];
+    }
+    static __device__ __forceinline__ float dot(const Q &q, const uint4 &r) {
+        float a = __uint_as_float(r.x) * q.f[0];
+        a = fmaf(__uint_as_float(r.y), q.f[1], a);
+        a = fmaf(__uint_as_float(r.z), q.f[2], a);
+        return fmaf(__uint_as_float(r.w), q.f[3], a);
+    }
+    static __device__ __forceinline__ void axpy(float *acc, float p, const uint4 &r) {
+        acc[0] = fmaf(p, __uint_as_float(r.x), acc[0]); acc[1] = fmaf(p, __uint_as_float(r.y), acc[1]);
+        acc[2] = fmaf(p, __uint_as_float(r.z), acc[2]); acc[3] = fmaf(p, __uint_as_float(r.w), acc[3]);
     }
 };
 template <> struct Elem<SH_F16> {
@@ -52,6 +90,29 @@ template <> struct Elem<SH_F16> {
             f[2 * i] = t.x; f[2 * i + 1] = t.y;
         }
     }
+    // With one CTA per unit and ~5 CTAs per SM this kernel is sensitive to register count:
+    // convert-then-FMA (48 registers) measured faster here than the mixed-precision and packed
+    // forms the pipelined kernel uses (62 registers, one CTA per SM fewer).
+    struct Q { float f[8]; };
+    static __device__ __forceinline__ void load_q(const void *row, int c, Q &q) { cvt(ld_plain(reinterpret_cast<const char *>(row) + c * 16), q.f); }
+    static __device__ __forceinline__ void q_floats(const Q &q, float *f) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) f[e] = q.f[e];
+    }
+    static __device__ __forceinline__ float dot(const Q &q, const uint4 &r) {
+        float f[8];
+        cvt(r, f);
+        float a = 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) a = fmaf(q.f[e], f[e], a);
+        return a;
+    }
+    static __device__ __forceinline__ void axpy(float *acc, float p, const uint4 &r) {
+        float f[8];
+        cvt(r, f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] = fmaf(p, f[e], acc[e]);
+    }
 };
 template <> struct Elem<SH_BF16> {
     static constexpr int EPL = 8;
@@ -62,6 +123,26 @@ template <> struct Elem<SH_BF16> {
             f[2 * i] = __uint_as_float(w[i] << 16);
             f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
         }
+    }
+    struct Q { float f[8]; };
+    static __device__ __forceinline__ void load_q(const void *row, int c, Q &q) { cvt(ld_plain(reinterpret_cast<const char *>(row) + c * 16), q.f); }
+    static __device__ __forceinline__ void q_floats(const Q &q, float *f) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) f[e] = q.f[e];
+    }
+    static __device__ __forceinline__ float dot(const Q &q, const uint4 &r) {
+        float f[8];
+        cvt(r, f);
+        float a = 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) a = fmaf(q.f[e], f[e], a);
+        return a;
+    }
+    static __device__ __forceinline__ void axpy(float *acc, float p, const uint4 &r) {
+        float f[8];
+        cvt(r, f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] = fmaf(p, f[e], acc[e]);
     }
 };
 // int4 store: a chunk is 32 codes.  Word k of the chunk holds elements 8k..8k+7;
@@ -80,6 +161,46 @@ template <> struct Elem<SH_INT4_G64_F16> {
                 __half2 h = __hsub2(*reinterpret_cast<__half2 *>(&bits), bias);
                 float2 t = __half22float2(h);
                 f[8 * k + 2 * i] = t.x; f[8 * k + 2 * i + 1] = t.y;
+            }
+        }
+    }
+    // the query's 32 fp16 elements of this chunk: word 4k+i holds elements 8k+2i, 8k+2i+1,
+    // the same pairing the code extraction below produces
+    struct Q { uint4 raw[4]; };
+    static __device__ __forceinline__ void load_q(const void *row, int c, Q &q) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) q.raw[k] = ld_plain(reinterpret_cast<const char *>(row) + c * 64 + 16 * k);
+    }
+    static __device__ __forceinline__ void q_floats(const Q &q, float *f) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) Elem<SH_F16>::cvt(q.raw[k], f + 8 * k);
+    }
+    static __device__ __forceinline__ float dot(const Q &q, const uint4 &r) {
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+        const __half2 bias = __floats2half2_rn(1032.f, 1032.f);
+        float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t qw[4] = {q.raw[k].x, q.raw[k].y, q.raw[k].z, q.raw[k].w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint32_t bits = ((w[k] >> (4 * i)) & 0x000F000Fu) | 0x64006400u;
+                const __half2 h = __hsub2(*reinterpret_cast<__half2 *>(&bits), bias);   // exact small integers
+                fma_pair_f16(a0, a1, qw[i], *reinterpret_cast<const uint32_t *>(&h));
+            }
+        }
+        return a0 + a1;
+    }
+    static __device__ __forceinline__ void axpy(float *acc, float p, const uint4 &r) {
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+        const __half2 bias = __floats2half2_rn(1032.f, 1032.f);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint32_t bits = ((w[k] >> (4 * i)) & 0x000F000Fu) | 0x64006400u;
+                const float2 t = __half22float2(__hsub2(*reinterpret_cast<__half2 *>(&bits), bias));
+                ffma2(acc[8 * k + 2 * i], acc[8 * k + 2 * i + 1], t.x, t.y, p);
             }
         }
     }
@@ -212,8 +333,8 @@ __global__ void __launch_bounds__(NW * 32) sh_decode_kernel(const DecodeParams p
     const int cnt = max(hi_all - lo, 0);
 
     // ---- q chunk of this lane, fp32
-    float qf[EPL];
-    load_input<DT>(reinterpret_cast<const char *>(p.q) + (size_t)u * INB, c, qf);
+    typename E::Q qv;
+    E::load_q(reinterpret_cast<const char *>(p.q) + (size_t)u * INB, c, qv);
 
     const char *Kb = p.K + (size_t)u * B * ROWB;
     const char *Vb = p.V + (size_t)u * B * ROWB;
@@ -238,11 +359,7 @@ __global__ void __launch_bounds__(NW * 32) sh_decode_kernel(const DecodeParams p
         float part[R];
 #pragma unroll
         for (int i = 0; i < R; ++i) {
-            float f[EPL];
-            E::cvt(raw[i], f);
-            float a = 0.f;
-#pragma unroll
-            for (int e = 0; e < EPL; ++e) a = fmaf(qf[e], f[e], a);
+            const float a = E::dot(qv, raw[i]);
             part[i] = Q4 ? a * rs[i] : a;
         }
         int rowi = 0;
@@ -289,8 +406,12 @@ __global__ void __launch_bounds__(NW * 32) sh_decode_kernel(const DecodeParams p
             st_plain(vdst, ld_plain(reinterpret_cast<const char *>(p.v_new) + (size_t)u * INB + c * 16));
         }
         float a = 0.f;
+        {
+            float qf[EPL];
+            E::q_floats(qv, qf);
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) a = fmaf(qf[e], fk[e], a);
+            for (int e = 0; e < EPL; ++e) a = fmaf(qf[e], fk[e], a);
+        }
 #pragma unroll
         for (int o = LPR / 2; o; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
         const float s = a * p.scale_log2e;
@@ -349,12 +470,7 @@ __global__ void __launch_bounds__(NW * 32) sh_decode_kernel(const DecodeParams p
             }
         }
 #pragma unroll
-        for (int i = 0; i < R; ++i) {
-            float f[EPL];
-            E::cvt(raw[i], f);
-#pragma unroll
-            for (int e = 0; e < EPL; ++e) acc[e] = fmaf(pe[i], f[e], acc[e]);
-        }
+        for (int i = 0; i < R; ++i) E::axpy(acc, pe[i], raw[i]);
     }
     if (has_new && warp == 0 && sub == 0) {
         const float e_new = s_sh[n_old - lo];
@@ -457,9 +573,11 @@ cudaError_t launch_split(const sh_context *c, const DecodeParams &p, cudaStream_
 }  // namespace
 
 cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches) {
-    // Large unit counts stream through the persistent pipelined kernel; small ones
-    // (where a cluster split is needed to fill the GPU) and the other dtypes use this file's.
-    if (c->kernel != 1 && sh_decode_tma_supported(c) && (c->kernel == 2 || c->U >= 2 * 148))
+    // fp16/bf16 rows of 256 bytes stream through the persistent pipelined kernel unless the
+    // caller asked for this one or for a cluster split, or there are too few units to give
+    // most SMs one; the other shapes and dtypes use this file's.
+    if (c->kernel != 1 && sh_decode_tma_supported(c) &&
+        (c->kernel == 2 || (c->U >= 128 && !(c->split_explicit && c->split > 1))))
         return sh_launch_decode_tma(c, p, s, launches);
     cudaError_t e = cudaErrorInvalidValue;
 #ifndef SH_DECODE_NW

@@ -95,9 +95,10 @@ __device__ __forceinline__ float ex2(float x) {
 }
 
 // DT dtype, D head_dim, NWC consumer warps, SR rows per tile, NST ring stages,
-// LR lanes per row (each lane owns CH = row_bytes/16/LR chunks of 16 bytes, LR apart).
-template <int DT, int D, int NWC, int SR, int NST, int LR>
-__global__ void __launch_bounds__(NWC * 32 + 32, 1) sh_decode_tma_kernel(const DecodeParams p, int *err) {
+// LR lanes per row (each lane owns CH = row_bytes/16/LR chunks of 16 bytes, LR apart),
+// CPS CTAs per SM the shared-memory footprint is sized for.
+template <int DT, int D, int NWC, int SR, int NST, int LR, int CPS>
+__global__ void __launch_bounds__(NWC * 32 + 32, CPS) sh_decode_tma_kernel(const DecodeParams p, int *err) {
     using E = ElemT<DT>;
     constexpr int EPL = E::EPL;
     constexpr int ROWB = D * E::BYTES;      // stored row == input row for these dtypes
@@ -346,7 +347,7 @@ __global__ void __launch_bounds__(NWC * 32 + 32, 1) sh_decode_tma_kernel(const D
     }
 }
 
-template <int DT, int D, int NWC, int SR, int NST, int LR>
+template <int DT, int D, int NWC, int SR, int NST, int LR, int CPS>
 cudaError_t launch_tma(const sh_context *c, const DecodeParams &p, cudaStream_t s) {
     using E = ElemT<DT>;
     constexpr int ROWB = D * E::BYTES;
@@ -354,13 +355,13 @@ cudaError_t launch_tma(const sh_context *c, const DecodeParams &p, cudaStream_t 
     const int capw = (c->B + 31) & ~31;
     const size_t smem = (size_t)NST * STAGE + sizeof(float) * ((size_t)2 * capw + (size_t)2 * NWC * D + (size_t)2 * NWC * 2);
     if (smem > 227 * 1024) return cudaErrorInvalidValue;
-    auto kern = sh_decode_tma_kernel<DT, D, NWC, SR, NST, LR>;
+    auto kern = sh_decode_tma_kernel<DT, D, NWC, SR, NST, LR, CPS>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int sms = 148;
     int dev = 0;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int grid = c->U < sms ? c->U : sms;
+    const int grid = c->U < sms * CPS ? c->U : sms * CPS;
     kern<<<grid, NWC * 32 + 32, smem, s>>>(p, reinterpret_cast<int *>(c->slab + c->L.err));
     return cudaGetLastError();
 }
@@ -379,10 +380,12 @@ cudaError_t launch_tma(const sh_context *c, const DecodeParams &p, cudaStream_t 
 #ifndef SH_TMA_LR
 #define SH_TMA_LR 8
 #endif
+#ifndef SH_TMA_CPS
+#define SH_TMA_CPS 1
+#endif
 
 // Whether the pipelined kernel can serve this handle (dtype, shape, shared memory).
 bool sh_decode_tma_supported(const sh_context *c) {
-    if (c->split != 1) return false;
     if (c->dtype != SH_F16 && c->dtype != SH_BF16) return false;
     if (c->D != 128) return false;
     const int capw = (c->B + 31) & ~31;
@@ -393,8 +396,8 @@ bool sh_decode_tma_supported(const sh_context *c) {
 
 cudaError_t sh_launch_decode_tma(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches) {
     cudaError_t e = cudaErrorInvalidValue;
-    if (c->dtype == SH_F16) e = launch_tma<SH_F16, 128, SH_TMA_NWC, SH_TMA_SR, SH_TMA_NST, SH_TMA_LR>(c, p, s);
-    else if (c->dtype == SH_BF16) e = launch_tma<SH_BF16, 128, SH_TMA_NWC, SH_TMA_SR, SH_TMA_NST, SH_TMA_LR>(c, p, s);
+    if (c->dtype == SH_F16) e = launch_tma<SH_F16, 128, SH_TMA_NWC, SH_TMA_SR, SH_TMA_NST, SH_TMA_LR, SH_TMA_CPS>(c, p, s);
+    else if (c->dtype == SH_BF16) e = launch_tma<SH_BF16, 128, SH_TMA_NWC, SH_TMA_SR, SH_TMA_NST, SH_TMA_LR, SH_TMA_CPS>(c, p, s);
     if (e == cudaSuccess) *launches += 1;
     return e;
 }

@@ -29,6 +29,7 @@ struct sh_context {
     long long t;     // tokens streamed per unit
     float scale;
     int split;
+    bool split_explicit;   // SH_OPT_SPLIT was set by the caller
     int auto_compress;
     int kernel;      // SH_OPT_DECODE_KERNEL: 0 automatic, 1 direct loads, 2 pipelined bulk copies
     bool started;    // a step has run: options are frozen
