@@ -105,6 +105,19 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def job_throughput(local_ms: float, steps: int, world: int, dist=None, device=None):
+    """Whole-job steps/s when every rank ran `steps` steps of its own replica of the
+    workload: the slowest rank's device time decides (max over ranks), and the job
+    processed world x the units of one replica.  Returns (ms_per_step, steps_per_s)."""
+    ms = float(local_ms)
+    if dist is not None and world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    per_step = ms / steps
+    return per_step, world * 1e3 / per_step
+
+
 def live_rows_schedule(cfg, first_step: int, count: int):
     """n (rows attended, new token included) at stream steps first_step.. ; the
     schedule is data-independent: n grows by one per step and drops by m when it reaches B."""
@@ -249,12 +262,7 @@ def cuda_arm(args, cfg, rank, world):
     else:
         total_ms = ev0.elapsed_time(ev1)
     kern_ms = [a.elapsed_time(b) for a, b in pairs]
-    if dist:
-        tt = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
-    ms_per_step = total_ms / K
-    value = world * 1e3 / ms_per_step
+    ms_per_step, value = job_throughput(total_ms, K, world, dist, dev)
 
     # ---- roofline of the fused decode kernel (one launch = one layer's units)
     n_sched = live_rows_schedule(cfg, cfg.prompt + W + 1, K)
@@ -299,13 +307,9 @@ def cuda_arm(args, cfg, rank, world):
                 h.compress()
         e1.record()
         barrier()
-        e_ms = e0.elapsed_time(e1)
-        if dist:
-            tt = torch.tensor([e_ms], device=dev)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e_ms = float(tt.item())
+        _, e_value = job_throughput(e0.elapsed_time(e1), Ke, world, dist, dev)
         in_b = Ly * U * d * (4 if cfg.dtype == "f32" else 2) * 3
-        e2e = {"value": world * Ke * 1e3 / e_ms, "unit": UNIT, "h2d_bytes_per_step": in_b,
+        e2e = {"value": e_value, "unit": UNIT, "h2d_bytes_per_step": in_b,
                "d2h_bytes_per_step": Ly * U * d * 4, "steps": Ke}
 
     if rank != 0:
