@@ -195,16 +195,22 @@ def cuda_arm(args, cfg, rank, world):
     U, d, Ly = cfg.units, cfg.head_dim, cfg.layers
     streams = [wl.Stream(cfg, device=dev, layer=l + 1000 * rank) for l in range(Ly)]
     handles = [sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, U, d, cfg.dtype, device=dev, auto_compress=False,
-                         split=args.split, kernel=args.kernel)
+                         split=args.split, kernel=args.kernel,
+                         prefill_chunk=False if args.no_prefill_chunk else None)
                for _ in range(Ly)]
 
     # ---- prompt: streamed through the same path, untimed
-    blk = max(1, min(64, (1 << 28) // (U * d * 2 * 3)))
+    blk = max(1, min(256, (1 << 31) // (U * d * 2 * 3)))
+    prompt_ms = 0.0
     for l, (h, st) in enumerate(zip(handles, streams)):
         for t0 in range(1, cfg.prompt + 1, blk):
             q, k, v = st.block(t0, min(t0 + blk, cfg.prompt + 1))
+            pa, pb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            pa.record()
             h.prefill(q, k, v)
-        torch.cuda.synchronize()
+            pb.record()
+            torch.cuda.synchronize()
+            prompt_ms += pa.elapsed_time(pb)
     # ---- decode inputs resident in HBM; cycle if the run is longer than the buffer
     n_in = min(W + K, max(1, int(6e9 // (Ly * U * d * 2 * 3))))
     dec = [st.block(cfg.prompt + 1, cfg.prompt + 1 + n_in) for st in streams]
@@ -329,6 +335,9 @@ def cuda_arm(args, cfg, rank, world):
                    "prompt": cfg.prompt, "l2": "flushed between steps" if flush else "inputs larger than L2",
                    "kv_bytes": kv_bytes, "parallelism": f"units replicated x{world}" if world > 1 else "1 GPU"},
         "attn_GBps": statistics.fmean(n_sched) * U * Ly * d * ES[cfg.dtype] * 2 / (ms_per_step * 1e-3) / 1e9,
+        "prompt": {"tokens": cfg.prompt, "ms": prompt_ms, "tokens_per_s": cfg.prompt * 1e3 / prompt_ms if prompt_ms else None,
+                   "chunked": bool(handles[0].prefill_chunk_max) and not args.no_prefill_chunk,
+                   "note": "untimed part of the benchmark; streamed through sh_prefill in blocks of %d tokens" % blk},
         "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": launches,
         "roofline": roofline, "cpu_baseline": cpu,
     }
@@ -347,6 +356,7 @@ def main():
     ap.add_argument("--oracle-units", type=int, default=2048)
     ap.add_argument("--split", type=int, default=None, help="CTAs per unit (default: chosen by the library)")
     ap.add_argument("--kernel", type=int, default=None, help="decode kernel: 1 direct loads, 2 pipelined bulk copies")
+    ap.add_argument("--no-prefill-chunk", action="store_true", help="stream the prompt one decode step per token")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (tuning runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup

@@ -62,6 +62,8 @@ typedef enum {
     SH_OPT_SPLIT = 1,         /* CTAs cooperating on one unit (1, 2, 4 or 8); default chosen from `heads` */
     SH_OPT_AUTO_COMPRESS = 2, /* 1 (default): sh_decode_step compresses by itself when the cache fills;
                                  0: the caller calls sh_compress */
+    SH_OPT_PREFILL_CHUNK = 4, /* 1 (default): sh_prefill hands the tokens between two compressions to the chunk
+                                 kernel where the shape allows it; 0: one decode step per token */
     SH_OPT_DECODE_KERNEL = 3  /* 0 (default): chosen from the shape; 1: one CTA (or cluster) per unit with
                                  direct loads; 2: persistent CTAs fed by bulk asynchronous copies
                                  (fp16/bf16 with head_dim 128 only, SH_OPT_SPLIT ignored; other shapes use 1) */
@@ -127,9 +129,26 @@ int sh_decode_step_host(sh_handle h, const void *q_host, const void *k_new_host,
  * sh_decode_step (each followed by a compression when the cache fills),
  * whatever SH_OPT_AUTO_COMPRESS says.  q_dev, k_dev, v_dev: time-major
  * [p][heads][head_dim].  out_dev: [p][heads][head_dim] fp32 or NULL to discard.
+ * Between two compressions the steps only append, so for fp16/bf16 stores with
+ * head_dim 128 they are evaluated up to 64 at a time by a tensor-core kernel
+ * (causal attention of the chunk over the cache and itself, one record
+ * bit-plane row per step); the results equal the per-token path up to fp32
+ * summation order.  SH_OPT_PREFILL_CHUNK = 0 forces the per-token path.
+ * At most 2^24 - 1 tokens may be streamed through a handle.
  */
 int sh_prefill(sh_handle h, const void *q_dev, const void *k_dev, const void *v_dev, int p,
                float *out_dev, void *stream);
+
+/*
+ * One chunk of the prompt without the compression: steps t+1 .. t+count for
+ * every unit in one launch (see sh_prefill).  Needs 1 <= count <=
+ * sh_prefill_chunk_max(h) and count <= B - n; returns SH_EINVAL otherwise
+ * (sh_prefill_chunk_max is 0 when the handle's dtype or shape is not served).
+ * Layout as sh_prefill.  The caller compresses when n reaches B.
+ */
+int sh_prefill_chunk(sh_handle h, const void *q_dev, const void *k_dev, const void *v_dev, int count,
+                     float *out_dev, void *stream);
+int sh_prefill_chunk_max(sh_handle h);
 
 /*
  * Algorithm 2 for every unit, if the cache is full (n == B): importance
@@ -189,6 +208,11 @@ int sh_select(const uint16_t *counters_dev, int units, int n, int r, int m, int3
  */
 int sh_state(sh_handle h, void *stream, int *n_out, long long *t_out, int32_t *pos_host,
              uint16_t *counters_host, uint32_t *low_host);
+
+/* The record bit-planes of one unit, [w][ceil(B/32)] uint32 on the host: row (s mod w) holds, for
+ * step s of the last w steps, bit j%32 of word j/32 = [alpha_j < 1/s] for the token now in slot j.
+ * Synchronises. */
+int sh_export_record(sh_handle h, int unit, uint32_t *planes_host, void *stream);
 
 /* Stored K and V rows of one unit as fp32 (int4: dequantised), [B][head_dim]
  * each on the host; rows beyond n are whatever the slots hold.  Synchronises. */

@@ -19,14 +19,15 @@ from . import build as _build
 SH_OK, SH_EINVAL, SH_EFULL, SH_ESTATE, SH_ECUDA, SH_ENOMEM, SH_ETOOBIG, SH_EDEVICE = 0, -1, -2, -3, -4, -5, -6, -7
 SH_STATIC_SCRATCH_MAX_ENTRIES = 1 << 20
 SH_F32, SH_F16, SH_BF16, SH_INT4_G64_F16 = 0, 1, 2, 3
-SH_OPT_SOFTMAX_SCALE, SH_OPT_SPLIT, SH_OPT_AUTO_COMPRESS, SH_OPT_DECODE_KERNEL = 0, 1, 2, 3
+SH_OPT_SOFTMAX_SCALE, SH_OPT_SPLIT, SH_OPT_AUTO_COMPRESS, SH_OPT_DECODE_KERNEL, SH_OPT_PREFILL_CHUNK = 0, 1, 2, 3, 4
 
 DTYPE_CODE = {"f32": SH_F32, "f16": SH_F16, "bf16": SH_BF16, "int4": SH_INT4_G64_F16}
 INPUT_TORCH_DTYPE = {SH_F32: torch.float32, SH_F16: torch.float16, SH_BF16: torch.bfloat16,
                      SH_INT4_G64_F16: torch.float16}
 
 EXPORTS = ["sh_create", "sh_destroy", "sh_workspace_bytes", "sh_bind", "sh_set_option", "sh_decode_step",
-           "sh_decode_step_host", "sh_prefill", "sh_compress", "sh_compress_static", "sh_select", "sh_state", "sh_export_unit",
+           "sh_decode_step_host", "sh_prefill", "sh_prefill_chunk", "sh_prefill_chunk_max", "sh_export_record",
+           "sh_compress", "sh_compress_static", "sh_select", "sh_state", "sh_export_unit",
            "sh_restore", "sh_launch_count", "sh_strerror", "sh_last_cuda_error"]
 
 
@@ -55,6 +56,9 @@ def _load() -> C.CDLL:
     lib.sh_decode_step.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.sh_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.sh_prefill.argtypes = [vp, vp, vp, vp, C.c_int, vp, vp]
+    lib.sh_prefill_chunk.argtypes = [vp, vp, vp, vp, C.c_int, vp, vp]
+    lib.sh_prefill_chunk_max.argtypes = [vp]
+    lib.sh_export_record.argtypes = [vp, C.c_int, vp, vp]
     lib.sh_compress.argtypes = [vp, vp, ip]
     lib.sh_compress_static.argtypes = [vp, vp, ip]
     lib.sh_select.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
@@ -100,7 +104,7 @@ class Handle:
 
     def __init__(self, B: int, r: int, w: int, m: int, heads: int, head_dim: int, dtype, device="cuda:0",
                  split: Optional[int] = None, scale: Optional[float] = None, auto_compress: bool = True,
-                 kernel: Optional[int] = None):
+                 kernel: Optional[int] = None, prefill_chunk: Optional[bool] = None):
         self.dtype = DTYPE_CODE[dtype] if isinstance(dtype, str) else int(dtype)
         self.B, self.r, self.w, self.m, self.U, self.D = B, r, w, m, heads, head_dim
         self.Bw = (B + 31) // 32
@@ -117,6 +121,8 @@ class Handle:
             self.set_option(SH_OPT_SPLIT, split)
         if kernel is not None:
             self.set_option(SH_OPT_DECODE_KERNEL, kernel)
+        if prefill_chunk is not None:
+            self.set_option(SH_OPT_PREFILL_CHUNK, 1.0 if prefill_chunk else 0.0)
         self.set_option(SH_OPT_AUTO_COMPRESS, 1.0 if auto_compress else 0.0)
         self.workspace_bytes = int(lib.sh_workspace_bytes(h))
         with torch.cuda.device(self.device):
@@ -171,6 +177,27 @@ class Handle:
         self._check(lib.sh_prefill(self._h, _dev(q, self.in_dtype, n, "q"), _dev(k, self.in_dtype, n, "k"),
                                    _dev(v, self.in_dtype, n, "v"), p, optr, _stream_ptr(stream)))
         return out
+
+    # -- sh_prefill_chunk --------------------------------------------------------
+    @property
+    def prefill_chunk_max(self) -> int:
+        return int(lib.sh_prefill_chunk_max(self._h))
+
+    def prefill_chunk(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: Optional[torch.Tensor] = None,
+                      stream=None):
+        c = q.shape[0]
+        n = c * self.U * self.D
+        optr = _dev(out, torch.float32, n, "out") if out is not None else None
+        self._check(lib.sh_prefill_chunk(self._h, _dev(q, self.in_dtype, n, "q"), _dev(k, self.in_dtype, n, "k"),
+                                         _dev(v, self.in_dtype, n, "v"), c, optr, _stream_ptr(stream)))
+        return out
+
+    # -- sh_export_record -----------------------------------------------------------
+    def export_record(self, unit: int, stream=None) -> np.ndarray:
+        """Bit-planes of one unit as a bool array [w, B]: entry (s mod w, j) is step s's comparison for slot j."""
+        planes = np.zeros((self.w, self.Bw), dtype=np.uint32)
+        self._check(lib.sh_export_record(self._h, unit, planes.ctypes.data, _stream_ptr(stream)))
+        return np.unpackbits(planes.view(np.uint8), axis=1, bitorder="little")[:, : self.B].astype(bool)
 
     # -- sh_compress -------------------------------------------------------------
     def compress(self, stream=None) -> int:

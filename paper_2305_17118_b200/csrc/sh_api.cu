@@ -152,6 +152,7 @@ int sh_create(int B, int r, int w, int m, int heads, int head_dim, int dtype, sh
     c->split_explicit = false;
     c->auto_compress = 1;
     c->kernel = 0;
+    c->prefill_chunk = 1;
     c->started = false;
     c->slab = nullptr; c->slab_bytes = 0;
     c->launches = 0;
@@ -196,6 +197,9 @@ int sh_set_option(sh_handle h, int key, double value) {
         case SH_OPT_AUTO_COMPRESS:
             h->auto_compress = value != 0.0;
             return SH_OK;
+        case SH_OPT_PREFILL_CHUNK:
+            h->prefill_chunk = value != 0.0;
+            return SH_OK;
         case SH_OPT_DECODE_KERNEL: {
             const int k = (int)value;
             if (k < 0 || k > 2) return SH_EINVAL;
@@ -212,6 +216,7 @@ int sh_decode_step(sh_handle h, const void *q_dev, const void *k_new_dev, const 
     if (misaligned(q_dev) || misaligned(k_new_dev) || misaligned(v_new_dev)) return SH_EINVAL;
     if (!h->slab) return SH_ESTATE;
     if (h->n >= h->B) return SH_EFULL;
+    if (h->t + 1 >= (1 << 24)) return SH_EINVAL;   // the threshold test multiplies by t in fp32
     return do_step(h, q_dev, k_new_dev, v_new_dev, attn_out_dev, (cudaStream_t)stream, h->auto_compress != 0);
 }
 
@@ -268,22 +273,74 @@ int sh_decode_step_host(sh_handle h, const void *q_host, const void *k_new_host,
     return SH_OK;
 }
 
+// Tokens [0, count) of a time-major block through the chunk kernel; no compression.
+static int do_chunk(sh_context *c, const char *q, const char *k, const char *v, float *out, int count, cudaStream_t s) {
+    cudaError_t e = sh_launch_prefill_chunk(c, q, k, v, out, count, s, &c->launches);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->started = true;
+    c->n += count;
+    c->t += count;
+    return SH_OK;
+}
+
+int sh_prefill_chunk(sh_handle h, const void *q_dev, const void *k_dev, const void *v_dev, int count, float *out_dev,
+                     void *stream) {
+    if (!h || !q_dev || !k_dev || !v_dev || count < 1) return SH_EINVAL;
+    if (misaligned(q_dev) || misaligned(k_dev) || misaligned(v_dev)) return SH_EINVAL;
+    if (!h->slab) return SH_ESTATE;
+    if (h->n >= h->B) return SH_EFULL;
+    const int cap = sh_prefill_chunk_capacity(h);
+    if (cap == 0 || count > cap || count > h->B - h->n) return SH_EINVAL;
+    if (h->t + count >= (1 << 24)) return SH_EINVAL;
+    return do_chunk(h, static_cast<const char *>(q_dev), static_cast<const char *>(k_dev),
+                    static_cast<const char *>(v_dev), out_dev, count, (cudaStream_t)stream);
+}
+
+int sh_prefill_chunk_max(sh_handle h) { return h ? sh_prefill_chunk_capacity(h) : 0; }
+
 int sh_prefill(sh_handle h, const void *q_dev, const void *k_dev, const void *v_dev, int p, float *out_dev,
                void *stream) {
     if (!h || !q_dev || !k_dev || !v_dev || p < 0) return SH_EINVAL;
     if (misaligned(q_dev) || misaligned(k_dev) || misaligned(v_dev)) return SH_EINVAL;
     if (!h->slab) return SH_ESTATE;
     if (h->n >= h->B) return SH_EFULL;
+    if (h->t + p >= (1 << 24)) return SH_EINVAL;
     const size_t in_stride = (size_t)h->U * h->in_bytes, out_stride = (size_t)h->U * h->D;
     float *sink = reinterpret_cast<float *>(h->slab + h->L.stage_out);
-    for (int i = 0; i < p; ++i) {
+    const int cap = h->prefill_chunk ? sh_prefill_chunk_capacity(h) : 0;
+    cudaStream_t s = (cudaStream_t)stream;
+    int i = 0;
+    while (i < p) {
         const char *q = static_cast<const char *>(q_dev) + i * in_stride;
         const char *k = static_cast<const char *>(k_dev) + i * in_stride;
         const char *v = static_cast<const char *>(v_dev) + i * in_stride;
-        float *o = out_dev ? out_dev + i * out_stride : sink;
-        int rc = do_step(h, q, k, v, o, (cudaStream_t)stream, true);
+        int cnt = p - i;
+        if (cnt > h->B - h->n) cnt = h->B - h->n;
+        if (cnt > cap) cnt = cap;
+        int rc;
+        if (cnt >= 2) {
+            // the steps up to the next compression only append: take them in one launch
+            rc = do_chunk(h, q, k, v, out_dev ? out_dev + i * out_stride : nullptr, cnt, s);
+        } else {
+            cnt = 1;
+            rc = do_step(h, q, k, v, out_dev ? out_dev + i * out_stride : sink, s, false);
+        }
         if (rc != SH_OK) return rc;
+        if (h->n == h->B && (rc = do_compress(h, s)) != SH_OK) return rc;
+        i += cnt;
     }
+    return SH_OK;
+}
+
+int sh_export_record(sh_handle h, int unit, uint32_t *planes_host, void *stream) {
+    if (!h || unit < 0 || unit >= h->U || !planes_host) return SH_EINVAL;
+    if (!h->slab) return SH_ESTATE;
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t bytes = (size_t)h->w * h->Bw * 4;
+    cudaError_t e = cudaMemcpyAsync(planes_host, h->slab + h->L.hist + (size_t)unit * bytes, bytes,
+                                    cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(h, e);
     return SH_OK;
 }
 

@@ -31,6 +31,7 @@ struct sh_context {
     int split;
     bool split_explicit;   // SH_OPT_SPLIT was set by the caller
     int auto_compress;
+    int prefill_chunk;  // SH_OPT_PREFILL_CHUNK: 1 = sh_prefill may batch tokens between compressions
     int kernel;      // SH_OPT_DECODE_KERNEL: 0 automatic, 1 direct loads, 2 pipelined bulk copies
     bool started;    // a step has run: options are frozen
     char *slab;
@@ -81,6 +82,10 @@ cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStr
 // Pipelined (bulk-copy ring) variant of the decode kernel and its applicability test.
 bool sh_decode_tma_supported(const sh_context *c);
 cudaError_t sh_launch_decode_tma(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches);
+// Chunked prompt kernel: tokens one launch can take for this handle (0 = unsupported), and its launcher.
+int sh_prefill_chunk_capacity(const sh_context *c);
+cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const void *k, const void *v, float *out,
+                                    int count, cudaStream_t s, long long *launches);
 cudaError_t sh_launch_select(const SelectParams &p, bool from_hist, cudaStream_t s, long long *launches);
 cudaError_t sh_launch_compact(const CompactParams &p, cudaStream_t s, long long *launches);
 cudaError_t sh_launch_counters(const uint32_t *hist, uint16_t *counters, int U, int B, int Bw, int w, int n,

@@ -1,0 +1,312 @@
+// Chunked prompt step: c consecutive tokens of the stream handled in one launch.
+//
+// Between two compressions the method's steps only append, so c steps can be
+// evaluated together: step i (0 <= i < c) attends with q_i over the n0 cached
+// rows plus the chunk's own tokens 0..i (causal), and records its comparison
+// bits in its own bit-plane row.  The results are those of c calls of the
+// decode step; K and V are read from HBM once per chunk instead of once per
+// token, and the two contractions S = Q.K^T  [c x n x d] and O = P.V [c x d x n]
+// are dense enough (about 50 FLOP per byte) to belong on the tensor cores.
+//
+// One CTA of 8 warps per unit.  S is kept whole in shared memory in fp32
+// ([CQ][n] - the record bits need every probability against the final row sum),
+// K and V pass through a 64-row tile buffer.  MMAs are warp-level
+// m16n8k16 with fp32 accumulation: q.k products of 16-bit inputs are exact;
+// P is fed as a high and a low 16-bit part so that P.V keeps ~fp32 accuracy.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "sh_internal.h"
+
+namespace {
+
+constexpr int D = 128;          // head_dim served by this kernel
+constexpr int KT = 64;          // keys per tile
+constexpr int ROWH = D + 8;     // padded row length in 16-bit elements (272 bytes: conflict-free ldmatrix)
+constexpr int NTHREADS = 256;
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void *row_ptr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(smem_addr(row_ptr)));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void *row_ptr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(smem_addr(row_ptr)));
+}
+
+template <int DT> struct Mma;
+template <> struct Mma<SH_F16> {
+    static __device__ __forceinline__ void run(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                     : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+    }
+    // p0, p1 in [0, 1] -> packed high parts and packed low parts (p = hi + lo up to ~2^-22)
+    static __device__ __forceinline__ void split(float p0, float p1, uint32_t &hi, uint32_t &lo) {
+        const __half2 h = __floats2half2_rn(p0, p1);
+        const float2 hf = __half22float2(h);
+        const __half2 l = __floats2half2_rn(p0 - hf.x, p1 - hf.y);
+        hi = *reinterpret_cast<const uint32_t *>(&h);
+        lo = *reinterpret_cast<const uint32_t *>(&l);
+    }
+};
+template <> struct Mma<SH_BF16> {
+    static __device__ __forceinline__ void run(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                     : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+    }
+    static __device__ __forceinline__ void split(float p0, float p1, uint32_t &hi, uint32_t &lo) {
+        const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+        const float2 hf = __bfloat1622float2(h);
+        const __nv_bfloat162 l = __floats2bfloat162_rn(p0 - hf.x, p1 - hf.y);
+        hi = *reinterpret_cast<const uint32_t *>(&h);
+        lo = *reinterpret_cast<const uint32_t *>(&l);
+    }
+};
+
+struct ChunkParams {
+    const char *q, *k, *v;   // [c][U][D] time-major, 16-bit elements
+    float *out;              // [c][U][D] fp32 or NULL
+    char *K, *V;             // caches [U][B][D]
+    uint32_t *hist;
+    int32_t *pos;
+    int U, B, Bw, w;
+    int n0;                  // live rows before the chunk
+    int c;                   // tokens in the chunk (<= CQ, <= w, n0 + c <= B)
+    int t0;                  // tokens streamed before the chunk
+    int SS;                  // row stride of S in floats
+    float scale_log2e;
+};
+
+// Fill the 64-row tile buffer with rows [j0, j0+64) of the unit's K or V as seen by
+// the chunk: cached rows, then the chunk's own tokens (which are also appended to the
+// cache here), zeros beyond.
+__device__ __forceinline__ void load_tile(uint16_t *tile, const char *cache_u, const char *chunk, char *append_u,
+                                          int j0, int n0, int n_tot, size_t chunk_stride) {
+    for (int idx = threadIdx.x; idx < KT * (D / 8); idx += NTHREADS) {
+        const int row = idx / (D / 8), ch = idx % (D / 8);
+        const int j = j0 + row;
+        uint4 val = make_uint4(0, 0, 0, 0);
+        if (j < n0) {
+            val = *reinterpret_cast<const uint4 *>(cache_u + (size_t)j * (D * 2) + ch * 16);
+        } else if (j < n_tot) {
+            val = *reinterpret_cast<const uint4 *>(chunk + (size_t)(j - n0) * chunk_stride + ch * 16);
+            *reinterpret_cast<uint4 *>(append_u + (size_t)j * (D * 2) + ch * 16) = val;
+        }
+        *reinterpret_cast<uint4 *>(tile + row * ROWH + ch * 8) = val;
+    }
+}
+
+// CQ queries per CTA (64 or 32).  Warps form a WM x WN grid: WM row blocks of 16 queries,
+// WN groups that split the 64 keys of a tile (logits) or the 128 output columns (P.V).
+template <int DT, int CQ>
+__global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const ChunkParams p) {
+    constexpr int WM = CQ / 16, WN = 8 / WM;
+    constexpr int NBK = KT / WN / 8;     // 8-key blocks per warp in the logits phase
+    constexpr int NBD = D / WN / 8;      // 8-column blocks per warp in the P.V phase
+    static_assert(NBK % 2 == 0 && NBD % 2 == 0, "ldmatrix.x4 covers two 8-wide blocks");
+    using M = Mma<DT>;
+
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint16_t *Qs = reinterpret_cast<uint16_t *>(smem_raw);              // [CQ][ROWH]
+    uint16_t *tile = Qs + CQ * ROWH;                                    // [KT][ROWH]
+    float *S = reinterpret_cast<float *>(tile + KT * ROWH);             // [CQ][SS]
+    float *rowL = S + (size_t)CQ * p.SS;                                // [CQ] row sums
+
+    const int u = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int wm = warp % WM, wn = warp / WM;
+    const int n0 = p.n0, c = p.c, n_tot = p.n0 + p.c, SS = p.SS;
+    const size_t tstride = (size_t)p.U * D * 2;          // bytes between consecutive tokens of one unit
+    const char *Kc = p.K + (size_t)u * p.B * D * 2;
+    const char *Vc = p.V + (size_t)u * p.B * D * 2;
+    const int ntiles = (n_tot + KT - 1) / KT;
+
+    // ---- queries of the chunk (rows beyond c are zero)
+    for (int idx = tid; idx < CQ * (D / 8); idx += NTHREADS) {
+        const int row = idx / (D / 8), ch = idx % (D / 8);
+        uint4 val = make_uint4(0, 0, 0, 0);
+        if (row < c) val = *reinterpret_cast<const uint4 *>(p.q + (size_t)row * tstride + (size_t)u * D * 2 + ch * 16);
+        *reinterpret_cast<uint4 *>(Qs + row * ROWH + ch * 8) = val;
+    }
+    if (tid < c) p.pos[(size_t)u * p.B + n0 + tid] = p.t0 + tid + 1;
+    __syncthreads();
+
+    // A fragments of this warp's 16 queries, all 8 k-steps, kept in registers
+    uint32_t qa[D / 16][4];
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+        const int mi = lane >> 3, r = lane & 7;   // matrix index, row within it
+        ldmatrix_x4(qa[ks], Qs + (wm * 16 + (mi & 1) * 8 + r) * ROWH + ks * 16 + (mi >> 1) * 8);
+    }
+
+    // ---- phase 1: S = scale * Q.K^T, causal inside the chunk
+    for (int kt = 0; kt < ntiles; ++kt) {
+        __syncthreads();      // previous tile consumed
+        load_tile(tile, Kc, p.k + (size_t)u * D * 2, p.K + (size_t)u * p.B * D * 2, kt * KT, n0, n_tot, tstride);
+        __syncthreads();
+        float acc[NBK][4];
+#pragma unroll
+        for (int nb = 0; nb < NBK; ++nb)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[nb][e] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+#pragma unroll
+            for (int nbp = 0; nbp < NBK / 2; ++nbp) {
+                uint32_t b[4];
+                const int mi = lane >> 3, r = lane & 7;
+                ldmatrix_x4(b, tile + (wn * (KT / WN) + nbp * 16 + (mi >> 1) * 8 + r) * ROWH + ks * 16 + (mi & 1) * 8);
+                M::run(acc[2 * nbp], qa[ks], b[0], b[1]);
+                M::run(acc[2 * nbp + 1], qa[ks], b[2], b[3]);
+            }
+        }
+#pragma unroll
+        for (int nb = 0; nb < NBK; ++nb) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int i = wm * 16 + (lane >> 2) + (e >> 1) * 8;                 // query row
+                const int j = kt * KT + wn * (KT / WN) + nb * 8 + (lane & 3) * 2 + (e & 1);   // key slot
+                const bool live = i < c && j < n0 + i + 1;                           // cached rows and chunk tokens 0..i
+                S[(size_t)i * SS + j] = live ? acc[nb][e] * p.scale_log2e : -INFINITY;
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- softmax rows and record bits: one warp per query row
+    for (int i = warp; i < CQ; i += NTHREADS / 32) {
+        float *Si = S + (size_t)i * SS;
+        const int nv = (i < c) ? n0 + i + 1 : 0;
+        float mx = -INFINITY;
+        for (int j = lane; j < nv; j += 32) mx = fmaxf(mx, Si[j]);
+#pragma unroll
+        for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        float sum = 0.f;
+        for (int j = lane; j < ntiles * KT; j += 32) {
+            const float e = (j < nv) ? exp2f(Si[j] - mx) : 0.f;
+            Si[j] = e;
+            sum += e;
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (lane == 0) rowL[i] = sum;
+        if (i < c) {
+            // step t = t0 + i + 1: low_j = [alpha_j < 1/t] = [e_j * t < L]
+            const int t = p.t0 + i + 1;
+            const float tf = (float)t;
+            uint32_t *hrow = p.hist + ((size_t)u * p.w + (t % p.w)) * p.Bw;
+            __syncwarp();
+            for (int wd = 0; wd < p.Bw; ++wd) {
+                const int j = (wd << 5) + lane;
+                const bool low = j < nv && Si[j] * tf < sum;
+                const uint32_t word = __ballot_sync(0xffffffffu, low);
+                if (lane == 0) hrow[wd] = word;
+            }
+        }
+    }
+
+    // ---- phase 2: O = P.V
+    float oacc[NBD][4];
+#pragma unroll
+    for (int nb = 0; nb < NBD; ++nb)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) oacc[nb][e] = 0.f;
+    for (int kt = 0; kt < ntiles; ++kt) {
+        __syncthreads();      // S complete (first pass) / previous tile consumed
+        load_tile(tile, Vc, p.v + (size_t)u * D * 2, p.V + (size_t)u * p.B * D * 2, kt * KT, n0, n_tot, tstride);
+        __syncthreads();
+#pragma unroll
+        for (int ks = 0; ks < KT / 16; ++ks) {
+            // A fragments of P: rows r0 = wm*16 + lane/4 and r0 + 8, key columns j0 + {0,1} and j0 + 8 + {0,1}
+            const int r0 = wm * 16 + (lane >> 2);
+            const int j0 = kt * KT + ks * 16 + (lane & 3) * 2;
+            const float2 p00 = *reinterpret_cast<const float2 *>(S + (size_t)r0 * SS + j0);
+            const float2 p10 = *reinterpret_cast<const float2 *>(S + (size_t)(r0 + 8) * SS + j0);
+            const float2 p01 = *reinterpret_cast<const float2 *>(S + (size_t)r0 * SS + j0 + 8);
+            const float2 p11 = *reinterpret_cast<const float2 *>(S + (size_t)(r0 + 8) * SS + j0 + 8);
+            uint32_t ahi[4], alo[4];
+            M::split(p00.x, p00.y, ahi[0], alo[0]);
+            M::split(p10.x, p10.y, ahi[1], alo[1]);
+            M::split(p01.x, p01.y, ahi[2], alo[2]);
+            M::split(p11.x, p11.y, ahi[3], alo[3]);
+#pragma unroll
+            for (int nbp = 0; nbp < NBD / 2; ++nbp) {
+                uint32_t b[4];
+                const int mi = lane >> 3, r = lane & 7;
+                ldmatrix_x4_trans(b, tile + (ks * 16 + (mi & 1) * 8 + r) * ROWH + wn * (D / WN) + nbp * 16 + (mi >> 1) * 8);
+                M::run(oacc[2 * nbp], ahi, b[0], b[1]);
+                M::run(oacc[2 * nbp], alo, b[0], b[1]);
+                M::run(oacc[2 * nbp + 1], ahi, b[2], b[3]);
+                M::run(oacc[2 * nbp + 1], alo, b[2], b[3]);
+            }
+        }
+    }
+    if (p.out) {
+#pragma unroll
+        for (int nb = 0; nb < NBD; ++nb) {
+#pragma unroll
+            for (int hrow = 0; hrow < 2; ++hrow) {
+                const int i = wm * 16 + (lane >> 2) + hrow * 8;
+                if (i < c) {
+                    const float inv = 1.f / rowL[i];
+                    const int col = wn * (D / WN) + nb * 8 + (lane & 3) * 2;
+                    float2 o2 = make_float2(oacc[nb][2 * hrow] * inv, oacc[nb][2 * hrow + 1] * inv);
+                    *reinterpret_cast<float2 *>(p.out + ((size_t)i * p.U + u) * D + col) = o2;
+                }
+            }
+        }
+    }
+}
+
+template <int DT, int CQ>
+cudaError_t launch_chunk(const ChunkParams &p, cudaStream_t s) {
+    const size_t smem = sizeof(uint16_t) * (size_t)(CQ + KT) * ROWH + sizeof(float) * ((size_t)CQ * p.SS + CQ);
+    auto kern = sh_prefill_chunk_kernel<DT, CQ>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kern<<<p.U, NTHREADS, smem, s>>>(p);
+    return cudaGetLastError();
+}
+
+int s_stride(int B) { return ((B + KT - 1) / KT) * KT + 8; }
+size_t smem_need(int CQ, int B) {
+    return sizeof(uint16_t) * (size_t)(CQ + KT) * ROWH + sizeof(float) * ((size_t)CQ * s_stride(B) + CQ);
+}
+
+}  // namespace
+
+// Largest number of tokens one chunk launch can take for this handle (0: not supported).
+int sh_prefill_chunk_capacity(const sh_context *c) {
+    if ((c->dtype != SH_F16 && c->dtype != SH_BF16) || c->D != 128) return 0;
+    int cq = 0;
+    if (smem_need(64, c->B) <= 200 * 1024) cq = 64;
+    else if (smem_need(32, c->B) <= 200 * 1024) cq = 32;
+    if (cq > c->w) cq = c->w;     // every step of a chunk needs its own bit-plane row
+    return cq;
+}
+
+// Steps t0+1 .. t0+count (count <= capacity, n0 + count <= B) in one launch.
+cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const void *k, const void *v, float *out,
+                                    int count, cudaStream_t s, long long *launches) {
+    ChunkParams p = {};
+    p.q = static_cast<const char *>(q); p.k = static_cast<const char *>(k); p.v = static_cast<const char *>(v);
+    p.out = out;
+    p.K = c->slab + c->L.K; p.V = c->slab + c->L.V;
+    p.hist = reinterpret_cast<uint32_t *>(c->slab + c->L.hist);
+    p.pos = reinterpret_cast<int32_t *>(c->slab + c->L.pos);
+    p.U = c->U; p.B = c->B; p.Bw = c->Bw; p.w = c->w;
+    p.n0 = c->n; p.c = count; p.t0 = (int)c->t;
+    p.SS = s_stride(c->B);
+    p.scale_log2e = (float)((double)c->scale * 1.4426950408889634);
+    cudaError_t e = cudaErrorInvalidValue;
+    if (count < 1 || count > sh_prefill_chunk_capacity(c)) return e;
+    if (count <= 32) e = c->dtype == SH_F16 ? launch_chunk<SH_F16, 32>(p, s) : launch_chunk<SH_BF16, 32>(p, s);
+    else e = c->dtype == SH_F16 ? launch_chunk<SH_F16, 64>(p, s) : launch_chunk<SH_BF16, 64>(p, s);
+    if (e == cudaSuccess) *launches += 1;
+    return e;
+}

@@ -82,3 +82,66 @@ def run_lockstep(handle, cfg_dtype: str, inputs, steps: int, units, tol: float, 
             res.compressions += 1
         res.steps += 1
     return res, orc
+
+
+def run_lockstep_chunked(handle, cfg_dtype: str, inputs_block, steps: int, units, tol: float, chunk_sizes=None,
+                         res: LockstepResult = None, orc=None):
+    """Same protocol as run_lockstep, driving the library through sh_prefill_chunk.
+
+    ``inputs_block(t0, t1)`` -> (q, k, v) CUDA tensors [t1-t0, U, d] for stream positions t0 .. t1-1
+    (1-based).  The library evaluates a whole chunk in one launch; the oracle then replays the chunk
+    step by step, and each step's record bits are read back from the unit's bit-planes (no
+    compression happens inside a chunk, so nothing has moved them).  ``chunk_sizes`` cycles through
+    requested chunk lengths (clipped to what the library and the remaining budget allow)."""
+    units = torch.as_tensor(units, dtype=torch.long)
+    un = units.numpy()
+    if orc is None:
+        orc = oracle_mod.Oracle(len(un), handle.B, handle.r, handle.w, handle.m, handle.D,
+                                quant=(cfg_dtype == "int4"))
+    res = res or LockstepResult()
+    dev_units = units.to(handle.device)
+    cap = handle.prefill_chunk_max
+    assert cap >= 2, "the chunk kernel does not serve this handle"
+    sizes = list(chunk_sizes or [cap])
+    done, k_i = 0, 0
+    while done < steps:
+        cnt = min(sizes[k_i % len(sizes)], cap, steps - done, handle.B - orc.n)
+        k_i += 1
+        t0 = orc.t + 1
+        q, k, v = inputs_block(t0, t0 + cnt)
+        out = torch.empty(cnt, handle.U, handle.D, device=handle.device)
+        handle.prefill_chunk(q, k, v, out)
+        n, tt, pos, cnt_rec, _ = handle.state(low=False)
+        planes = [handle.export_record(int(u)) for u in un]      # [w, B] bool per sampled unit
+        for i in range(cnt):
+            t = t0 + i
+            o_out, alpha, o_low, amb = orc.attend(to_oracle(q[i], dev_units), to_oracle(k[i], dev_units),
+                                                  to_oracle(v[i], dev_units))
+            err = float(np.abs(out[i][dev_units].double().cpu().numpy() - o_out).max())
+            res.max_abs_err = max(res.max_abs_err, err)
+            assert err <= tol, f"step {t}: attention output off by {err:.3e} > {tol}"
+            nn = orc.n
+            g_low = np.stack([pl[t % handle.w, :nn] for pl in planes])
+            beyond = np.stack([pl[t % handle.w, nn:] for pl in planes])
+            assert not beyond.any(), f"step {t}: record bits set beyond the slots live at that step"
+            diff = g_low != o_low
+            bad = diff & ~amb
+            assert not bad.any(), (f"step {t}: {int(bad.sum())} record bits differ outside the 1e-6 window; "
+                                   f"first at (unit, slot) {np.argwhere(bad)[0].tolist()}")
+            res.adoptions += int(diff.sum())
+            res.slot_steps += g_low.size
+            orc.record(g_low)
+            res.steps += 1
+        assert n == orc.n and tt == orc.t
+        assert (pos[un] == orc.positions()).all(), f"after step {orc.t}: positions differ"
+        assert (cnt_rec[un].astype(np.int32) == orc.counters()).all(), f"after step {orc.t}: records differ"
+        if orc.full:
+            orc.compress()
+            assert handle.compress() == handle.m
+            n2, _, pos2, cnt2, _ = handle.state(low=False)
+            assert n2 == orc.n
+            assert (pos2[un] == orc.positions()).all(), f"after step {orc.t}: kept sets differ"
+            assert (cnt2[un].astype(np.int32) == orc.counters()).all()
+            res.compressions += 1
+        done += cnt
+    return res, orc

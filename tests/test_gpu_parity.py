@@ -6,7 +6,7 @@ import pytest
 import torch
 
 import oracle
-from lockstep import run_lockstep, to_oracle
+from lockstep import run_lockstep, run_lockstep_chunked, to_oracle
 from paper_2305_17118_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -59,6 +59,49 @@ def test_lockstep_pipelined_kernel(sh, dtype, U, B, r, w, m):
     res, _ = run_lockstep(h, dtype, _stream_fn(q, k, v), T, torch.arange(U), TOL[dtype])
     assert res.compressions >= 3
     assert res.adoptions <= 1e-4 * res.slot_steps + 2
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("U,B,r,w,m,sizes", [(5, 150, 9, 37, 41, [64, 7, 33, 1, 50]), (3, 410, 64, 128, 64, [64]),
+                                             (2, 700, 5, 64, 300, [32, 17]), (4, 40, 3, 9, 20, [5, 9, 2]),
+                                             (130, 96, 8, 70, 30, [64, 31])])
+def test_lockstep_chunked_prompt_kernel(sh, dtype, U, B, r, w, m, sizes):
+    """sh_prefill_chunk against the oracle replaying the same steps one by one: outputs of
+    every step, its record bits, positions, counters and kept sets."""
+    d, T = 128, 2 * B + 2 * m + 11
+    q, k, v = wl.random_stream(U, d, T, seed=17 + U, dtype=dtype, peaked=3.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
+    res, orc = run_lockstep_chunked(h, dtype, blk, T, torch.arange(U), TOL[dtype], chunk_sizes=sizes)
+    assert res.steps == T and res.compressions >= 3
+    assert res.adoptions <= 1e-4 * res.slot_steps + 2
+    # and the decode step carries on from the state the chunks left
+    q2, k2, v2 = wl.random_stream(U, d, 40, seed=99, dtype=dtype, peaked=3.0, device="cuda")
+    run_lockstep(h, dtype, lambda t: (q2[t - T - 1], k2[t - T - 1], v2[t - T - 1]), 40, torch.arange(U), TOL[dtype], orc=orc)
+
+
+def test_prefill_uses_chunks_and_matches_oracle(sh):
+    """sh_prefill with its automatic chunking on the OPT-6.7B-shaped stream, then decode steps in lockstep."""
+    cfg = wl.CONFIGS["opt6b"].scaled(units=24, prompt=700)
+    st = wl.Stream(cfg, device="cuda")
+    h = sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, cfg.units, cfg.head_dim, cfg.dtype, auto_compress=False)
+    orc = oracle.Oracle(cfg.units, cfg.B, cfg.r, cfg.w, cfg.m, cfg.head_dim)
+    q, k, v = st.block(1, cfg.prompt + 1)
+    out = torch.empty(cfg.prompt, cfg.units, cfg.head_dim, device="cuda")
+    before = h.launch_count
+    h.prefill(q, k, v, out)
+    assert h.launch_count - before < cfg.prompt // 8        # chunks, not one launch per token
+    idx = torch.arange(cfg.units, device="cuda")
+    worst = 0.0
+    for t in range(cfg.prompt):
+        o, _ = orc.step(to_oracle(q[t], idx), to_oracle(k[t], idx), to_oracle(v[t], idx))
+        worst = max(worst, float(np.abs(out[t].double().cpu().numpy() - o).max()))
+    assert worst <= TOL[cfg.dtype]
+    n, t, pos, cnt, _ = h.state(low=False)
+    assert n == orc.n and t == orc.t
+    same = (pos == orc.positions()).all(axis=1)
+    assert same.mean() >= 0.9      # units without a threshold-ambiguous flip must agree exactly
+    assert (cnt[same].astype(np.int32) == orc.counters()[same]).all()
 
 
 # ---- the benchmark's own configurations ----------------------------------------------------
@@ -160,7 +203,7 @@ def test_compaction_moves_rows_bit_identically(sh, dtype):
 def test_prefill_equals_token_by_token_steps(sh):
     U, d, B, r, w, m, T, dtype = 6, 128, 80, 8, 24, 30, 260, "f16"
     q, k, v = wl.random_stream(U, d, T, seed=5, dtype=dtype, peaked=3.0, device="cuda")
-    a = sh.Handle(B, r, w, m, U, d, dtype)
+    a = sh.Handle(B, r, w, m, U, d, dtype, prefill_chunk=False)    # one decode step per prompt token
     b = sh.Handle(B, r, w, m, U, d, dtype)
     out_a = torch.empty(T, U, d, device="cuda")
     a.prefill(q, k, v, out_a)
