@@ -83,22 +83,24 @@ struct ChunkParams {
     float scale_log2e;
 };
 
-// Fill the 64-row tile buffer with rows [j0, j0+64) of the unit's K or V as seen by
-// the chunk: cached rows, then the chunk's own tokens (which are also appended to the
-// cache here), zeros beyond.
-__device__ __forceinline__ void load_tile(uint16_t *tile, const char *cache_u, const char *chunk, char *append_u,
-                                          int j0, int n0, int n_tot, size_t chunk_stride) {
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Start filling a 64-row tile buffer with rows [j0, j0+64) of the unit's K or V as seen by
+// the chunk: cached rows, then the chunk's own tokens, zeros beyond.  Asynchronous: the
+// caller commits the group and waits for it before reading the tile.
+__device__ __forceinline__ void load_tile_async(uint16_t *tile, const char *cache_u, const char *chunk, int j0, int n0,
+                                                int n_tot, size_t chunk_stride) {
     for (int idx = threadIdx.x; idx < KT * (D / 8); idx += NTHREADS) {
         const int row = idx / (D / 8), ch = idx % (D / 8);
         const int j = j0 + row;
-        uint4 val = make_uint4(0, 0, 0, 0);
-        if (j < n0) {
-            val = *reinterpret_cast<const uint4 *>(cache_u + (size_t)j * (D * 2) + ch * 16);
-        } else if (j < n_tot) {
-            val = *reinterpret_cast<const uint4 *>(chunk + (size_t)(j - n0) * chunk_stride + ch * 16);
-            *reinterpret_cast<uint4 *>(append_u + (size_t)j * (D * 2) + ch * 16) = val;
-        }
-        *reinterpret_cast<uint4 *>(tile + row * ROWH + ch * 8) = val;
+        uint16_t *dst = tile + row * ROWH + ch * 8;
+        if (j < n0) cp_async16(dst, cache_u + (size_t)j * (D * 2) + ch * 16);
+        else if (j < n_tot) cp_async16(dst, chunk + (size_t)(j - n0) * chunk_stride + ch * 16);
+        else *reinterpret_cast<uint4 *>(dst) = make_uint4(0, 0, 0, 0);
     }
 }
 
@@ -114,8 +116,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
 
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint16_t *Qs = reinterpret_cast<uint16_t *>(smem_raw);              // [CQ][ROWH]
-    uint16_t *tile = Qs + CQ * ROWH;                                    // [KT][ROWH]
-    float *S = reinterpret_cast<float *>(tile + KT * ROWH);             // [CQ][SS]
+    uint16_t *tile0 = Qs + CQ * ROWH;                                   // [2][KT][ROWH] double-buffered K/V tiles
+    float *S = reinterpret_cast<float *>(tile0 + 2 * KT * ROWH);        // [CQ][SS]
     float *rowL = S + (size_t)CQ * p.SS;                                // [CQ] row sums
 
     const int u = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -134,6 +136,17 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
         *reinterpret_cast<uint4 *>(Qs + row * ROWH + ch * 8) = val;
     }
     if (tid < c) p.pos[(size_t)u * p.B + n0 + tid] = p.t0 + tid + 1;
+    // append the chunk's keys and values to the cache (nothing in this launch reads them back from there)
+    for (int idx = tid; idx < c * (D / 8); idx += NTHREADS) {
+        const int row = idx / (D / 8), ch = idx % (D / 8);
+        const size_t src = (size_t)row * tstride + (size_t)u * D * 2 + ch * 16;
+        const size_t dst = ((size_t)u * p.B + n0 + row) * (D * 2) + ch * 16;
+        *reinterpret_cast<uint4 *>(p.K + dst) = *reinterpret_cast<const uint4 *>(p.k + src);
+        *reinterpret_cast<uint4 *>(p.V + dst) = *reinterpret_cast<const uint4 *>(p.v + src);
+    }
+    const char *kchunk = p.k + (size_t)u * D * 2, *vchunk = p.v + (size_t)u * D * 2;
+    load_tile_async(tile0, Kc, kchunk, 0, n0, n_tot, tstride);      // first K tile is on its way
+    cp_async_commit();
     __syncthreads();
 
     // A fragments of this warp's 16 queries, all 8 k-steps, kept in registers
@@ -146,8 +159,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
 
     // ---- phase 1: S = scale * Q.K^T, causal inside the chunk
     for (int kt = 0; kt < ntiles; ++kt) {
-        __syncthreads();      // previous tile consumed
-        load_tile(tile, Kc, p.k + (size_t)u * D * 2, p.K + (size_t)u * p.B * D * 2, kt * KT, n0, n_tot, tstride);
+        uint16_t *tile = tile0 + (kt & 1) * KT * ROWH;
+        // prefetch the next K tile (or the first V tile) into the other buffer, then wait for this one
+        if (kt + 1 < ntiles) load_tile_async(tile0 + ((kt + 1) & 1) * KT * ROWH, Kc, kchunk, (kt + 1) * KT, n0, n_tot, tstride);
+        else load_tile_async(tile0 + ((kt + 1) & 1) * KT * ROWH, Vc, vchunk, 0, n0, n_tot, tstride);
+        cp_async_commit();
+        cp_async_wait<1>();
         __syncthreads();
         float acc[NBK][4];
 #pragma unroll
@@ -175,8 +192,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
                 S[(size_t)i * SS + j] = live ? acc[nb][e] * p.scale_log2e : -INFINITY;
             }
         }
+        __syncthreads();      // tile consumed: its buffer may be refilled by the next iteration's prefetch
     }
-    __syncthreads();
 
     // ---- softmax rows and record bits: one warp per query row
     for (int i = warp; i < CQ; i += NTHREADS / 32) {
@@ -217,9 +234,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
 #pragma unroll
         for (int e = 0; e < 4; ++e) oacc[nb][e] = 0.f;
     for (int kt = 0; kt < ntiles; ++kt) {
-        __syncthreads();      // S complete (first pass) / previous tile consumed
-        load_tile(tile, Vc, p.v + (size_t)u * D * 2, p.V + (size_t)u * p.B * D * 2, kt * KT, n0, n_tot, tstride);
-        __syncthreads();
+        // V tile kt sits in buffer (ntiles + kt) & 1: the first one was prefetched behind the last K tile
+        uint16_t *tile = tile0 + ((ntiles + kt) & 1) * KT * ROWH;
+        if (kt + 1 < ntiles) load_tile_async(tile0 + ((ntiles + kt + 1) & 1) * KT * ROWH, Vc, vchunk, (kt + 1) * KT, n0, n_tot, tstride);
+        cp_async_commit();
+        cp_async_wait<1>();
+        __syncthreads();      // tile landed for everyone; on the first pass also: P complete
 #pragma unroll
         for (int ks = 0; ks < KT / 16; ++ks) {
             // A fragments of P: rows r0 = wm*16 + lane/4 and r0 + 8, key columns j0 + {0,1} and j0 + 8 + {0,1}
@@ -245,7 +265,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
                 M::run(oacc[2 * nbp + 1], alo, b[2], b[3]);
             }
         }
+        __syncthreads();      // tile consumed before the next prefetch overwrites the other buffer's partner
     }
+    cp_async_wait<0>();
     if (p.out) {
 #pragma unroll
         for (int nb = 0; nb < NBD; ++nb) {
@@ -265,7 +287,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
 
 template <int DT, int CQ>
 cudaError_t launch_chunk(const ChunkParams &p, cudaStream_t s) {
-    const size_t smem = sizeof(uint16_t) * (size_t)(CQ + KT) * ROWH + sizeof(float) * ((size_t)CQ * p.SS + CQ);
+    const size_t smem = sizeof(uint16_t) * (size_t)(CQ + 2 * KT) * ROWH + sizeof(float) * ((size_t)CQ * p.SS + CQ);
     auto kern = sh_prefill_chunk_kernel<DT, CQ>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -275,7 +297,7 @@ cudaError_t launch_chunk(const ChunkParams &p, cudaStream_t s) {
 
 int s_stride(int B) { return ((B + KT - 1) / KT) * KT + 8; }
 size_t smem_need(int CQ, int B) {
-    return sizeof(uint16_t) * (size_t)(CQ + KT) * ROWH + sizeof(float) * ((size_t)CQ * s_stride(B) + CQ);
+    return sizeof(uint16_t) * (size_t)(CQ + 2 * KT) * ROWH + sizeof(float) * ((size_t)CQ * s_stride(B) + CQ);
 }
 
 }  // namespace
