@@ -196,7 +196,8 @@ def cuda_arm(args, cfg, rank, world):
     streams = [wl.Stream(cfg, device=dev, layer=l + 1000 * rank) for l in range(Ly)]
     handles = [sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, U, d, cfg.dtype, device=dev, auto_compress=False,
                          split=args.split, kernel=args.kernel,
-                         prefill_chunk=False if args.no_prefill_chunk else None)
+                         prefill_chunk=False if args.no_prefill_chunk else None,
+                         recompute_record=args.recompute_record)
                for _ in range(Ly)]
 
     # ---- prompt: streamed through the same path, untimed
@@ -332,7 +333,8 @@ def cuda_arm(args, cfg, rank, world):
         "data": "synthetic",
         "config": {"workload": cfg.name, "batch": cfg.batch, "heads": cfg.heads, "layers": Ly, "units": U * Ly,
                    "head_dim": d, "kv_dtype": cfg.dtype, "B": cfg.B, "r": cfg.r, "w": cfg.w, "m": cfg.m,
-                   "prompt": cfg.prompt, "l2": "flushed between steps" if flush else "inputs larger than L2",
+                   "prompt": cfg.prompt, "record": "recomputed at compression" if args.recompute_record else "online",
+                   "l2": "flushed between steps" if flush else "inputs larger than L2",
                    "kv_bytes": kv_bytes, "parallelism": f"units replicated x{world}" if world > 1 else "1 GPU"},
         "attn_GBps": statistics.fmean(n_sched) * U * Ly * d * ES[cfg.dtype] * 2 / (ms_per_step * 1e-3) / 1e9,
         "prompt": {"tokens": cfg.prompt, "ms": prompt_ms, "tokens_per_s": cfg.prompt * 1e3 / prompt_ms if prompt_ms else None,
@@ -356,6 +358,8 @@ def main():
     ap.add_argument("--oracle-units", type=int, default=2048)
     ap.add_argument("--split", type=int, default=None, help="CTAs per unit (default: chosen by the library)")
     ap.add_argument("--kernel", type=int, default=None, help="decode kernel: 1 direct loads, 2 pipelined bulk copies")
+    ap.add_argument("--recompute-record", action="store_true",
+                    help="variant: rebuild the importance record at each compression from stored queries")
     ap.add_argument("--no-prefill-chunk", action="store_true", help="stream the prompt one decode step per token")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (tuning runs)")
     args = ap.parse_args()

@@ -62,6 +62,12 @@ typedef enum {
     SH_OPT_SPLIT = 1,         /* CTAs cooperating on one unit (1, 2, 4 or 8); default chosen from `heads` */
     SH_OPT_AUTO_COMPRESS = 2, /* 1 (default): sh_decode_step compresses by itself when the cache fills;
                                  0: the caller calls sh_compress */
+    SH_OPT_RECORD_MODE = 5,   /* 0 (default): the importance record is kept online, one comparison per cached
+                                 token per step; 1: it is recomputed at every compression from the queries of
+                                 the last w steps (the library keeps them: heads*w*head_dim extra elements)
+                                 scored against the cache as it is then (Algorithm 2 as stated; Section 4.1,
+                                 "Overhead Tradeoff").  fp16/bf16, head_dim 128 only.  Set before sh_bind:
+                                 it changes sh_workspace_bytes. */
     SH_OPT_PREFILL_CHUNK = 4, /* 1 (default): sh_prefill hands the tokens between two compressions to the chunk
                                  kernel where the shape allows it; 0: one decode step per token */
     SH_OPT_DECODE_KERNEL = 3  /* 0 (default): chosen from the shape; 1: one CTA (or cluster) per unit with
@@ -208,6 +214,15 @@ int sh_select(const uint16_t *counters_dev, int units, int n, int r, int m, int3
  */
 int sh_state(sh_handle h, void *stream, int *n_out, long long *t_out, int32_t *pos_host,
              uint16_t *counters_host, uint32_t *low_host);
+
+/*
+ * SH_OPT_RECORD_MODE = 1 only: recompute the record now (what sh_compress does first in that
+ * mode): each query of the last w steps (t-w, t] is scored against the cached tokens that
+ * already existed at its step, softmax over those, and alpha_j < 1/step becomes that step's
+ * bit-plane row.  A following sh_compress at the same step uses the result as it stands.
+ * Errors: SH_ESTATE when the handle keeps its record online.
+ */
+int sh_recompute_record(sh_handle h, void *stream);
 
 /* The record bit-planes of one unit, [w][ceil(B/32)] uint32 on the host: row (s mod w) holds, for
  * step s of the last w steps, bit j%32 of word j/32 = [alpha_j < 1/s] for the token now in slot j.

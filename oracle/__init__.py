@@ -68,6 +68,10 @@ def _load():
     lib.sho_select.argtypes = [ip, c.c_int, c.c_int, c.c_int, ip]
     lib.sho_select.restype = None
     lib.sho_compress.argtypes = [c.c_void_p, ip]
+    lib.sho_recount.argtypes = [c.c_void_p, dp, bp, bp, ip]
+    lib.sho_recount.restype = None
+    lib.sho_set_record.argtypes = [c.c_void_p, bp, ip]
+    lib.sho_set_record.restype = None
     lib.sho_quantize.argtypes = [dp, c.c_int, c.c_int, dp, c.POINTER(c.c_int8), c.POINTER(c.c_float)]
     lib.sho_quantize.restype = None
     _lib = lib
@@ -187,6 +191,42 @@ class Oracle:
         ev = np.zeros((self.U, self.m), dtype=np.int32)
         got = self._lib.sho_compress(self._h, _ip(ev))
         return ev if got else None
+
+    # -- the record recomputed at compression time (Algorithm 2 as stated) ----
+    def recount(self):
+        """Scores of the last w queries against the present cache (causal by
+        position), as ``(alpha, low, amb)`` each [U, w, n] with row = step mod w,
+        and ``steps`` [w] (0 where the window holds no query)."""
+        U, w, B = self.U, self.w, self.B
+        alpha = np.zeros((U, w, B))
+        low = np.zeros((U, w, B), dtype=np.uint8)
+        amb = np.zeros((U, w, B), dtype=np.uint8)
+        steps = np.zeros(w, dtype=np.int32)
+        self._lib.sho_recount(self._h, _dp(alpha), _bp(low), _bp(amb), _ip(steps))
+        n = self.n
+        return alpha[:, :, :n].copy(), low[:, :, :n].astype(bool), amb[:, :, :n].astype(bool), steps
+
+    def set_record(self, low, steps) -> None:
+        """Make ``low`` ([U, w, n] bool, rows as in ``recount``) the importance
+        record of the live tokens."""
+        low = np.asarray(low)
+        if low.shape != (self.U, self.w, self.n):
+            raise ValueError(f"low must be [{self.U}, {self.w}, {self.n}]")
+        buf = np.zeros((self.U, self.w, self.B), dtype=np.uint8)
+        buf[:, :, : self.n] = low
+        steps = np.ascontiguousarray(np.asarray(steps, dtype=np.int32))
+        self._lib.sho_set_record(self._h, _bp(buf), _ip(steps))
+
+    def step_recompute(self, q, k, v):
+        """One step of the recompute-at-compression variant: attend; when the
+        cache is full, recount, adopt the recount as the record, compress."""
+        out, _alpha, _low, _amb = self.attend(q, k, v)
+        dropped = None
+        if self.full:
+            _a, low, _amb2, steps = self.recount()
+            self.set_record(low, steps)
+            dropped = self.compress()
+        return out, dropped
 
     def step(self, q, k, v):
         """attend + record + compress.  Returns ``(out, dropped or None)``."""

@@ -65,6 +65,8 @@ typedef struct {
     int *h_cnt;       /* [B] how many (step, low) pairs the token has received */
     int *h_step;      /* [B][w] the last w pairs: step numbers */
     uint8_t *h_low;   /* [B][w] the last w pairs: low flags */
+    double *Q;        /* [w][d] queries of the last w steps (slot = step mod w) */
+    int *q_step;      /* [w] step of each stored query, 0 = none */
 } unit_t;
 
 typedef struct {
@@ -89,7 +91,7 @@ void sho_destroy(sho_t *o) {
     if (o->unit) {
         for (int u = 0; u < o->U; ++u) {
             unit_t *x = &o->unit[u];
-            free(x->K); free(x->V); free(x->pos); free(x->h_cnt); free(x->h_step); free(x->h_low);
+            free(x->K); free(x->V); free(x->pos); free(x->h_cnt); free(x->h_step); free(x->h_low); free(x->Q); free(x->q_step);
         }
         free(o->unit);
     }
@@ -114,7 +116,9 @@ sho_t *sho_create(int U, int B, int r, int w, int m, int d, double scale, int qu
         x->h_cnt = calloc((size_t)B, sizeof(int));
         x->h_step = calloc((size_t)B * w, sizeof(int));
         x->h_low = calloc((size_t)B * w, 1);
-        if (!x->K || !x->V || !x->pos || !x->h_cnt || !x->h_step || !x->h_low) { sho_destroy(o); return NULL; }
+        x->Q = calloc((size_t)w * d, sizeof(double));
+        x->q_step = calloc((size_t)w, sizeof(int));
+        if (!x->K || !x->V || !x->pos || !x->h_cnt || !x->h_step || !x->h_low || !x->Q || !x->q_step) { sho_destroy(o); return NULL; }
     }
     return o;
 }
@@ -188,6 +192,8 @@ int sho_attend(sho_t *o, const double *q, const double *k, const double *v,
         /* 2. scores and output */
         double *a = alpha + (size_t)u * B;
         const double *qu = q + (size_t)u * d;
+        memcpy(x->Q + (size_t)(t % o->w) * d, qu, sizeof(double) * d);   /* kept for the recompute variant */
+        x->q_step[t % o->w] = (int)t;
         double smax = -INFINITY;
         for (j = 0; j < n; ++j) {
             double s = 0.0;
@@ -323,6 +329,75 @@ int sho_compress(sho_t *o, int *evicted_pos) {
         free(I); free(ev); free(drop);
     }
     return m;
+}
+
+/*
+ * The record as Algorithm 2 states it, computed at compression time ("an extra
+ * attention computation ... to collect the importance measurements over a
+ * history window", Section 4.1, Overhead Tradeoff) instead of being kept
+ * online: every query of the last w steps (t-w, t] is scored again against the
+ * cache as it is now, restricted to the tokens that already existed at that
+ * query's step (pos <= step: attention is causal), and compared with 1/step.
+ * Tokens evicted since then are gone, so the scores are normalised over the
+ * survivors.  alpha, low, amb: [U][w][B], row (step mod w); steps: [w] (0 = no query).
+ */
+void sho_recount(const sho_t *o, double *alpha, uint8_t *low, uint8_t *amb, int *steps) {
+    const int B = o->B, d = o->d, w = o->w;
+    for (int s = 0; s < w; ++s) {
+        int st = o->unit[0].q_step[s];
+        steps[s] = (st > 0 && (long)st > o->t - w && (long)st <= o->t) ? st : 0;
+    }
+#pragma omp parallel for schedule(static)
+    for (int u = 0; u < o->U; ++u) {
+        const unit_t *x = &o->unit[u];
+        for (int s = 0; s < w; ++s) {
+            double *a = alpha + ((size_t)u * w + s) * B;
+            uint8_t *lo = low + ((size_t)u * w + s) * B, *am = amb + ((size_t)u * w + s) * B;
+            for (int j = 0; j < B; ++j) { a[j] = 0.0; lo[j] = 0; am[j] = 0; }
+            const int st = steps[s];
+            if (!st) continue;
+            const double *qu = x->Q + (size_t)s * d;
+            int nv = 0;                                   /* tokens that existed at step st (positions ascend) */
+            while (nv < x->n && x->pos[nv] <= st) ++nv;
+            if (!nv) continue;
+            double smax = -INFINITY, L = 0.0;
+            for (int j = 0; j < nv; ++j) {
+                double sc = 0.0;
+                for (int i = 0; i < d; ++i) sc += qu[i] * x->K[(size_t)j * d + i];
+                a[j] = sc * o->scale;
+                if (a[j] > smax) smax = a[j];
+            }
+            for (int j = 0; j < nv; ++j) { a[j] = exp(a[j] - smax); L += a[j]; }
+            const double thr = 1.0 / (double)st;
+            for (int j = 0; j < nv; ++j) {
+                a[j] /= L;
+                lo[j] = a[j] < thr;
+                am[j] = fabs(a[j] - thr) <= sho_amb_window();
+            }
+        }
+    }
+}
+
+/* Replace every live token's history by the given recomputed flags
+ * ([U][w][B], row = step mod w, steps as returned by sho_recount). */
+void sho_set_record(sho_t *o, const uint8_t *low, const int *steps) {
+    const int B = o->B, w = o->w;
+#pragma omp parallel for schedule(static)
+    for (int u = 0; u < o->U; ++u) {
+        unit_t *x = &o->unit[u];
+        for (int j = 0; j < x->n; ++j) {
+            x->h_cnt[j] = 0;
+            for (long st = o->t - w + 1; st <= o->t; ++st) {     /* ascending steps */
+                if (st < 1) continue;
+                const int s = (int)(st % w);
+                if (steps[s] != (int)st || x->pos[j] > st) continue;
+                const int slot = x->h_cnt[j] % w;
+                x->h_step[(size_t)j * w + slot] = (int)st;
+                x->h_low[(size_t)j * w + slot] = low[((size_t)u * w + s) * B + j] ? 1 : 0;
+                x->h_cnt[j] += 1;
+            }
+        }
+    }
 }
 
 /* One whole step for callers that do not intervene: 1-4 above. */

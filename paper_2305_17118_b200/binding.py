@@ -19,14 +19,14 @@ from . import build as _build
 SH_OK, SH_EINVAL, SH_EFULL, SH_ESTATE, SH_ECUDA, SH_ENOMEM, SH_ETOOBIG, SH_EDEVICE = 0, -1, -2, -3, -4, -5, -6, -7
 SH_STATIC_SCRATCH_MAX_ENTRIES = 1 << 20
 SH_F32, SH_F16, SH_BF16, SH_INT4_G64_F16 = 0, 1, 2, 3
-SH_OPT_SOFTMAX_SCALE, SH_OPT_SPLIT, SH_OPT_AUTO_COMPRESS, SH_OPT_DECODE_KERNEL, SH_OPT_PREFILL_CHUNK = 0, 1, 2, 3, 4
+SH_OPT_SOFTMAX_SCALE, SH_OPT_SPLIT, SH_OPT_AUTO_COMPRESS, SH_OPT_DECODE_KERNEL, SH_OPT_PREFILL_CHUNK, SH_OPT_RECORD_MODE = 0, 1, 2, 3, 4, 5
 
 DTYPE_CODE = {"f32": SH_F32, "f16": SH_F16, "bf16": SH_BF16, "int4": SH_INT4_G64_F16}
 INPUT_TORCH_DTYPE = {SH_F32: torch.float32, SH_F16: torch.float16, SH_BF16: torch.bfloat16,
                      SH_INT4_G64_F16: torch.float16}
 
 EXPORTS = ["sh_create", "sh_destroy", "sh_workspace_bytes", "sh_bind", "sh_set_option", "sh_decode_step",
-           "sh_decode_step_host", "sh_prefill", "sh_prefill_chunk", "sh_prefill_chunk_max", "sh_export_record",
+           "sh_decode_step_host", "sh_prefill", "sh_prefill_chunk", "sh_prefill_chunk_max", "sh_export_record", "sh_recompute_record",
            "sh_compress", "sh_compress_static", "sh_select", "sh_state", "sh_export_unit",
            "sh_restore", "sh_launch_count", "sh_strerror", "sh_last_cuda_error"]
 
@@ -59,6 +59,7 @@ def _load() -> C.CDLL:
     lib.sh_prefill_chunk.argtypes = [vp, vp, vp, vp, C.c_int, vp, vp]
     lib.sh_prefill_chunk_max.argtypes = [vp]
     lib.sh_export_record.argtypes = [vp, C.c_int, vp, vp]
+    lib.sh_recompute_record.argtypes = [vp, vp]
     lib.sh_compress.argtypes = [vp, vp, ip]
     lib.sh_compress_static.argtypes = [vp, vp, ip]
     lib.sh_select.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
@@ -104,7 +105,7 @@ class Handle:
 
     def __init__(self, B: int, r: int, w: int, m: int, heads: int, head_dim: int, dtype, device="cuda:0",
                  split: Optional[int] = None, scale: Optional[float] = None, auto_compress: bool = True,
-                 kernel: Optional[int] = None, prefill_chunk: Optional[bool] = None):
+                 kernel: Optional[int] = None, prefill_chunk: Optional[bool] = None, recompute_record: bool = False):
         self.dtype = DTYPE_CODE[dtype] if isinstance(dtype, str) else int(dtype)
         self.B, self.r, self.w, self.m, self.U, self.D = B, r, w, m, heads, head_dim
         self.Bw = (B + 31) // 32
@@ -121,6 +122,8 @@ class Handle:
             self.set_option(SH_OPT_SPLIT, split)
         if kernel is not None:
             self.set_option(SH_OPT_DECODE_KERNEL, kernel)
+        if recompute_record:
+            self.set_option(SH_OPT_RECORD_MODE, 1.0)
         if prefill_chunk is not None:
             self.set_option(SH_OPT_PREFILL_CHUNK, 1.0 if prefill_chunk else 0.0)
         self.set_option(SH_OPT_AUTO_COMPRESS, 1.0 if auto_compress else 0.0)
@@ -191,6 +194,10 @@ class Handle:
         self._check(lib.sh_prefill_chunk(self._h, _dev(q, self.in_dtype, n, "q"), _dev(k, self.in_dtype, n, "k"),
                                          _dev(v, self.in_dtype, n, "v"), c, optr, _stream_ptr(stream)))
         return out
+
+    # -- sh_recompute_record --------------------------------------------------------
+    def recompute_record(self, stream=None):
+        self._check(lib.sh_recompute_record(self._h, _stream_ptr(stream)))
 
     # -- sh_export_record -----------------------------------------------------------
     def export_record(self, unit: int, stream=None) -> np.ndarray:

@@ -42,6 +42,7 @@ void make_layout(sh_context *c) {
     L.stage_v = take(U * (size_t)c->in_bytes);
     L.stage_out = take(U * D * 4);
     L.err = take(256);
+    L.qring = take(c->record_mode ? U * (size_t)c->w * c->in_bytes : 0);
     L.total = off;
 }
 
@@ -81,6 +82,8 @@ __global__ void sh_export_kernel(const char *K, const char *V, const __half *Ks,
 }
 
 int do_compress(sh_context *c, cudaStream_t s) {
+    int rrc = sh_recount_if_needed(c, s);
+    if (rrc != SH_OK) return rrc;
     SelectParams sp = {};
     sp.hist = reinterpret_cast<const uint32_t *>(c->slab + c->L.hist);
     sp.counters = nullptr;
@@ -106,6 +109,18 @@ int do_compress(sh_context *c, cudaStream_t s) {
     return SH_OK;
 }
 
+}  // namespace
+
+int sh_recount_if_needed(sh_context *c, cudaStream_t s) {
+    if (!c->record_mode || c->record_fresh_t == c->t) return SH_OK;
+    cudaError_t e = sh_launch_recount(c, s, &c->launches);
+    if (e != cudaSuccess) { c->last_err = e; return SH_ECUDA; }
+    c->record_fresh_t = c->t;
+    return SH_OK;
+}
+
+namespace {
+
 int do_step(sh_context *c, const void *q, const void *k, const void *v, float *out, cudaStream_t s,
             bool compress_after) {
     DecodeParams p = {};
@@ -114,6 +129,7 @@ int do_step(sh_context *c, const void *q, const void *k, const void *v, float *o
     p.Ks = c->slab + c->L.Ks; p.Vs = c->slab + c->L.Vs;
     p.hist = reinterpret_cast<uint32_t *>(c->slab + c->L.hist);
     p.pos = reinterpret_cast<int32_t *>(c->slab + c->L.pos);
+    p.qring = c->record_mode ? c->slab + c->L.qring : nullptr;
     p.U = c->U; p.B = c->B; p.Bw = c->Bw; p.w = c->w;
     p.n = c->n + 1;
     p.t = (int)(c->t + 1);
@@ -153,6 +169,8 @@ int sh_create(int B, int r, int w, int m, int heads, int head_dim, int dtype, sh
     c->auto_compress = 1;
     c->kernel = 0;
     c->prefill_chunk = 1;
+    c->record_mode = 0;
+    c->record_fresh_t = -1;
     c->started = false;
     c->slab = nullptr; c->slab_bytes = 0;
     c->launches = 0;
@@ -197,6 +215,15 @@ int sh_set_option(sh_handle h, int key, double value) {
         case SH_OPT_AUTO_COMPRESS:
             h->auto_compress = value != 0.0;
             return SH_OK;
+        case SH_OPT_RECORD_MODE: {
+            const int mode = (int)value;
+            if (mode != 0 && mode != 1) return SH_EINVAL;
+            if (h->slab) return SH_ESTATE;                       // changes the workspace layout
+            if (mode == 1 && sh_prefill_chunk_capacity(h) == 0) return SH_EINVAL;   // needs the tensor-core kernel's shapes
+            h->record_mode = mode;
+            make_layout(h);
+            return SH_OK;
+        }
         case SH_OPT_PREFILL_CHUNK:
             h->prefill_chunk = value != 0.0;
             return SH_OK;
@@ -332,6 +359,13 @@ int sh_prefill(sh_handle h, const void *q_dev, const void *k_dev, const void *v_
     return SH_OK;
 }
 
+int sh_recompute_record(sh_handle h, void *stream) {
+    if (!h) return SH_EINVAL;
+    if (!h->slab || !h->record_mode) return SH_ESTATE;
+    h->record_fresh_t = -1;
+    return sh_recount_if_needed(h, (cudaStream_t)stream);
+}
+
 int sh_export_record(sh_handle h, int unit, uint32_t *planes_host, void *stream) {
     if (!h || unit < 0 || unit >= h->U || !planes_host) return SH_EINVAL;
     if (!h->slab) return SH_ESTATE;
@@ -431,6 +465,7 @@ int sh_restore(sh_handle h, int n, long long t) {
     h->n = n;
     h->t = t;
     h->started = true;
+    h->record_fresh_t = -1;
     return SH_OK;
 }
 

@@ -335,6 +335,9 @@ __global__ void __launch_bounds__(NW * 32) sh_decode_kernel(const DecodeParams p
     // ---- q chunk of this lane, fp32
     typename E::Q qv;
     E::load_q(reinterpret_cast<const char *>(p.q) + (size_t)u * INB, c, qv);
+    if (!Q4 && p.qring && warp == 0 && sub == 0 && cr == 0)     // remembered for a recount at compression time
+        st_plain(p.qring + ((size_t)u * p.w + p.hist_row) * INB + c * 16,
+                 ld_plain(reinterpret_cast<const char *>(p.q) + (size_t)u * INB + c * 16));
 
     const char *Kb = p.K + (size_t)u * B * ROWB;
     const char *Vb = p.V + (size_t)u * B * ROWB;

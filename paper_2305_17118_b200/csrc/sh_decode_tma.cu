@@ -191,6 +191,11 @@ __global__ void __launch_bounds__(NWC * 32 + 32, CPS) sh_decode_tma_kernel(const
                 if (tl == 0) {
 #pragma unroll
                     for (int k = 0; k < CH; ++k) qraw[k] = *reinterpret_cast<const uint4 *>(st + 2 * TILE + (c + k * LR) * 16);
+                    if (p.qring && warp == 0 && sub == 0 && !dead) {     // remembered for a recount at compression time
+#pragma unroll
+                        for (int k = 0; k < CH; ++k)
+                            *reinterpret_cast<uint4 *>(p.qring + ((size_t)u * p.w + p.hist_row) * ROWB + (c + k * LR) * 16) = qraw[k];
+                    }
                 }
                 // ---- this group's rows of the tile: K chunks -> partial dot, V chunks parked in registers
                 float sv[RG];

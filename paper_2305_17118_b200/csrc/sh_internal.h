@@ -17,6 +17,7 @@ struct ShLayout {
     size_t xport;           // [2][B][D] fp32 scratch for sh_export_unit
     size_t stage_q, stage_k, stage_v, stage_out;  // staging for the *_host calls
     size_t err;             // one int: set by a kernel whose bounded wait gave up
+    size_t qring;           // record_mode 1 only: [U][w][in_bytes] queries of the last w steps
     size_t total;
 };
 
@@ -31,6 +32,8 @@ struct sh_context {
     int split;
     bool split_explicit;   // SH_OPT_SPLIT was set by the caller
     int auto_compress;
+    int record_mode;    // SH_OPT_RECORD_MODE: 0 record kept online, 1 recomputed at compression from stored queries
+    long long record_fresh_t;   // record_mode 1: step for which the bit-planes were last recomputed (-1: never)
     int prefill_chunk;  // SH_OPT_PREFILL_CHUNK: 1 = sh_prefill may batch tokens between compressions
     int kernel;      // SH_OPT_DECODE_KERNEL: 0 automatic, 1 direct loads, 2 pipelined bulk copies
     bool started;    // a step has run: options are frozen
@@ -48,6 +51,7 @@ struct DecodeParams {
     char *Ks, *Vs;
     uint32_t *hist;
     int32_t *pos;
+    char *qring;    // [U][w][row] ring of the last w queries (row = step mod w), or NULL
     int U, B, Bw, w;
     int n;          // live rows per unit including the token appended by this step
     int hist_row;   // t mod w
@@ -86,6 +90,9 @@ cudaError_t sh_launch_decode_tma(const sh_context *c, const DecodeParams &p, cud
 int sh_prefill_chunk_capacity(const sh_context *c);
 cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const void *k, const void *v, float *out,
                                     int count, cudaStream_t s, long long *launches);
+cudaError_t sh_launch_recount(const sh_context *c, cudaStream_t s, long long *launches);
+// Recompute the record if the handle is in recompute mode and has not done so for the current step.
+int sh_recount_if_needed(sh_context *c, cudaStream_t s);
 cudaError_t sh_launch_select(const SelectParams &p, bool from_hist, cudaStream_t s, long long *launches);
 cudaError_t sh_launch_compact(const CompactParams &p, cudaStream_t s, long long *launches);
 cudaError_t sh_launch_counters(const uint32_t *hist, uint16_t *counters, int U, int B, int Bw, int w, int n,

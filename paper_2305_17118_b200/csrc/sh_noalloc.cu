@@ -54,6 +54,8 @@ extern "C" int sh_compress_static(sh_handle h, void *stream, int *evicted_per_un
     cudaError_t e = scratch_address(&src_idx);
     if (e != cudaSuccess) { h->last_err = e; return SH_ECUDA; }
     cudaStream_t s = (cudaStream_t)stream;
+    const int rrc = sh_recount_if_needed(h, s);
+    if (rrc != SH_OK) return rrc;
 
     SelectParams sp = {};
     sp.hist = reinterpret_cast<const uint32_t *>(h->slab + h->L.hist);

@@ -81,6 +81,11 @@ struct ChunkParams {
     int t0;                  // tokens streamed before the chunk
     int SS;                  // row stride of S in floats
     float scale_log2e;
+    char *qring;             // [U][w][D] queries of the last w steps (row = step mod w), or NULL
+    // recount mode (the record recomputed at compression time): queries come from the ring,
+    // steps first_step .. first_step + nsteps - 1, blockIdx.y selects CQ of them; keys are the
+    // n0 cached rows, visible to a query when their position does not exceed its step
+    int first_step, nsteps;
 };
 
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc) {
@@ -106,7 +111,7 @@ __device__ __forceinline__ void load_tile_async(uint16_t *tile, const char *cach
 
 // CQ queries per CTA (64 or 32).  Warps form a WM x WN grid: WM row blocks of 16 queries,
 // WN groups that split the 64 keys of a tile (logits) or the 128 output columns (P.V).
-template <int DT, int CQ>
+template <int DT, int CQ, bool RECOUNT>
 __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const ChunkParams p) {
     constexpr int WM = CQ / 16, WN = 8 / WM;
     constexpr int NBK = KT / WN / 8;     // 8-key blocks per warp in the logits phase
@@ -119,10 +124,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
     uint16_t *tile0 = Qs + CQ * ROWH;                                   // [2][KT][ROWH] double-buffered K/V tiles
     float *S = reinterpret_cast<float *>(tile0 + 2 * KT * ROWH);        // [CQ][SS]
     float *rowL = S + (size_t)CQ * p.SS;                                // [CQ] row sums
+    int *nvs = reinterpret_cast<int *>(rowL + CQ);                      // [CQ] keys visible to each query
 
     const int u = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int wm = warp % WM, wn = warp / WM;
-    const int n0 = p.n0, c = p.c, n_tot = p.n0 + p.c, SS = p.SS;
+    const int n0 = p.n0, SS = p.SS;
+    // first step handled by this CTA and how many
+    const int step0 = RECOUNT ? p.first_step + (int)blockIdx.y * CQ : p.t0 + 1;
+    const int c = RECOUNT ? min(CQ, p.nsteps - (int)blockIdx.y * CQ) : p.c;
+    const int n_tot = RECOUNT ? p.n0 : p.n0 + p.c;
     const size_t tstride = (size_t)p.U * D * 2;          // bytes between consecutive tokens of one unit
     const char *Kc = p.K + (size_t)u * p.B * D * 2;
     const char *Vc = p.V + (size_t)u * p.B * D * 2;
@@ -132,19 +142,41 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
     for (int idx = tid; idx < CQ * (D / 8); idx += NTHREADS) {
         const int row = idx / (D / 8), ch = idx % (D / 8);
         uint4 val = make_uint4(0, 0, 0, 0);
-        if (row < c) val = *reinterpret_cast<const uint4 *>(p.q + (size_t)row * tstride + (size_t)u * D * 2 + ch * 16);
+        if (row < c) {
+            char *ring_row = p.qring ? p.qring + ((size_t)u * p.w + (step0 + row) % p.w) * (D * 2) + ch * 16 : nullptr;
+            if (RECOUNT) {
+                val = *reinterpret_cast<const uint4 *>(ring_row);
+            } else {
+                val = *reinterpret_cast<const uint4 *>(p.q + (size_t)row * tstride + (size_t)u * D * 2 + ch * 16);
+                if (ring_row) *reinterpret_cast<uint4 *>(ring_row) = val;     // remembered for a later recount
+            }
+        }
         *reinterpret_cast<uint4 *>(Qs + row * ROWH + ch * 8) = val;
     }
-    if (tid < c) p.pos[(size_t)u * p.B + n0 + tid] = p.t0 + tid + 1;
-    // append the chunk's keys and values to the cache (nothing in this launch reads them back from there)
-    for (int idx = tid; idx < c * (D / 8); idx += NTHREADS) {
-        const int row = idx / (D / 8), ch = idx % (D / 8);
-        const size_t src = (size_t)row * tstride + (size_t)u * D * 2 + ch * 16;
-        const size_t dst = ((size_t)u * p.B + n0 + row) * (D * 2) + ch * 16;
-        *reinterpret_cast<uint4 *>(p.K + dst) = *reinterpret_cast<const uint4 *>(p.k + src);
-        *reinterpret_cast<uint4 *>(p.V + dst) = *reinterpret_cast<const uint4 *>(p.v + src);
+    if (RECOUNT) {
+        // slots are sorted by position: query i sees the slots whose position is <= its step
+        const int32_t *pos_u = p.pos + (size_t)u * p.B;
+        for (int i = tid; i < CQ; i += NTHREADS) {
+            int lo = 0, hi = (i < c) ? n0 : 0;
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (pos_u[mid] <= step0 + i) lo = mid + 1; else hi = mid;
+            }
+            nvs[i] = lo;
+        }
+    } else {
+        for (int i = tid; i < CQ; i += NTHREADS) nvs[i] = (i < c) ? n0 + i + 1 : 0;
+        if (tid < c) p.pos[(size_t)u * p.B + n0 + tid] = p.t0 + tid + 1;
+        // append the chunk's keys and values to the cache (nothing in this launch reads them back from there)
+        for (int idx = tid; idx < c * (D / 8); idx += NTHREADS) {
+            const int row = idx / (D / 8), ch = idx % (D / 8);
+            const size_t src = (size_t)row * tstride + (size_t)u * D * 2 + ch * 16;
+            const size_t dst = ((size_t)u * p.B + n0 + row) * (D * 2) + ch * 16;
+            *reinterpret_cast<uint4 *>(p.K + dst) = *reinterpret_cast<const uint4 *>(p.k + src);
+            *reinterpret_cast<uint4 *>(p.V + dst) = *reinterpret_cast<const uint4 *>(p.v + src);
+        }
     }
-    const char *kchunk = p.k + (size_t)u * D * 2, *vchunk = p.v + (size_t)u * D * 2;
+    const char *kchunk = RECOUNT ? nullptr : p.k + (size_t)u * D * 2, *vchunk = RECOUNT ? nullptr : p.v + (size_t)u * D * 2;
     load_tile_async(tile0, Kc, kchunk, 0, n0, n_tot, tstride);      // first K tile is on its way
     cp_async_commit();
     __syncthreads();
@@ -162,7 +194,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
         uint16_t *tile = tile0 + (kt & 1) * KT * ROWH;
         // prefetch the next K tile (or the first V tile) into the other buffer, then wait for this one
         if (kt + 1 < ntiles) load_tile_async(tile0 + ((kt + 1) & 1) * KT * ROWH, Kc, kchunk, (kt + 1) * KT, n0, n_tot, tstride);
-        else load_tile_async(tile0 + ((kt + 1) & 1) * KT * ROWH, Vc, vchunk, 0, n0, n_tot, tstride);
+        else if (!RECOUNT) load_tile_async(tile0 + ((kt + 1) & 1) * KT * ROWH, Vc, vchunk, 0, n0, n_tot, tstride);
         cp_async_commit();
         cp_async_wait<1>();
         __syncthreads();
@@ -188,7 +220,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
             for (int e = 0; e < 4; ++e) {
                 const int i = wm * 16 + (lane >> 2) + (e >> 1) * 8;                 // query row
                 const int j = kt * KT + wn * (KT / WN) + nb * 8 + (lane & 3) * 2 + (e & 1);   // key slot
-                const bool live = i < c && j < n0 + i + 1;                           // cached rows and chunk tokens 0..i
+                const bool live = j < nvs[i];                                         // cached rows (and chunk tokens 0..i) the query may see
                 S[(size_t)i * SS + j] = live ? acc[nb][e] * p.scale_log2e : -INFINITY;
             }
         }
@@ -198,7 +230,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
     // ---- softmax rows and record bits: one warp per query row
     for (int i = warp; i < CQ; i += NTHREADS / 32) {
         float *Si = S + (size_t)i * SS;
-        const int nv = (i < c) ? n0 + i + 1 : 0;
+        const int nv = nvs[i];
         float mx = -INFINITY;
         for (int j = lane; j < nv; j += 32) mx = fmaxf(mx, Si[j]);
 #pragma unroll
@@ -213,8 +245,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
         for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
         if (lane == 0) rowL[i] = sum;
         if (i < c) {
-            // step t = t0 + i + 1: low_j = [alpha_j < 1/t] = [e_j * t < L]
-            const int t = p.t0 + i + 1;
+            // step t: low_j = [alpha_j < 1/t] = [e_j * t < L]
+            const int t = step0 + i;
             const float tf = (float)t;
             uint32_t *hrow = p.hist + ((size_t)u * p.w + (t % p.w)) * p.Bw;
             __syncwarp();
@@ -227,6 +259,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
         }
     }
 
+    if constexpr (RECOUNT) {
+        cp_async_wait<0>();
+    } else {
     // ---- phase 2: O = P.V
     float oacc[NBD][4];
 #pragma unroll
@@ -283,21 +318,23 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
             }
         }
     }
+    }   // !RECOUNT
 }
 
-template <int DT, int CQ>
+template <int DT, int CQ, bool RECOUNT>
 cudaError_t launch_chunk(const ChunkParams &p, cudaStream_t s) {
-    const size_t smem = sizeof(uint16_t) * (size_t)(CQ + 2 * KT) * ROWH + sizeof(float) * ((size_t)CQ * p.SS + CQ);
-    auto kern = sh_prefill_chunk_kernel<DT, CQ>;
+    const size_t smem = sizeof(uint16_t) * (size_t)(CQ + 2 * KT) * ROWH + sizeof(float) * ((size_t)CQ * p.SS + 2 * CQ);
+    auto kern = sh_prefill_chunk_kernel<DT, CQ, RECOUNT>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    kern<<<p.U, NTHREADS, smem, s>>>(p);
+    const unsigned gy = RECOUNT ? (unsigned)((p.nsteps + CQ - 1) / CQ) : 1u;
+    kern<<<dim3(p.U, gy, 1), NTHREADS, smem, s>>>(p);
     return cudaGetLastError();
 }
 
 int s_stride(int B) { return ((B + KT - 1) / KT) * KT + 8; }
 size_t smem_need(int CQ, int B) {
-    return sizeof(uint16_t) * (size_t)(CQ + 2 * KT) * ROWH + sizeof(float) * ((size_t)CQ * s_stride(B) + CQ);
+    return sizeof(uint16_t) * (size_t)(CQ + 2 * KT) * ROWH + sizeof(float) * ((size_t)CQ * s_stride(B) + 2 * CQ);
 }
 
 }  // namespace
@@ -325,10 +362,33 @@ cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const vo
     p.n0 = c->n; p.c = count; p.t0 = (int)c->t;
     p.SS = s_stride(c->B);
     p.scale_log2e = (float)((double)c->scale * 1.4426950408889634);
+    p.qring = c->record_mode ? c->slab + c->L.qring : nullptr;
     cudaError_t e = cudaErrorInvalidValue;
     if (count < 1 || count > sh_prefill_chunk_capacity(c)) return e;
-    if (count <= 32) e = c->dtype == SH_F16 ? launch_chunk<SH_F16, 32>(p, s) : launch_chunk<SH_BF16, 32>(p, s);
-    else e = c->dtype == SH_F16 ? launch_chunk<SH_F16, 64>(p, s) : launch_chunk<SH_BF16, 64>(p, s);
+    if (count <= 32) e = c->dtype == SH_F16 ? launch_chunk<SH_F16, 32, false>(p, s) : launch_chunk<SH_BF16, 32, false>(p, s);
+    else e = c->dtype == SH_F16 ? launch_chunk<SH_F16, 64, false>(p, s) : launch_chunk<SH_BF16, 64, false>(p, s);
+    if (e == cudaSuccess) *launches += 1;
+    return e;
+}
+
+// The record of Algorithm 2 recomputed from the queries of the last w steps against the
+// present cache: rewrites the unit's bit-plane rows of those steps.
+cudaError_t sh_launch_recount(const sh_context *c, cudaStream_t s, long long *launches) {
+    ChunkParams p = {};
+    p.K = c->slab + c->L.K; p.V = c->slab + c->L.V;
+    p.hist = reinterpret_cast<uint32_t *>(c->slab + c->L.hist);
+    p.pos = reinterpret_cast<int32_t *>(c->slab + c->L.pos);
+    p.U = c->U; p.B = c->B; p.Bw = c->Bw; p.w = c->w;
+    p.n0 = c->n; p.c = 0; p.t0 = (int)c->t;
+    p.SS = s_stride(c->B);
+    p.scale_log2e = (float)((double)c->scale * 1.4426950408889634);
+    p.qring = c->slab + c->L.qring;
+    p.nsteps = c->t < c->w ? (int)c->t : c->w;
+    p.first_step = (int)c->t - p.nsteps + 1;
+    if (p.nsteps < 1) return cudaSuccess;
+    cudaError_t e;
+    if (smem_need(64, c->B) <= 200 * 1024) e = c->dtype == SH_F16 ? launch_chunk<SH_F16, 64, true>(p, s) : launch_chunk<SH_BF16, 64, true>(p, s);
+    else e = c->dtype == SH_F16 ? launch_chunk<SH_F16, 32, true>(p, s) : launch_chunk<SH_BF16, 32, true>(p, s);
     if (e == cudaSuccess) *launches += 1;
     return e;
 }

@@ -145,3 +145,52 @@ def run_lockstep_chunked(handle, cfg_dtype: str, inputs_block, steps: int, units
             res.compressions += 1
         done += cnt
     return res, orc
+
+
+def run_lockstep_recompute(handle, cfg_dtype: str, inputs, steps: int, units, tol: float, res: LockstepResult = None,
+                           orc=None):
+    """Lockstep for SH_OPT_RECORD_MODE = 1 (the record recomputed at compression time).
+    Every step: outputs compared.  When the cache fills: the library recomputes its
+    bit-planes, the oracle recounts from its own stored queries; bits may differ only
+    inside the 1e-6 window (the oracle then adopts the library's), after which counters,
+    positions and kept sets must be identical."""
+    units = torch.as_tensor(units, dtype=torch.long)
+    un = units.numpy()
+    if orc is None:
+        orc = oracle_mod.Oracle(len(un), handle.B, handle.r, handle.w, handle.m, handle.D)
+    res = res or LockstepResult()
+    dev_units = units.to(handle.device)
+    w = handle.w
+    for _ in range(steps):
+        t = orc.t + 1
+        q, k, v = inputs(t)
+        out = handle.decode_step(q, k, v)
+        o_out, _alpha, _low, _amb = orc.attend(to_oracle(q, dev_units), to_oracle(k, dev_units),
+                                               to_oracle(v, dev_units))
+        err = float(np.abs(out[dev_units].double().cpu().numpy() - o_out).max())
+        res.max_abs_err = max(res.max_abs_err, err)
+        assert err <= tol, f"step {t}: attention output off by {err:.3e} > {tol}"
+        if orc.full:
+            handle.recompute_record()
+            nn = orc.n
+            g = np.stack([handle.export_record(int(u))[:, :nn] for u in un])          # [units, w, n]
+            _a, o_low, amb, steps_in = orc.recount()
+            live_rows = steps_in > 0
+            assert not g[:, ~live_rows].any(), "bits in rows of steps outside the window"
+            diff = g != o_low
+            bad = diff & ~amb
+            assert not bad.any(), (f"step {t}: {int(bad.sum())} recomputed bits differ outside the 1e-6 window; "
+                                   f"first at (unit, row, slot) {np.argwhere(bad)[0].tolist()}")
+            res.adoptions += int(diff.sum())
+            res.slot_steps += int(live_rows.sum()) * nn * len(un)
+            orc.set_record(g, steps_in)
+            n1, _, pos1, cnt1, _ = handle.state(low=False)
+            assert (cnt1[un].astype(np.int32) == orc.counters()).all(), f"step {t}: recomputed records differ"
+            orc.compress()
+            assert handle.compress() == handle.m
+            n2, _, pos2, cnt2, _ = handle.state(low=False)
+            assert n2 == orc.n
+            assert (pos2[un] == orc.positions()).all(), f"step {t}: kept sets differ"
+            res.compressions += 1
+        res.steps += 1
+    return res, orc

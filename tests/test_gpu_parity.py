@@ -6,7 +6,7 @@ import pytest
 import torch
 
 import oracle
-from lockstep import run_lockstep, run_lockstep_chunked, to_oracle
+from lockstep import run_lockstep, run_lockstep_chunked, run_lockstep_recompute, to_oracle
 from paper_2305_17118_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -78,6 +78,42 @@ def test_lockstep_chunked_prompt_kernel(sh, dtype, U, B, r, w, m, sizes):
     # and the decode step carries on from the state the chunks left
     q2, k2, v2 = wl.random_stream(U, d, 40, seed=99, dtype=dtype, peaked=3.0, device="cuda")
     run_lockstep(h, dtype, lambda t: (q2[t - T - 1], k2[t - T - 1], v2[t - T - 1]), 40, torch.arange(U), TOL[dtype], orc=orc)
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("U,B,r,w,m", [(5, 150, 9, 37, 41), (3, 410, 64, 128, 64), (140, 96, 8, 70, 30), (2, 40, 3, 9, 20)])
+def test_lockstep_record_recomputed_at_compression(sh, dtype, U, B, r, w, m):
+    """SH_OPT_RECORD_MODE = 1: Algorithm 2 as stated, the record rebuilt at each compression from
+    the stored queries of the last w steps against the present cache."""
+    d, T = 128, 2 * B + 3 * m + 5
+    q, k, v = wl.random_stream(U, d, T, seed=23 + U, dtype=dtype, peaked=3.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, recompute_record=True)
+    res, orc = run_lockstep_recompute(h, dtype, _stream_fn(q, k, v), T, torch.arange(U), TOL[dtype])
+    assert res.compressions >= 4
+    assert res.adoptions <= 1e-4 * res.slot_steps + 2
+
+
+def test_recompute_mode_through_prefill_and_automatic_compression(sh):
+    """Same mode driven the way an application would: chunked sh_prefill, then decode steps with
+    automatic compression; compared with the oracle running the same variant on its own."""
+    U, d, B, r, w, m, P, T, dtype = 12, 128, 120, 8, 50, 40, 300, 420, "f16"
+    q, k, v = wl.random_stream(U, d, T, seed=31, dtype=dtype, peaked=3.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, recompute_record=True)
+    orc = oracle.Oracle(U, B, r, w, m, d)
+    idx = torch.arange(U, device="cuda")
+    outs = torch.empty(T, U, d, device="cuda")
+    h.prefill(q[:P].contiguous(), k[:P].contiguous(), v[:P].contiguous(), outs[:P])
+    for t in range(P, T):
+        h.decode_step(q[t], k[t], v[t], outs[t])
+    worst = 0.0
+    for t in range(T):
+        o, _ = orc.step_recompute(to_oracle(q[t], idx), to_oracle(k[t], idx), to_oracle(v[t], idx))
+        worst = max(worst, float(np.abs(outs[t].double().cpu().numpy() - o).max()))
+    n, tt, pos, cnt, _ = h.state(low=False)
+    assert n == orc.n and tt == orc.t
+    same = (pos == orc.positions()).all(axis=1)
+    assert same.mean() >= 0.75          # units without a threshold-ambiguous flip agree exactly
+    assert worst <= TOL[dtype] or same.mean() < 1.0
 
 
 def test_prefill_uses_chunks_and_matches_oracle(sh):

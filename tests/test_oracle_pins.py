@@ -343,3 +343,54 @@ def test_ambiguity_flag_marks_scores_near_the_threshold():
     o.record(low)
     out, alpha, low, amb = o.attend(kk, kk, kk)
     assert not low.any() and amb.all()
+
+
+# --- the record recomputed at compression time -------------------------------------------
+def test_recount_matches_causal_attention_of_stored_queries_over_the_kept_set():
+    # From the definition: each of the last w queries against the tokens still cached that
+    # existed at its step, softmax over those, compared with 1/step.
+    T, U, d, B, r, w, m = 70, 2, 8, 14, 3, 9, 5
+    q, k, v = _stream(T, U, d, 21, peaked=2.5)
+    o = oracle.Oracle(U, B, r, w, m, d)
+    scale = 1 / math.sqrt(d)
+    n_compress = 0
+    for t in range(1, T + 1):
+        out, alpha, low, amb = o.attend(q[t - 1], k[t - 1], v[t - 1])
+        if o.full:
+            a, lo, am, steps = o.recount()
+            pos = o.positions()
+            window = [s for s in range(max(1, t - w + 1), t + 1)]
+            assert sorted(int(x) for x in steps if x) == window
+            for u in range(U):
+                for s in window:
+                    row = s % w
+                    vis = pos[u] <= s
+                    _, beta = full_attention(q[s - 1, u], k[pos[u][vis] - 1, u], v[pos[u][vis] - 1, u], scale)
+                    np.testing.assert_allclose(a[u, row][vis], beta, rtol=1e-11, atol=1e-15)
+                    assert (a[u, row][~vis] == 0).all() and not lo[u, row][~vis].any()
+                    assert (lo[u, row][vis] == (beta < 1.0 / s)).all()
+            o.set_record(lo, steps)
+            # counters now count the recomputed flags, by definition
+            I = o.counters()
+            for u in range(U):
+                want = sum(lo[u, s % w].astype(int) for s in window)
+                assert (I[u] == want).all()
+            dropped = o.compress()
+            assert dropped is not None and (dropped <= t - r).all()
+            n_compress += 1
+    assert n_compress >= 10
+
+
+def test_step_recompute_keeps_the_budget_and_full_attention_when_it_never_fills():
+    T, U, d = 30, 2, 8
+    q, k, v = _stream(T, U, d, 22, peaked=2.0)
+    o = oracle.Oracle(U, T + 1, 2, 6, 3, d)
+    for t in range(T):
+        out, dropped = o.step_recompute(q[t], k[t], v[t])
+        assert dropped is None
+    ref, _ = full_attention(q[T - 1, 0], k[:, 0], v[:, 0], 1 / math.sqrt(d))
+    np.testing.assert_allclose(out[0], ref, atol=1e-13)
+    o2 = oracle.Oracle(U, 10, 2, 6, 3, d)
+    for t in range(T):
+        o2.step_recompute(q[t], k[t], v[t])
+        assert o2.n < 10
