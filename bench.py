@@ -132,11 +132,12 @@ def live_rows_schedule(cfg, first_step: int, count: int):
 
 
 # --------------------------------------------------------------------------- CPU oracle arm
-def oracle_run(cfg, steps: int, warmup: int, sample_units: int, budget_s: float = 60.0):
+def oracle_run(cfg, steps: int, warmup: int, sample_units: int, min_seconds: float = 0.0, budget_s: float = 60.0):
     """Times the CPU oracle (as it stands) on `sample_units` units: an untimed
-    run-in of B + warmup tokens to reach the steady-state saw-tooth, then up to
-    `steps` timed steps.  Returns (steps/s scaled to all units, info)."""
-    import numpy as np
+    run-in of B + warmup tokens to reach the steady-state saw-tooth, then at least
+    `steps` timed steps (more, until `min_seconds` of CPU work, never beyond
+    `budget_s`).  Inputs cycle through 64 pre-drawn steps.  Returns (steps/s scaled
+    to all units, info, seconds per step)."""
     import oracle
     U = min(sample_units, cfg.units)
     st = wl.Stream(cfg.scaled(units=U), device="cpu")
@@ -146,12 +147,14 @@ def oracle_run(cfg, steps: int, warmup: int, sample_units: int, budget_s: float 
     for t in range(1, run_in + 1):
         q, k, v = st.step(t)
         orc.step(f64(q), f64(k), f64(v))
-    pre = [tuple(f64(x) for x in st.step(run_in + 1 + i)) for i in range(steps)]
+    pre = [tuple(f64(x) for x in st.step(run_in + 1 + i)) for i in range(min(64, max(steps, 1)))]
     done, t0 = 0, time.perf_counter()
-    for q, k, v in pre:
+    while True:
+        q, k, v = pre[done % len(pre)]
         orc.step(q, k, v)
         done += 1
-        if time.perf_counter() - t0 > budget_s:
+        el = time.perf_counter() - t0
+        if el > budget_s or (done >= steps and el >= min_seconds):
             break
     dt = time.perf_counter() - t0
     unit_steps_per_s = done * U / dt
@@ -325,7 +328,7 @@ def cuda_arm(args, cfg, rank, world):
         return
     cpu = None
     if (world == 1 or rank == 0) and not args.no_cpu_baseline:
-        _, cpu, _ = oracle_run(cfg, min(K, 256), 0, args.oracle_units, budget_s=20.0)
+        _, cpu, _ = oracle_run(cfg, min(K, 64), 0, args.oracle_units, min_seconds=10.0, budget_s=30.0)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
