@@ -1,0 +1,64 @@
+"""Persistence-of-importance diagnostics on synthetic streams (Section 3.2).
+
+A token is *pivotal* for position t when the query at t gives it a score above
+1/t; S_{a->b} is the union of the pivotal sets of positions a..b.  For a
+sentence of length l the paper measures, with t = l/2,
+
+    persistence ratio = |S_{t+1->l} n S_{1->t}| / |{x in S_{t+1->l} : x among x_1..x_t}|
+
+and the relative size |S_{1->t}| / t.  Both come straight out of the library's
+importance record: a handle whose budget holds the whole sentence never
+compresses, and with a history window of l steps its bit-planes keep, for every
+step, which cached tokens scored below 1/t.  The attention itself runs in the
+CUDA kernels; only the set algebra on the exported bits is done here.
+
+The paper measures these on trained OPT models over text; here the inputs are
+the synthetic streams of ``workloads`` (there are no weights or corpora in this
+repository), so the numbers characterise those streams, not a language model.
+"""
+from __future__ import annotations
+
+import dataclasses
+
+import numpy as np
+import torch
+
+from . import binding as sh
+
+
+@dataclasses.dataclass
+class Persistence:
+    ratio: np.ndarray        # [units] persistence ratio (nan where the later half has no pivotal token in the first half)
+    pivotal_frac: np.ndarray # [units] |S_{1->t}| / t
+    t: int
+    l: int
+
+
+def pivotal_table(handle: "sh.Handle", unit: int, l: int) -> np.ndarray:
+    """[l, l] bool: entry (s-1, j) = token j+1 was pivotal for position s (score not below 1/s).
+    Needs a handle that has streamed exactly l tokens with B > l and w >= l (no compression, every
+    step's bit-plane row still present)."""
+    planes = handle.export_record(unit)              # [w, B]: row s mod w, slot j; bit set = "low"
+    rows = np.arange(1, l + 1) % handle.w
+    low = planes[rows][:, :l]
+    seen = np.tril(np.ones((l, l), dtype=bool))      # position s only sees tokens 1..s
+    return seen & ~low
+
+
+def persistence(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, dtype: str, device="cuda:0") -> Persistence:
+    """q, k, v: [l, units, head_dim] CUDA tensors in the storage dtype.  Runs full-cache attention
+    over the stream (budget l + 1, window l) and evaluates the two measures per unit."""
+    l, U, d = q.shape
+    h = sh.Handle(l + 1, 0, l, 1, U, d, dtype, device=device, auto_compress=False, prefill_chunk=False)
+    h.prefill(q, k, v)
+    t = l // 2
+    ratio = np.full(U, np.nan)
+    frac = np.zeros(U)
+    for u in range(U):
+        piv = pivotal_table(h, u, l)
+        first = piv[:t, :t].any(axis=0)              # S_{1->t}
+        later = piv[t:, :t].any(axis=0)              # S_{t+1->l} restricted to x_1..x_t
+        if later.any():
+            ratio[u] = (first & later).sum() / later.sum()
+        frac[u] = first.sum() / t
+    return Persistence(ratio, frac, t, l)

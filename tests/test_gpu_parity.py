@@ -285,6 +285,36 @@ def test_snapshot_restore_replays_identically(sh):
     assert s1[0] == s2[0] and s1[1] == s2[1] and all((x == y).all() for x, y in zip(s1[2:], s2[2:]))
 
 
+def test_persistence_diagnostics_match_oracle_scores(sh):
+    """Persistence ratio and pivotal-set size (Section 3.2) from the library's record bits, against
+    the same quantities from the oracle's fp64 scores on a full (never compressed) cache."""
+    from paper_2305_17118_b200 import diagnostics
+    l, U, d, dtype = 96, 6, 128, "f16"
+    q, k, v = wl.random_stream(U, d, l, seed=41, dtype=dtype, peaked=3.0, device="cuda")
+    got = diagnostics.persistence(q, k, v, dtype)
+    orc = oracle.Oracle(U, l + 1, 0, l, 1, d)
+    idx = torch.arange(U, device="cuda")
+    piv = np.zeros((U, l, l), dtype=bool)
+    amb_any = np.zeros(U, dtype=bool)
+    for s in range(l):
+        _o, alpha, low, amb = orc.attend(to_oracle(q[s], idx), to_oracle(k[s], idx), to_oracle(v[s], idx))
+        orc.record(low)
+        piv[:, s, : s + 1] = ~low
+        if s > 0:                                      # at the first step alpha = 1 = 1/t exactly, on both sides
+            amb_any |= amb.any(axis=1)
+    t = l // 2
+    assert got.t == t and got.l == l
+    for u in range(U):
+        if amb_any[u]:
+            continue                                   # a score within 1e-6 of 1/t may legitimately flip
+        first, later = piv[u, :t, :t].any(axis=0), piv[u, t:, :t].any(axis=0)
+        want = (first & later).sum() / later.sum() if later.any() else np.nan
+        assert (np.isnan(want) and np.isnan(got.ratio[u])) or abs(got.ratio[u] - want) < 1e-12
+        assert abs(got.pivotal_frac[u] - first.sum() / t) < 1e-12
+    assert (~amb_any).sum() >= U - 1
+    assert np.nanmin(got.ratio) >= 0 and np.nanmax(got.ratio) <= 1
+
+
 def test_error_codes(sh):
     import ctypes as C
     lib = sh.lib
