@@ -146,6 +146,27 @@ int sh_prefill(sh_handle h, const void *q_dev, const void *k_dev, const void *v_
                float *out_dev, void *stream);
 
 /*
+ * Prompts of different lengths (Section 4.1 treats one head of one sequence; a batch is many such
+ * streams, and real batches are ragged).  The handle's units are n_sequences groups of
+ * heads / n_sequences consecutive units; sequence i consumes the first lengths_host[i] <= p_max
+ * tokens of its units' columns of the time-major blocks q/k/v [p_max][heads][head_dim] (the rest
+ * is ignored), with compressions whenever its own cache fills.  Afterwards n and t differ per
+ * sequence: they live in per-unit device arrays that the kernels read and advance, every
+ * sh_decode_step appends one token to every sequence, a compression runs whenever some sequence's
+ * cache is full and touches only those, and sh_sequence_state reports the per-sequence counters.
+ * Needs a freshly bound handle (nothing streamed yet) and heads % n_sequences == 0.
+ * Not available with SH_OPT_RECORD_MODE = 1; sh_prefill, sh_prefill_chunk and sh_restore are not
+ * available afterwards (SH_ESTATE).  out_dev as for sh_prefill (rows past a sequence's length are
+ * not written).
+ */
+int sh_prefill_ragged(sh_handle h, const void *q_dev, const void *k_dev, const void *v_dev, int p_max,
+                      const int *lengths_host, int n_sequences, float *out_dev, void *stream);
+
+/* Per-sequence live tokens and tokens streamed (one entry, the common values, unless
+ * sh_prefill_ragged was used).  Fills at most `capacity` entries; returns the number of sequences. */
+int sh_sequence_state(sh_handle h, int *n_host, long long *t_host, int capacity);
+
+/*
  * One chunk of the prompt without the compression: steps t+1 .. t+count for
  * every unit in one launch (see sh_prefill).  Needs 1 <= count <=
  * sh_prefill_chunk_max(h) and count <= B - n; returns SH_EINVAL otherwise
@@ -205,7 +226,8 @@ int sh_select(const uint16_t *counters_dev, int units, int n, int r, int m, int3
 
 /*
  * Snapshot for checking and checkpointing; synchronises `stream`.  Any output
- * pointer may be NULL.  n_out: live tokens per unit.  t_out: tokens streamed.
+ * pointer may be NULL.  n_out: live tokens per unit (-1 after sh_prefill_ragged: they differ).
+ * t_out: tokens streamed (the largest, after sh_prefill_ragged).
  * pos_host [heads][B] int32: stream positions (1-based) of slots [0,n), 0 beyond.
  * counters_host [heads][B] uint16: importance record I of Algorithm 2 at the
  * current step, 0 beyond n.  low_host [heads][ceil(B/32)] uint32: bit j%32 of

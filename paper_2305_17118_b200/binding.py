@@ -26,7 +26,8 @@ INPUT_TORCH_DTYPE = {SH_F32: torch.float32, SH_F16: torch.float16, SH_BF16: torc
                      SH_INT4_G64_F16: torch.float16}
 
 EXPORTS = ["sh_create", "sh_destroy", "sh_workspace_bytes", "sh_bind", "sh_set_option", "sh_decode_step",
-           "sh_decode_step_host", "sh_prefill", "sh_prefill_chunk", "sh_prefill_chunk_max", "sh_export_record", "sh_recompute_record",
+           "sh_decode_step_host", "sh_prefill", "sh_prefill_chunk", "sh_prefill_chunk_max", "sh_export_record", "sh_recompute_record", "sh_prefill_ragged",
+           "sh_sequence_state",
            "sh_compress", "sh_compress_static", "sh_select", "sh_state", "sh_export_unit",
            "sh_restore", "sh_launch_count", "sh_strerror", "sh_last_cuda_error"]
 
@@ -60,6 +61,8 @@ def _load() -> C.CDLL:
     lib.sh_prefill_chunk_max.argtypes = [vp]
     lib.sh_export_record.argtypes = [vp, C.c_int, vp, vp]
     lib.sh_recompute_record.argtypes = [vp, vp]
+    lib.sh_prefill_ragged.argtypes = [vp, vp, vp, vp, C.c_int, ip, C.c_int, vp, vp]
+    lib.sh_sequence_state.argtypes = [vp, ip, llp, C.c_int]
     lib.sh_compress.argtypes = [vp, vp, ip]
     lib.sh_compress_static.argtypes = [vp, vp, ip]
     lib.sh_select.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
@@ -180,6 +183,35 @@ class Handle:
         self._check(lib.sh_prefill(self._h, _dev(q, self.in_dtype, n, "q"), _dev(k, self.in_dtype, n, "k"),
                                    _dev(v, self.in_dtype, n, "v"), p, optr, _stream_ptr(stream)))
         return out
+
+    # -- sh_prefill_ragged / sh_sequence_state -----------------------------------
+    def prefill_ragged(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, lengths, out: Optional[torch.Tensor] = None,
+                       stream=None):
+        p = q.shape[0]
+        n = p * self.U * self.D
+        lens = (C.c_int * len(lengths))(*[int(x) for x in lengths])
+        optr = _dev(out, torch.float32, n, "out") if out is not None else None
+        self._check(lib.sh_prefill_ragged(self._h, _dev(q, self.in_dtype, n, "q"), _dev(k, self.in_dtype, n, "k"),
+                                          _dev(v, self.in_dtype, n, "v"), p, lens, len(lengths), optr,
+                                          _stream_ptr(stream)))
+        return out
+
+    def sequence_state(self):
+        """(n [sequences], t [sequences]) host counters."""
+        ns = lib.sh_sequence_state(self._h, None, None, 0)
+        n_a, t_a = (C.c_int * ns)(), (C.c_longlong * ns)()
+        lib.sh_sequence_state(self._h, n_a, t_a, ns)
+        return np.array(n_a[:], dtype=np.int64), np.array(t_a[:], dtype=np.int64)
+
+    def state_full(self, stream=None):
+        """sh_state without trimming to a common n: (pos [U,B], counters [U,B], low [U,B] bool)."""
+        pos_a = np.zeros((self.U, self.B), dtype=np.int32)
+        cnt_a = np.zeros((self.U, self.B), dtype=np.uint16)
+        low_a = np.zeros((self.U, self.Bw), dtype=np.uint32)
+        self._check(lib.sh_state(self._h, _stream_ptr(stream), None, None, pos_a.ctypes.data, cnt_a.ctypes.data,
+                                 low_a.ctypes.data))
+        bits = np.unpackbits(low_a.view(np.uint8), axis=1, bitorder="little")[:, : self.B].astype(bool)
+        return pos_a, cnt_a, bits
 
     # -- sh_prefill_chunk --------------------------------------------------------
     @property

@@ -43,6 +43,8 @@ void make_layout(sh_context *c) {
     L.stage_out = take(U * D * 4);
     L.err = take(256);
     L.qring = take(c->record_mode ? U * (size_t)c->w * c->in_bytes : 0);
+    L.n_arr = take(U * 4);
+    L.t_arr = take(U * 4);
     L.total = off;
 }
 
@@ -81,35 +83,55 @@ __global__ void sh_export_kernel(const char *K, const char *V, const __half *Ks,
     }
 }
 
+__global__ void sh_fill_counts_kernel(int *n_arr, int *t_arr, int count, int n, int t) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < count) { n_arr[i] = n; t_arr[i] = t; }
+}
+
 int do_compress(sh_context *c, cudaStream_t s) {
     int rrc = sh_recount_if_needed(c, s);
     if (rrc != SH_OK) return rrc;
     SelectParams sp = {};
-    sp.hist = reinterpret_cast<const uint32_t *>(c->slab + c->L.hist);
+    sp.hist = sh_phist(c);
     sp.counters = nullptr;
-    sp.src_idx = reinterpret_cast<int32_t *>(c->slab + c->L.src_idx);
+    sp.src_idx = sh_psrc(c);
     sp.evicted = nullptr;
-    sp.U = c->U; sp.B = c->B; sp.Bw = c->Bw; sp.w = c->w; sp.n = c->n; sp.r = c->r; sp.m = c->m;
+    sp.U = c->ucount; sp.B = c->B; sp.Bw = c->Bw; sp.w = c->w; sp.n = c->B; sp.r = c->r; sp.m = c->m;
     sp.cmax = c->w;
+    sp.n_arr = sh_pnarr(c);
     cudaError_t e = sh_launch_select(sp, true, s, &c->launches);
     if (e != cudaSuccess) return cuda_fail(c, e);
     CompactParams cp = {};
-    cp.K = c->slab + c->L.K; cp.V = c->slab + c->L.V;
-    cp.Ks = c->slab + c->L.Ks; cp.Vs = c->slab + c->L.Vs;
-    cp.hist = reinterpret_cast<uint32_t *>(c->slab + c->L.hist);
-    cp.pos = reinterpret_cast<int32_t *>(c->slab + c->L.pos);
+    cp.K = sh_pK(c); cp.V = sh_pV(c);
+    cp.Ks = sh_pKs(c); cp.Vs = sh_pVs(c);
+    cp.hist = sh_phist(c);
+    cp.pos = sh_ppos(c);
     cp.src_idx = sp.src_idx;
-    cp.U = c->U; cp.B = c->B; cp.Bw = c->Bw; cp.w = c->w; cp.n = c->n; cp.m = c->m;
+    cp.U = c->ucount; cp.B = c->B; cp.Bw = c->Bw; cp.w = c->w; cp.n = c->B; cp.m = c->m;
     cp.row_bytes = c->row_bytes;
     cp.scale_bytes = c->dtype == SH_INT4_G64_F16 ? (c->D / 64) * 2 : 0;
     cp.err = reinterpret_cast<int *>(c->slab + c->L.err);
+    cp.n_arr = sh_pnarr(c);
     e = sh_launch_compact(cp, s, &c->launches);
     if (e != cudaSuccess) return cuda_fail(c, e);
-    c->n -= c->m;
+    sh_after_compression(c);
     return SH_OK;
 }
 
 }  // namespace
+
+bool sh_compression_due(const sh_context *c) {
+    if (!c->ragged) return c->n == c->B;
+    for (int n : c->n_seq)
+        if (n == c->B) return true;
+    return false;
+}
+
+void sh_after_compression(sh_context *c) {
+    if (!c->ragged) { c->n -= c->m; return; }
+    for (int &n : c->n_seq)
+        if (n == c->B) n -= c->m;
+}
 
 int sh_recount_if_needed(sh_context *c, cudaStream_t s) {
     if (!c->record_mode || c->record_fresh_t == c->t) return SH_OK;
@@ -125,12 +147,13 @@ int do_step(sh_context *c, const void *q, const void *k, const void *v, float *o
             bool compress_after) {
     DecodeParams p = {};
     p.q = q; p.k_new = k; p.v_new = v; p.out = out;
-    p.K = c->slab + c->L.K; p.V = c->slab + c->L.V;
-    p.Ks = c->slab + c->L.Ks; p.Vs = c->slab + c->L.Vs;
-    p.hist = reinterpret_cast<uint32_t *>(c->slab + c->L.hist);
-    p.pos = reinterpret_cast<int32_t *>(c->slab + c->L.pos);
-    p.qring = c->record_mode ? c->slab + c->L.qring : nullptr;
-    p.U = c->U; p.B = c->B; p.Bw = c->Bw; p.w = c->w;
+    p.K = sh_pK(c); p.V = sh_pV(c);
+    p.Ks = sh_pKs(c); p.Vs = sh_pVs(c);
+    p.hist = sh_phist(c);
+    p.pos = sh_ppos(c);
+    p.qring = sh_pqring(c);
+    p.n_arr = sh_pnarr(c); p.t_arr = sh_ptarr(c);
+    p.U = c->ucount; p.B = c->B; p.Bw = c->Bw; p.w = c->w;
     p.n = c->n + 1;
     p.t = (int)(c->t + 1);
     p.hist_row = (int)((c->t + 1) % c->w);
@@ -138,11 +161,18 @@ int do_step(sh_context *c, const void *q, const void *k, const void *v, float *o
     cudaError_t e = sh_launch_decode(c, p, s, &c->launches);
     if (e != cudaSuccess) return cuda_fail(c, e);
     c->started = true;
-    c->n += 1;
     c->t += 1;
-    if (compress_after && c->n == c->B) return do_compress(c, s);
+    if (c->ragged) {
+        for (size_t i = 0; i < c->n_seq.size(); ++i) { c->n_seq[i] += 1; c->t_seq[i] += 1; }
+    } else {
+        c->n += 1;
+    }
+    if (compress_after && sh_compression_due(c)) return do_compress(c, s);
     return SH_OK;
 }
+
+// Is any cache full (the next step would overflow it)?
+bool cache_full(const sh_context *c) { return sh_compression_due(c); }
 
 bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
@@ -175,6 +205,9 @@ int sh_create(int B, int r, int w, int m, int heads, int head_dim, int dtype, sh
     c->slab = nullptr; c->slab_bytes = 0;
     c->launches = 0;
     c->last_err = cudaSuccess;
+    c->u0 = 0; c->ucount = heads;
+    c->ragged = false;
+    c->units_per_seq = heads;
     make_layout(c);
     *out = c;
     return SH_OK;
@@ -194,6 +227,10 @@ int sh_bind(sh_handle h, void *slab_dev, size_t bytes, void *stream) {
     h->slab_bytes = bytes;
     h->n = 0; h->t = 0;
     h->started = false;
+    h->ragged = false;
+    h->n_seq.clear(); h->t_seq.clear();
+    h->u0 = 0; h->ucount = h->U;
+    h->record_fresh_t = -1;
     return SH_OK;
 }
 
@@ -242,7 +279,7 @@ int sh_decode_step(sh_handle h, const void *q_dev, const void *k_new_dev, const 
     if (!h || !q_dev || !k_new_dev || !v_new_dev || !attn_out_dev) return SH_EINVAL;
     if (misaligned(q_dev) || misaligned(k_new_dev) || misaligned(v_new_dev)) return SH_EINVAL;
     if (!h->slab) return SH_ESTATE;
-    if (h->n >= h->B) return SH_EFULL;
+    if (cache_full(h)) return SH_EFULL;
     if (h->t + 1 >= (1 << 24)) return SH_EINVAL;   // the threshold test multiplies by t in fp32
     return do_step(h, q_dev, k_new_dev, v_new_dev, attn_out_dev, (cudaStream_t)stream, h->auto_compress != 0);
 }
@@ -265,7 +302,8 @@ int sh_decode_step_host(sh_handle h, const void *q_host, const void *k_new_host,
                         float *attn_out_host, void *stream) {
     if (!h || !q_host || !k_new_host || !v_new_host || !attn_out_host) return SH_EINVAL;
     if (!h->slab) return SH_ESTATE;
-    if (h->n >= h->B) return SH_EFULL;
+    if (cache_full(h)) return SH_EFULL;
+    if (h->t + 1 >= (1 << 24)) return SH_EINVAL;
     cudaStream_t s = (cudaStream_t)stream;
     const size_t inb = (size_t)h->U * h->in_bytes, outb = (size_t)h->U * h->D * 4;
     cudaError_t e;
@@ -292,7 +330,7 @@ int sh_decode_step_host(sh_handle h, const void *q_host, const void *k_new_host,
     if (stage_out &&
         (e = cudaMemcpyAsync(attn_out_host, out, outb, cudaMemcpyDeviceToHost, s)) != cudaSuccess)
         return cuda_fail(h, e);
-    if (h->auto_compress && h->n == h->B) {
+    if (h->auto_compress && sh_compression_due(h)) {
         rc = do_compress(h, s);
         if (rc != SH_OK) return rc;
     }
@@ -314,7 +352,7 @@ int sh_prefill_chunk(sh_handle h, const void *q_dev, const void *k_dev, const vo
                      void *stream) {
     if (!h || !q_dev || !k_dev || !v_dev || count < 1) return SH_EINVAL;
     if (misaligned(q_dev) || misaligned(k_dev) || misaligned(v_dev)) return SH_EINVAL;
-    if (!h->slab) return SH_ESTATE;
+    if (!h->slab || h->ragged) return SH_ESTATE;
     if (h->n >= h->B) return SH_EFULL;
     const int cap = sh_prefill_chunk_capacity(h);
     if (cap == 0 || count > cap || count > h->B - h->n) return SH_EINVAL;
@@ -325,22 +363,17 @@ int sh_prefill_chunk(sh_handle h, const void *q_dev, const void *k_dev, const vo
 
 int sh_prefill_chunk_max(sh_handle h) { return h ? sh_prefill_chunk_capacity(h) : 0; }
 
-int sh_prefill(sh_handle h, const void *q_dev, const void *k_dev, const void *v_dev, int p, float *out_dev,
-               void *stream) {
-    if (!h || !q_dev || !k_dev || !v_dev || p < 0) return SH_EINVAL;
-    if (misaligned(q_dev) || misaligned(k_dev) || misaligned(v_dev)) return SH_EINVAL;
-    if (!h->slab) return SH_ESTATE;
-    if (h->n >= h->B) return SH_EFULL;
-    if (h->t + p >= (1 << 24)) return SH_EINVAL;
+// p tokens of the active unit range (q, k, v, out already point at that range's first unit;
+// consecutive tokens are h->U rows apart): chunks where the shape allows, decode steps otherwise,
+// a compression whenever the cache fills.
+static int prefill_range(sh_context *h, const char *q_dev, const char *k_dev, const char *v_dev, int p, float *out_dev,
+                         cudaStream_t s) {
     const size_t in_stride = (size_t)h->U * h->in_bytes, out_stride = (size_t)h->U * h->D;
     float *sink = reinterpret_cast<float *>(h->slab + h->L.stage_out);
     const int cap = h->prefill_chunk ? sh_prefill_chunk_capacity(h) : 0;
-    cudaStream_t s = (cudaStream_t)stream;
     int i = 0;
     while (i < p) {
-        const char *q = static_cast<const char *>(q_dev) + i * in_stride;
-        const char *k = static_cast<const char *>(k_dev) + i * in_stride;
-        const char *v = static_cast<const char *>(v_dev) + i * in_stride;
+        const char *q = q_dev + i * in_stride, *k = k_dev + i * in_stride, *v = v_dev + i * in_stride;
         int cnt = p - i;
         if (cnt > h->B - h->n) cnt = h->B - h->n;
         if (cnt > cap) cnt = cap;
@@ -357,6 +390,76 @@ int sh_prefill(sh_handle h, const void *q_dev, const void *k_dev, const void *v_
         i += cnt;
     }
     return SH_OK;
+}
+
+int sh_prefill(sh_handle h, const void *q_dev, const void *k_dev, const void *v_dev, int p, float *out_dev,
+               void *stream) {
+    if (!h || !q_dev || !k_dev || !v_dev || p < 0) return SH_EINVAL;
+    if (misaligned(q_dev) || misaligned(k_dev) || misaligned(v_dev)) return SH_EINVAL;
+    if (!h->slab || h->ragged) return SH_ESTATE;
+    if (h->n >= h->B) return SH_EFULL;
+    if (h->t + p >= (1 << 24)) return SH_EINVAL;
+    return prefill_range(h, static_cast<const char *>(q_dev), static_cast<const char *>(k_dev),
+                         static_cast<const char *>(v_dev), p, out_dev, (cudaStream_t)stream);
+}
+
+int sh_prefill_ragged(sh_handle h, const void *q_dev, const void *k_dev, const void *v_dev, int p_max,
+                      const int *lengths_host, int n_sequences, float *out_dev, void *stream) {
+    if (!h || !q_dev || !k_dev || !v_dev || !lengths_host || p_max < 0 || n_sequences < 1) return SH_EINVAL;
+    if (misaligned(q_dev) || misaligned(k_dev) || misaligned(v_dev)) return SH_EINVAL;
+    if (!h->slab) return SH_ESTATE;
+    if (h->ragged || h->t != 0 || h->n != 0) return SH_ESTATE;       // a fresh handle only
+    if (h->record_mode) return SH_EINVAL;                            // the recompute variant assumes one schedule
+    if (h->U % n_sequences) return SH_EINVAL;
+    for (int sq = 0; sq < n_sequences; ++sq)
+        if (lengths_host[sq] < 0 || lengths_host[sq] > p_max) return SH_EINVAL;
+    if (p_max >= (1 << 24)) return SH_EINVAL;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int ups = h->U / n_sequences;
+    h->units_per_seq = ups;
+    h->n_seq.assign(n_sequences, 0);
+    h->t_seq.assign(n_sequences, 0);
+    long long t_max = 0;
+    int rc = SH_OK;
+    for (int sq = 0; sq < n_sequences && rc == SH_OK; ++sq) {
+        // this sequence's units alone, with its own n and t: the uniform machinery on a sub-range
+        h->u0 = sq * ups; h->ucount = ups; h->n = 0; h->t = 0;
+        const size_t in_off = (size_t)h->u0 * h->in_bytes;
+        rc = prefill_range(h, static_cast<const char *>(q_dev) + in_off, static_cast<const char *>(k_dev) + in_off,
+                           static_cast<const char *>(v_dev) + in_off, lengths_host[sq],
+                           out_dev ? out_dev + (size_t)h->u0 * h->D : nullptr, s);
+        if (rc != SH_OK) break;
+        h->n_seq[sq] = h->n;
+        h->t_seq[sq] = h->t;
+        if (h->t > t_max) t_max = h->t;
+        int *na = reinterpret_cast<int *>(h->slab + h->L.n_arr) + h->u0;
+        int *ta = reinterpret_cast<int *>(h->slab + h->L.t_arr) + h->u0;
+        sh_fill_counts_kernel<<<(ups + 255) / 256, 256, 0, s>>>(na, ta, ups, h->n, (int)h->t);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) rc = cuda_fail(h, e);
+        else h->launches += 1;
+    }
+    h->u0 = 0; h->ucount = h->U;
+    h->n = 0;
+    h->t = t_max;
+    if (rc != SH_OK) return rc;
+    h->ragged = true;
+    h->started = true;
+    return SH_OK;
+}
+
+int sh_sequence_state(sh_handle h, int *n_host, long long *t_host, int capacity) {
+    if (!h || capacity < 0) return SH_EINVAL;
+    if (!h->ragged) {
+        if (capacity >= 1) { if (n_host) n_host[0] = h->n; if (t_host) t_host[0] = h->t; }
+        return 1;
+    }
+    const int ns = (int)h->n_seq.size();
+    for (int i = 0; i < ns && i < capacity; ++i) {
+        if (n_host) n_host[i] = h->n_seq[i];
+        if (t_host) t_host[i] = h->t_seq[i];
+    }
+    return ns;
 }
 
 int sh_recompute_record(sh_handle h, void *stream) {
@@ -382,7 +485,7 @@ int sh_compress(sh_handle h, void *stream, int *evicted_per_unit) {
     if (!h) return SH_EINVAL;
     if (!h->slab) return SH_ESTATE;
     if (evicted_per_unit) *evicted_per_unit = 0;
-    if (h->n < h->B) return SH_OK;
+    if (!sh_compression_due(h)) return SH_OK;
     int rc = do_compress(h, (cudaStream_t)stream);
     if (rc == SH_OK && evicted_per_unit) *evicted_per_unit = h->m;
     return rc;
@@ -408,7 +511,7 @@ int sh_state(sh_handle h, void *stream, int *n_out, long long *t_out, int32_t *p
     if (!h->slab) return SH_ESTATE;
     cudaStream_t s = (cudaStream_t)stream;
     cudaError_t e;
-    if (n_out) *n_out = h->n;
+    if (n_out) *n_out = h->ragged ? -1 : h->n;      // sequences differ: see sh_sequence_state
     if (t_out) *t_out = h->t;
     const size_t U = h->U, B = h->B;
     if (pos_host) {
@@ -418,17 +521,22 @@ int sh_state(sh_handle h, void *stream, int *n_out, long long *t_out, int32_t *p
     if (counters_host) {
         uint16_t *cd = reinterpret_cast<uint16_t *>(h->slab + h->L.counters);
         e = sh_launch_counters(reinterpret_cast<const uint32_t *>(h->slab + h->L.hist), cd, h->U, h->B, h->Bw, h->w,
-                               h->n, s, &h->launches);
+                               h->n, sh_pnarr(h), s, &h->launches);
         if (e != cudaSuccess) return cuda_fail(h, e);
         e = cudaMemcpyAsync(counters_host, cd, U * B * 2, cudaMemcpyDeviceToHost, s);
         if (e != cudaSuccess) return cuda_fail(h, e);
     }
     if (low_host) {
-        const int row = (int)(h->t % h->w);
-        const char *src = h->slab + h->L.hist + (size_t)row * h->Bw * 4;
-        e = cudaMemcpy2DAsync(low_host, (size_t)h->Bw * 4, src, (size_t)h->w * h->Bw * 4, (size_t)h->Bw * 4, U,
-                              cudaMemcpyDeviceToHost, s);
-        if (e != cudaSuccess) return cuda_fail(h, e);
+        // the bit-plane row of each sequence's own last step
+        const size_t row_b = (size_t)h->Bw * 4, unit_b = (size_t)h->w * row_b;
+        const int nsq = h->ragged ? (int)h->t_seq.size() : 1, ups = h->ragged ? h->units_per_seq : h->U;
+        for (int sq = 0; sq < nsq; ++sq) {
+            const int row = (int)((h->ragged ? h->t_seq[sq] : h->t) % h->w);
+            const char *src = h->slab + h->L.hist + (size_t)sq * ups * unit_b + (size_t)row * row_b;
+            e = cudaMemcpy2DAsync(reinterpret_cast<char *>(low_host) + (size_t)sq * ups * row_b, row_b, src, unit_b, row_b,
+                                  ups, cudaMemcpyDeviceToHost, s);
+            if (e != cudaSuccess) return cuda_fail(h, e);
+        }
     }
     int dev_err = 0;
     e = cudaMemcpyAsync(&dev_err, h->slab + h->L.err, sizeof(int), cudaMemcpyDeviceToHost, s);
@@ -466,6 +574,8 @@ int sh_restore(sh_handle h, int n, long long t) {
     h->t = t;
     h->started = true;
     h->record_fresh_t = -1;
+    h->ragged = false;
+    h->n_seq.clear(); h->t_seq.clear();
     return SH_OK;
 }
 

@@ -54,6 +54,7 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
     uint32_t *planes = reinterpret_cast<uint32_t *>(cut + 2);   // [w * Bw] when staged, then [G][5][Bw] partial sums
     const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
     const int n = p.n, ncand = p.n - p.r, m = p.m;
+    if (p.n_arr && p.n_arr[u] != n) return;      // this unit's cache is not full (whole CTA leaves)
 
     for (int i = tid; i <= p.cmax; i += SEL_THREADS) bins[i] = 0;
     if (FROM_HIST) {
@@ -164,6 +165,7 @@ __global__ void __launch_bounds__(ROWS_THREADS) sh_compact_rows_kernel(const Com
     __shared__ int first_moved;
     const int u = blockIdx.x, what = blockIdx.y, tid = threadIdx.x;
     const int n_keep = p.n - p.m, rb = p.row_bytes;
+    if (p.n_arr && p.n_arr[u] != p.n) return;    // this unit's cache is not full (whole CTA leaves)
     const int32_t *src = p.src_idx + (size_t)u * p.B;
     char *rows = (what == 0 ? p.K : p.V) + (size_t)u * p.B * rb;
 
@@ -252,6 +254,7 @@ __global__ void __launch_bounds__(CMP_THREADS) sh_compact_record_kernel(const Co
     extern __shared__ uint32_t rec_sm[];
     const int u = blockIdx.x, tid = threadIdx.x;
     const int n_keep = p.n - p.m, Bw = p.Bw, w = p.w;
+    if (p.n_arr && p.n_arr[u] != p.n) return;        // this unit's cache is not full (whole CTA leaves)
     const int stride = Bw | 1;                       // odd row stride: no bank conflicts
     const int32_t *src = p.src_idx + (size_t)u * p.B;
     uint32_t *hist_u = p.hist + (size_t)u * w * Bw;
@@ -314,11 +317,13 @@ __global__ void __launch_bounds__(CMP_THREADS) sh_compact_record_kernel(const Co
         __syncthreads();
         if (d < p.n) pos[d] = val;
     }
+    if (p.n_arr && tid == 0) p.n_arr[u] = n_keep;    // last kernel of the compression: the unit is compacted
 }
 
 __global__ void __launch_bounds__(256) sh_counters_kernel(const uint32_t *hist, uint16_t *counters, int B, int Bw,
-                                                          int w, int n) {
+                                                          int w, int n_all, const int *n_arr) {
     const int u = blockIdx.x;
+    const int n = n_arr ? n_arr[u] : n_all;
     for (int j = threadIdx.x; j < B; j += blockDim.x) {
         int I = 0;
         if (j < n) I = slot_counter(hist + (size_t)u * w * Bw, w, Bw, j);
@@ -392,8 +397,8 @@ cudaError_t sh_launch_compact(const CompactParams &p_in, cudaStream_t s, long lo
 }
 
 cudaError_t sh_launch_counters(const uint32_t *hist, uint16_t *counters, int U, int B, int Bw, int w, int n,
-                               cudaStream_t s, long long *launches) {
-    sh_counters_kernel<<<U, 256, 0, s>>>(hist, counters, B, Bw, w, n);
+                               const int *n_arr, cudaStream_t s, long long *launches) {
+    sh_counters_kernel<<<U, 256, 0, s>>>(hist, counters, B, Bw, w, n, n_arr);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess && launches) *launches += 1;
     return e;

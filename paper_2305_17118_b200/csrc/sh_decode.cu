@@ -307,7 +307,16 @@ __global__ void __launch_bounds__(NW * 32) sh_decode_kernel(const DecodeParams p
     const int sub = lane / LPR, c = lane % LPR;
     const int u = blockIdx.x / S;
     const int cr = (S > 1) ? (int)(blockIdx.x % S) : 0;
-    const int n = p.n, n_old = p.n - 1, B = p.B;
+    const int B = p.B;
+    // live rows including this step's token, the step number and its bit-plane row: the same for
+    // every unit (kernel arguments) unless the handle serves sequences of different lengths
+    int n = p.n, t_step = p.t, hist_row = p.hist_row;
+    if (p.n_arr) {
+        n = p.n_arr[u] + 1;
+        t_step = p.t_arr[u] + 1;
+        hist_row = t_step % p.w;
+    }
+    const int n_old = n - 1;
 
     int chunk, lo;
     if constexpr (S > 1) {
@@ -336,7 +345,7 @@ __global__ void __launch_bounds__(NW * 32) sh_decode_kernel(const DecodeParams p
     typename E::Q qv;
     E::load_q(reinterpret_cast<const char *>(p.q) + (size_t)u * INB, c, qv);
     if (!Q4 && p.qring && warp == 0 && sub == 0 && cr == 0)     // remembered for a recount at compression time
-        st_plain(p.qring + ((size_t)u * p.w + p.hist_row) * INB + c * 16,
+        st_plain(p.qring + ((size_t)u * p.w + hist_row) * INB + c * 16,
                  ld_plain(reinterpret_cast<const char *>(p.q) + (size_t)u * INB + c * 16));
 
     const char *Kb = p.K + (size_t)u * B * ROWB;
@@ -420,7 +429,7 @@ __global__ void __launch_bounds__(NW * 32) sh_decode_kernel(const DecodeParams p
         const float s = a * p.scale_log2e;
         if (lane == 0) s_sh[n_old - lo] = s;
         lmax = fmaxf(lmax, s);
-        if (lane == 0) p.pos[(size_t)u * B + n_old] = p.t;
+        if (lane == 0) p.pos[(size_t)u * B + n_old] = t_step;
     }
 
     // ---- max over the unit
@@ -517,8 +526,8 @@ __global__ void __launch_bounds__(NW * 32) sh_decode_kernel(const DecodeParams p
 
     // ---- record: low_j = [alpha_j < 1/t] = [e_j * t < L], one bit-plane row per step
     {
-        const float tf = (float)p.t;
-        uint32_t *hrow = p.hist + ((size_t)u * p.w + p.hist_row) * p.Bw;
+        const float tf = (float)t_step;
+        uint32_t *hrow = p.hist + ((size_t)u * p.w + hist_row) * p.Bw;
         const int w_lo = lo >> 5;
         const int w_hi = (S > 1 && cr != S - 1) ? min(p.Bw, (lo + chunk) >> 5) : p.Bw;
         for (int wd = w_lo + warp; wd < w_hi; wd += NW) {
@@ -533,6 +542,10 @@ __global__ void __launch_bounds__(NW * 32) sh_decode_kernel(const DecodeParams p
         // peers may still be reading this CTA's shared memory
         cg::this_cluster().sync();
     }
+    if (p.n_arr && tid == 0 && cr == 0) {    // every CTA of the unit has read the old values
+        p.n_arr[u] = n;
+        p.t_arr[u] = t_step;
+    }
 }
 
 template <int DT, int D, int NW, int R, int S>
@@ -546,7 +559,7 @@ cudaError_t launch_one(const sh_context *c, const DecodeParams &p, cudaStream_t 
         if (e != cudaSuccess) return e;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(c->U * S), 1, 1);
+    cfg.gridDim = dim3((unsigned)(p.U * S), 1, 1);
     cfg.blockDim = dim3(NW * 32, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
@@ -580,7 +593,7 @@ cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStr
     // caller asked for this one or for a cluster split, or there are too few units to give
     // most SMs one; the other shapes and dtypes use this file's.
     if (c->kernel != 1 && sh_decode_tma_supported(c) &&
-        (c->kernel == 2 || (c->U >= 128 && !(c->split_explicit && c->split > 1))))
+        (c->kernel == 2 || (p.U >= 128 && !(c->split_explicit && c->split > 1))))
         return sh_launch_decode_tma(c, p, s, launches);
     cudaError_t e = cudaErrorInvalidValue;
 #ifndef SH_DECODE_NW

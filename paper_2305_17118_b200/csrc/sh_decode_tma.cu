@@ -118,7 +118,7 @@ __global__ void __launch_bounds__(NWC * 32 + 32, CPS) sh_decode_tma_kernel(const
     __shared__ __align__(8) uint64_t full[NST], empty[NST];
     __shared__ int drain;                   // set once any bounded wait has given up
     __shared__ int issued;                  // tiles the producer has armed
-    const int B = p.B, n = p.n, n_old = p.n - 1;
+    const int B = p.B;
     const int capw = (B + 31) & ~31;
     unsigned char *ring = smem;
     float *s_all = reinterpret_cast<float *>(smem + (size_t)NST * STAGE);   // [2][capw] scaled logits
@@ -126,7 +126,9 @@ __global__ void __launch_bounds__(NWC * 32 + 32, CPS) sh_decode_tma_kernel(const
     float *ml = part + 2 * NWC * D;                                         // [2][NWC][2] (max, sum)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int ntiles = n_old > 0 ? (n_old + SR - 1) / SR : 1;   // the first tile also carries q and the new token
+    // rows already cached for unit u (the same for all units unless sequences differ in length)
+    auto cached_rows = [&](int u) { return p.n_arr ? p.n_arr[u] : p.n - 1; };
+    auto tiles_of = [](int n_old) { return n_old > 0 ? (n_old + SR - 1) / SR : 1; };   // the first tile also carries q and the new token
 
     if (tid == 0) {
         for (int s = 0; s < NST; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], NWC); }
@@ -145,6 +147,7 @@ __global__ void __launch_bounds__(NWC * 32 + 32, CPS) sh_decode_tma_kernel(const
             for (int u = blockIdx.x; u < p.U && !stop; u += gridDim.x) {
                 const char *Kb = p.K + (size_t)u * B * ROWB;
                 const char *Vb = p.V + (size_t)u * B * ROWB;
+                const int n_old = cached_rows(u), ntiles = tiles_of(n_old);
                 for (int tl = 0; tl < ntiles; ++tl) {
                     if (it >= NST && !mbar_wait(&empty[s], ph, err, 2)) *(volatile int *)&drain = 1;
                     if (*(volatile int *)&drain) { stop = true; break; }
@@ -170,13 +173,16 @@ __global__ void __launch_bounds__(NWC * 32 + 32, CPS) sh_decode_tma_kernel(const
         // ------------------------------------------------------------ consumers
         const int sub = lane / LR, c = lane % LR;
         const int g = warp * RPW + sub;                 // row group of this lane
-        const float tf = (float)p.t;
         const float sc = p.scale_log2e;
         int s = 0, par = 0;
         uint32_t ph = 0;
         bool dead = false;                              // this thread has given up a wait: touch no more data
         for (int u = blockIdx.x; u < p.U; u += gridDim.x, par ^= 1) {
             float *s_sh = s_all + par * capw;
+            const int n_old = cached_rows(u), ntiles = tiles_of(n_old), n = n_old + 1;
+            const int t_step = p.t_arr ? p.t_arr[u] + 1 : p.t;
+            const int hist_row = p.t_arr ? t_step % p.w : p.hist_row;
+            const float tf = (float)t_step;
             uint4 qraw[CH];
             float m_run = -INFINITY, l_run = 0.f;
             float acc[EL];
@@ -194,7 +200,7 @@ __global__ void __launch_bounds__(NWC * 32 + 32, CPS) sh_decode_tma_kernel(const
                     if (p.qring && warp == 0 && sub == 0 && !dead) {     // remembered for a recount at compression time
 #pragma unroll
                         for (int k = 0; k < CH; ++k)
-                            *reinterpret_cast<uint4 *>(p.qring + ((size_t)u * p.w + p.hist_row) * ROWB + (c + k * LR) * 16) = qraw[k];
+                            *reinterpret_cast<uint4 *>(p.qring + ((size_t)u * p.w + hist_row) * ROWB + (c + k * LR) * 16) = qraw[k];
                     }
                 }
                 // ---- this group's rows of the tile: K chunks -> partial dot, V chunks parked in registers
@@ -243,7 +249,7 @@ __global__ void __launch_bounds__(NWC * 32 + 32, CPS) sh_decode_tma_kernel(const
                         }
                         if (c == 0) {
                             s_sh[n_old] = s_new;
-                            p.pos[(size_t)u * B + n_old] = p.t;
+                            p.pos[(size_t)u * B + n_old] = t_step;
                         }
                     }
                 }
@@ -332,13 +338,17 @@ __global__ void __launch_bounds__(NWC * 32 + 32, CPS) sh_decode_tma_kernel(const
                 if (tid < D) p.out[(size_t)u * D + tid] = o / L;
             }
             // ---- record bits of every slot, one ballot word per 32 slots
-            uint32_t *hrow = p.hist + ((size_t)u * p.w + p.hist_row) * p.Bw;
+            uint32_t *hrow = p.hist + ((size_t)u * p.w + hist_row) * p.Bw;
             for (int wd = warp; wd < p.Bw; wd += NWC) {
                 const int j = (wd << 5) + lane;
                 bool low = false;
                 if (j < n && !dead) low = ex2(s_sh[j] - M) * tf < L;
                 const uint32_t word = __ballot_sync(0xffffffffu, low);
                 if (lane == 0) hrow[wd] = word;
+            }
+            if (p.n_arr && tid == 0) {      // all warps are past the barrier: everyone has used the old values
+                p.n_arr[u] = n;
+                p.t_arr[u] = t_step;
             }
         }
     }
@@ -366,7 +376,7 @@ cudaError_t launch_tma(const sh_context *c, const DecodeParams &p, cudaStream_t 
     int sms = 148;
     int dev = 0;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int grid = c->U < sms * CPS ? c->U : sms * CPS;
+    const int grid = p.U < sms * CPS ? p.U : sms * CPS;
     kern<<<grid, NWC * 32 + 32, smem, s>>>(p, reinterpret_cast<int *>(c->slab + c->L.err));
     return cudaGetLastError();
 }

@@ -4,6 +4,8 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "scissorhands.h"
 
 // Byte offsets of the regions inside the caller's workspace slab.
@@ -18,6 +20,7 @@ struct ShLayout {
     size_t stage_q, stage_k, stage_v, stage_out;  // staging for the *_host calls
     size_t err;             // one int: set by a kernel whose bounded wait gave up
     size_t qring;           // record_mode 1 only: [U][w][in_bytes] queries of the last w steps
+    size_t n_arr, t_arr;    // [U] int32 each: per-unit live rows / tokens streamed (sequences of different lengths)
     size_t total;
 };
 
@@ -42,7 +45,32 @@ struct sh_context {
     ShLayout L;
     long long launches;
     cudaError_t last_err;
+    // Active range of units: normally all of them.  While a ragged prompt is streamed, one
+    // sequence's units at a time, with n and t above holding for that sequence.
+    int u0, ucount;
+    // Sequences of different lengths (after sh_prefill_ragged): per-sequence mirrors of the
+    // device arrays n_arr / t_arr; units_per_seq consecutive units form a sequence.
+    bool ragged;
+    int units_per_seq;
+    std::vector<int> n_seq;
+    std::vector<long long> t_seq;
 };
+
+// Base pointers of the active unit range inside the workspace.
+inline char *sh_pK(const sh_context *c) { return c->slab + c->L.K + (size_t)c->u0 * c->B * c->row_bytes; }
+inline char *sh_pV(const sh_context *c) { return c->slab + c->L.V + (size_t)c->u0 * c->B * c->row_bytes; }
+inline char *sh_pKs(const sh_context *c) { return c->slab + c->L.Ks + (size_t)c->u0 * c->B * (c->D / 64) * 2; }
+inline char *sh_pVs(const sh_context *c) { return c->slab + c->L.Vs + (size_t)c->u0 * c->B * (c->D / 64) * 2; }
+inline uint32_t *sh_phist(const sh_context *c) {
+    return reinterpret_cast<uint32_t *>(c->slab + c->L.hist) + (size_t)c->u0 * c->w * c->Bw;
+}
+inline int32_t *sh_ppos(const sh_context *c) { return reinterpret_cast<int32_t *>(c->slab + c->L.pos) + (size_t)c->u0 * c->B; }
+inline int32_t *sh_psrc(const sh_context *c) { return reinterpret_cast<int32_t *>(c->slab + c->L.src_idx) + (size_t)c->u0 * c->B; }
+inline char *sh_pqring(const sh_context *c) {
+    return c->record_mode ? c->slab + c->L.qring + (size_t)c->u0 * c->w * c->in_bytes : nullptr;
+}
+inline int *sh_pnarr(const sh_context *c) { return c->ragged ? reinterpret_cast<int *>(c->slab + c->L.n_arr) + c->u0 : nullptr; }
+inline int *sh_ptarr(const sh_context *c) { return c->ragged ? reinterpret_cast<int *>(c->slab + c->L.t_arr) + c->u0 : nullptr; }
 
 struct DecodeParams {
     const void *q, *k_new, *v_new;
@@ -52,6 +80,8 @@ struct DecodeParams {
     uint32_t *hist;
     int32_t *pos;
     char *qring;    // [U][w][row] ring of the last w queries (row = step mod w), or NULL
+    int *n_arr, *t_arr;   // per-unit live rows / tokens streamed before this step (sequences of different
+                          // lengths), updated by the kernel; NULL when n and t below hold for every unit
     int U, B, Bw, w;
     int n;          // live rows per unit including the token appended by this step
     int hist_row;   // t mod w
@@ -66,6 +96,7 @@ struct SelectParams {
     int32_t *evicted;           // [U][m] or NULL
     int U, B, Bw, w, n, r, m;
     int cmax;                   // largest possible counter value
+    const int *n_arr;           // per-unit live rows, or NULL: units whose cache is not full are skipped
     int stage_planes;           // set by the launcher: copy the unit's bit-planes to shared memory first
 };
 
@@ -79,6 +110,8 @@ struct CompactParams {
     int chunk_bytes;            // set by the launcher: shared-memory gather buffer of the row kernel
     int rec_rows;               // set by the launcher: bit-plane rows staged per pass of the record kernel
     int *err;                   // device error word (a bounded wait gave up)
+    int *n_arr;                 // per-unit live rows, or NULL: units whose cache is not full are skipped;
+                                // the record kernel, which runs last, takes m off the ones it compacted
 };
 
 // Launchers (each returns the cudaError_t of its launch and adds to *launches).
@@ -90,10 +123,14 @@ cudaError_t sh_launch_decode_tma(const sh_context *c, const DecodeParams &p, cud
 int sh_prefill_chunk_capacity(const sh_context *c);
 cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const void *k, const void *v, float *out,
                                     int count, cudaStream_t s, long long *launches);
+// Host bookkeeping shared by the compression entry points: is a compression due (some cache full),
+// and the counter update once its kernels have been enqueued.
+bool sh_compression_due(const sh_context *c);
+void sh_after_compression(sh_context *c);
 cudaError_t sh_launch_recount(const sh_context *c, cudaStream_t s, long long *launches);
 // Recompute the record if the handle is in recompute mode and has not done so for the current step.
 int sh_recount_if_needed(sh_context *c, cudaStream_t s);
 cudaError_t sh_launch_select(const SelectParams &p, bool from_hist, cudaStream_t s, long long *launches);
 cudaError_t sh_launch_compact(const CompactParams &p, cudaStream_t s, long long *launches);
 cudaError_t sh_launch_counters(const uint32_t *hist, uint16_t *counters, int U, int B, int Bw, int w, int n,
-                               cudaStream_t s, long long *launches);
+                               const int *n_arr, cudaStream_t s, long long *launches);

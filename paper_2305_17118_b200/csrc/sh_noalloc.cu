@@ -49,7 +49,7 @@ extern "C" int sh_compress_static(sh_handle h, void *stream, int *evicted_per_un
     if (!h->slab) return SH_ESTATE;
     if (evicted_per_unit) *evicted_per_unit = 0;
     if ((size_t)h->U * (size_t)h->B > SH_STATIC_SCRATCH_ENTRIES) return SH_ETOOBIG;
-    if (h->n < h->B) return SH_OK;
+    if (!sh_compression_due(h)) return SH_OK;
     int32_t *src_idx = nullptr;
     cudaError_t e = scratch_address(&src_idx);
     if (e != cudaSuccess) { h->last_err = e; return SH_ECUDA; }
@@ -58,28 +58,30 @@ extern "C" int sh_compress_static(sh_handle h, void *stream, int *evicted_per_un
     if (rrc != SH_OK) return rrc;
 
     SelectParams sp = {};
-    sp.hist = reinterpret_cast<const uint32_t *>(h->slab + h->L.hist);
+    sp.hist = sh_phist(h);
     sp.counters = nullptr;
     sp.src_idx = src_idx;
     sp.evicted = nullptr;
-    sp.U = h->U; sp.B = h->B; sp.Bw = h->Bw; sp.w = h->w; sp.n = h->n; sp.r = h->r; sp.m = h->m;
+    sp.U = h->U; sp.B = h->B; sp.Bw = h->Bw; sp.w = h->w; sp.n = h->B; sp.r = h->r; sp.m = h->m;
     sp.cmax = h->w;
+    sp.n_arr = sh_pnarr(h);
     e = sh_launch_select(sp, true, s, &h->launches);
     if (e != cudaSuccess) { h->last_err = e; return SH_ECUDA; }
 
     CompactParams cp = {};
-    cp.K = h->slab + h->L.K; cp.V = h->slab + h->L.V;
-    cp.Ks = h->slab + h->L.Ks; cp.Vs = h->slab + h->L.Vs;
-    cp.hist = reinterpret_cast<uint32_t *>(h->slab + h->L.hist);
-    cp.pos = reinterpret_cast<int32_t *>(h->slab + h->L.pos);
+    cp.K = sh_pK(h); cp.V = sh_pV(h);
+    cp.Ks = sh_pKs(h); cp.Vs = sh_pVs(h);
+    cp.hist = sh_phist(h);
+    cp.pos = sh_ppos(h);
     cp.src_idx = src_idx;
-    cp.U = h->U; cp.B = h->B; cp.Bw = h->Bw; cp.w = h->w; cp.n = h->n; cp.m = h->m;
+    cp.U = h->U; cp.B = h->B; cp.Bw = h->Bw; cp.w = h->w; cp.n = h->B; cp.m = h->m;
+    cp.n_arr = sh_pnarr(h);
     cp.row_bytes = h->row_bytes;
     cp.scale_bytes = h->dtype == SH_INT4_G64_F16 ? (h->D / 64) * 2 : 0;
     cp.err = reinterpret_cast<int *>(h->slab + h->L.err);
     e = sh_launch_compact(cp, s, &h->launches);
     if (e != cudaSuccess) { h->last_err = e; return SH_ECUDA; }
-    h->n -= h->m;
+    sh_after_compression(h);
     if (evicted_per_unit) *evicted_per_unit = h->m;
     return SH_OK;
 }

@@ -76,6 +76,7 @@ struct ChunkParams {
     uint32_t *hist;
     int32_t *pos;
     int U, B, Bw, w;
+    int Utot;                // units of the whole handle: tokens of q/k/v/out are Utot rows apart
     int n0;                  // live rows before the chunk
     int c;                   // tokens in the chunk (<= CQ, <= w, n0 + c <= B)
     int t0;                  // tokens streamed before the chunk
@@ -133,7 +134,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
     const int step0 = RECOUNT ? p.first_step + (int)blockIdx.y * CQ : p.t0 + 1;
     const int c = RECOUNT ? min(CQ, p.nsteps - (int)blockIdx.y * CQ) : p.c;
     const int n_tot = RECOUNT ? p.n0 : p.n0 + p.c;
-    const size_t tstride = (size_t)p.U * D * 2;          // bytes between consecutive tokens of one unit
+    const size_t tstride = (size_t)p.Utot * D * 2;       // bytes between consecutive tokens of one unit
     const char *Kc = p.K + (size_t)u * p.B * D * 2;
     const char *Vc = p.V + (size_t)u * p.B * D * 2;
     const int ntiles = (n_tot + KT - 1) / KT;
@@ -313,7 +314,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
                     const float inv = 1.f / rowL[i];
                     const int col = wn * (D / WN) + nb * 8 + (lane & 3) * 2;
                     float2 o2 = make_float2(oacc[nb][2 * hrow] * inv, oacc[nb][2 * hrow + 1] * inv);
-                    *reinterpret_cast<float2 *>(p.out + ((size_t)i * p.U + u) * D + col) = o2;
+                    *reinterpret_cast<float2 *>(p.out + ((size_t)i * p.Utot + u) * D + col) = o2;
                 }
             }
         }
@@ -355,14 +356,14 @@ cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const vo
     ChunkParams p = {};
     p.q = static_cast<const char *>(q); p.k = static_cast<const char *>(k); p.v = static_cast<const char *>(v);
     p.out = out;
-    p.K = c->slab + c->L.K; p.V = c->slab + c->L.V;
-    p.hist = reinterpret_cast<uint32_t *>(c->slab + c->L.hist);
-    p.pos = reinterpret_cast<int32_t *>(c->slab + c->L.pos);
-    p.U = c->U; p.B = c->B; p.Bw = c->Bw; p.w = c->w;
+    p.K = sh_pK(c); p.V = sh_pV(c);
+    p.hist = sh_phist(c);
+    p.pos = sh_ppos(c);
+    p.U = c->ucount; p.Utot = c->U; p.B = c->B; p.Bw = c->Bw; p.w = c->w;
     p.n0 = c->n; p.c = count; p.t0 = (int)c->t;
     p.SS = s_stride(c->B);
     p.scale_log2e = (float)((double)c->scale * 1.4426950408889634);
-    p.qring = c->record_mode ? c->slab + c->L.qring : nullptr;
+    p.qring = sh_pqring(c);
     cudaError_t e = cudaErrorInvalidValue;
     if (count < 1 || count > sh_prefill_chunk_capacity(c)) return e;
     if (count <= 32) e = c->dtype == SH_F16 ? launch_chunk<SH_F16, 32, false>(p, s) : launch_chunk<SH_BF16, 32, false>(p, s);
@@ -375,14 +376,14 @@ cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const vo
 // present cache: rewrites the unit's bit-plane rows of those steps.
 cudaError_t sh_launch_recount(const sh_context *c, cudaStream_t s, long long *launches) {
     ChunkParams p = {};
-    p.K = c->slab + c->L.K; p.V = c->slab + c->L.V;
-    p.hist = reinterpret_cast<uint32_t *>(c->slab + c->L.hist);
-    p.pos = reinterpret_cast<int32_t *>(c->slab + c->L.pos);
-    p.U = c->U; p.B = c->B; p.Bw = c->Bw; p.w = c->w;
+    p.K = sh_pK(c); p.V = sh_pV(c);
+    p.hist = sh_phist(c);
+    p.pos = sh_ppos(c);
+    p.U = c->ucount; p.Utot = c->U; p.B = c->B; p.Bw = c->Bw; p.w = c->w;
     p.n0 = c->n; p.c = 0; p.t0 = (int)c->t;
     p.SS = s_stride(c->B);
     p.scale_log2e = (float)((double)c->scale * 1.4426950408889634);
-    p.qring = c->slab + c->L.qring;
+    p.qring = sh_pqring(c);
     p.nsteps = c->t < c->w ? (int)c->t : c->w;
     p.first_step = (int)c->t - p.nsteps + 1;
     if (p.nsteps < 1) return cudaSuccess;

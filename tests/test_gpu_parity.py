@@ -285,6 +285,74 @@ def test_snapshot_restore_replays_identically(sh):
     assert s1[0] == s2[0] and s1[1] == s2[1] and all((x == y).all() for x, y in zip(s1[2:], s2[2:]))
 
 
+@pytest.mark.parametrize("dtype,kernel", [("f16", None), ("bf16", 2), ("f16", 1), ("f32", None)])
+def test_ragged_sequences_lockstep(sh, dtype, kernel):
+    """Sequences of different prompt lengths in one handle (sh_prefill_ragged), then decode steps in
+    lockstep: one oracle per sequence, each with its own n, t and compression schedule."""
+    d = 128 if dtype != "f32" else 64
+    lengths = [0, 37, 150, 96, 211, 95]            # empty, short, several compressions, exactly full, long, one short of full
+    nseq, ups, B, r, w, m, T_dec = len(lengths), 3, 96, 8, 40, 30, 170
+    U, p_max = nseq * ups, max(lengths)
+    q, k, v = wl.random_stream(U, d, p_max + T_dec, seed=51, dtype=dtype, peaked=3.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, kernel=kernel)
+    out_p = torch.zeros(p_max, U, d, device="cuda")
+    h.prefill_ragged(q[:p_max].contiguous(), k[:p_max].contiguous(), v[:p_max].contiguous(), lengths, out_p)
+    orcs, ok = [], []
+    for sq in range(nseq):
+        o = oracle.Oracle(ups, B, r, w, m, d)
+        idx = torch.arange(sq * ups, (sq + 1) * ups, device="cuda")
+        for t in range(lengths[sq]):
+            oo, _ = o.step(to_oracle(q[t], idx), to_oracle(k[t], idx), to_oracle(v[t], idx))
+            assert np.abs(out_p[t][idx].double().cpu().numpy() - oo).max() <= TOL[dtype]
+        orcs.append(o)
+    n_seq, t_seq = h.sequence_state()
+    assert n_seq.tolist() == [o.n for o in orcs] and t_seq.tolist() == lengths
+    pos, cnt, _ = h.state_full()
+    for sq, o in enumerate(orcs):
+        sl = slice(sq * ups, (sq + 1) * ups)
+        same = (pos[sl, : o.n] == o.positions()).all() and (cnt[sl, : o.n].astype(np.int32) == o.counters()).all()
+        ok.append(bool(same))                     # a threshold-ambiguous flip in the prompt may change a kept set
+        assert (pos[sl, o.n:] == 0).all()
+    assert sum(ok) >= nseq - 1
+    compressions = 0
+    for step in range(T_dec):
+        ti = p_max + step
+        out = h.decode_step(q[ti], k[ti], v[ti])
+        pos, cnt, low = h.state_full()
+        for sq, o in enumerate(orcs):
+            if not ok[sq]:
+                continue
+            idx = torch.arange(sq * ups, (sq + 1) * ups, device="cuda")
+            sl = slice(sq * ups, (sq + 1) * ups)
+            oo, alpha, o_low, amb = o.attend(to_oracle(q[ti], idx), to_oracle(k[ti], idx), to_oracle(v[ti], idx))
+            assert np.abs(out[idx].double().cpu().numpy() - oo).max() <= TOL[dtype]
+            g_low = low[sl, : o.n]
+            assert not low[sl, o.n:].any()
+            diff = g_low != o_low
+            assert not (diff & ~amb).any(), f"sequence {sq}, step {step}: record bits differ outside the 1e-6 window"
+            o.record(g_low)
+            assert (pos[sl, : o.n] == o.positions()).all() and (cnt[sl, : o.n].astype(np.int32) == o.counters()).all()
+        n_seq, t_seq = h.sequence_state()
+        due = [sq for sq in range(nseq) if n_seq[sq] == B]
+        assert h.compress() == (m if due else 0)
+        if due:
+            compressions += 1
+            pos, cnt, _ = h.state_full()
+            for sq in due:
+                if not ok[sq]:
+                    continue
+                o = orcs[sq]
+                assert o.full
+                o.compress()
+                sl = slice(sq * ups, (sq + 1) * ups)
+                assert (pos[sl, : o.n] == o.positions()).all() and (pos[sl, o.n:] == 0).all()
+                assert (cnt[sl, : o.n].astype(np.int32) == o.counters()).all()
+        n_seq, t_seq = h.sequence_state()
+        assert all(n_seq[sq] == orcs[sq].n for sq in range(nseq) if ok[sq])
+        assert t_seq.tolist() == [lengths[sq] + step + 1 for sq in range(nseq)]
+    assert compressions >= 12                    # the sequences fill at different steps
+
+
 def test_persistence_diagnostics_match_oracle_scores(sh):
     """Persistence ratio and pivotal-set size (Section 3.2) from the library's record bits, against
     the same quantities from the oracle's fp64 scores on a full (never compressed) cache."""
