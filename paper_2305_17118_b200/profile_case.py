@@ -27,6 +27,7 @@ def main():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--rows", type=int, default=None, help="live rows before the first step")
     ap.add_argument("--compress", action="store_true")
+    ap.add_argument("--chunk", type=int, default=0, help="instead of decode steps, run one prompt chunk of this many tokens")
     ap.add_argument("--split", type=int, default=None)
     ap.add_argument("--kernel", type=int, default=None, help="1 direct loads, 2 pipelined bulk copies")
     args = ap.parse_args()
@@ -35,6 +36,8 @@ def main():
     torch.cuda.set_device(0)
     h = sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, U, d, cfg.dtype, split=args.split, kernel=args.kernel, auto_compress=True)
     rows = args.rows if args.rows is not None else (cfg.B - 1 if args.compress else cfg.B - cfg.m // 2)
+    if args.chunk:
+        rows = args.rows if args.rows is not None else cfg.B - args.chunk
     # K then V sit at the start of the workspace, [U][B][row_bytes] each.
     row_bytes = {"f32": 4 * d, "f16": 2 * d, "bf16": 2 * d, "int4": d // 2}[cfg.dtype]
     kv = h.slab[h._slab_off: h._slab_off + 2 * U * cfg.B * row_bytes]
@@ -50,6 +53,20 @@ def main():
     x = torch.randn(3, args.steps, U, d, generator=g, device="cuda").to(cfg.torch_dtype)
     out = torch.empty(U, d, device="cuda")
     torch.cuda.synchronize()
+    if args.chunk:
+        c = args.chunk
+        xc = torch.randn(3, c, U, d, generator=g, device="cuda").to(cfg.torch_dtype)
+        oc = torch.empty(c, U, d, device="cuda")
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        h.prefill_chunk(xc[0], xc[1], xc[2], oc)
+        b.record()
+        torch.cuda.synchronize()
+        flops = 2 * 2 * c * (rows + (c + 1) / 2) * d * U
+        byts = U * (2 * rows * row_bytes + 3 * c * row_bytes + c * d * 4)
+        print(f"chunk of {c} tokens over {rows} cached rows: {a.elapsed_time(b) * 1e3:.1f} us, "
+              f"{flops / 1e9:.1f} GFLOP (algorithmic), {byts / 1e6:.1f} MB")
+        return
     for i in range(args.steps):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
