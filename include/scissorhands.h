@@ -80,7 +80,7 @@ typedef enum {
  * B = token budget per unit, r = recent window (never evicted), w = history
  * window of the importance record in steps, m = tokens dropped per
  * compression, heads = number of units, head_dim = d.
- * Requires B >= 1, r >= 0, 1 <= w <= 16384, 1 <= m <= B - r, B <= 65535,
+ * Requires 1 <= B <= 32768, r >= 0, 1 <= w <= 16384, 1 <= m <= B - r,
  * head_dim in {64, 128} (int4: 128 or 64), dtype an sh_dtype.
  * Errors: SH_EINVAL, SH_ENOMEM.
  */

@@ -183,7 +183,8 @@ extern "C" {
 int sh_create(int B, int r, int w, int m, int heads, int head_dim, int dtype, sh_handle *out) {
     if (!out) return SH_EINVAL;
     *out = nullptr;
-    if (B < 1 || B > 65535 || r < 0 || w < 1 || w > 16384 || m < 1 || m > B - r || heads < 1) return SH_EINVAL;
+    // B is bounded by the shared memory that holds one unit's logits (4 bytes per slot)
+    if (B < 1 || B > 32768 || r < 0 || w < 1 || w > 16384 || m < 1 || m > B - r || heads < 1) return SH_EINVAL;
     if (head_dim != 64 && head_dim != 128) return SH_EINVAL;
     if (dtype < SH_F32 || dtype > SH_INT4_G64_F16) return SH_EINVAL;
     sh_context *c = new (std::nothrow) sh_context();

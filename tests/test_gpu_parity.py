@@ -38,10 +38,10 @@ def test_lockstep_small(sh, dtype, d, split):
 
 
 @pytest.mark.parametrize("B,r,w,m", [(33, 0, 1, 33), (64, 63, 5, 1), (32, 4, 100, 7), (1000, 10, 400, 500),
-                                     (2, 1, 3, 1), (97, 5, 64, 92)])
+                                     (2, 1, 3, 1), (97, 5, 64, 92), (3000, 10, 400, 1500)])
 def test_lockstep_edge_parameters(sh, B, r, w, m):
     U, d, dtype = 3, 64, "f16"
-    T = min(3 * B + 50, 1300)
+    T = min(3 * B + 50, 1300) if B <= 1000 else B + 100
     q, k, v = wl.random_stream(U, d, T, seed=B, dtype=dtype, peaked=2.0, device="cuda")
     h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
     res, _ = run_lockstep(h, dtype, _stream_fn(q, k, v), T, torch.arange(U), TOL[dtype])
@@ -114,6 +114,20 @@ def test_recompute_mode_through_prefill_and_automatic_compression(sh):
     same = (pos == orc.positions()).all(axis=1)
     assert same.mean() >= 0.75          # units without a threshold-ambiguous flip agree exactly
     assert worst <= TOL[dtype] or same.mean() < 1.0
+
+
+def test_paper_hyperparameters_chunked_prompt_then_decode(sh):
+    """The values the paper uses in all its experiments (Section 4.1: r = 10, w = 400, m = 0.5 B), on a
+    budget large enough that the chunk kernel has to fall back to 32 queries per launch."""
+    U, d, B, r, w, m, dtype = 3, 128, 600, 10, 400, 300, "bf16"
+    T = B + 2 * m + 40
+    q, k, v = wl.random_stream(U, d, T + 60, seed=61, dtype=dtype, peaked=3.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    assert h.prefill_chunk_max == 32
+    blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
+    res, orc = run_lockstep_chunked(h, dtype, blk, T, torch.arange(U), TOL[dtype])
+    assert res.compressions == 3
+    run_lockstep(h, dtype, _stream_fn(q, k, v), 60, torch.arange(U), TOL[dtype], orc=orc)
 
 
 def test_prefill_uses_chunks_and_matches_oracle(sh):
