@@ -38,6 +38,13 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void *
                  : "r"(smem_addr(row_ptr)));
 }
 
+// 2^x (one MUFU instruction; 2^-inf = 0)
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 template <int DT> struct Mma;
 template <> struct Mma<SH_F16> {
     static __device__ __forceinline__ void run(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
@@ -113,7 +120,7 @@ __device__ __forceinline__ void load_tile_async(uint16_t *tile, const char *cach
 // CQ queries per CTA (64 or 32).  Warps form a WM x WN grid: WM row blocks of 16 queries,
 // WN groups that split the 64 keys of a tile (logits) or the 128 output columns (P.V).
 template <int DT, int CQ, bool RECOUNT>
-__global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const ChunkParams p) {
+__global__ void __launch_bounds__(NTHREADS, CQ == 32 ? 2 : 1) sh_prefill_chunk_kernel(const ChunkParams p) {
     constexpr int WM = CQ / 16, WN = 8 / WM;
     constexpr int NBK = KT / WN / 8;     // 8-key blocks per warp in the logits phase
     constexpr int NBD = D / WN / 8;      // 8-column blocks per warp in the P.V phase
@@ -131,9 +138,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
     const int wm = warp % WM, wn = warp / WM;
     const int n0 = p.n0, SS = p.SS;
     // first step handled by this CTA and how many
-    const int step0 = RECOUNT ? p.first_step + (int)blockIdx.y * CQ : p.t0 + 1;
-    const int c = RECOUNT ? min(CQ, p.nsteps - (int)blockIdx.y * CQ) : p.c;
-    const int n_tot = RECOUNT ? p.n0 : p.n0 + p.c;
+    // blockIdx.y selects CQ consecutive queries (of the window in recount mode, of the chunk otherwise)
+    const int qoff = (int)blockIdx.y * CQ;
+    const int step0 = (RECOUNT ? p.first_step : p.t0 + 1) + qoff;
+    const int c = min(CQ, (RECOUNT ? p.nsteps : p.c) - qoff);
+    // keys this CTA needs: the cache, and the chunk's tokens up to its own last query
+    const int n_tot = RECOUNT ? p.n0 : p.n0 + qoff + c;
     const size_t tstride = (size_t)p.Utot * D * 2;       // bytes between consecutive tokens of one unit
     const char *Kc = p.K + (size_t)u * p.B * D * 2;
     const char *Vc = p.V + (size_t)u * p.B * D * 2;
@@ -148,7 +158,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
             if (RECOUNT) {
                 val = *reinterpret_cast<const uint4 *>(ring_row);
             } else {
-                val = *reinterpret_cast<const uint4 *>(p.q + (size_t)row * tstride + (size_t)u * D * 2 + ch * 16);
+                val = *reinterpret_cast<const uint4 *>(p.q + (size_t)(qoff + row) * tstride + (size_t)u * D * 2 + ch * 16);
                 if (ring_row) *reinterpret_cast<uint4 *>(ring_row) = val;     // remembered for a later recount
             }
         }
@@ -166,13 +176,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
             nvs[i] = lo;
         }
     } else {
-        for (int i = tid; i < CQ; i += NTHREADS) nvs[i] = (i < c) ? n0 + i + 1 : 0;
-        if (tid < c) p.pos[(size_t)u * p.B + n0 + tid] = p.t0 + tid + 1;
+        for (int i = tid; i < CQ; i += NTHREADS) nvs[i] = (i < c) ? n0 + qoff + i + 1 : 0;
+        if (tid < c) p.pos[(size_t)u * p.B + n0 + qoff + tid] = step0 + tid;
         // append the chunk's keys and values to the cache (nothing in this launch reads them back from there)
         for (int idx = tid; idx < c * (D / 8); idx += NTHREADS) {
             const int row = idx / (D / 8), ch = idx % (D / 8);
-            const size_t src = (size_t)row * tstride + (size_t)u * D * 2 + ch * 16;
-            const size_t dst = ((size_t)u * p.B + n0 + row) * (D * 2) + ch * 16;
+            const size_t src = (size_t)(qoff + row) * tstride + (size_t)u * D * 2 + ch * 16;
+            const size_t dst = ((size_t)u * p.B + n0 + qoff + row) * (D * 2) + ch * 16;
             *reinterpret_cast<uint4 *>(p.K + dst) = *reinterpret_cast<const uint4 *>(p.k + src);
             *reinterpret_cast<uint4 *>(p.V + dst) = *reinterpret_cast<const uint4 *>(p.v + src);
         }
@@ -238,7 +248,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
         for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
         float sum = 0.f;
         for (int j = lane; j < ntiles * KT; j += 32) {
-            const float e = (j < nv) ? exp2f(Si[j] - mx) : 0.f;
+            const float e = (j < nv) ? ex2_approx(Si[j] - mx) : 0.f;
             Si[j] = e;
             sum += e;
         }
@@ -314,7 +324,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) sh_prefill_chunk_kernel(const Chu
                     const float inv = 1.f / rowL[i];
                     const int col = wn * (D / WN) + nb * 8 + (lane & 3) * 2;
                     float2 o2 = make_float2(oacc[nb][2 * hrow] * inv, oacc[nb][2 * hrow + 1] * inv);
-                    *reinterpret_cast<float2 *>(p.out + ((size_t)i * p.Utot + u) * D + col) = o2;
+                    *reinterpret_cast<float2 *>(p.out + ((size_t)(qoff + i) * p.Utot + u) * D + col) = o2;
                 }
             }
         }
@@ -328,7 +338,7 @@ cudaError_t launch_chunk(const ChunkParams &p, cudaStream_t s) {
     auto kern = sh_prefill_chunk_kernel<DT, CQ, RECOUNT>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    const unsigned gy = RECOUNT ? (unsigned)((p.nsteps + CQ - 1) / CQ) : 1u;
+    const unsigned gy = (unsigned)(((RECOUNT ? p.nsteps : p.c) + CQ - 1) / CQ);
     kern<<<dim3(p.U, gy, 1), NTHREADS, smem, s>>>(p);
     return cudaGetLastError();
 }
@@ -344,8 +354,7 @@ size_t smem_need(int CQ, int B) {
 int sh_prefill_chunk_capacity(const sh_context *c) {
     if ((c->dtype != SH_F16 && c->dtype != SH_BF16) || c->D != 128) return 0;
     int cq = 0;
-    if (smem_need(64, c->B) <= 200 * 1024) cq = 64;
-    else if (smem_need(32, c->B) <= 200 * 1024) cq = 32;
+    if (smem_need(32, c->B) <= 200 * 1024) cq = 64;      // one or two CTAs of 32 queries, or one of 64
     if (cq > c->w) cq = c->w;     // every step of a chunk needs its own bit-plane row
     return cq;
 }
@@ -366,7 +375,12 @@ cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const vo
     p.qring = sh_pqring(c);
     cudaError_t e = cudaErrorInvalidValue;
     if (count < 1 || count > sh_prefill_chunk_capacity(c)) return e;
-    if (count <= 32) e = c->dtype == SH_F16 ? launch_chunk<SH_F16, 32, false>(p, s) : launch_chunk<SH_BF16, 32, false>(p, s);
+    // 32 queries per CTA when two such CTAs fit on an SM (the second half of a longer chunk goes to a
+    // sibling CTA that re-reads the keys): more warps in flight hide the latencies of this kernel better
+    // than sharing the K/V tiles between 64 queries does
+    const bool two_per_sm = smem_need(32, c->B) <= 112 * 1024;
+    if (count <= 32 || two_per_sm || smem_need(64, c->B) > 200 * 1024)
+        e = c->dtype == SH_F16 ? launch_chunk<SH_F16, 32, false>(p, s) : launch_chunk<SH_BF16, 32, false>(p, s);
     else e = c->dtype == SH_F16 ? launch_chunk<SH_F16, 64, false>(p, s) : launch_chunk<SH_BF16, 64, false>(p, s);
     if (e == cudaSuccess) *launches += 1;
     return e;

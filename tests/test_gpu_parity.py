@@ -123,7 +123,7 @@ def test_paper_hyperparameters_chunked_prompt_then_decode(sh):
     T = B + 2 * m + 40
     q, k, v = wl.random_stream(U, d, T + 60, seed=61, dtype=dtype, peaked=3.0, device="cuda")
     h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
-    assert h.prefill_chunk_max == 32
+    assert h.prefill_chunk_max == 64
     blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
     res, orc = run_lockstep_chunked(h, dtype, blk, T, torch.arange(U), TOL[dtype])
     assert res.compressions == 3
