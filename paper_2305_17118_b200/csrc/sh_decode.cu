@@ -1,5 +1,8 @@
 // Fused decode step: append + logits + stable softmax + P.V + importance-record
-// bits, one CTA (or one cluster of S CTAs) per (sequence, head) unit.
+// bits, one CTA (or one cluster of S CTAs) per (sequence, head) unit.  This is
+// the kernel for fp32 and int4 stores, head_dim 64, and launches with few units;
+// fp16/bf16 rows of 256 bytes at scale go through the pipelined kernel of
+// sh_decode_tma.cu (sh_launch_decode picks).
 //
 // The work is a GEMV per unit (one query against n cached rows), so it is bound
 // by HBM bandwidth and runs on CUDA cores.  Layout of the work inside a CTA:

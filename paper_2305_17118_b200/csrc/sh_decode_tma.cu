@@ -9,8 +9,8 @@
 // (bounded by registers, drained at every CTA boundary) cannot.  A read-only
 // stream measured 7.1 TB/s on B200 this way.
 //
-// Per unit each group of LPR lanes (one stored row = LPR x 16 bytes) keeps its
-// own running softmax state (max, sum, weighted V sum) over the rows it is
+// Per unit each group of LR lanes (a stored row is split over LR lanes, two
+// 16-byte chunks each for 256-byte rows) keeps its own running softmax state (max, sum, weighted V sum) over the rows it is
 // dealt, flash-decoding style, so K and V tiles are consumed together and no
 // barrier sits between the logits and P.V.  Scaled logits are parked in shared
 // memory; once the groups' states are merged, the record bits
