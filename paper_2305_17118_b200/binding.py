@@ -174,6 +174,13 @@ class Handle:
                                             _stream_ptr(stream)))
         return out
 
+    def decode_step_host_raw(self, q_ptr: int, k_ptr: int, v_ptr: int, out_ptr: int, stream_ptr: int = 0):
+        """sh_decode_step_host on raw host addresses the caller has validated once (contiguous rows of
+        the handle's dtype, [heads, head_dim]; out fp32): no per-call tensor checks."""
+        rc = lib.sh_decode_step_host(self._h, q_ptr, k_ptr, v_ptr, out_ptr, stream_ptr)
+        if rc:
+            self._check(rc)
+
     # -- sh_prefill ------------------------------------------------------------
     def prefill(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: Optional[torch.Tensor] = None,
                 stream=None):
