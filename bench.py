@@ -283,7 +283,7 @@ def cuda_arm(args, cfg, rank, world):
     traffic = None
     try:
         with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
-            tr = json.load(f).get(cfg.name)
+            tr = json.load(f).get(cfg.name)      # shape variants have no capture: traffic stays null
             if tr:
                 traffic = tr["dram_bytes_per_unit_row"] * statistics.fmean(n_sched) * U
     except Exception:
@@ -373,11 +373,16 @@ def main():
     ap.add_argument("--kernel", type=int, default=None, help="decode kernel: 1 direct loads, 2 pipelined bulk copies")
     ap.add_argument("--recompute-record", action="store_true",
                     help="variant: rebuild the importance record at each compression from stored queries")
+    ap.add_argument("--kv-dtype", default=None, choices=["f32", "f16", "bf16", "int4"], help="override the workload's K/V dtype")
+    ap.add_argument("--head-dim", type=int, default=None, choices=[64, 128], help="override the workload's head_dim")
     ap.add_argument("--no-prefill-chunk", action="store_true", help="stream the prompt one decode step per token")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (tuning runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     cfg = wl.CONFIGS[args.config]
+    if args.kv_dtype or args.head_dim:      # shape variants of a named workload (not the benchmark's own lines)
+        cfg = cfg.scaled(name=f"{cfg.name}[{args.kv_dtype or cfg.dtype},d{args.head_dim or cfg.head_dim}]",
+                         dtype=args.kv_dtype or cfg.dtype, head_dim=args.head_dim or cfg.head_dim)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":

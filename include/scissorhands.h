@@ -72,7 +72,8 @@ typedef enum {
                                  kernel where the shape allows it; 0: one decode step per token */
     SH_OPT_DECODE_KERNEL = 3  /* 0 (default): chosen from the shape; 1: one CTA (or cluster) per unit with
                                  direct loads; 2: persistent CTAs fed by bulk asynchronous copies
-                                 (fp16/bf16 with head_dim 128 only, SH_OPT_SPLIT ignored; other shapes use 1) */
+                                 (stored rows of 256 bytes or more: fp32, and fp16/bf16 with head_dim 128; SH_OPT_SPLIT
+                                 ignored; other shapes use 1) */
 } sh_option;
 
 /*

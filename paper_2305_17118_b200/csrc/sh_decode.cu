@@ -1,8 +1,8 @@
 // Fused decode step: append + logits + stable softmax + P.V + importance-record
 // bits, one CTA (or one cluster of S CTAs) per (sequence, head) unit.  This is
-// the kernel for fp32 and int4 stores, head_dim 64, and launches with few units;
-// fp16/bf16 rows of 256 bytes at scale go through the pipelined kernel of
-// sh_decode_tma.cu (sh_launch_decode picks).
+// the kernel for the int4 store, for 16-bit stores with head_dim 64 and for
+// launches with few units; stores with rows of 256 bytes or more go through the
+// pipelined kernel of sh_decode_tma.cu at scale (sh_launch_decode picks).
 //
 // The work is a GEMV per unit (one query against n cached rows), so it is bound
 // by HBM bandwidth and runs on CUDA cores.  Layout of the work inside a CTA:
@@ -592,9 +592,8 @@ cudaError_t launch_split(const sh_context *c, const DecodeParams &p, cudaStream_
 }  // namespace
 
 cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches) {
-    // fp16/bf16 rows of 256 bytes stream through the persistent pipelined kernel unless the
-    // caller asked for this one or for a cluster split, or there are too few units to give
-    // most SMs one; the other shapes and dtypes use this file's.
+    // Rows of 256 bytes or more stream through the persistent pipelined kernel unless the caller
+    // asked for this one or for a cluster split, or there are too few units to give most SMs one.
     if (c->kernel != 1 && sh_decode_tma_supported(c) &&
         (c->kernel == 2 || (p.U >= 128 && !(c->split_explicit && c->split > 1))))
         return sh_launch_decode_tma(c, p, s, launches);

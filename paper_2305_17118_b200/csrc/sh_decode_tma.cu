@@ -45,6 +45,19 @@ __device__ __forceinline__ void ffma2(float &d0, float &d1, float a0, float a1, 
 //         separate conversions).
 //   axpy: acc[0..EPL) += p * v for one chunk: convert pairs, then packed fp32 FMAs.
 template <int DT> struct ElemT;
+template <> struct ElemT<SH_F32> {
+    static constexpr int EPL = 4, BYTES = 4;
+    static __device__ __forceinline__ void dot(const uint4 &q, const uint4 &k, float &a0, float &a1) {
+        a0 = fmaf(__uint_as_float(q.x), __uint_as_float(k.x), a0);
+        a1 = fmaf(__uint_as_float(q.y), __uint_as_float(k.y), a1);
+        a0 = fmaf(__uint_as_float(q.z), __uint_as_float(k.z), a0);
+        a1 = fmaf(__uint_as_float(q.w), __uint_as_float(k.w), a1);
+    }
+    static __device__ __forceinline__ void axpy(float *acc, float pe, const uint4 &v) {
+        ffma2(acc[0], acc[1], __uint_as_float(v.x), __uint_as_float(v.y), pe);
+        ffma2(acc[2], acc[3], __uint_as_float(v.z), __uint_as_float(v.w), pe);
+    }
+};
 template <> struct ElemT<SH_F16> {
     static constexpr int EPL = 8, BYTES = 2;
     static __device__ __forceinline__ void dot(const uint4 &q, const uint4 &k, float &a0, float &a1) {
@@ -399,20 +412,57 @@ cudaError_t launch_tma(const sh_context *c, const DecodeParams &p, cudaStream_t 
 #define SH_TMA_CPS 1
 #endif
 
+namespace {
+
+// Tile shapes per stored row size; 256-byte rows take the tuned (overridable) defaults.
+//   row bytes   SR    NST   LR   stage     row groups x rows per group per tile
+//   256        128     3     8   64 KB     32 x 4
+//   512         64     3    16   64 KB     16 x 4
+// 128-byte rows (16-bit stores with head_dim 64) are left to the direct-load kernel: with half
+// the bytes per row the per-row work of this one dominates (best of four shapes tried on B200:
+// 190 us against 184 us for the OPT-66B-shaped workload with head_dim 64).
+template <int DT, int D> struct Shape {
+    static constexpr int RB = D * ElemT<DT>::BYTES;
+    static constexpr int SR = RB == 512 ? 64 : SH_TMA_SR, NST = SH_TMA_NST, LR = RB == 512 ? 16 : SH_TMA_LR;
+};
+
+template <int DT, int D> size_t shape_smem(int B) {
+    using S = Shape<DT, D>;
+    const int capw = (B + 31) & ~31;
+    return (size_t)S::NST * (2 * S::SR * S::RB + 3 * S::RB) +
+           sizeof(float) * ((size_t)2 * capw + (size_t)2 * SH_TMA_NWC * D + (size_t)2 * SH_TMA_NWC * 2);
+}
+
+template <int DT> size_t smem_for(int D, int B) { return D == 64 ? shape_smem<DT, 64>(B) : shape_smem<DT, 128>(B); }
+
+template <int DT>
+cudaError_t launch_dt(const sh_context *c, const DecodeParams &p, cudaStream_t s) {
+    if constexpr (DT == SH_F32) {
+        if (c->D == 64)
+            return launch_tma<DT, 64, SH_TMA_NWC, Shape<DT, 64>::SR, Shape<DT, 64>::NST, Shape<DT, 64>::LR, SH_TMA_CPS>(c, p, s);
+    }
+    return launch_tma<DT, 128, SH_TMA_NWC, Shape<DT, 128>::SR, Shape<DT, 128>::NST, Shape<DT, 128>::LR, SH_TMA_CPS>(c, p, s);
+}
+
+}  // namespace
+
 // Whether the pipelined kernel can serve this handle (dtype, shape, shared memory).
 bool sh_decode_tma_supported(const sh_context *c) {
-    if (c->dtype != SH_F16 && c->dtype != SH_BF16) return false;
-    if (c->D != 128) return false;
-    const int capw = (c->B + 31) & ~31;
-    const size_t ring = (size_t)SH_TMA_NST * (2 * SH_TMA_SR * 256 + 3 * 256);
-    const size_t rest = sizeof(float) * ((size_t)2 * capw + (size_t)2 * SH_TMA_NWC * 128 + 4 * SH_TMA_NWC);
-    return ring + rest <= 227 * 1024;
+    if (c->D != 64 && c->D != 128) return false;
+    if (c->row_bytes < 256) return false;
+    size_t need;
+    if (c->dtype == SH_F32) need = smem_for<SH_F32>(c->D, c->B);
+    else if (c->dtype == SH_F16) need = smem_for<SH_F16>(c->D, c->B);
+    else if (c->dtype == SH_BF16) need = smem_for<SH_BF16>(c->D, c->B);
+    else return false;
+    return need <= 227 * 1024;
 }
 
 cudaError_t sh_launch_decode_tma(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches) {
     cudaError_t e = cudaErrorInvalidValue;
-    if (c->dtype == SH_F16) e = launch_tma<SH_F16, 128, SH_TMA_NWC, SH_TMA_SR, SH_TMA_NST, SH_TMA_LR, SH_TMA_CPS>(c, p, s);
-    else if (c->dtype == SH_BF16) e = launch_tma<SH_BF16, 128, SH_TMA_NWC, SH_TMA_SR, SH_TMA_NST, SH_TMA_LR, SH_TMA_CPS>(c, p, s);
+    if (c->dtype == SH_F32) e = launch_dt<SH_F32>(c, p, s);
+    else if (c->dtype == SH_F16) e = launch_dt<SH_F16>(c, p, s);
+    else if (c->dtype == SH_BF16) e = launch_dt<SH_BF16>(c, p, s);
     if (e == cudaSuccess) *launches += 1;
     return e;
 }

@@ -48,12 +48,13 @@ def test_lockstep_edge_parameters(sh, B, r, w, m):
     assert res.compressions >= 1
 
 
-@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("dtype,d", [("f16", 128), ("bf16", 128), ("f32", 128), ("f32", 64)])
 @pytest.mark.parametrize("U,B,r,w,m", [(5, 150, 9, 37, 41), (301, 130, 16, 33, 50), (3, 700, 5, 64, 300), (2, 40, 3, 9, 20)])
-def test_lockstep_pipelined_kernel(sh, dtype, U, B, r, w, m):
+def test_lockstep_pipelined_kernel(sh, dtype, d, U, B, r, w, m):
     """The persistent bulk-copy variant of the decode kernel, forced on shapes that
-    cover fewer units than CTAs, more units than SMs, ragged last tiles and tiny caches."""
-    d, T = 128, 2 * B + 2 * m + 7
+    cover fewer units than CTAs, more units than SMs, ragged last tiles and tiny caches,
+    for every row size it serves (256 and 512 bytes)."""
+    T = 2 * B + 2 * m + 7
     q, k, v = wl.random_stream(U, d, T, seed=11 + U, dtype=dtype, peaked=3.0, device="cuda")
     h = sh.Handle(B, r, w, m, U, d, dtype, split=1, kernel=2, auto_compress=False)
     res, _ = run_lockstep(h, dtype, _stream_fn(q, k, v), T, torch.arange(U), TOL[dtype])
