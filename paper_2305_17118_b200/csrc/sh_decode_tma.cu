@@ -433,7 +433,12 @@ template <int DT, int D> size_t shape_smem(int B) {
            sizeof(float) * ((size_t)2 * capw + (size_t)2 * SH_TMA_NWC * D + (size_t)2 * SH_TMA_NWC * 2);
 }
 
-template <int DT> size_t smem_for(int D, int B) { return D == 64 ? shape_smem<DT, 64>(B) : shape_smem<DT, 128>(B); }
+template <int DT> size_t smem_for(int D, int B) {
+    if constexpr (DT == SH_F32) {
+        if (D == 64) return shape_smem<DT, 64>(B);
+    }
+    return shape_smem<DT, 128>(B);
+}
 
 template <int DT>
 cudaError_t launch_dt(const sh_context *c, const DecodeParams &p, cudaStream_t s) {
