@@ -29,7 +29,7 @@ void make_layout(sh_context *c) {
     };
     L.K = take(U * B * c->row_bytes);
     L.V = take(U * B * c->row_bytes);
-    const size_t sc = c->dtype == SH_INT4_G64_F16 ? U * B * (D / 64) * 2 : 0;
+    const size_t sc = c->dtype == SH_INT4_G64_F16 ? U * (size_t)c->Bs * (D / 64) * 2 : 0;
     L.Ks = take(sc);
     L.Vs = take(sc);
     L.hist = take(U * (size_t)c->w * c->Bw * 4);
@@ -110,6 +110,7 @@ int do_compress(sh_context *c, cudaStream_t s) {
     cp.U = c->ucount; cp.B = c->B; cp.Bw = c->Bw; cp.w = c->w; cp.n = c->B; cp.m = c->m;
     cp.row_bytes = c->row_bytes;
     cp.scale_bytes = c->dtype == SH_INT4_G64_F16 ? (c->D / 64) * 2 : 0;
+    cp.Bs = c->Bs;
     cp.err = reinterpret_cast<int *>(c->slab + c->L.err);
     cp.n_arr = sh_pnarr(c);
     e = sh_launch_compact(cp, s, &c->launches);
@@ -153,7 +154,7 @@ int do_step(sh_context *c, const void *q, const void *k, const void *v, float *o
     p.pos = sh_ppos(c);
     p.qring = sh_pqring(c);
     p.n_arr = sh_pnarr(c); p.t_arr = sh_ptarr(c);
-    p.U = c->ucount; p.B = c->B; p.Bw = c->Bw; p.w = c->w;
+    p.U = c->ucount; p.B = c->B; p.Bw = c->Bw; p.w = c->w; p.Bs = c->Bs;
     p.n = c->n + 1;
     p.t = (int)(c->t + 1);
     p.hist_row = (int)((c->t + 1) % c->w);
@@ -191,6 +192,7 @@ int sh_create(int B, int r, int w, int m, int heads, int head_dim, int dtype, sh
     if (!c) return SH_ENOMEM;
     c->B = B; c->r = r; c->w = w; c->m = m; c->U = heads; c->D = head_dim; c->dtype = dtype;
     c->Bw = (B + 31) / 32;
+    c->Bs = (B + 7) / 8 * 8;
     c->row_bytes = dtype == SH_F32 ? head_dim * 4 : (dtype == SH_INT4_G64_F16 ? head_dim / 2 : head_dim * 2);
     c->in_bytes = dtype == SH_F32 ? head_dim * 4 : head_dim * 2;
     c->n = 0; c->t = 0;
@@ -555,8 +557,8 @@ int sh_export_unit(sh_handle h, int unit, float *K_host, float *V_host, void *st
     const size_t B = h->B, D = h->D;
     const char *K = h->slab + h->L.K + (size_t)unit * B * h->row_bytes;
     const char *V = h->slab + h->L.V + (size_t)unit * B * h->row_bytes;
-    const __half *Ks = reinterpret_cast<const __half *>(h->slab + h->L.Ks) + (size_t)unit * B * (D / 64);
-    const __half *Vs = reinterpret_cast<const __half *>(h->slab + h->L.Vs) + (size_t)unit * B * (D / 64);
+    const __half *Ks = reinterpret_cast<const __half *>(h->slab + h->L.Ks) + (size_t)unit * h->Bs * (D / 64);
+    const __half *Vs = reinterpret_cast<const __half *>(h->slab + h->L.Vs) + (size_t)unit * h->Bs * (D / 64);
     sh_export_kernel<<<64, 256, 0, s>>>(K, V, Ks, Vs, dst, h->B, h->D, h->dtype, h->row_bytes);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);

@@ -213,7 +213,7 @@ __global__ void __launch_bounds__(ROWS_THREADS) sh_compact_rows_kernel(const Com
     if (p.scale_bytes) {
         __syncthreads();
         if (p.scale_bytes == 4) {
-            uint32_t *sc = reinterpret_cast<uint32_t *>(what == 0 ? p.Ks : p.Vs) + (size_t)u * p.B;
+            uint32_t *sc = reinterpret_cast<uint32_t *>(what == 0 ? p.Ks : p.Vs) + (size_t)u * p.Bs;
             for (int base = 0; base < p.n; base += ROWS_THREADS) {
                 const int d = base + tid;
                 uint32_t val = 0;
@@ -222,7 +222,7 @@ __global__ void __launch_bounds__(ROWS_THREADS) sh_compact_rows_kernel(const Com
                 if (d < p.n) sc[d] = val;
             }
         } else {
-            uint16_t *sc = reinterpret_cast<uint16_t *>(what == 0 ? p.Ks : p.Vs) + (size_t)u * p.B;
+            uint16_t *sc = reinterpret_cast<uint16_t *>(what == 0 ? p.Ks : p.Vs) + (size_t)u * p.Bs;
             for (int base = 0; base < p.n; base += ROWS_THREADS) {
                 const int d = base + tid;
                 uint16_t val = 0;

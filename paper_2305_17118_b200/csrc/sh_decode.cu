@@ -353,8 +353,8 @@ __global__ void __launch_bounds__(NW * 32) sh_decode_kernel(const DecodeParams p
 
     const char *Kb = p.K + (size_t)u * B * ROWB;
     const char *Vb = p.V + (size_t)u * B * ROWB;
-    const __half *Ksb = Q4 ? reinterpret_cast<const __half *>(p.Ks) + (size_t)u * B * (D / 64) : nullptr;
-    const __half *Vsb = Q4 ? reinterpret_cast<const __half *>(p.Vs) + (size_t)u * B * (D / 64) : nullptr;
+    const __half *Ksb = Q4 ? reinterpret_cast<const __half *>(p.Ks) + (size_t)u * p.Bs * (D / 64) : nullptr;
+    const __half *Vsb = Q4 ? reinterpret_cast<const __half *>(p.Vs) + (size_t)u * p.Bs * (D / 64) : nullptr;
 
     // ---- logits of the cached rows
     float lmax = -INFINITY;
@@ -412,8 +412,8 @@ __global__ void __launch_bounds__(NW * 32) sh_decode_kernel(const DecodeParams p
                 st_plain(kdst, ck);
                 st_plain(vdst, cv);
                 if ((c & 1) == 0) {
-                    reinterpret_cast<__half *>(p.Ks)[((size_t)u * B + n_old) * (D / 64) + (c >> 1)] = __float2half_rn(sck);
-                    reinterpret_cast<__half *>(p.Vs)[((size_t)u * B + n_old) * (D / 64) + (c >> 1)] = __float2half_rn(scv);
+                    reinterpret_cast<__half *>(p.Ks)[((size_t)u * p.Bs + n_old) * (D / 64) + (c >> 1)] = __float2half_rn(sck);
+                    reinterpret_cast<__half *>(p.Vs)[((size_t)u * p.Bs + n_old) * (D / 64) + (c >> 1)] = __float2half_rn(scv);
                 }
             }
         } else if (sub == 0) {

@@ -11,7 +11,7 @@
 // Byte offsets of the regions inside the caller's workspace slab.
 struct ShLayout {
     size_t K, V;            // [U][B][row_bytes]
-    size_t Ks, Vs;          // int4 only: [U][B][D/64] fp16 group scales
+    size_t Ks, Vs;          // int4 only: [U][Bs][D/64] fp16 group scales (Bs = B rounded up to 8: every unit 16-byte aligned)
     size_t hist;            // [U][w][Bw] u32 bit-planes: row (step mod w), bit j = "slot j was low at that step"
     size_t pos;             // [U][B] int32 stream positions
     size_t src_idx;         // [U][B] int32 selection result: source slot of each surviving destination slot
@@ -27,6 +27,7 @@ struct ShLayout {
 struct sh_context {
     int B, r, w, m, U, D, dtype;
     int Bw;          // ceil(B / 32)
+    int Bs;          // scale rows per unit of the int4 store: B rounded up to a multiple of 8
     int row_bytes;   // bytes of one stored K (or V) row, without int4 scales
     int in_bytes;    // bytes of one q / k_new / v_new row
     int n;           // live tokens per unit
@@ -59,8 +60,8 @@ struct sh_context {
 // Base pointers of the active unit range inside the workspace.
 inline char *sh_pK(const sh_context *c) { return c->slab + c->L.K + (size_t)c->u0 * c->B * c->row_bytes; }
 inline char *sh_pV(const sh_context *c) { return c->slab + c->L.V + (size_t)c->u0 * c->B * c->row_bytes; }
-inline char *sh_pKs(const sh_context *c) { return c->slab + c->L.Ks + (size_t)c->u0 * c->B * (c->D / 64) * 2; }
-inline char *sh_pVs(const sh_context *c) { return c->slab + c->L.Vs + (size_t)c->u0 * c->B * (c->D / 64) * 2; }
+inline char *sh_pKs(const sh_context *c) { return c->slab + c->L.Ks + (size_t)c->u0 * c->Bs * (c->D / 64) * 2; }
+inline char *sh_pVs(const sh_context *c) { return c->slab + c->L.Vs + (size_t)c->u0 * c->Bs * (c->D / 64) * 2; }
 inline uint32_t *sh_phist(const sh_context *c) {
     return reinterpret_cast<uint32_t *>(c->slab + c->L.hist) + (size_t)c->u0 * c->w * c->Bw;
 }
@@ -83,6 +84,7 @@ struct DecodeParams {
     int *n_arr, *t_arr;   // per-unit live rows / tokens streamed before this step (sequences of different
                           // lengths), updated by the kernel; NULL when n and t below hold for every unit
     int U, B, Bw, w;
+    int Bs;         // scale rows per unit (int4 store)
     int n;          // live rows per unit including the token appended by this step
     int hist_row;   // t mod w
     int t;          // 1-based stream position of this step's token
@@ -107,6 +109,7 @@ struct CompactParams {
     const int32_t *src_idx;
     int U, B, Bw, w, n, m;
     int row_bytes, scale_bytes;
+    int Bs;                     // scale rows per unit (int4 store)
     int chunk_bytes;            // set by the launcher: shared-memory gather buffer of the row kernel
     int rec_rows;               // set by the launcher: bit-plane rows staged per pass of the record kernel
     int *err;                   // device error word (a bounded wait gave up)

@@ -78,6 +78,7 @@ extern "C" int sh_compress_static(sh_handle h, void *stream, int *evicted_per_un
     cp.n_arr = sh_pnarr(h);
     cp.row_bytes = h->row_bytes;
     cp.scale_bytes = h->dtype == SH_INT4_G64_F16 ? (h->D / 64) * 2 : 0;
+    cp.Bs = h->Bs;
     cp.err = reinterpret_cast<int *>(h->slab + h->L.err);
     e = sh_launch_compact(cp, s, &h->launches);
     if (e != cudaSuccess) { h->last_err = e; return SH_ECUDA; }
