@@ -200,7 +200,7 @@ def cuda_arm(args, cfg, rank, world):
     handles = [sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, U, d, cfg.dtype, device=dev, auto_compress=False,
                          split=args.split, kernel=args.kernel,
                          prefill_chunk=False if args.no_prefill_chunk else None,
-                         recompute_record=args.recompute_record)
+                         recompute_record=args.recompute_record, unordered=args.unordered_compaction)
                for _ in range(Ly)]
 
     # ---- prompt: streamed through the same path, untimed
@@ -347,6 +347,7 @@ def cuda_arm(args, cfg, rank, world):
         "config": {"workload": cfg.name, "batch": cfg.batch, "heads": cfg.heads, "layers": Ly, "units": U * Ly,
                    "head_dim": d, "kv_dtype": cfg.dtype, "B": cfg.B, "r": cfg.r, "w": cfg.w, "m": cfg.m,
                    "prompt": cfg.prompt, "record": "recomputed at compression" if args.recompute_record else "online",
+                   "compaction": "unordered" if args.unordered_compaction else "stable",
                    "l2": "flushed between steps" if flush else "inputs larger than L2",
                    "kv_bytes": kv_bytes, "parallelism": f"units replicated x{world}" if world > 1 else "1 GPU"},
         "attn_GBps": statistics.fmean(n_sched) * U * Ly * d * ES[cfg.dtype] * 2 / (ms_per_step * 1e-3) / 1e9,
@@ -375,6 +376,8 @@ def main():
                     help="variant: rebuild the importance record at each compression from stored queries")
     ap.add_argument("--kv-dtype", default=None, choices=["f32", "f16", "bf16", "int4"], help="override the workload's K/V dtype")
     ap.add_argument("--head-dim", type=int, default=None, choices=[64, 128], help="override the workload's head_dim")
+    ap.add_argument("--unordered-compaction", action="store_true",
+                    help="SH_OPT_COMPACTION = 1: holes filled from the tail, at most m rows move per compression")
     ap.add_argument("--no-prefill-chunk", action="store_true", help="stream the prompt one decode step per token")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (tuning runs)")
     args = ap.parse_args()

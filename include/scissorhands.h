@@ -22,8 +22,9 @@
  *   - Every function returns an sh_status (0 = SH_OK, negative = error) and
  *     never aborts, throws or prints.  On error nothing has been enqueued
  *     unless stated otherwise.
- *   - Slots [0, n) of a unit's cache are live and sorted by stream position;
- *     compaction is stable, so "the r newest" are slots [n-r, n).
+ *   - Slots [0, n) of a unit's cache are live.  By default they are sorted by
+ *     stream position (compaction is stable, so "the r newest" are slots
+ *     [n-r, n)); with SH_OPT_COMPACTION = 1 their order is arbitrary.
  */
 #ifndef SCISSORHANDS_H_
 #define SCISSORHANDS_H_
@@ -68,6 +69,11 @@ typedef enum {
                                  scored against the cache as it is then (Algorithm 2 as stated; Section 4.1,
                                  "Overhead Tradeoff").  fp16/bf16, head_dim 128 only.  Set before sh_bind:
                                  it changes sh_workspace_bytes. */
+    SH_OPT_COMPACTION = 6,    /* 0 (default): stable left-compaction, slots stay sorted by stream position;
+                                 1: every hole left by a dropped token below n-m is filled with a kept row from
+                                 the tail (at most m rows move instead of nearly all); slots are then in no
+                                 particular order: sh_state's pos tells which token sits where.  The kept set is
+                                 the same either way. */
     SH_OPT_PREFILL_CHUNK = 4, /* 1 (default): sh_prefill hands the tokens between two compressions to the chunk
                                  kernel where the shape allows it; 0: one decode step per token */
     SH_OPT_DECODE_KERNEL = 3  /* 0 (default): chosen from the shape; 1: one CTA (or cluster) per unit with

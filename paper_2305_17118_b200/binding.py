@@ -20,6 +20,7 @@ SH_OK, SH_EINVAL, SH_EFULL, SH_ESTATE, SH_ECUDA, SH_ENOMEM, SH_ETOOBIG, SH_EDEVI
 SH_STATIC_SCRATCH_MAX_ENTRIES = 1 << 20
 SH_F32, SH_F16, SH_BF16, SH_INT4_G64_F16 = 0, 1, 2, 3
 SH_OPT_SOFTMAX_SCALE, SH_OPT_SPLIT, SH_OPT_AUTO_COMPRESS, SH_OPT_DECODE_KERNEL, SH_OPT_PREFILL_CHUNK, SH_OPT_RECORD_MODE = 0, 1, 2, 3, 4, 5
+SH_OPT_COMPACTION = 6
 
 DTYPE_CODE = {"f32": SH_F32, "f16": SH_F16, "bf16": SH_BF16, "int4": SH_INT4_G64_F16}
 INPUT_TORCH_DTYPE = {SH_F32: torch.float32, SH_F16: torch.float16, SH_BF16: torch.bfloat16,
@@ -108,7 +109,8 @@ class Handle:
 
     def __init__(self, B: int, r: int, w: int, m: int, heads: int, head_dim: int, dtype, device="cuda:0",
                  split: Optional[int] = None, scale: Optional[float] = None, auto_compress: bool = True,
-                 kernel: Optional[int] = None, prefill_chunk: Optional[bool] = None, recompute_record: bool = False):
+                 kernel: Optional[int] = None, prefill_chunk: Optional[bool] = None, recompute_record: bool = False,
+                 unordered: bool = False):
         self.dtype = DTYPE_CODE[dtype] if isinstance(dtype, str) else int(dtype)
         self.B, self.r, self.w, self.m, self.U, self.D = B, r, w, m, heads, head_dim
         self.Bw = (B + 31) // 32
@@ -127,6 +129,8 @@ class Handle:
             self.set_option(SH_OPT_DECODE_KERNEL, kernel)
         if recompute_record:
             self.set_option(SH_OPT_RECORD_MODE, 1.0)
+        if unordered:
+            self.set_option(SH_OPT_COMPACTION, 1.0)
         if prefill_chunk is not None:
             self.set_option(SH_OPT_PREFILL_CHUNK, 1.0 if prefill_chunk else 0.0)
         self.set_option(SH_OPT_AUTO_COMPRESS, 1.0 if auto_compress else 0.0)

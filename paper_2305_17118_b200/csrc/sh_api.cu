@@ -100,6 +100,11 @@ int do_compress(sh_context *c, cudaStream_t s) {
     sp.U = c->ucount; sp.B = c->B; sp.Bw = c->Bw; sp.w = c->w; sp.n = c->B; sp.r = c->r; sp.m = c->m;
     sp.cmax = c->w;
     sp.n_arr = sh_pnarr(c);
+    sp.unordered = c->unordered;
+    sp.pos = sh_ppos(c);
+    sp.t_arr = sh_ptarr(c);
+    sp.t = (int)c->t;
+    sp.n_moves = reinterpret_cast<uint16_t *>(c->slab + c->L.counters) + (size_t)c->u0 * c->B;
     cudaError_t e = sh_launch_select(sp, true, s, &c->launches);
     if (e != cudaSuccess) return cuda_fail(c, e);
     CompactParams cp = {};
@@ -114,6 +119,8 @@ int do_compress(sh_context *c, cudaStream_t s) {
     cp.Bs = c->Bs;
     cp.err = reinterpret_cast<int *>(c->slab + c->L.err);
     cp.n_arr = sh_pnarr(c);
+    cp.unordered = c->unordered;
+    cp.n_moves = sp.n_moves;
     e = sh_launch_compact(cp, s, &c->launches);
     if (e != cudaSuccess) return cuda_fail(c, e);
     sh_after_compression(c);
@@ -204,6 +211,7 @@ int sh_create(int B, int r, int w, int m, int heads, int head_dim, int dtype, sh
     c->kernel = 0;
     c->prefill_chunk = 1;
     c->record_mode = 0;
+    c->unordered = 0;
     c->record_fresh_t = -1;
     c->started = false;
     c->slab = nullptr; c->slab_bytes = 0;
@@ -263,6 +271,12 @@ int sh_set_option(sh_handle h, int key, double value) {
             if (mode == 1 && sh_prefill_chunk_capacity(h) == 0) return SH_EINVAL;   // needs the tensor-core kernel's shapes
             h->record_mode = mode;
             make_layout(h);
+            return SH_OK;
+        }
+        case SH_OPT_COMPACTION: {
+            const int mode = (int)value;
+            if (mode != 0 && mode != 1) return SH_EINVAL;
+            h->unordered = mode;
             return SH_OK;
         }
         case SH_OPT_PREFILL_CHUNK:

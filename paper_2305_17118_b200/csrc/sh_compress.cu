@@ -10,6 +10,7 @@ namespace {
 
 constexpr int SEL_THREADS = 256;
 constexpr int CMP_THREADS = 256;
+constexpr int SEL_TIE_CAP = 1024;     // tie classes up to this size are searched from a shared-memory list
 
 // Exclusive prefix count of a per-thread flag over the CTA.  `wsum` is shared
 // scratch of >= 32 ints.  Returns this thread's rank; total in *total.
@@ -50,11 +51,15 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
     int *cnt_sh = sm;                      // [n]
     int *bins = cnt_sh + p.n;              // [cmax + 1]
     int *wsum = bins + (p.cmax + 1);       // [32]
-    int *cut = wsum + 32;                  // [2] = {cstar, need}
-    uint32_t *planes = reinterpret_cast<uint32_t *>(cut + 2);   // [w * Bw] when staged, then [G][5][Bw] partial sums
+    int *cut = wsum + 32;                  // [8] = {cstar, need, size of the tie class, pstar, tie list fill}
+    int *tie_list = cut + 8;               // [SEL_TIE_CAP] positions of the tie class (unordered mode only)
+    uint32_t *planes = reinterpret_cast<uint32_t *>(tie_list + (p.unordered ? SEL_TIE_CAP : 0));   // [w * Bw] when staged, then [G][5][Bw] partial sums
     const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
     const int n = p.n, ncand = p.n - p.r, m = p.m;
-    if (p.n_arr && p.n_arr[u] != n) return;      // this unit's cache is not full (whole CTA leaves)
+    if (p.n_arr && p.n_arr[u] != n) {            // this unit's cache is not full (whole CTA leaves)
+        if (tid == 0 && p.unordered && p.n_moves) p.n_moves[(size_t)u * p.B] = 0;   // tells the move kernel to skip it too
+        return;
+    }
 
     for (int i = tid; i <= p.cmax; i += SEL_THREADS) bins[i] = 0;
     if (FROM_HIST) {
@@ -100,7 +105,13 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
         for (int j = tid; j < n; j += SEL_THREADS) cnt_sh[j] = min((int)p.counters[(size_t)u * n + j], p.cmax);
     }
     __syncthreads();
-    for (int j = tid; j < ncand; j += SEL_THREADS) atomicAdd(&bins[cnt_sh[j]], 1);
+    // Candidates: everything but the r most recent tokens.  With position-sorted slots those are the
+    // last r slots; otherwise the positions say (one token per step: the r newest have pos > t - r).
+    const int32_t *pos_u = p.unordered ? p.pos + (size_t)u * p.B : nullptr;
+    const int t_cut = p.unordered ? (p.t_arr ? p.t_arr[u] : p.t) - p.r : 0;
+    auto is_cand = [&](int j) { return p.unordered ? (j < n && pos_u[j] <= t_cut) : j < ncand; };
+    for (int j = tid; j < n; j += SEL_THREADS)
+        if (is_cand(j)) atomicAdd(&bins[cnt_sh[j]], 1);
     __syncthreads();
 
     // Cut: largest c with #{I >= c} >= m.  Warp 0 scans the bins from the top, 32 at a time.
@@ -121,6 +132,8 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
                 if (lane == f) {
                     cut[0] = cidx;
                     cut[1] = m - (above + incl - v);   // how many of the tie class go
+                    cut[2] = v;
+                    cut[4] = 0;
                 }
                 break;
             }
@@ -130,6 +143,69 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
     __syncthreads();
     const int cstar = cut[0], need = cut[1];
 
+    if (p.unordered) {
+        // Tie class at the cut: the `need` members with the smallest positions go.  Positions are unique
+        // and at most t_cut, so a binary search on the position value finds the largest one that goes.
+        const int tie_size = cut[2];
+        int pstar = -1;
+        if (need >= tie_size) {
+            pstar = t_cut;                   // the whole class goes
+        } else if (need > 0 && tie_size <= SEL_TIE_CAP) {
+            // small class (the usual case): its positions are listed in shared memory and one warp searches
+            for (int j = tid; j < n; j += SEL_THREADS)
+                if (is_cand(j) && cnt_sh[j] == cstar) tie_list[atomicAdd(&cut[4], 1)] = pos_u[j];
+            __syncthreads();
+            if (tid < 32) {
+                int lo = 0, hi = t_cut;      // smallest value with #{tie, pos <= value} >= need lies in (lo, hi]
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    int cntv = 0;
+                    for (int i = lane; i < tie_size; i += 32) cntv += tie_list[i] <= mid;
+                    cntv = __reduce_add_sync(0xffffffffu, cntv);
+                    if (cntv >= need) hi = mid; else lo = mid;
+                }
+                if (lane == 0) cut[3] = hi;
+            }
+            __syncthreads();
+            pstar = cut[3];
+        } else if (need > 0) {
+            int lo = 0, hi = t_cut;          // same search with block-wide counts over all slots
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                int cntv = 0;
+                for (int j0 = 0; j0 < n; j0 += SEL_THREADS) {
+                    const int j = j0 + tid;
+                    const bool in = j < n && is_cand(j) && cnt_sh[j] == cstar && pos_u[j] <= mid;
+                    cntv += __syncthreads_count(in);
+                }
+                if (cntv >= need) hi = mid; else lo = mid;
+            }
+            pstar = hi;
+        }
+        // Holes (dropped slots below n - m) are filled, in order, by the kept slots at or beyond n - m.
+        const int n_keep = n - m;
+        int hole_carry = 0, fill_carry = 0, ev_carry = 0;
+        for (int j0 = 0; j0 < n; j0 += SEL_THREADS) {
+            const int j = j0 + tid;
+            const int I = j < n ? cnt_sh[j] : -1;
+            const bool ev = j < n && is_cand(j) && (I > cstar || (I == cstar && pos_u[j] <= pstar));
+            const bool hole = ev && j < n_keep, filler = j >= n_keep && j < n && !ev;
+            int tot;
+            const int hk = hole_carry + block_flag_scan(hole, wsum, &tot);
+            hole_carry += tot;
+            const int fk = fill_carry + block_flag_scan(filler, wsum, &tot);
+            fill_carry += tot;
+            const int eidx = ev_carry + block_flag_scan(ev, wsum, &tot);
+            ev_carry += tot;
+            if (p.src_idx) {
+                if (hole) p.src_idx[(size_t)u * p.B + hk] = j;
+                if (filler) p.src_idx[(size_t)u * p.B + (p.B - 1 - fk)] = j;
+            }
+            if (ev && p.evicted) p.evicted[(size_t)u * m + eidx] = j;
+        }
+        if (tid == 0 && p.n_moves) p.n_moves[(size_t)u * p.B] = (uint16_t)(0x8000 | hole_carry);   // bit 15: unit selected
+        return;
+    }
     int tie_carry = 0, keep_carry = 0, ev_carry = 0;
     for (int j0 = 0; j0 < n; j0 += SEL_THREADS) {
         const int j = j0 + tid;
@@ -256,6 +332,8 @@ __global__ void __launch_bounds__(CMP_THREADS) sh_compact_record_kernel(const Co
     const int n_keep = p.n - p.m, Bw = p.Bw, w = p.w;
     if (p.n_arr && p.n_arr[u] != p.n) return;        // this unit's cache is not full (whole CTA leaves)
     const int stride = Bw | 1;                       // odd row stride: no bank conflicts
+    const uint32_t bw_magic = p.bw_magic;
+    auto row_of = [&](int i) { return Bw > 1 ? (int)__umulhi((uint32_t)i, bw_magic) : i; };   // i / Bw
     const int32_t *src = p.src_idx + (size_t)u * p.B;
     uint32_t *hist_u = p.hist + (size_t)u * w * Bw;
     uint32_t *keep = rec_sm;                         // [Bw] keep mask per source word
@@ -284,7 +362,7 @@ __global__ void __launch_bounds__(CMP_THREADS) sh_compact_record_kernel(const Co
     __syncthreads();
     for (int s0 = 0; s0 < w; s0 += p.rec_rows) {
         const int nr = min(p.rec_rows, w - s0);
-        for (int i = tid; i < nr * Bw; i += CMP_THREADS) rows[(i / Bw) * stride + (i % Bw)] = hist_u[(size_t)s0 * Bw + i];
+        for (int i = tid; i < nr * Bw; i += CMP_THREADS) { const int rr = row_of(i); rows[rr * stride + (i - rr * Bw)] = hist_u[(size_t)s0 * Bw + i]; }
         __syncthreads();
         for (int r = tid; r < nr; r += CMP_THREADS) {
             uint32_t *row = rows + r * stride;
@@ -305,7 +383,7 @@ __global__ void __launch_bounds__(CMP_THREADS) sh_compact_record_kernel(const Co
             for (; o < Bw; ++o) row[o] = 0;
         }
         __syncthreads();
-        for (int i = tid; i < nr * Bw; i += CMP_THREADS) hist_u[(size_t)s0 * Bw + i] = rows[(i / Bw) * stride + (i % Bw)];
+        for (int i = tid; i < nr * Bw; i += CMP_THREADS) { const int rr = row_of(i); hist_u[(size_t)s0 * Bw + i] = rows[rr * stride + (i - rr * Bw)]; }
         __syncthreads();
     }
     // positions: read a batch, barrier, write it (destinations never pass sources)
@@ -317,6 +395,139 @@ __global__ void __launch_bounds__(CMP_THREADS) sh_compact_record_kernel(const Co
         __syncthreads();
         if (d < p.n) pos[d] = val;
     }
+    if (p.n_arr && tid == 0) p.n_arr[u] = n_keep;    // last kernel of the compression: the unit is compacted
+}
+
+// Inverse of compress_bits: the low popc(m) bits of x spread to the set bits of m (same masks, reverse order).
+__device__ __forceinline__ uint32_t expand_bits(uint32_t x, uint32_t m, const uint32_t *mv) {
+#pragma unroll
+    for (int i = 4; i >= 0; --i) {
+        const uint32_t t = x << (1 << i);
+        x = (x & ~mv[i]) | (t & mv[i]);
+    }
+    return x & m;
+}
+
+__device__ __forceinline__ void compress_masks(uint32_t m, uint32_t *mv_out) {
+    uint32_t mk = ~m << 1;
+#pragma unroll
+    for (int i = 0; i < 5; ++i) {
+        uint32_t mp = mk ^ (mk << 1);
+        mp ^= mp << 2; mp ^= mp << 4; mp ^= mp << 8; mp ^= mp << 16;
+        const uint32_t mv = mp & m;
+        mv_out[i] = mv;
+        m = (m ^ mv) | (mv >> (1 << i));
+        mk &= ~mp;
+    }
+}
+
+// Unordered compaction: each hole takes the row of its filler.  Holes lie below n - m, fillers at or
+// beyond it, so sources and destinations are disjoint and the moves are independent.  blockIdx.y:
+// 0 = K rows (+ int4 scales), 1 = V rows (+ scales), 2 = record bit-planes and positions.
+__global__ void __launch_bounds__(CMP_THREADS) sh_fill_holes_kernel(const CompactParams p) {
+    extern __shared__ uint32_t fh_sm[];
+    const int u = blockIdx.x, what = blockIdx.y, tid = threadIdx.x;
+    // The selection kernel marked the units it handled (the three CTAs of a unit must agree, and the
+    // third one updates the unit's row count, so that count cannot be the test here).
+    const int marked = p.n_moves[(size_t)u * p.B];
+    if (!(marked & 0x8000)) return;
+    const int n_keep = p.n - p.m, h = marked & 0x7fff;
+    const int32_t *row = p.src_idx + (size_t)u * p.B;
+    auto hole_of = [&](int k) { return row[k]; };
+    auto filler_of = [&](int k) { return row[p.B - 1 - k]; };
+    if (what < 2) {
+        char *rows = (what == 0 ? p.K : p.V) + (size_t)u * p.B * p.row_bytes;
+        const int lpr = p.row_bytes >> 4, lsh = __ffs(lpr) - 1;     // 16-byte chunks per row: a power of two
+        for (int idx = tid; idx < h * lpr; idx += CMP_THREADS) {
+            const int k = idx >> lsh, ch = idx & (lpr - 1);
+            *reinterpret_cast<uint4 *>(rows + (size_t)hole_of(k) * p.row_bytes + ch * 16) =
+                *reinterpret_cast<const uint4 *>(rows + (size_t)filler_of(k) * p.row_bytes + ch * 16);
+        }
+        if (p.scale_bytes == 4) {
+            uint32_t *sc = reinterpret_cast<uint32_t *>(what == 0 ? p.Ks : p.Vs) + (size_t)u * p.Bs;
+            for (int k = tid; k < h; k += CMP_THREADS) sc[hole_of(k)] = sc[filler_of(k)];
+        } else if (p.scale_bytes == 2) {
+            uint16_t *sc = reinterpret_cast<uint16_t *>(what == 0 ? p.Ks : p.Vs) + (size_t)u * p.Bs;
+            for (int k = tid; k < h; k += CMP_THREADS) sc[hole_of(k)] = sc[filler_of(k)];
+        }
+        return;
+    }
+    // Record.  In every bit-plane row the fillers' bits, taken in slot order, go to the holes in slot
+    // order: the tail words are compressed by the filler mask into a bit stream (written over the tail,
+    // which is dead afterwards), and each head word takes its share of the stream expanded to its holes.
+    const int Bw = p.Bw, w = p.w, stride = Bw | 1;
+    const uint32_t bw_magic = p.bw_magic;
+    auto row_of = [&](int i) { return Bw > 1 ? (int)__umulhi((uint32_t)i, bw_magic) : i; };   // i / Bw
+    uint32_t *hist_u = p.hist + (size_t)u * w * Bw;
+    uint32_t *hmask = fh_sm;                 // [Bw] holes per word
+    uint32_t *fmask = hmask + Bw;            // [Bw] fillers per word
+    uint32_t *hoff = fmask + Bw;             // [Bw] holes before this word
+    uint32_t *hmv = hoff + Bw;               // [Bw][5]
+    uint32_t *fmv = hmv + 5 * Bw;            // [Bw][5]
+    uint32_t *rows_sh = fmv + 5 * Bw;        // [p.rec_rows][stride]
+    for (int k = tid; k < 2 * Bw; k += CMP_THREADS) hmask[k] = 0;
+    __syncthreads();
+    for (int k = tid; k < h; k += CMP_THREADS) {
+        const int d = hole_of(k), sj = filler_of(k);
+        atomicOr(&hmask[d >> 5], 1u << (d & 31));
+        atomicOr(&fmask[sj >> 5], 1u << (sj & 31));
+    }
+    __syncthreads();
+    for (int k = tid; k < Bw; k += CMP_THREADS) {
+        compress_masks(hmask[k], hmv + k * 5);
+        compress_masks(fmask[k], fmv + k * 5);
+    }
+    if (tid == 0) {
+        uint32_t run = 0;
+        for (int k = 0; k < Bw; ++k) { hoff[k] = run; run += __popc(hmask[k]); }
+    }
+    __syncthreads();
+    const int k0 = n_keep >> 5, k_end = (p.n + 31) >> 5;         // tail words: [k0, k_end)
+    const uint32_t low0 = (n_keep & 31) ? ((1u << (n_keep & 31)) - 1u) : 0u;   // head bits of word k0
+    for (int s0 = 0; s0 < w; s0 += p.rec_rows) {
+        const int nr = min(p.rec_rows, w - s0);
+        for (int i = tid; i < nr * Bw; i += CMP_THREADS) { const int rr = row_of(i); rows_sh[rr * stride + (i - rr * Bw)] = hist_u[(size_t)s0 * Bw + i]; }
+        __syncthreads();
+        for (int r = tid; r < nr; r += CMP_THREADS) {
+            uint32_t *rw = rows_sh + r * stride;
+            const uint32_t saved0 = k0 < Bw ? rw[k0] & low0 : 0u;
+            unsigned long long acc = 0;
+            int fill = 0, o = k0;
+            for (int k = k0; k < k_end; ++k) {
+                const uint32_t mk = fmask[k];
+                const uint32_t c = compress_bits(rw[k], mk, fmv + k * 5);
+                acc |= (unsigned long long)c << fill;
+                fill += __popc(mk);
+                if (fill >= 32) {
+                    rw[o++] = (uint32_t)acc;      // o <= k: the word was already consumed
+                    acc >>= 32;
+                    fill -= 32;
+                }
+            }
+            if (o < Bw) rw[o] = (uint32_t)acc;
+            const int head_words = low0 ? k0 + 1 : k0;
+            for (int wd = 0; wd < head_words; ++wd) {
+                const uint32_t hm = hmask[wd];
+                uint32_t val = (wd == k0) ? saved0 : rw[wd];
+                if (hm) {
+                    const int off = hoff[wd], sw = k0 + (off >> 5), sb = off & 31;
+                    const uint32_t lo = rw[sw], hi = (sw + 1 < Bw) ? rw[sw + 1] : 0u;
+                    const uint32_t bits = __funnelshift_r(lo, hi, sb);          // stream bits off .. off+31
+                    val = (val & ~hm) | expand_bits(bits, hm, hmv + wd * 5);
+                }
+                if (wd == k0) val &= low0;
+                if (wd != k0) rw[wd] = val; else rw[k0] = val;
+            }
+            for (int wd = head_words; wd < Bw; ++wd) rw[wd] = 0;
+        }
+        __syncthreads();
+        for (int i = tid; i < nr * Bw; i += CMP_THREADS) { const int rr = row_of(i); hist_u[(size_t)s0 * Bw + i] = rows_sh[rr * stride + (i - rr * Bw)]; }
+        __syncthreads();
+    }
+    int32_t *pos = p.pos + (size_t)u * p.B;
+    for (int k = tid; k < h; k += CMP_THREADS) pos[hole_of(k)] = pos[filler_of(k)];
+    __syncthreads();                                 // every filler is read before the tail is zeroed
+    for (int j = n_keep + tid; j < p.n; j += CMP_THREADS) pos[j] = 0;
     if (p.n_arr && tid == 0) p.n_arr[u] = n_keep;    // last kernel of the compression: the unit is compacted
 }
 
@@ -335,7 +546,7 @@ __global__ void __launch_bounds__(256) sh_counters_kernel(const uint32_t *hist, 
 
 cudaError_t sh_launch_select(const SelectParams &p_in, bool from_hist, cudaStream_t s, long long *launches) {
     SelectParams p = p_in;
-    size_t smem = sizeof(int) * ((size_t)p.n + p.cmax + 1 + 32 + 2);
+    size_t smem = sizeof(int) * ((size_t)p.n + p.cmax + 1 + 32 + 8 + (p.unordered ? SEL_TIE_CAP : 0));
     const size_t planes = from_hist ? sizeof(uint32_t) * ((size_t)p.w * p.Bw + (size_t)((p.w + 30) / 31) * 5 * p.Bw) : 0;
     p.stage_planes = from_hist && smem + planes <= 96 * 1024;
     if (p.stage_planes) smem += planes;
@@ -360,6 +571,26 @@ cudaError_t sh_launch_select(const SelectParams &p_in, bool from_hist, cudaStrea
 
 cudaError_t sh_launch_compact(const CompactParams &p_in, cudaStream_t s, long long *launches) {
     CompactParams p = p_in;
+    // i / Bw as a multiply-high: exact while i * Bw < 2^32 (i stays below rows-per-pass * Bw <= 2^18)
+    p.bw_magic = p.Bw > 1 ? (uint32_t)(0x100000000ULL / (unsigned)p.Bw) + 1u : 0u;
+    if (p.unordered) {
+        const int stride = p.Bw | 1;
+        const size_t fixed = sizeof(uint32_t) * 13 * (size_t)p.Bw;     // masks, offsets, butterfly masks
+        int rec_rows = (int)((96 * 1024 - fixed) / (stride * 4));
+        if (rec_rows > CMP_THREADS) rec_rows = CMP_THREADS;
+        if (rec_rows > p.w) rec_rows = p.w;
+        if (rec_rows < 1) rec_rows = 1;
+        p.rec_rows = rec_rows;
+        const size_t smem = fixed + sizeof(uint32_t) * (size_t)rec_rows * stride;
+        if (smem > 48 * 1024) {
+            cudaError_t e = cudaFuncSetAttribute(sh_fill_holes_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+        }
+        sh_fill_holes_kernel<<<dim3(p.U, 3, 1), CMP_THREADS, smem, s>>>(p);
+        cudaError_t e = cudaGetLastError();
+        if (e == cudaSuccess && launches) *launches += 1;
+        return e;
+    }
     // K/V rows: chunks of ~32 KB keep several CTAs per SM, so the reads of one
     // overlap the writes of another (measured best on B200 among 16..100 KB)
     const int max_chunk = p.row_bytes > 32 * 1024 ? p.row_bytes : 32 * 1024;

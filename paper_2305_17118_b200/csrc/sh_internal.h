@@ -36,6 +36,7 @@ struct sh_context {
     int split;
     bool split_explicit;   // SH_OPT_SPLIT was set by the caller
     int auto_compress;
+    int unordered;      // SH_OPT_COMPACTION: 0 stable left-compaction, 1 holes filled from the tail (slots unordered)
     int record_mode;    // SH_OPT_RECORD_MODE: 0 record kept online, 1 recomputed at compression from stored queries
     long long record_fresh_t;   // record_mode 1: step for which the bit-planes were last recomputed (-1: never)
     int prefill_chunk;  // SH_OPT_PREFILL_CHUNK: 1 = sh_prefill may batch tokens between compressions
@@ -99,6 +100,13 @@ struct SelectParams {
     int U, B, Bw, w, n, r, m;
     int cmax;                   // largest possible counter value
     const int *n_arr;           // per-unit live rows, or NULL: units whose cache is not full are skipped
+    // unordered mode (holes are filled from the tail, so slots are not sorted by position): the recent
+    // window and the tie-break go by the position array; the result is a list of (hole, filler) moves
+    int unordered;
+    const int32_t *pos;         // [U][B] stream positions
+    const int *t_arr;           // per-unit tokens streamed, or NULL: t below holds for every unit
+    int t;
+    uint16_t *n_moves;          // [U][B] u16 scratch: entry u*B receives the number of moves of unit u
     int stage_planes;           // set by the launcher: copy the unit's bit-planes to shared memory first
 };
 
@@ -112,7 +120,11 @@ struct CompactParams {
     int Bs;                     // scale rows per unit (int4 store)
     int chunk_bytes;            // set by the launcher: shared-memory gather buffer of the row kernel
     int rec_rows;               // set by the launcher: bit-plane rows staged per pass of the record kernel
+    uint32_t bw_magic;          // set by the launcher: floor(2^32 / Bw) + 1
     int *err;                   // device error word (a bounded wait gave up)
+    int unordered;              // moves (hole <- filler) listed in src_idx: holes from the front of the row, fillers
+                                // from its back, their number in n_moves[u*B]
+    const uint16_t *n_moves;
     int *n_arr;                 // per-unit live rows, or NULL: units whose cache is not full are skipped;
                                 // the record kernel, which runs last, takes m off the ones it compacted
 };

@@ -65,6 +65,11 @@ extern "C" int sh_compress_static(sh_handle h, void *stream, int *evicted_per_un
     sp.U = h->U; sp.B = h->B; sp.Bw = h->Bw; sp.w = h->w; sp.n = h->B; sp.r = h->r; sp.m = h->m;
     sp.cmax = h->w;
     sp.n_arr = sh_pnarr(h);
+    sp.unordered = h->unordered;
+    sp.pos = sh_ppos(h);
+    sp.t_arr = sh_ptarr(h);
+    sp.t = (int)h->t;
+    sp.n_moves = reinterpret_cast<uint16_t *>(h->slab + h->L.counters);
     e = sh_launch_select(sp, true, s, &h->launches);
     if (e != cudaSuccess) { h->last_err = e; return SH_ECUDA; }
 
@@ -76,6 +81,8 @@ extern "C" int sh_compress_static(sh_handle h, void *stream, int *evicted_per_un
     cp.src_idx = src_idx;
     cp.U = h->U; cp.B = h->B; cp.Bw = h->Bw; cp.w = h->w; cp.n = h->B; cp.m = h->m;
     cp.n_arr = sh_pnarr(h);
+    cp.unordered = h->unordered;
+    cp.n_moves = sp.n_moves;
     cp.row_bytes = h->row_bytes;
     cp.scale_bytes = h->dtype == SH_INT4_G64_F16 ? (h->D / 64) * 2 : 0;
     cp.Bs = h->Bs;

@@ -164,17 +164,11 @@ __global__ void __launch_bounds__(NTHREADS, CQ == 32 ? 2 : 1) sh_prefill_chunk_k
         }
         *reinterpret_cast<uint4 *>(Qs + row * ROWH + ch * 8) = val;
     }
+    const int32_t *pos_u = p.pos + (size_t)u * p.B;
     if (RECOUNT) {
-        // slots are sorted by position: query i sees the slots whose position is <= its step
-        const int32_t *pos_u = p.pos + (size_t)u * p.B;
-        for (int i = tid; i < CQ; i += NTHREADS) {
-            int lo = 0, hi = (i < c) ? n0 : 0;
-            while (lo < hi) {
-                const int mid = (lo + hi) >> 1;
-                if (pos_u[mid] <= step0 + i) lo = mid + 1; else hi = mid;
-            }
-            nvs[i] = lo;
-        }
+        // a query sees the cached slots whose position does not exceed its step (slots need not be sorted);
+        // every cached slot is scanned, the invisible ones carry a logit of -inf
+        for (int i = tid; i < CQ; i += NTHREADS) nvs[i] = (i < c) ? n0 : 0;
     } else {
         for (int i = tid; i < CQ; i += NTHREADS) nvs[i] = (i < c) ? n0 + qoff + i + 1 : 0;
         if (tid < c) p.pos[(size_t)u * p.B + n0 + qoff + tid] = step0 + tid;
@@ -231,7 +225,8 @@ __global__ void __launch_bounds__(NTHREADS, CQ == 32 ? 2 : 1) sh_prefill_chunk_k
             for (int e = 0; e < 4; ++e) {
                 const int i = wm * 16 + (lane >> 2) + (e >> 1) * 8;                 // query row
                 const int j = kt * KT + wn * (KT / WN) + nb * 8 + (lane & 3) * 2 + (e & 1);   // key slot
-                const bool live = j < nvs[i];                                         // cached rows (and chunk tokens 0..i) the query may see
+                // cached rows (and chunk tokens 0..i) the query may see
+                const bool live = RECOUNT ? (j < nvs[i] && pos_u[j] <= step0 + i) : j < nvs[i];
                 S[(size_t)i * SS + j] = live ? acc[nb][e] * p.scale_log2e : -INFINITY;
             }
         }
@@ -248,7 +243,7 @@ __global__ void __launch_bounds__(NTHREADS, CQ == 32 ? 2 : 1) sh_prefill_chunk_k
         for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
         float sum = 0.f;
         for (int j = lane; j < ntiles * KT; j += 32) {
-            const float e = (j < nv) ? ex2_approx(Si[j] - mx) : 0.f;
+            const float e = (j < nv && Si[j] != -INFINITY) ? ex2_approx(Si[j] - mx) : 0.f;
             Si[j] = e;
             sum += e;
         }
@@ -263,7 +258,7 @@ __global__ void __launch_bounds__(NTHREADS, CQ == 32 ? 2 : 1) sh_prefill_chunk_k
             __syncwarp();
             for (int wd = 0; wd < p.Bw; ++wd) {
                 const int j = (wd << 5) + lane;
-                const bool low = j < nv && Si[j] * tf < sum;
+                const bool low = j < nv && (!RECOUNT || pos_u[j] <= t) && Si[j] * tf < sum;
                 const uint32_t word = __ballot_sync(0xffffffffu, low);
                 if (lane == 0) hrow[wd] = word;
             }

@@ -29,6 +29,52 @@ class LockstepResult:
     max_abs_err: float = 0.0
 
 
+class SortedView:
+    """A handle whose slots are read back in position order.
+
+    With SH_OPT_COMPACTION = 1 the library keeps the surviving tokens in no particular slot order,
+    while the oracle keeps them oldest first.  What each side holds per token (position, record,
+    this step's bit, key and value row) is unique, so the comparison sorts the library's slots by
+    position and stays element by element.  For an ordered handle the permutation is the identity."""
+
+    def __init__(self, handle):
+        self._h = handle
+
+    def __getattr__(self, name):
+        return getattr(self._h, name)
+
+    def _perm(self):
+        n, _, pos, _, _ = self._h.state(pos=True, counters=False, low=False)
+        perm = np.argsort(pos, axis=1, kind="stable")
+        assert (np.diff(np.take_along_axis(pos, perm, axis=1), axis=1) > 0).all(), "duplicate positions in a unit"
+        return n, perm
+
+    def state(self, pos=True, counters=True, low=True, stream=None):
+        n, t, p, c, l = self._h.state(pos=True, counters=counters, low=low, stream=stream)
+        perm = np.argsort(p, axis=1, kind="stable")
+        srt = lambda a: np.take_along_axis(a, perm, axis=1) if a is not None else None
+        return n, t, (srt(p) if pos else None), srt(c), srt(l)
+
+    def state_full(self, stream=None):
+        p, c, l = self._h.state_full(stream)
+        key = np.where(p > 0, p, np.iinfo(np.int32).max)          # free slots (position 0) go last
+        perm = np.argsort(key, axis=1, kind="stable")
+        return tuple(np.take_along_axis(a, perm, axis=1) for a in (p, c, l))
+
+    def export_record(self, unit, stream=None):
+        n, perm = self._perm()
+        planes = self._h.export_record(unit, stream)
+        out = planes.copy()
+        out[:, :n] = planes[:, perm[unit]]
+        return out
+
+    def export_unit(self, unit, stream=None):
+        n, perm = self._perm()
+        K, V = self._h.export_unit(unit, stream)
+        K[:n], V[:n] = K[perm[unit]], V[perm[unit]]
+        return K, V
+
+
 def to_oracle(x: torch.Tensor, units) -> np.ndarray:
     """Rows ``units`` of a [U, d] storage-dtype tensor as exact fp64."""
     return x[units].to(torch.float64).cpu().numpy()

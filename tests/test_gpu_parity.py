@@ -6,7 +6,7 @@ import pytest
 import torch
 
 import oracle
-from lockstep import run_lockstep, run_lockstep_chunked, run_lockstep_recompute, to_oracle
+from lockstep import SortedView, run_lockstep, run_lockstep_chunked, run_lockstep_recompute, to_oracle
 from paper_2305_17118_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -251,6 +251,77 @@ def test_compaction_moves_rows_bit_identically(sh, dtype):
         assert (K[:n].astype(np.float64) == oK).all() and (V[:n].astype(np.float64) == oV).all()
 
 
+# ---- SH_OPT_COMPACTION = 1: holes filled from the tail, slots in no particular order -------------
+@pytest.mark.parametrize("dtype,d,kernel", [("f32", 64, None), ("f16", 128, None), ("bf16", 128, 2), ("int4", 128, None),
+                                             ("f16", 64, 1)])
+@pytest.mark.parametrize("U,B,r,w,m", [(5, 150, 9, 37, 41), (3, 700, 5, 64, 300), (4, 96, 0, 20, 1), (2, 64, 63, 5, 1),
+                                       (3, 33, 0, 1, 33), (2, 1100, 10, 400, 550), (2, 2400, 10, 1, 1200)])
+def test_lockstep_unordered_compaction(sh, dtype, d, kernel, U, B, r, w, m):
+    """Same protocol as the ordered mode; the library's slots are read back in position order.
+    The last shape (w = 1: counters of 0 or 1) has tie classes beyond the shared-memory list of the
+    selection kernel, the others stay inside it."""
+    T = min(2 * B + 4 * m + 9, 2 * B + 300) if B < 2000 else B + m + 20
+    q, k, v = wl.random_stream(U, d, T, seed=71 + B, dtype=dtype, peaked=3.0, device="cuda")
+    h = SortedView(sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, kernel=kernel, unordered=True))
+    res, _ = run_lockstep(h, dtype, _stream_fn(q, k, v), T, torch.arange(U), TOL[dtype])
+    assert res.compressions >= 2
+    assert res.adoptions <= 1e-4 * res.slot_steps + 2
+
+
+@pytest.mark.parametrize("U,B,r,w,m,sizes", [(5, 150, 9, 37, 41, [64, 7, 33, 1, 50]), (3, 410, 64, 128, 64, [64]),
+                                             (130, 96, 8, 70, 30, [64, 31])])
+def test_lockstep_unordered_chunked_prompt(sh, U, B, r, w, m, sizes):
+    dtype, d, T = "f16", 128, 2 * B + 2 * m + 11
+    q, k, v = wl.random_stream(U, d, T, seed=19 + U, dtype=dtype, peaked=3.0, device="cuda")
+    h = SortedView(sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, unordered=True))
+    blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
+    res, orc = run_lockstep_chunked(h, dtype, blk, T, torch.arange(U), TOL[dtype], chunk_sizes=sizes)
+    assert res.steps == T and res.compressions >= 3
+    q2, k2, v2 = wl.random_stream(U, d, 40, seed=98, dtype=dtype, peaked=3.0, device="cuda")
+    run_lockstep(h, dtype, lambda t: (q2[t - T - 1], k2[t - T - 1], v2[t - T - 1]), 40, torch.arange(U), TOL[dtype], orc=orc)
+
+
+@pytest.mark.parametrize("U,B,r,w,m", [(5, 150, 9, 37, 41), (3, 410, 64, 128, 64), (140, 96, 8, 70, 30)])
+def test_lockstep_unordered_record_recomputed(sh, U, B, r, w, m):
+    dtype, d, T = "bf16", 128, 2 * B + 3 * m + 5
+    q, k, v = wl.random_stream(U, d, T, seed=29 + U, dtype=dtype, peaked=3.0, device="cuda")
+    h = SortedView(sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, recompute_record=True, unordered=True))
+    res, orc = run_lockstep_recompute(h, dtype, _stream_fn(q, k, v), T, torch.arange(U), TOL[dtype])
+    assert res.compressions >= 4
+
+
+def test_unordered_compaction_moves_at_most_m_rows_and_keeps_them_bit_identical(sh):
+    """Rows that stay are not touched: a slot below n - m that survives a compression holds the same
+    token before and after; and every kept token's key and value rows equal the oracle's."""
+    U, d, B, r, w, m, T, dtype = 4, 128, 96, 8, 20, 40, 200, "f16"
+    q, k, v = wl.random_stream(U, d, T, seed=3, dtype=dtype, peaked=3.0, device="cuda")
+    raw = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, unordered=True)
+    h = SortedView(raw)
+    orc = oracle.Oracle(U, B, r, w, m, d)
+    idx = torch.arange(U, device="cuda")
+    for t in range(T):
+        h.decode_step(q[t], k[t], v[t])
+        out, alpha, low, amb = orc.attend(to_oracle(q[t], idx), to_oracle(k[t], idx), to_oracle(v[t], idx))
+        glow = h.state()[4]
+        orc.record(glow if not ((glow != low) & ~amb).any() else low)
+        if orc.full:
+            before = raw.state(counters=False, low=False)[2].copy()
+            orc.compress()
+            assert raw.compress() == m
+            n2, _, after, _, _ = raw.state(counters=False, low=False)
+            assert n2 == B - m
+            for u in range(U):
+                head = before[u, : B - m]
+                kept = np.isin(head, orc.positions()[u])
+                assert (after[u][kept] == head[kept]).all()          # survivors in the head did not move
+            assert (np.sort(after, axis=1) == orc.positions()).all()
+    n = h.n
+    for u in range(U):
+        K, V = h.export_unit(u)
+        oK, oV = orc.cache(u)
+        assert (K[:n].astype(np.float64) == oK).all() and (V[:n].astype(np.float64) == oV).all()
+
+
 def test_prefill_equals_token_by_token_steps(sh):
     U, d, B, r, w, m, T, dtype = 6, 128, 80, 8, 24, 30, 260, "f16"
     q, k, v = wl.random_stream(U, d, T, seed=5, dtype=dtype, peaked=3.0, device="cuda")
@@ -300,8 +371,9 @@ def test_snapshot_restore_replays_identically(sh):
     assert s1[0] == s2[0] and s1[1] == s2[1] and all((x == y).all() for x, y in zip(s1[2:], s2[2:]))
 
 
-@pytest.mark.parametrize("dtype,kernel", [("f16", None), ("bf16", 2), ("f16", 1), ("f32", None)])
-def test_ragged_sequences_lockstep(sh, dtype, kernel):
+@pytest.mark.parametrize("dtype,kernel,unordered", [("f16", None, False), ("bf16", 2, False), ("f16", 1, False),
+                                                    ("f32", None, False), ("f16", None, True), ("bf16", 2, True)])
+def test_ragged_sequences_lockstep(sh, dtype, kernel, unordered):
     """Sequences of different prompt lengths in one handle (sh_prefill_ragged), then decode steps in
     lockstep: one oracle per sequence, each with its own n, t and compression schedule."""
     d = 128 if dtype != "f32" else 64
@@ -309,7 +381,7 @@ def test_ragged_sequences_lockstep(sh, dtype, kernel):
     nseq, ups, B, r, w, m, T_dec = len(lengths), 3, 96, 8, 40, 30, 170
     U, p_max = nseq * ups, max(lengths)
     q, k, v = wl.random_stream(U, d, p_max + T_dec, seed=51, dtype=dtype, peaked=3.0, device="cuda")
-    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, kernel=kernel)
+    h = SortedView(sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, kernel=kernel, unordered=unordered))
     out_p = torch.zeros(p_max, U, d, device="cuda")
     h.prefill_ragged(q[:p_max].contiguous(), k[:p_max].contiguous(), v[:p_max].contiguous(), lengths, out_p)
     orcs, ok = [], []

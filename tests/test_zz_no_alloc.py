@@ -18,14 +18,14 @@ from paper_2305_17118_b200 import workloads as wl
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("dtype", ["f16", "int4"])
-def test_static_scratch_compress_matches_regular_compress_twice(dtype):
+@pytest.mark.parametrize("dtype,unordered", [("f16", False), ("int4", False), ("f16", True)])
+def test_static_scratch_compress_matches_regular_compress_twice(dtype, unordered):
     from paper_2305_17118_b200 import binding as sh
     U, d, B, r, w, m = 37, 128, 100, 8, 24, 30
     T = B + m + 5     # fills once at step B, again at step B + m
     q, k, v = wl.random_stream(U, d, T, seed=21, dtype=dtype, peaked=3.0, device="cuda")
-    a = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
-    b = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    a = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, unordered=unordered)
+    b = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, unordered=unordered)
     calls = 0
     for t in range(T):
         oa = a.decode_step(q[t], k[t], v[t])
