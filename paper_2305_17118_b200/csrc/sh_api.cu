@@ -105,8 +105,6 @@ int do_compress(sh_context *c, cudaStream_t s) {
     sp.t_arr = sh_ptarr(c);
     sp.t = (int)c->t;
     sp.n_moves = reinterpret_cast<uint16_t *>(c->slab + c->L.counters) + (size_t)c->u0 * c->B;
-    cudaError_t e = sh_launch_select(sp, true, s, &c->launches);
-    if (e != cudaSuccess) return cuda_fail(c, e);
     CompactParams cp = {};
     cp.K = sh_pK(c); cp.V = sh_pV(c);
     cp.Ks = sh_pKs(c); cp.Vs = sh_pVs(c);
@@ -121,7 +119,13 @@ int do_compress(sh_context *c, cudaStream_t s) {
     cp.n_arr = sh_pnarr(c);
     cp.unordered = c->unordered;
     cp.n_moves = sp.n_moves;
-    e = sh_launch_compact(cp, s, &c->launches);
+    cudaError_t e;
+    if (c->unordered) {
+        e = sh_launch_compress_unordered(sp, cp, s, &c->launches);
+    } else {
+        e = sh_launch_select(sp, true, s, &c->launches);
+        if (e == cudaSuccess) e = sh_launch_compact(cp, s, &c->launches);
+    }
     if (e != cudaSuccess) return cuda_fail(c, e);
     sh_after_compression(c);
     return SH_OK;

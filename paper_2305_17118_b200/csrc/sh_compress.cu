@@ -41,6 +41,160 @@ __device__ __forceinline__ int slot_counter(const uint32_t *hist_u, int w, int B
     return cnt;
 }
 
+// Bit compress of one word (keep the bits under mask m, squeezed to the right) with the five
+// butterfly masks of the classic network, which depend on m alone.
+__device__ __forceinline__ uint32_t compress_bits(uint32_t x, uint32_t m, const uint32_t *mv) {
+    x &= m;
+#pragma unroll
+    for (int i = 0; i < 5; ++i) {
+        const uint32_t t = x & mv[i];
+        x = (x ^ t) | (t >> (1 << i));
+    }
+    return x;
+}
+
+// Inverse of compress_bits: the low popc(m) bits of x spread to the set bits of m (same masks, reverse order).
+__device__ __forceinline__ uint32_t expand_bits(uint32_t x, uint32_t m, const uint32_t *mv) {
+#pragma unroll
+    for (int i = 4; i >= 0; --i) {
+        const uint32_t t = x << (1 << i);
+        x = (x & ~mv[i]) | (t & mv[i]);
+    }
+    return x & m;
+}
+
+__device__ __forceinline__ void compress_masks(uint32_t m, uint32_t *mv_out) {
+    uint32_t mk = ~m << 1;
+#pragma unroll
+    for (int i = 0; i < 5; ++i) {
+        uint32_t mp = mk ^ (mk << 1);
+        mp ^= mp << 2; mp ^= mp << 4; mp ^= mp << 8; mp ^= mp << 16;
+        const uint32_t mv = mp & m;
+        mv_out[i] = mv;
+        m = (m ^ mv) | (mv >> (1 << i));
+        mk &= ~mp;
+    }
+}
+
+// Unordered compaction, record part.  Per-word masks of the holes (slots below n - m that were dropped)
+// and of the fillers (kept slots at or beyond n - m), their butterfly masks, and the number of holes
+// before each word.  hmask..fmv: shared arrays of Bw, Bw, Bw, 5 Bw, 5 Bw words.  Ends with a barrier.
+template <class HoleOf, class FillerOf>
+__device__ __forceinline__ void build_fill_masks(HoleOf hole_of, FillerOf filler_of, int h, int Bw, uint32_t *hmask,
+                                                 uint32_t *fmask, uint32_t *hoff, uint32_t *hmv, uint32_t *fmv) {
+    const int tid = threadIdx.x, nt = blockDim.x;
+    for (int k = tid; k < Bw; k += nt) { hmask[k] = 0; fmask[k] = 0; }
+    __syncthreads();
+    for (int k = tid; k < h; k += nt) {
+        const int d = hole_of(k), sj = filler_of(k);
+        atomicOr(&hmask[d >> 5], 1u << (d & 31));
+        atomicOr(&fmask[sj >> 5], 1u << (sj & 31));
+    }
+    __syncthreads();
+    for (int k = tid; k < Bw; k += nt) {
+        compress_masks(hmask[k], hmv + k * 5);
+        compress_masks(fmask[k], fmv + k * 5);
+    }
+    if (tid == 0) {
+        uint32_t run = 0;
+        for (int k = 0; k < Bw; ++k) { hoff[k] = run; run += __popc(hmask[k]); }
+    }
+    __syncthreads();
+}
+
+// In every one of the nr staged bit-plane rows (row stride `stride` words, one thread per row) the
+// fillers' bits, taken in slot order, go to the holes in slot order: the tail words are compressed by the
+// filler mask into a bit stream (written over the tail, which is dead afterwards), each head word takes
+// its share of the stream expanded to its holes, and the bits from n_keep on are cleared.
+__device__ __forceinline__ void fill_record_rows(uint32_t *rows_sh, int stride, int nr, int n, int n_keep, int Bw,
+                                                 const uint32_t *hmask, const uint32_t *fmask, const uint32_t *hoff,
+                                                 const uint32_t *hmv, const uint32_t *fmv) {
+    const int k0 = n_keep >> 5, k_end = (n + 31) >> 5;         // tail words: [k0, k_end)
+    const uint32_t low0 = (n_keep & 31) ? ((1u << (n_keep & 31)) - 1u) : 0u;   // head bits of word k0
+    for (int r = threadIdx.x; r < nr; r += blockDim.x) {
+        uint32_t *rw = rows_sh + r * stride;
+        const uint32_t saved0 = rw[k0] & low0;
+        unsigned long long acc = 0;
+        int fill = 0, o = k0;
+        for (int k = k0; k < k_end; ++k) {
+            const uint32_t mk = fmask[k];
+            const uint32_t c = compress_bits(rw[k], mk, fmv + k * 5);
+            acc |= (unsigned long long)c << fill;
+            fill += __popc(mk);
+            if (fill >= 32) {
+                rw[o++] = (uint32_t)acc;      // o <= k: the word was already consumed
+                acc >>= 32;
+                fill -= 32;
+            }
+        }
+        if (o < Bw) rw[o] = (uint32_t)acc;
+        const int head_words = low0 ? k0 + 1 : k0;
+        for (int wd = 0; wd < head_words; ++wd) {
+            const uint32_t hm = hmask[wd];
+            uint32_t val = (wd == k0) ? saved0 : rw[wd];
+            if (hm) {
+                const int off = hoff[wd], sw = k0 + (off >> 5), sb = off & 31;
+                const uint32_t lo = rw[sw], hi = (sw + 1 < Bw) ? rw[sw + 1] : 0u;
+                const uint32_t bits = __funnelshift_r(lo, hi, sb);          // stream bits off .. off+31
+                val = (val & ~hm) | expand_bits(bits, hm, hmv + wd * 5);
+            }
+            if (wd == k0) val &= low0;
+            rw[wd] = val;               // word k0 comes last: the stream's first word is no longer needed
+        }
+        for (int wd = head_words; wd < Bw; ++wd) rw[wd] = 0;
+    }
+}
+
+// K and V rows (and int4 scales) of the h moves of one unit: hole <- filler.  Sources and destinations
+// are disjoint.  Four independent 16-byte pieces per thread are in flight: the loads of a batch are
+// issued before its stores.  what: 0 = K, 1 = V, 2 = both.
+template <class HoleOf, class FillerOf>
+__device__ __forceinline__ void fill_rows(const CompactParams &p, int u, int what, int h, HoleOf hole_of, FillerOf filler_of) {
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int lpr = p.row_bytes >> 4, lsh = __ffs(lpr) - 1;     // 16-byte chunks per row: a power of two
+    const int per = h * lpr, first = what == 1 ? per : 0, last = what == 0 ? per : 2 * per;
+    char *Kr = p.K + (size_t)u * p.B * p.row_bytes, *Vr = p.V + (size_t)u * p.B * p.row_bytes;
+    for (int base = first + tid; base < last; base += 4 * nt) {
+        uint4 val[4];
+        char *dst[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int idx = base + i * nt;
+            dst[i] = nullptr;
+            if (idx < last) {
+                char *rows = idx >= per ? Vr : Kr;
+                const int rem = idx >= per ? idx - per : idx;
+                const int k = rem >> lsh, ch = rem & (lpr - 1);
+                dst[i] = rows + (size_t)hole_of(k) * p.row_bytes + ch * 16;
+                val[i] = *reinterpret_cast<const uint4 *>(rows + (size_t)filler_of(k) * p.row_bytes + ch * 16);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (dst[i]) *reinterpret_cast<uint4 *>(dst[i]) = val[i];
+    }
+    for (int side = (what == 1 ? 1 : 0); side <= (what == 0 ? 0 : 1); ++side) {
+        if (p.scale_bytes == 4) {
+            uint32_t *sc = reinterpret_cast<uint32_t *>(side == 0 ? p.Ks : p.Vs) + (size_t)u * p.Bs;
+            for (int k = tid; k < h; k += nt) sc[hole_of(k)] = sc[filler_of(k)];
+        } else if (p.scale_bytes == 2) {
+            uint16_t *sc = reinterpret_cast<uint16_t *>(side == 0 ? p.Ks : p.Vs) + (size_t)u * p.Bs;
+            for (int k = tid; k < h; k += nt) sc[hole_of(k)] = sc[filler_of(k)];
+        }
+    }
+}
+
+// Positions of the h moves of one unit, then the freed tail is zeroed and the unit's row count updated.
+template <class HoleOf, class FillerOf>
+__device__ __forceinline__ void fill_positions(const CompactParams &p, int u, int h, HoleOf hole_of, FillerOf filler_of) {
+    const int tid = threadIdx.x, nt = blockDim.x, n_keep = p.n - p.m;
+    int32_t *pos = p.pos + (size_t)u * p.B;
+    for (int k = tid; k < h; k += nt) pos[hole_of(k)] = pos[filler_of(k)];
+    __syncthreads();                                 // every filler is read before the tail is zeroed
+    for (int j = n_keep + tid; j < p.n; j += nt) pos[j] = 0;
+    if (p.n_arr && tid == 0) p.n_arr[u] = n_keep;    // the unit is compacted
+}
+
 // Selection: among slots [0, n-r) drop the m with the largest key
 // (counter descending, slot ascending).  Radix-select on the counter value by
 // a shared-memory histogram, then an exact prefix count in slot order inside
@@ -69,15 +223,23 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
             // rows are summed 32 slots at a time: thread (g, k) adds rows g, g+G, ... of
             // word column k into a 5-plane bit-sliced counter (at most 31 rows each), and
             // every slot finally picks its bits out of the G partial counters.
-            const int Bw = p.Bw, w = p.w, G = (w + 30) / 31;
-            for (int i = tid; i < w * Bw; i += SEL_THREADS) planes[i] = hist_u[i];
+            // (the fused path works on the staged rows later, one thread per row: odd row stride there)
+            const int Bw = p.Bw, w = p.w, G = (w + 30) / 31, pst = p.fuse ? (Bw | 1) : Bw;
+            if (p.fuse) {
+                for (int i = tid; i < w * Bw; i += SEL_THREADS) {
+                    const int rr = Bw > 1 ? (int)__umulhi((uint32_t)i, p.bw_magic) : i;      // i / Bw
+                    planes[rr * pst + (i - rr * Bw)] = hist_u[i];
+                }
+            } else {
+                for (int i = tid; i < w * Bw; i += SEL_THREADS) planes[i] = hist_u[i];
+            }
             __syncthreads();
-            uint32_t *part = planes + w * Bw;
+            uint32_t *part = planes + w * pst;
             for (int item = tid; item < G * Bw; item += SEL_THREADS) {
                 const int g = item / Bw, k = item % Bw;
                 uint32_t c0 = 0, c1 = 0, c2 = 0, c3 = 0, c4 = 0;
                 for (int s = g; s < w; s += G) {
-                    uint32_t x = planes[s * Bw + k], t;
+                    uint32_t x = planes[s * pst + k], t;
                     t = c0 & x; c0 ^= x; x = t;
                     t = c1 & x; c1 ^= x; x = t;
                     t = c2 & x; c2 ^= x; x = t;
@@ -197,13 +359,40 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
             fill_carry += tot;
             const int eidx = ev_carry + block_flag_scan(ev, wsum, &tot);
             ev_carry += tot;
-            if (p.src_idx) {
+            if (p.fuse) {
+                if (hole) sm[p.fuse_off + hk] = j;
+                if (filler) sm[p.fuse_off + m + fk] = j;
+            } else if (p.src_idx) {
                 if (hole) p.src_idx[(size_t)u * p.B + hk] = j;
                 if (filler) p.src_idx[(size_t)u * p.B + (p.B - 1 - fk)] = j;
             }
             if (ev && p.evicted) p.evicted[(size_t)u * m + eidx] = j;
         }
-        if (tid == 0 && p.n_moves) p.n_moves[(size_t)u * p.B] = (uint16_t)(0x8000 | hole_carry);   // bit 15: unit selected
+        if (!p.fuse) {
+            if (tid == 0 && p.n_moves) p.n_moves[(size_t)u * p.B] = (uint16_t)(0x8000 | hole_carry);   // bit 15: unit selected
+            return;
+        }
+        // Fused path: the move list stays in shared memory and this CTA carries the moves out.
+        __syncthreads();
+        const int h = hole_carry;
+        const int *hole_sh = sm + p.fuse_off, *fill_sh = hole_sh + m;
+        auto hole_of = [&](int k) { return hole_sh[k]; };
+        auto filler_of = [&](int k) { return fill_sh[k]; };
+        fill_rows(p.mv, u, 2, h, hole_of, filler_of);       // K and V rows: loads in flight during the record work
+        {
+            const int Bw = p.Bw, w = p.w, pst = Bw | 1;
+            uint32_t *hmask = reinterpret_cast<uint32_t *>(sm + p.fuse_off + 2 * m);
+            uint32_t *fmask = hmask + Bw, *hoff = fmask + Bw, *hmv = hoff + Bw, *fmv = hmv + 5 * Bw;
+            build_fill_masks(hole_of, filler_of, h, Bw, hmask, fmask, hoff, hmv, fmv);
+            fill_record_rows(planes, pst, w, n, n_keep, Bw, hmask, fmask, hoff, hmv, fmv);   // the rows staged for counting
+            __syncthreads();
+            uint32_t *hist_w = p.mv.hist + (size_t)u * w * Bw;
+            for (int i = tid; i < w * Bw; i += SEL_THREADS) {
+                const int rr = Bw > 1 ? (int)__umulhi((uint32_t)i, p.bw_magic) : i;
+                hist_w[i] = planes[rr * pst + (i - rr * Bw)];
+            }
+        }
+        fill_positions(p.mv, u, h, hole_of, filler_of);
         return;
     }
     int tie_carry = 0, keep_carry = 0, ev_carry = 0;
@@ -316,16 +505,6 @@ __global__ void __launch_bounds__(ROWS_THREADS) sh_compact_rows_kernel(const Com
 // masks of the classic compress network are computed once per 32-slot word and
 // every row is then handled by one thread: 20 logic operations per source word
 // plus a funnel shift into the output stream.  Bits of the freed slots become 0.
-__device__ __forceinline__ uint32_t compress_bits(uint32_t x, uint32_t m, const uint32_t *mv) {
-    x &= m;
-#pragma unroll
-    for (int i = 0; i < 5; ++i) {
-        const uint32_t t = x & mv[i];
-        x = (x ^ t) | (t >> (1 << i));
-    }
-    return x;
-}
-
 __global__ void __launch_bounds__(CMP_THREADS) sh_compact_record_kernel(const CompactParams p) {
     extern __shared__ uint32_t rec_sm[];
     const int u = blockIdx.x, tid = threadIdx.x;
@@ -398,35 +577,14 @@ __global__ void __launch_bounds__(CMP_THREADS) sh_compact_record_kernel(const Co
     if (p.n_arr && tid == 0) p.n_arr[u] = n_keep;    // last kernel of the compression: the unit is compacted
 }
 
-// Inverse of compress_bits: the low popc(m) bits of x spread to the set bits of m (same masks, reverse order).
-__device__ __forceinline__ uint32_t expand_bits(uint32_t x, uint32_t m, const uint32_t *mv) {
-#pragma unroll
-    for (int i = 4; i >= 0; --i) {
-        const uint32_t t = x << (1 << i);
-        x = (x & ~mv[i]) | (t & mv[i]);
-    }
-    return x & m;
-}
-
-__device__ __forceinline__ void compress_masks(uint32_t m, uint32_t *mv_out) {
-    uint32_t mk = ~m << 1;
-#pragma unroll
-    for (int i = 0; i < 5; ++i) {
-        uint32_t mp = mk ^ (mk << 1);
-        mp ^= mp << 2; mp ^= mp << 4; mp ^= mp << 8; mp ^= mp << 16;
-        const uint32_t mv = mp & m;
-        mv_out[i] = mv;
-        m = (m ^ mv) | (mv >> (1 << i));
-        mk &= ~mp;
-    }
-}
-
 // Unordered compaction: each hole takes the row of its filler.  Holes lie below n - m, fillers at or
-// beyond it, so sources and destinations are disjoint and the moves are independent.  blockIdx.y:
+// beyond it, so sources and destinations are disjoint and the moves are independent.  blockIdx.x % 3:
 // 0 = K rows (+ int4 scales), 1 = V rows (+ scales), 2 = record bit-planes and positions.
 __global__ void __launch_bounds__(CMP_THREADS) sh_fill_holes_kernel(const CompactParams p) {
     extern __shared__ uint32_t fh_sm[];
-    const int u = blockIdx.x, what = blockIdx.y, tid = threadIdx.x;
+    // the three jobs of a unit sit next to each other in the grid: row traffic and the latency-bound
+    // record work then overlap on every SM instead of running one after the other
+    const int u = blockIdx.x / 3, what = blockIdx.x % 3, tid = threadIdx.x;
     // The selection kernel marked the units it handled (the three CTAs of a unit must agree, and the
     // third one updates the unit's row count, so that count cannot be the test here).
     const int marked = p.n_moves[(size_t)u * p.B];
@@ -436,25 +594,9 @@ __global__ void __launch_bounds__(CMP_THREADS) sh_fill_holes_kernel(const Compac
     auto hole_of = [&](int k) { return row[k]; };
     auto filler_of = [&](int k) { return row[p.B - 1 - k]; };
     if (what < 2) {
-        char *rows = (what == 0 ? p.K : p.V) + (size_t)u * p.B * p.row_bytes;
-        const int lpr = p.row_bytes >> 4, lsh = __ffs(lpr) - 1;     // 16-byte chunks per row: a power of two
-        for (int idx = tid; idx < h * lpr; idx += CMP_THREADS) {
-            const int k = idx >> lsh, ch = idx & (lpr - 1);
-            *reinterpret_cast<uint4 *>(rows + (size_t)hole_of(k) * p.row_bytes + ch * 16) =
-                *reinterpret_cast<const uint4 *>(rows + (size_t)filler_of(k) * p.row_bytes + ch * 16);
-        }
-        if (p.scale_bytes == 4) {
-            uint32_t *sc = reinterpret_cast<uint32_t *>(what == 0 ? p.Ks : p.Vs) + (size_t)u * p.Bs;
-            for (int k = tid; k < h; k += CMP_THREADS) sc[hole_of(k)] = sc[filler_of(k)];
-        } else if (p.scale_bytes == 2) {
-            uint16_t *sc = reinterpret_cast<uint16_t *>(what == 0 ? p.Ks : p.Vs) + (size_t)u * p.Bs;
-            for (int k = tid; k < h; k += CMP_THREADS) sc[hole_of(k)] = sc[filler_of(k)];
-        }
+        fill_rows(p, u, what, h, hole_of, filler_of);
         return;
     }
-    // Record.  In every bit-plane row the fillers' bits, taken in slot order, go to the holes in slot
-    // order: the tail words are compressed by the filler mask into a bit stream (written over the tail,
-    // which is dead afterwards), and each head word takes its share of the stream expanded to its holes.
     const int Bw = p.Bw, w = p.w, stride = Bw | 1;
     const uint32_t bw_magic = p.bw_magic;
     auto row_of = [&](int i) { return Bw > 1 ? (int)__umulhi((uint32_t)i, bw_magic) : i; };   // i / Bw
@@ -465,70 +607,24 @@ __global__ void __launch_bounds__(CMP_THREADS) sh_fill_holes_kernel(const Compac
     uint32_t *hmv = hoff + Bw;               // [Bw][5]
     uint32_t *fmv = hmv + 5 * Bw;            // [Bw][5]
     uint32_t *rows_sh = fmv + 5 * Bw;        // [p.rec_rows][stride]
-    for (int k = tid; k < 2 * Bw; k += CMP_THREADS) hmask[k] = 0;
-    __syncthreads();
-    for (int k = tid; k < h; k += CMP_THREADS) {
-        const int d = hole_of(k), sj = filler_of(k);
-        atomicOr(&hmask[d >> 5], 1u << (d & 31));
-        atomicOr(&fmask[sj >> 5], 1u << (sj & 31));
-    }
-    __syncthreads();
-    for (int k = tid; k < Bw; k += CMP_THREADS) {
-        compress_masks(hmask[k], hmv + k * 5);
-        compress_masks(fmask[k], fmv + k * 5);
-    }
-    if (tid == 0) {
-        uint32_t run = 0;
-        for (int k = 0; k < Bw; ++k) { hoff[k] = run; run += __popc(hmask[k]); }
-    }
-    __syncthreads();
-    const int k0 = n_keep >> 5, k_end = (p.n + 31) >> 5;         // tail words: [k0, k_end)
-    const uint32_t low0 = (n_keep & 31) ? ((1u << (n_keep & 31)) - 1u) : 0u;   // head bits of word k0
-    for (int s0 = 0; s0 < w; s0 += p.rec_rows) {
+    auto stage_rows = [&](int s0) {
         const int nr = min(p.rec_rows, w - s0);
         for (int i = tid; i < nr * Bw; i += CMP_THREADS) { const int rr = row_of(i); rows_sh[rr * stride + (i - rr * Bw)] = hist_u[(size_t)s0 * Bw + i]; }
-        __syncthreads();
-        for (int r = tid; r < nr; r += CMP_THREADS) {
-            uint32_t *rw = rows_sh + r * stride;
-            const uint32_t saved0 = k0 < Bw ? rw[k0] & low0 : 0u;
-            unsigned long long acc = 0;
-            int fill = 0, o = k0;
-            for (int k = k0; k < k_end; ++k) {
-                const uint32_t mk = fmask[k];
-                const uint32_t c = compress_bits(rw[k], mk, fmv + k * 5);
-                acc |= (unsigned long long)c << fill;
-                fill += __popc(mk);
-                if (fill >= 32) {
-                    rw[o++] = (uint32_t)acc;      // o <= k: the word was already consumed
-                    acc >>= 32;
-                    fill -= 32;
-                }
-            }
-            if (o < Bw) rw[o] = (uint32_t)acc;
-            const int head_words = low0 ? k0 + 1 : k0;
-            for (int wd = 0; wd < head_words; ++wd) {
-                const uint32_t hm = hmask[wd];
-                uint32_t val = (wd == k0) ? saved0 : rw[wd];
-                if (hm) {
-                    const int off = hoff[wd], sw = k0 + (off >> 5), sb = off & 31;
-                    const uint32_t lo = rw[sw], hi = (sw + 1 < Bw) ? rw[sw + 1] : 0u;
-                    const uint32_t bits = __funnelshift_r(lo, hi, sb);          // stream bits off .. off+31
-                    val = (val & ~hm) | expand_bits(bits, hm, hmv + wd * 5);
-                }
-                if (wd == k0) val &= low0;
-                if (wd != k0) rw[wd] = val; else rw[k0] = val;
-            }
-            for (int wd = head_words; wd < Bw; ++wd) rw[wd] = 0;
+    };
+    stage_rows(0);                           // does not depend on the move list: in flight while the masks are built
+    build_fill_masks(hole_of, filler_of, h, Bw, hmask, fmask, hoff, hmv, fmv);
+    for (int s0 = 0; s0 < w; s0 += p.rec_rows) {
+        const int nr = min(p.rec_rows, w - s0);
+        if (s0) {
+            stage_rows(s0);
+            __syncthreads();
         }
+        fill_record_rows(rows_sh, stride, nr, p.n, n_keep, Bw, hmask, fmask, hoff, hmv, fmv);
         __syncthreads();
         for (int i = tid; i < nr * Bw; i += CMP_THREADS) { const int rr = row_of(i); hist_u[(size_t)s0 * Bw + i] = rows_sh[rr * stride + (i - rr * Bw)]; }
         __syncthreads();
     }
-    int32_t *pos = p.pos + (size_t)u * p.B;
-    for (int k = tid; k < h; k += CMP_THREADS) pos[hole_of(k)] = pos[filler_of(k)];
-    __syncthreads();                                 // every filler is read before the tail is zeroed
-    for (int j = n_keep + tid; j < p.n; j += CMP_THREADS) pos[j] = 0;
-    if (p.n_arr && tid == 0) p.n_arr[u] = n_keep;    // last kernel of the compression: the unit is compacted
+    fill_positions(p, u, h, hole_of, filler_of);     // last job of the compression for this unit
 }
 
 __global__ void __launch_bounds__(256) sh_counters_kernel(const uint32_t *hist, uint16_t *counters, int B, int Bw,
@@ -544,12 +640,32 @@ __global__ void __launch_bounds__(256) sh_counters_kernel(const uint32_t *hist, 
 
 }  // namespace
 
-cudaError_t sh_launch_select(const SelectParams &p_in, bool from_hist, cudaStream_t s, long long *launches) {
+namespace {
+// fuse_with != NULL: take the fused unordered path if its shared arrays fit (reported in *fused)
+cudaError_t launch_select(const SelectParams &p_in, bool from_hist, cudaStream_t s, long long *launches,
+                          const CompactParams *fuse_with, bool *fused) {
     SelectParams p = p_in;
+    p.fuse = 0;
+    p.bw_magic = p.Bw > 1 ? (uint32_t)(0x100000000ULL / (unsigned)p.Bw) + 1u : 0u;
     size_t smem = sizeof(int) * ((size_t)p.n + p.cmax + 1 + 32 + 8 + (p.unordered ? SEL_TIE_CAP : 0));
-    const size_t planes = from_hist ? sizeof(uint32_t) * ((size_t)p.w * p.Bw + (size_t)((p.w + 30) / 31) * 5 * p.Bw) : 0;
-    p.stage_planes = from_hist && smem + planes <= 96 * 1024;
-    if (p.stage_planes) smem += planes;
+    const size_t partial = sizeof(uint32_t) * (size_t)((p.w + 30) / 31) * 5 * p.Bw;
+    const size_t planes = from_hist ? sizeof(uint32_t) * (size_t)p.w * p.Bw + partial : 0;
+    if (fuse_with && from_hist && p.unordered) {
+        const size_t planes_odd = sizeof(uint32_t) * (size_t)p.w * (p.Bw | 1) + partial;
+        const size_t lists = sizeof(int) * (2 * (size_t)p.m + 13 * (size_t)p.Bw);
+        if (smem + planes_odd + lists <= 96 * 1024) {
+            p.fuse = 1;
+            p.stage_planes = 1;
+            p.fuse_off = (int)((smem + planes_odd) / sizeof(int));
+            p.mv = *fuse_with;
+            smem += planes_odd + lists;
+        }
+    }
+    if (!p.fuse) {
+        p.stage_planes = from_hist && smem + planes <= 96 * 1024;
+        if (p.stage_planes) smem += planes;
+    }
+    if (fused) *fused = p.fuse != 0;
     cudaError_t e;
     if (from_hist) {
         if (smem > 48 * 1024) {
@@ -567,6 +683,18 @@ cudaError_t sh_launch_select(const SelectParams &p_in, bool from_hist, cudaStrea
     e = cudaGetLastError();
     if (e == cudaSuccess && launches) *launches += 1;
     return e;
+}
+}  // namespace
+
+cudaError_t sh_launch_select(const SelectParams &p, bool from_hist, cudaStream_t s, long long *launches) {
+    return launch_select(p, from_hist, s, launches, nullptr, nullptr);
+}
+
+cudaError_t sh_launch_compress_unordered(const SelectParams &sp, const CompactParams &cp, cudaStream_t s, long long *launches) {
+    bool fused = false;
+    cudaError_t e = launch_select(sp, true, s, launches, &cp, &fused);
+    if (e != cudaSuccess || fused) return e;
+    return sh_launch_compact(cp, s, launches);
 }
 
 cudaError_t sh_launch_compact(const CompactParams &p_in, cudaStream_t s, long long *launches) {
@@ -586,7 +714,7 @@ cudaError_t sh_launch_compact(const CompactParams &p_in, cudaStream_t s, long lo
             cudaError_t e = cudaFuncSetAttribute(sh_fill_holes_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
         }
-        sh_fill_holes_kernel<<<dim3(p.U, 3, 1), CMP_THREADS, smem, s>>>(p);
+        sh_fill_holes_kernel<<<3 * p.U, CMP_THREADS, smem, s>>>(p);
         cudaError_t e = cudaGetLastError();
         if (e == cudaSuccess && launches) *launches += 1;
         return e;

@@ -92,24 +92,6 @@ struct DecodeParams {
     float scale_log2e;
 };
 
-struct SelectParams {
-    const uint32_t *hist;       // bit-planes, or
-    const uint16_t *counters;   // [U][n] caller-supplied records
-    int32_t *src_idx;           // [U][B] or NULL
-    int32_t *evicted;           // [U][m] or NULL
-    int U, B, Bw, w, n, r, m;
-    int cmax;                   // largest possible counter value
-    const int *n_arr;           // per-unit live rows, or NULL: units whose cache is not full are skipped
-    // unordered mode (holes are filled from the tail, so slots are not sorted by position): the recent
-    // window and the tie-break go by the position array; the result is a list of (hole, filler) moves
-    int unordered;
-    const int32_t *pos;         // [U][B] stream positions
-    const int *t_arr;           // per-unit tokens streamed, or NULL: t below holds for every unit
-    int t;
-    uint16_t *n_moves;          // [U][B] u16 scratch: entry u*B receives the number of moves of unit u
-    int stage_planes;           // set by the launcher: copy the unit's bit-planes to shared memory first
-};
-
 struct CompactParams {
     char *K, *V, *Ks, *Vs;
     uint32_t *hist;
@@ -129,6 +111,31 @@ struct CompactParams {
                                 // the record kernel, which runs last, takes m off the ones it compacted
 };
 
+struct SelectParams {
+    const uint32_t *hist;       // bit-planes, or
+    const uint16_t *counters;   // [U][n] caller-supplied records
+    int32_t *src_idx;           // [U][B] or NULL
+    int32_t *evicted;           // [U][m] or NULL
+    int U, B, Bw, w, n, r, m;
+    int cmax;                   // largest possible counter value
+    const int *n_arr;           // per-unit live rows, or NULL: units whose cache is not full are skipped
+    // unordered mode (holes are filled from the tail, so slots are not sorted by position): the recent
+    // window and the tie-break go by the position array; the result is a list of (hole, filler) moves
+    int unordered;
+    const int32_t *pos;         // [U][B] stream positions
+    const int *t_arr;           // per-unit tokens streamed, or NULL: t below holds for every unit
+    int t;
+    uint16_t *n_moves;          // [U][B] u16 scratch: entry u*B receives the number of moves of unit u
+    int stage_planes;           // set by the launcher: copy the unit's bit-planes to shared memory first
+    // fused unordered compression (set by the launcher when everything fits in shared memory): the selecting CTA
+    // also moves the rows, the record bits and the positions of its unit; no move list leaves the CTA
+    int fuse;
+    int fuse_off;               // offset (in ints) of the fused path's shared arrays
+    uint32_t bw_magic;          // floor(2^32 / Bw) + 1
+    CompactParams mv;
+};
+
+
 // Launchers (each returns the cudaError_t of its launch and adds to *launches).
 cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches);
 // Pipelined (bulk-copy ring) variant of the decode kernel and its applicability test.
@@ -146,6 +153,9 @@ cudaError_t sh_launch_recount(const sh_context *c, cudaStream_t s, long long *la
 // Recompute the record if the handle is in recompute mode and has not done so for the current step.
 int sh_recount_if_needed(sh_context *c, cudaStream_t s);
 cudaError_t sh_launch_select(const SelectParams &p, bool from_hist, cudaStream_t s, long long *launches);
+// Unordered compression (SH_OPT_COMPACTION = 1): one fused launch where the unit's bit-planes fit in shared
+// memory, else the selection followed by the hole-filling kernel.
+cudaError_t sh_launch_compress_unordered(const SelectParams &sp, const CompactParams &cp, cudaStream_t s, long long *launches);
 cudaError_t sh_launch_compact(const CompactParams &p, cudaStream_t s, long long *launches);
 cudaError_t sh_launch_counters(const uint32_t *hist, uint16_t *counters, int U, int B, int Bw, int w, int n,
                                const int *n_arr, cudaStream_t s, long long *launches);

@@ -70,9 +70,6 @@ extern "C" int sh_compress_static(sh_handle h, void *stream, int *evicted_per_un
     sp.t_arr = sh_ptarr(h);
     sp.t = (int)h->t;
     sp.n_moves = reinterpret_cast<uint16_t *>(h->slab + h->L.counters);
-    e = sh_launch_select(sp, true, s, &h->launches);
-    if (e != cudaSuccess) { h->last_err = e; return SH_ECUDA; }
-
     CompactParams cp = {};
     cp.K = sh_pK(h); cp.V = sh_pV(h);
     cp.Ks = sh_pKs(h); cp.Vs = sh_pVs(h);
@@ -87,7 +84,12 @@ extern "C" int sh_compress_static(sh_handle h, void *stream, int *evicted_per_un
     cp.scale_bytes = h->dtype == SH_INT4_G64_F16 ? (h->D / 64) * 2 : 0;
     cp.Bs = h->Bs;
     cp.err = reinterpret_cast<int *>(h->slab + h->L.err);
-    e = sh_launch_compact(cp, s, &h->launches);
+    if (h->unordered) {
+        e = sh_launch_compress_unordered(sp, cp, s, &h->launches);
+    } else {
+        e = sh_launch_select(sp, true, s, &h->launches);
+        if (e == cudaSuccess) e = sh_launch_compact(cp, s, &h->launches);
+    }
     if (e != cudaSuccess) { h->last_err = e; return SH_ECUDA; }
     sh_after_compression(h);
     if (evicted_per_unit) *evicted_per_unit = h->m;

@@ -255,11 +255,13 @@ def test_compaction_moves_rows_bit_identically(sh, dtype):
 @pytest.mark.parametrize("dtype,d,kernel", [("f32", 64, None), ("f16", 128, None), ("bf16", 128, 2), ("int4", 128, None),
                                              ("f16", 64, 1)])
 @pytest.mark.parametrize("U,B,r,w,m", [(5, 150, 9, 37, 41), (3, 700, 5, 64, 300), (4, 96, 0, 20, 1), (2, 64, 63, 5, 1),
-                                       (3, 33, 0, 1, 33), (2, 1100, 10, 400, 550), (2, 2400, 10, 1, 1200)])
+                                       (3, 33, 0, 1, 33), (2, 1100, 10, 400, 550), (2, 2400, 10, 1, 1200),
+                                       (2, 3000, 10, 400, 1500)])
 def test_lockstep_unordered_compaction(sh, dtype, d, kernel, U, B, r, w, m):
     """Same protocol as the ordered mode; the library's slots are read back in position order.
-    The last shape (w = 1: counters of 0 or 1) has tie classes beyond the shared-memory list of the
-    selection kernel, the others stay inside it."""
+    The shape with w = 1 (counters of 0 or 1) has tie classes beyond the shared-memory list of the
+    selection kernel; the last one is too large for the fused single-launch compression and takes the
+    selection + hole-filling pair; the others run fused."""
     T = min(2 * B + 4 * m + 9, 2 * B + 300) if B < 2000 else B + m + 20
     q, k, v = wl.random_stream(U, d, T, seed=71 + B, dtype=dtype, peaked=3.0, device="cuda")
     h = SortedView(sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, kernel=kernel, unordered=True))
