@@ -376,8 +376,10 @@ def main():
                     help="variant: rebuild the importance record at each compression from stored queries")
     ap.add_argument("--kv-dtype", default=None, choices=["f32", "f16", "bf16", "int4"], help="override the workload's K/V dtype")
     ap.add_argument("--head-dim", type=int, default=None, choices=[64, 128], help="override the workload's head_dim")
-    ap.add_argument("--unordered-compaction", action="store_true",
-                    help="SH_OPT_COMPACTION = 1: holes filled from the tail, at most m rows move per compression")
+    ap.add_argument("--stable-compaction", dest="unordered_compaction", action="store_false",
+                    help="SH_OPT_COMPACTION = 0 (the library's default): stable left-compaction, slots stay sorted by "
+                         "position.  The benchmark runs SH_OPT_COMPACTION = 1 (holes filled from the tail, at most m "
+                         "rows move per compression; same kept sets)")
     ap.add_argument("--no-prefill-chunk", action="store_true", help="stream the prompt one decode step per token")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (tuning runs)")
     args = ap.parse_args()

@@ -35,30 +35,41 @@ class SortedView:
     With SH_OPT_COMPACTION = 1 the library keeps the surviving tokens in no particular slot order,
     while the oracle keeps them oldest first.  What each side holds per token (position, record,
     this step's bit, key and value row) is unique, so the comparison sorts the library's slots by
-    position and stays element by element.  For an ordered handle the permutation is the identity."""
+    position and stays element by element.  For an ordered handle the permutation is the identity.
+    ``units``: sort only these units' rows (the others come back as stored), for large handles of
+    which a test checks a sample."""
 
-    def __init__(self, handle):
+    def __init__(self, handle, units=None):
         self._h = handle
+        self._units = None if units is None else np.asarray(units, dtype=np.int64)
+
+    def _argsort(self, key):
+        if self._units is None:
+            return np.argsort(key, axis=1, kind="stable")
+        perm = np.broadcast_to(np.arange(key.shape[1]), key.shape).copy()
+        perm[self._units] = np.argsort(key[self._units], axis=1, kind="stable")
+        return perm
 
     def __getattr__(self, name):
         return getattr(self._h, name)
 
     def _perm(self):
         n, _, pos, _, _ = self._h.state(pos=True, counters=False, low=False)
-        perm = np.argsort(pos, axis=1, kind="stable")
-        assert (np.diff(np.take_along_axis(pos, perm, axis=1), axis=1) > 0).all(), "duplicate positions in a unit"
+        perm = self._argsort(pos)
+        rows = slice(None) if self._units is None else self._units
+        assert (np.diff(np.take_along_axis(pos, perm, axis=1)[rows], axis=1) > 0).all(), "duplicate positions in a unit"
         return n, perm
 
     def state(self, pos=True, counters=True, low=True, stream=None):
         n, t, p, c, l = self._h.state(pos=True, counters=counters, low=low, stream=stream)
-        perm = np.argsort(p, axis=1, kind="stable")
+        perm = self._argsort(p)
         srt = lambda a: np.take_along_axis(a, perm, axis=1) if a is not None else None
         return n, t, (srt(p) if pos else None), srt(c), srt(l)
 
     def state_full(self, stream=None):
         p, c, l = self._h.state_full(stream)
         key = np.where(p > 0, p, np.iinfo(np.int32).max)          # free slots (position 0) go last
-        perm = np.argsort(key, axis=1, kind="stable")
+        perm = self._argsort(key)
         return tuple(np.take_along_axis(a, perm, axis=1) for a in (p, c, l))
 
     def export_record(self, unit, stream=None):

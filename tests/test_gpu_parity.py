@@ -178,13 +178,16 @@ def test_config_opt6b_shapes(sh, name):
     assert res.adoptions <= 1e-4 * res.slot_steps + 2
 
 
-def test_config_opt66b_full_size_sampled_units(sh):
-    """The workload the benchmark times, in its launch configuration, checked on
-    a sample of units all the way through prompt and decode."""
+@pytest.mark.parametrize("unordered", [True, False])
+def test_config_opt66b_full_size_sampled_units(sh, unordered):
+    """The workload the benchmark times, in its launch configuration (unordered compaction; the
+    library's default stable compaction as well), checked on a sample of units all the way through
+    prompt and decode."""
     cfg = wl.CONFIGS["opt66b"]
     st = wl.Stream(cfg, device="cuda")
     units = wl.sample_units(cfg, 24)
-    h = sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, cfg.units, cfg.head_dim, cfg.dtype, auto_compress=False)
+    h = SortedView(sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, cfg.units, cfg.head_dim, cfg.dtype, auto_compress=False,
+                             unordered=unordered), units=units)
     res, _ = run_lockstep(h, cfg.dtype, st.step, cfg.total_steps, units, TOL[cfg.dtype], state_every=64)
     assert res.compressions == 30
     assert res.adoptions <= 1e-4 * res.slot_steps + 2
