@@ -31,6 +31,25 @@ __device__ __forceinline__ int block_flag_scan(bool flag, int *wsum, int *total)
     return before + in_warp;
 }
 
+// Three flags at once: ranks and totals packed 10 bits each (a CTA of at most 1023 threads), one barrier pair.
+__device__ __forceinline__ int block_flag_scan3(bool a, bool b, bool c, int *wsum, int *total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    const uint32_t lt = (1u << lane) - 1u;
+    const uint32_t ba = __ballot_sync(0xffffffffu, a), bb = __ballot_sync(0xffffffffu, b), bc = __ballot_sync(0xffffffffu, c);
+    const int in_warp = __popc(ba & lt) | (__popc(bb & lt) << 10) | (__popc(bc & lt) << 20);
+    __syncthreads();                 // wsum free for reuse
+    if (lane == 0) wsum[warp] = __popc(ba) | (__popc(bb) << 10) | (__popc(bc) << 20);
+    __syncthreads();
+    int before = 0, tot = 0;
+    for (int i = 0; i < nw; ++i) {
+        const int v = wsum[i];
+        if (i < warp) before += v;
+        tot += v;
+    }
+    *total = tot;
+    return before + in_warp;
+}
+
 // I_j = number of set bits of slot j over the w bit-plane rows of its unit.
 __device__ __forceinline__ int slot_counter(const uint32_t *hist_u, int w, int Bw, int j) {
     const uint32_t *col = hist_u + (j >> 5);
@@ -225,7 +244,7 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
             // every slot finally picks its bits out of the G partial counters.
             // (the fused path works on the staged rows later, one thread per row: odd row stride there)
             const int Bw = p.Bw, w = p.w, G = (w + 30) / 31, pst = p.fuse ? (Bw | 1) : Bw;
-            if (p.fuse) {
+            if (pst != Bw) {
                 for (int i = tid; i < w * Bw; i += SEL_THREADS) {
                     const int rr = Bw > 1 ? (int)__umulhi((uint32_t)i, p.bw_magic) : i;      // i / Bw
                     planes[rr * pst + (i - rr * Bw)] = hist_u[i];
@@ -353,12 +372,11 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
             const bool ev = j < n && is_cand(j) && (I > cstar || (I == cstar && pos_u[j] <= pstar));
             const bool hole = ev && j < n_keep, filler = j >= n_keep && j < n && !ev;
             int tot;
-            const int hk = hole_carry + block_flag_scan(hole, wsum, &tot);
-            hole_carry += tot;
-            const int fk = fill_carry + block_flag_scan(filler, wsum, &tot);
-            fill_carry += tot;
-            const int eidx = ev_carry + block_flag_scan(ev, wsum, &tot);
-            ev_carry += tot;
+            const int rk = block_flag_scan3(hole, filler, ev, wsum, &tot);
+            const int hk = hole_carry + (rk & 1023), fk = fill_carry + ((rk >> 10) & 1023), eidx = ev_carry + (rk >> 20);
+            hole_carry += tot & 1023;
+            fill_carry += (tot >> 10) & 1023;
+            ev_carry += tot >> 20;
             if (p.fuse) {
                 if (hole) sm[p.fuse_off + hk] = j;
                 if (filler) sm[p.fuse_off + m + fk] = j;
@@ -387,9 +405,13 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
             fill_record_rows(planes, pst, w, n, n_keep, Bw, hmask, fmask, hoff, hmv, fmv);   // the rows staged for counting
             __syncthreads();
             uint32_t *hist_w = p.mv.hist + (size_t)u * w * Bw;
-            for (int i = tid; i < w * Bw; i += SEL_THREADS) {
-                const int rr = Bw > 1 ? (int)__umulhi((uint32_t)i, p.bw_magic) : i;
-                hist_w[i] = planes[rr * pst + (i - rr * Bw)];
+            if (pst != Bw) {
+                for (int i = tid; i < w * Bw; i += SEL_THREADS) {
+                    const int rr = (int)__umulhi((uint32_t)i, p.bw_magic);
+                    hist_w[i] = planes[rr * pst + (i - rr * Bw)];
+                }
+            } else {
+                for (int i = tid; i < w * Bw; i += SEL_THREADS) hist_w[i] = planes[i];
             }
         }
         fill_positions(p.mv, u, h, hole_of, filler_of);
@@ -406,10 +428,10 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
         tie_carry += tot;
         const bool ev = cand && (I > cstar || (tie && tie_rank < need));
         const bool keep = j < n && !ev;
-        const int dst = keep_carry + block_flag_scan(keep, wsum, &tot);
-        keep_carry += tot;
-        const int eidx = ev_carry + block_flag_scan(ev, wsum, &tot);
-        ev_carry += tot;
+        const int rk = block_flag_scan3(keep, ev, false, wsum, &tot);
+        const int dst = keep_carry + (rk & 1023), eidx = ev_carry + ((rk >> 10) & 1023);
+        keep_carry += tot & 1023;
+        ev_carry += (tot >> 10) & 1023;
         if (keep && p.src_idx) p.src_idx[(size_t)u * p.B + dst] = j;
         if (ev && p.evicted) p.evicted[(size_t)u * m + eidx] = j;
     }
