@@ -253,6 +253,17 @@ int sh_state(sh_handle h, void *stream, int *n_out, long long *t_out, int32_t *p
  */
 int sh_recompute_record(sh_handle h, void *stream);
 
+/*
+ * Analysis entry point (paper, "Ablation on Attention Score Error": the change ratio
+ * (alpha_s - alpha_o) / alpha_o between the scores over a budgeted cache and over the full one).
+ * Attention scores of query q ([heads][head_dim], device, the handle's input dtype) over each unit's
+ * present cache: alpha_out[u][j] = softmax_j(scale * q_u . k_j) over the live slots j < n of unit u,
+ * 0 for the other slots; alpha_out is device memory, fp32, [heads][B].  Nothing is appended, the
+ * record and the counters do not change.  Asynchronous on `stream`.  int4 caches are scored on their
+ * dequantised keys.  Errors: SH_EINVAL (NULL argument), SH_ESTATE (not bound), SH_ECUDA.
+ */
+int sh_scores(sh_handle h, const void *q, float *alpha_out, void *stream);
+
 /* The record bit-planes of one unit, [w][ceil(B/32)] uint32 on the host: row (s mod w) holds, for
  * step s of the last w steps, bit j%32 of word j/32 = [alpha_j < 1/s] for the token now in slot j.
  * Synchronises. */

@@ -29,7 +29,7 @@ INPUT_TORCH_DTYPE = {SH_F32: torch.float32, SH_F16: torch.float16, SH_BF16: torc
 EXPORTS = ["sh_create", "sh_destroy", "sh_workspace_bytes", "sh_bind", "sh_set_option", "sh_decode_step",
            "sh_decode_step_host", "sh_prefill", "sh_prefill_chunk", "sh_prefill_chunk_max", "sh_export_record", "sh_recompute_record", "sh_prefill_ragged",
            "sh_sequence_state",
-           "sh_compress", "sh_compress_static", "sh_select", "sh_state", "sh_export_unit",
+           "sh_compress", "sh_compress_static", "sh_scores", "sh_select", "sh_state", "sh_export_unit",
            "sh_restore", "sh_launch_count", "sh_strerror", "sh_last_cuda_error"]
 
 
@@ -55,6 +55,7 @@ def _load() -> C.CDLL:
     lib.sh_workspace_bytes.restype = C.c_size_t
     lib.sh_bind.argtypes = [vp, vp, C.c_size_t, vp]
     lib.sh_set_option.argtypes = [vp, C.c_int, C.c_double]
+    lib.sh_scores.argtypes = [vp, vp, vp, vp]
     lib.sh_decode_step.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.sh_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.sh_prefill.argtypes = [vp, vp, vp, vp, C.c_int, vp, vp]
@@ -248,6 +249,15 @@ class Handle:
         planes = np.zeros((self.w, self.Bw), dtype=np.uint32)
         self._check(lib.sh_export_record(self._h, unit, planes.ctypes.data, _stream_ptr(stream)))
         return np.unpackbits(planes.view(np.uint8), axis=1, bitorder="little")[:, : self.B].astype(bool)
+
+    # -- sh_scores ---------------------------------------------------------------
+    def scores(self, q: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """Attention scores of ``q`` [U, d] over each unit's present cache: fp32 [U, B], 0 beyond the live slots."""
+        if out is None:
+            out = torch.empty(self.U, self.B, dtype=torch.float32, device=self.device)
+        self._check(lib.sh_scores(self._h, _dev(q, self.in_dtype, self.U * self.D, "q"),
+                                  _dev(out, torch.float32, self.U * self.B, "out"), _stream_ptr(stream)))
+        return out
 
     # -- sh_compress -------------------------------------------------------------
     def compress(self, stream=None) -> int:

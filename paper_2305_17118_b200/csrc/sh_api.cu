@@ -503,6 +503,21 @@ int sh_export_record(sh_handle h, int unit, uint32_t *planes_host, void *stream)
     return SH_OK;
 }
 
+int sh_scores(sh_handle h, const void *q, float *alpha_out, void *stream) {
+    if (!h || !q || !alpha_out) return SH_EINVAL;
+    if (!h->slab) return SH_ESTATE;
+    DecodeParams p = {};
+    p.q = q;
+    p.K = sh_pK(h); p.Ks = sh_pKs(h);
+    p.n_arr = sh_pnarr(h);
+    p.U = h->ucount; p.B = h->B; p.Bs = h->Bs;
+    p.n = h->n;
+    p.scale_log2e = (float)((double)h->scale * LOG2E);
+    cudaError_t e = sh_launch_scores(h, p, alpha_out, (cudaStream_t)stream, &h->launches);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    return SH_OK;
+}
+
 int sh_compress(sh_handle h, void *stream, int *evicted_per_unit) {
     if (!h) return SH_EINVAL;
     if (!h->slab) return SH_ESTATE;

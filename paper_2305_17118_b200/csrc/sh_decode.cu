@@ -578,6 +578,78 @@ cudaError_t launch_one(const sh_context *c, const DecodeParams &p, cudaStream_t 
     return cudaLaunchKernelEx(&cfg, kern, p);
 }
 
+// Attention scores of one query over each unit's present cache, written out in full: alpha_j =
+// softmax_j(scale * q.k_j) over the live slots, 0 beyond them.  Nothing is appended and no state
+// changes.  Analysis only (the score change ratio of the paper's "Ablation on Attention Score Error"
+// compares these between a budgeted cache and a full one); one CTA per unit, plain loads.
+template <int DT, int D>
+__global__ void __launch_bounds__(256) sh_scores_kernel(const DecodeParams p, float *alpha_out) {
+    using E = Elem<DT>;
+    constexpr int EPL = E::EPL, LPR = D / EPL, RPW = 32 / LPR, NW = 8;
+    constexpr bool Q4 = (DT == SH_INT4_G64_F16);
+    const int ROWB = stored_row_bytes<DT>(D);
+    const int INB = (DT == SH_F32) ? D * 4 : D * 2;
+    extern __shared__ __align__(16) float smem[];
+    float *s_sh = smem;                       // [B rounded up]
+    float *wred = s_sh + ((p.B + 31) & ~31);  // [NW]
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int sub = lane / LPR, c = lane % LPR;
+    const int u = blockIdx.x, B = p.B;
+    const int n = p.n_arr ? p.n_arr[u] : p.n;
+    typename E::Q qv;
+    E::load_q(reinterpret_cast<const char *>(p.q) + (size_t)u * INB, c, qv);
+    const char *Kb = p.K + (size_t)u * B * ROWB;
+    const __half *Ksb = Q4 ? reinterpret_cast<const __half *>(p.Ks) + (size_t)u * p.Bs * (D / 64) : nullptr;
+    float lmax = -INFINITY;
+    for (int j0 = warp * RPW; j0 < n; j0 += NW * RPW) {
+        const int j = j0 + sub;
+        float a = 0.f;
+        if (j < n) {
+            a = E::dot(qv, ld_plain(Kb + (size_t)j * ROWB + c * 16));
+            if constexpr (Q4) a *= __half2float(Ksb[(size_t)j * (D / 64) + (c >> 1)]);
+        }
+#pragma unroll
+        for (int o = LPR / 2; o; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        if (j < n && c == 0) {
+            const float sc = a * p.scale_log2e;
+            s_sh[j] = sc;
+            lmax = fmaxf(lmax, sc);
+        }
+    }
+    lmax = warp_max(lmax);
+    if (lane == 0) wred[warp] = lmax;
+    __syncthreads();
+    float M = wred[0];
+#pragma unroll
+    for (int i = 1; i < NW; ++i) M = fmaxf(M, wred[i]);
+    __syncthreads();
+    float lsum = 0.f;
+    for (int j = tid; j < n; j += NW * 32) {
+        const float e = exp2f(s_sh[j] - M);
+        s_sh[j] = e;
+        lsum += e;
+    }
+    lsum = warp_sum(lsum);
+    if (lane == 0) wred[warp] = lsum;
+    __syncthreads();
+    float L = 0.f;
+#pragma unroll
+    for (int i = 0; i < NW; ++i) L += wred[i];
+    for (int j = tid; j < B; j += NW * 32) alpha_out[(size_t)u * B + j] = j < n ? s_sh[j] / L : 0.f;
+}
+
+template <int DT, int D>
+cudaError_t launch_scores(const DecodeParams &p, float *alpha_out, cudaStream_t s) {
+    const size_t smem = sizeof(float) * ((size_t)((p.B + 31) & ~31) + 8);
+    auto kern = sh_scores_kernel<DT, D>;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    kern<<<p.U, 256, smem, s>>>(p, alpha_out);
+    return cudaGetLastError();
+}
+
 template <int DT, int D, int NW, int R>
 cudaError_t launch_split(const sh_context *c, const DecodeParams &p, cudaStream_t s) {
     switch (c->split) {
@@ -590,6 +662,21 @@ cudaError_t launch_split(const sh_context *c, const DecodeParams &p, cudaStream_
 }
 
 }  // namespace
+
+cudaError_t sh_launch_scores(const sh_context *c, const DecodeParams &p, float *alpha_out, cudaStream_t s, long long *launches) {
+    cudaError_t e = cudaErrorInvalidValue;
+    switch (c->dtype) {
+        case SH_F32: e = c->D == 64 ? launch_scores<SH_F32, 64>(p, alpha_out, s) : launch_scores<SH_F32, 128>(p, alpha_out, s); break;
+        case SH_F16: e = c->D == 64 ? launch_scores<SH_F16, 64>(p, alpha_out, s) : launch_scores<SH_F16, 128>(p, alpha_out, s); break;
+        case SH_BF16: e = c->D == 64 ? launch_scores<SH_BF16, 64>(p, alpha_out, s) : launch_scores<SH_BF16, 128>(p, alpha_out, s); break;
+        case SH_INT4_G64_F16:
+            e = c->D == 64 ? launch_scores<SH_INT4_G64_F16, 64>(p, alpha_out, s) : launch_scores<SH_INT4_G64_F16, 128>(p, alpha_out, s);
+            break;
+        default: break;
+    }
+    if (e == cudaSuccess) *launches += 1;
+    return e;
+}
 
 cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches) {
     // Rows of 256 bytes or more stream through the persistent pipelined kernel unless the caller

@@ -138,6 +138,8 @@ struct SelectParams {
 
 // Launchers (each returns the cudaError_t of its launch and adds to *launches).
 cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches);
+// Scores of a query over the present caches (analysis; p.n = live rows, nothing appended).
+cudaError_t sh_launch_scores(const sh_context *c, const DecodeParams &p, float *alpha_out, cudaStream_t s, long long *launches);
 // Pipelined (bulk-copy ring) variant of the decode kernel and its applicability test.
 bool sh_decode_tma_supported(const sh_context *c);
 cudaError_t sh_launch_decode_tma(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches);

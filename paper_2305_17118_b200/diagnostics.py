@@ -62,3 +62,36 @@ def persistence(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, dtype: str, d
             ratio[u] = (first & later).sum() / later.sum()
         frac[u] = first.sum() / t
     return Persistence(ratio, frac, t, l)
+
+
+@dataclasses.dataclass
+class ScoreChange:
+    ratio: np.ndarray        # [units, t] (alpha_s - alpha_o) / alpha_o per stream position 1..t; -1 where the token was dropped
+    kept: np.ndarray         # [units, t] bool: the token is still in the budgeted cache
+    alpha_s: np.ndarray      # [units, t] score over the budgeted cache (0 where dropped)
+    alpha_o: np.ndarray      # [units, t] score over the full cache
+    t: int
+
+
+def score_change_ratio(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, dtype: str, B: int, r: int, w: int, m: int,
+                       device="cuda:0", unordered: bool = False) -> ScoreChange:
+    """Change ratio of the attention scores (the paper's ablation on attention score error):
+    the t tokens of ``q, k, v`` ([t, units, head_dim], storage dtype, CUDA) are streamed through a
+    handle with budget ``B`` (compressing as it goes) and through one that keeps everything; the
+    last step's query is then scored over both caches (``sh_scores``) and compared token by token,
+    a dropped token counting as a score of 0 (ratio -1).  Scores come from the CUDA kernels; only
+    the scatter by position and the division are done here."""
+    t, U, d = q.shape
+    hs = sh.Handle(B, r, w, m, U, d, dtype, device=device, unordered=unordered)
+    ho = sh.Handle(t + 1, 0, 1, 1, U, d, dtype, device=device)          # never fills: the original cache
+    hs.prefill(q, k, v)
+    ho.prefill(q, k, v)
+    a_s = hs.scores(q[t - 1].contiguous()).cpu().numpy().astype(np.float64)
+    a_o = ho.scores(q[t - 1].contiguous()).cpu().numpy().astype(np.float64)[:, :t]
+    n, _, pos, _, _ = hs.state(counters=False, low=False)
+    alpha_s = np.zeros((U, t))
+    kept = np.zeros((U, t), dtype=bool)
+    rows = np.arange(U)[:, None]
+    alpha_s[rows, pos - 1] = a_s[:, :n]
+    kept[rows, pos - 1] = True
+    return ScoreChange((alpha_s - a_o) / a_o, kept, alpha_s, a_o, t)

@@ -475,6 +475,65 @@ def test_persistence_diagnostics_match_oracle_scores(sh):
     assert np.nanmin(got.ratio) >= 0 and np.nanmax(got.ratio) <= 1
 
 
+@pytest.mark.parametrize("dtype,d", [("f32", 64), ("f16", 128), ("bf16", 64), ("int4", 128)])
+@pytest.mark.parametrize("unordered", [False, True])
+def test_scores_entry_point_matches_oracle_scores(sh, dtype, d, unordered):
+    """sh_scores against the oracle's fp64 alpha of the same step, on caches that have been through
+    several compressions, at several fill levels (n not a multiple of anything)."""
+    U, B, r, w, m, T = 5, 150, 9, 37, 41, 330
+    q, k, v = wl.random_stream(U, d, T + 1, seed=83, dtype=dtype, peaked=3.0, device="cuda")
+    h = SortedView(sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, unordered=unordered))
+    _, orc = run_lockstep(h, dtype, _stream_fn(q, k, v), T - 3, torch.arange(U), TOL[dtype])
+    idx = torch.arange(U, device="cuda")
+    for t in range(T - 3, T):
+        h.decode_step(q[t], k[t], v[t])
+        got = h.scores(q[t]).cpu().numpy().astype(np.float64)
+        n, _, pos, _, low = h.state(counters=False)
+        _o, alpha, o_low, amb = orc.attend(to_oracle(q[t], idx), to_oracle(k[t], idx), to_oracle(v[t], idx))
+        assert not ((low != o_low) & ~amb).any()
+        orc.record(low)
+        assert n == orc.n and (pos == orc.positions()).all()
+        raw_pos = h._h.state(counters=False, low=False)[2]
+        by_pos = np.take_along_axis(got[:, :n], np.argsort(raw_pos, axis=1), axis=1)      # slot order -> position order
+        assert np.abs(by_pos - alpha).max() <= 2e-5 * alpha.max() + 1e-9
+        assert (np.abs(by_pos - alpha) <= 1e-4 * alpha + 1e-9).all()
+        assert (got[:, n:] == 0).all() and abs(got.sum(axis=1) - 1).max() < 1e-5
+        assert not orc.full
+
+
+def test_score_change_ratio_diagnostic(sh):
+    """(alpha_s - alpha_o) / alpha_o of the last step's query, budgeted cache against full cache, from
+    the library; the same from two oracles' caches with the softmax written out here.  Units whose
+    kept set differs from the oracle's (a threshold-ambiguous flip on the way) are left out."""
+    from paper_2305_17118_b200 import diagnostics
+    U, d, B, r, w, m, t, dtype = 8, 128, 64, 6, 24, 20, 173, "f16"
+    q, k, v = wl.random_stream(U, d, t, seed=87, dtype=dtype, peaked=3.0, device="cuda")
+    got = diagnostics.score_change_ratio(q, k, v, dtype, B, r, w, m)
+    o_s, o_o = oracle.Oracle(U, B, r, w, m, d), oracle.Oracle(U, t + 1, 0, 1, 1, d)
+    idx = torch.arange(U, device="cuda")
+    for s in range(t):
+        for o in (o_s, o_o):
+            o.step(to_oracle(q[s], idx), to_oracle(k[s], idx), to_oracle(v[s], idx))
+    qf = to_oracle(q[t - 1], idx)
+    checked = 0
+    for u in range(U):
+        def scores(o):
+            K, _ = o.cache(u)
+            z = K @ qf[u] / math.sqrt(d)
+            e = np.exp(z - z.max())
+            return e / e.sum()
+        pos_s = o_s.positions()[u]
+        if got.kept[u].sum() != len(pos_s) or not got.kept[u][pos_s - 1].all():
+            continue
+        want = np.full(t, -1.0)
+        a_o = scores(o_o)
+        want[pos_s - 1] = (scores(o_s) - a_o[pos_s - 1]) / a_o[pos_s - 1]
+        assert np.abs(got.ratio[u] - want).max() <= 2e-4
+        assert (got.ratio[u][~got.kept[u]] == -1).all() and (got.ratio[u][got.kept[u]] >= -1e-4).all()
+        checked += 1
+    assert checked >= U - 2
+
+
 def test_error_codes(sh):
     import ctypes as C
     lib = sh.lib
