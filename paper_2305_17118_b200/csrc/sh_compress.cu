@@ -291,6 +291,76 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
     const int32_t *pos_u = p.unordered ? p.pos + (size_t)u * p.B : nullptr;
     const int t_cut = p.unordered ? (p.t_arr ? p.t_arr[u] : p.t) - p.r : 0;
     auto is_cand = [&](int j) { return p.unordered ? (j < n && pos_u[j] <= t_cut) : j < ncand; };
+    if (p.unordered && p.fuse && m == 1) {
+        // Steady state with one token dropped per step: the candidate with the largest counter goes,
+        // the oldest among equals; the newest row takes its slot.  No histogram, no lists, no bit
+        // networks: a block-wide maximum of (counter, -position), one row pair to move, and in every
+        // bit-plane row one bit to carry from the last slot to the freed one.
+        unsigned long long key = 0;                       // 0: no candidate seen
+        for (int j = tid; j < n; j += SEL_THREADS)
+            if (is_cand(j)) {
+                const unsigned long long kj = ((unsigned long long)(cnt_sh[j] + 1) << 32) | (uint32_t)(0x7fffffff - pos_u[j]);
+                key = kj > key ? kj : key;
+            }
+        unsigned long long best = key;
+#pragma unroll
+        for (int o = 16; o; o >>= 1) {
+            const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+            best = other > best ? other : best;
+        }
+        if (lane == 0) {                                  // per-warp maxima as two words each in the scan scratch
+            wsum[tid >> 5] = (int)(uint32_t)(best >> 32);
+            wsum[16 + (tid >> 5)] = (int)(uint32_t)best;
+        }
+        __syncthreads();
+        best = 0;
+        for (int i = 0; i < SEL_THREADS / 32; ++i) {
+            const unsigned long long bi = ((unsigned long long)(uint32_t)wsum[i] << 32) | (uint32_t)wsum[16 + i];
+            best = bi > best ? bi : best;
+        }
+        for (int j = tid; j < n; j += SEL_THREADS)
+            if (is_cand(j) && (((unsigned long long)(cnt_sh[j] + 1) << 32) | (uint32_t)(0x7fffffff - pos_u[j])) == best) cut[0] = j;
+        __syncthreads();
+        const int hole = cut[0], last = n - 1;            // positions are unique: exactly one thread wrote
+        const CompactParams &c = p.mv;
+        if (tid == 0 && p.evicted) p.evicted[u] = hole;
+        if (hole != last) {
+            const int lpr = c.row_bytes >> 4;
+            if (tid < 2 * lpr) {
+                char *rows = (tid < lpr ? c.K : c.V) + (size_t)u * c.B * c.row_bytes;
+                const int ch = tid < lpr ? tid : tid - lpr;
+                *reinterpret_cast<uint4 *>(rows + (size_t)hole * c.row_bytes + ch * 16) =
+                    *reinterpret_cast<const uint4 *>(rows + (size_t)last * c.row_bytes + ch * 16);
+            }
+            if (tid >= 64 && tid < 66 && c.scale_bytes) {
+                char *sc = (tid == 64 ? c.Ks : c.Vs) + (size_t)u * c.Bs * c.scale_bytes;
+                for (int b = 0; b < c.scale_bytes; ++b) sc[(size_t)hole * c.scale_bytes + b] = sc[(size_t)last * c.scale_bytes + b];
+            }
+        }
+        {
+            const int Bw = p.Bw, pst = Bw | 1;
+            uint32_t *hist_w = c.hist + (size_t)u * p.w * Bw;
+            for (int rr = tid; rr < p.w; rr += SEL_THREADS) {
+                const uint32_t *rw = planes + rr * pst;
+                const uint32_t bit = (rw[last >> 5] >> (last & 31)) & 1u;
+                if ((hole >> 5) == (last >> 5)) {
+                    uint32_t x = rw[last >> 5] & ~(1u << (last & 31));
+                    if (hole != last) x = (x & ~(1u << (hole & 31))) | (bit << (hole & 31));
+                    hist_w[(size_t)rr * Bw + (last >> 5)] = x;
+                } else {
+                    hist_w[(size_t)rr * Bw + (last >> 5)] = rw[last >> 5] & ~(1u << (last & 31));
+                    hist_w[(size_t)rr * Bw + (hole >> 5)] = (rw[hole >> 5] & ~(1u << (hole & 31))) | (bit << (hole & 31));
+                }
+            }
+        }
+        if (tid == 0) {
+            int32_t *pos_w = c.pos + (size_t)u * c.B;
+            if (hole != last) pos_w[hole] = pos_w[last];
+            pos_w[last] = 0;
+            if (c.n_arr) c.n_arr[u] = n - 1;
+        }
+        return;
+    }
     for (int j = tid; j < n; j += SEL_THREADS)
         if (is_cand(j)) atomicAdd(&bins[cnt_sh[j]], 1);
     __syncthreads();

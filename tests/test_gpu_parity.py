@@ -259,7 +259,7 @@ def test_compaction_moves_rows_bit_identically(sh, dtype):
                                              ("f16", 64, 1)])
 @pytest.mark.parametrize("U,B,r,w,m", [(5, 150, 9, 37, 41), (3, 700, 5, 64, 300), (4, 96, 0, 20, 1), (2, 64, 63, 5, 1),
                                        (3, 33, 0, 1, 33), (2, 1100, 10, 400, 550), (2, 2400, 10, 1, 1200),
-                                       (2, 3000, 10, 400, 1500)])
+                                       (2, 3000, 10, 400, 1500), (3, 130, 7, 40, 1)])
 def test_lockstep_unordered_compaction(sh, dtype, d, kernel, U, B, r, w, m):
     """Same protocol as the ordered mode; the library's slots are read back in position order.
     The shape with w = 1 (counters of 0 or 1) has tie classes beyond the shared-memory list of the
