@@ -447,15 +447,18 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
             hole_carry += tot & 1023;
             fill_carry += (tot >> 10) & 1023;
             ev_carry += tot >> 20;
+            // (ranks stay below m as long as the positions of a unit are distinct, which the library
+            // maintains; the bounds keep a workspace restored from foreign data from writing out of range)
             if (p.fuse) {
-                if (hole) sm[p.fuse_off + hk] = j;
-                if (filler) sm[p.fuse_off + m + fk] = j;
+                if (hole && hk < m) sm[p.fuse_off + hk] = j;
+                if (filler && fk < m) sm[p.fuse_off + m + fk] = j;
             } else if (p.src_idx) {
-                if (hole) p.src_idx[(size_t)u * p.B + hk] = j;
-                if (filler) p.src_idx[(size_t)u * p.B + (p.B - 1 - fk)] = j;
+                if (hole && hk < m) p.src_idx[(size_t)u * p.B + hk] = j;
+                if (filler && fk < m) p.src_idx[(size_t)u * p.B + (p.B - 1 - fk)] = j;
             }
-            if (ev && p.evicted) p.evicted[(size_t)u * m + eidx] = j;
+            if (ev && eidx < m && p.evicted) p.evicted[(size_t)u * m + eidx] = j;
         }
+        hole_carry = min(min(hole_carry, fill_carry), m);
         if (!p.fuse) {
             if (tid == 0 && p.n_moves) p.n_moves[(size_t)u * p.B] = (uint16_t)(0x8000 | hole_carry);   // bit 15: unit selected
             return;

@@ -133,6 +133,7 @@ __global__ void __launch_bounds__(NTHREADS, CQ == 32 ? 2 : 1) sh_prefill_chunk_k
     float *S = reinterpret_cast<float *>(tile0 + 2 * KT * ROWH);        // [CQ][SS]
     float *rowL = S + (size_t)CQ * p.SS;                                // [CQ] row sums
     int *nvs = reinterpret_cast<int *>(rowL + CQ);                      // [CQ] keys visible to each query
+    int *pos_sh = nvs + CQ;                                             // [SS] stream positions of the cached slots (recount mode)
 
     const int u = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int wm = warp % WM, wn = warp / WM;
@@ -169,6 +170,7 @@ __global__ void __launch_bounds__(NTHREADS, CQ == 32 ? 2 : 1) sh_prefill_chunk_k
         // a query sees the cached slots whose position does not exceed its step (slots need not be sorted);
         // every cached slot is scanned, the invisible ones carry a logit of -inf
         for (int i = tid; i < CQ; i += NTHREADS) nvs[i] = (i < c) ? n0 : 0;
+        for (int j = tid; j < n0; j += NTHREADS) pos_sh[j] = pos_u[j];
     } else {
         for (int i = tid; i < CQ; i += NTHREADS) nvs[i] = (i < c) ? n0 + qoff + i + 1 : 0;
         if (tid < c) p.pos[(size_t)u * p.B + n0 + qoff + tid] = step0 + tid;
@@ -226,7 +228,7 @@ __global__ void __launch_bounds__(NTHREADS, CQ == 32 ? 2 : 1) sh_prefill_chunk_k
                 const int i = wm * 16 + (lane >> 2) + (e >> 1) * 8;                 // query row
                 const int j = kt * KT + wn * (KT / WN) + nb * 8 + (lane & 3) * 2 + (e & 1);   // key slot
                 // cached rows (and chunk tokens 0..i) the query may see
-                const bool live = RECOUNT ? (j < nvs[i] && pos_u[j] <= step0 + i) : j < nvs[i];
+                const bool live = RECOUNT ? (j < nvs[i] && pos_sh[j] <= step0 + i) : j < nvs[i];
                 S[(size_t)i * SS + j] = live ? acc[nb][e] * p.scale_log2e : -INFINITY;
             }
         }
@@ -258,7 +260,7 @@ __global__ void __launch_bounds__(NTHREADS, CQ == 32 ? 2 : 1) sh_prefill_chunk_k
             __syncwarp();
             for (int wd = 0; wd < p.Bw; ++wd) {
                 const int j = (wd << 5) + lane;
-                const bool low = j < nv && (!RECOUNT || pos_u[j] <= t) && Si[j] * tf < sum;
+                const bool low = j < nv && (!RECOUNT || pos_sh[j] <= t) && Si[j] * tf < sum;
                 const uint32_t word = __ballot_sync(0xffffffffu, low);
                 if (lane == 0) hrow[wd] = word;
             }
@@ -329,7 +331,7 @@ __global__ void __launch_bounds__(NTHREADS, CQ == 32 ? 2 : 1) sh_prefill_chunk_k
 
 template <int DT, int CQ, bool RECOUNT>
 cudaError_t launch_chunk(const ChunkParams &p, cudaStream_t s) {
-    const size_t smem = sizeof(uint16_t) * (size_t)(CQ + 2 * KT) * ROWH + sizeof(float) * ((size_t)CQ * p.SS + 2 * CQ);
+    const size_t smem = sizeof(uint16_t) * (size_t)(CQ + 2 * KT) * ROWH + sizeof(float) * ((size_t)CQ * p.SS + 2 * CQ) + sizeof(int) * (size_t)p.SS;
     auto kern = sh_prefill_chunk_kernel<DT, CQ, RECOUNT>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -340,7 +342,7 @@ cudaError_t launch_chunk(const ChunkParams &p, cudaStream_t s) {
 
 int s_stride(int B) { return ((B + KT - 1) / KT) * KT + 8; }
 size_t smem_need(int CQ, int B) {
-    return sizeof(uint16_t) * (size_t)(CQ + 2 * KT) * ROWH + sizeof(float) * ((size_t)CQ * s_stride(B) + 2 * CQ);
+    return sizeof(uint16_t) * (size_t)(CQ + 2 * KT) * ROWH + sizeof(float) * ((size_t)CQ * s_stride(B) + 2 * CQ) + sizeof(int) * (size_t)s_stride(B);
 }
 
 }  // namespace

@@ -27,6 +27,9 @@ def main():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--rows", type=int, default=None, help="live rows before the first step")
     ap.add_argument("--compress", action="store_true")
+    ap.add_argument("--unordered", action="store_true",
+                    help="SH_OPT_COMPACTION = 1; the cache is then filled by streaming a random prompt through sh_prefill "
+                         "(the selection needs real positions), a few launches before the ones of interest")
     ap.add_argument("--chunk", type=int, default=0, help="instead of decode steps, run one prompt chunk of this many tokens")
     ap.add_argument("--split", type=int, default=None)
     ap.add_argument("--kernel", type=int, default=None, help="1 direct loads, 2 pipelined bulk copies")
@@ -34,7 +37,8 @@ def main():
     cfg = wl.CONFIGS[args.config]
     U, d = args.units, cfg.head_dim
     torch.cuda.set_device(0)
-    h = sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, U, d, cfg.dtype, split=args.split, kernel=args.kernel, auto_compress=True)
+    h = sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, U, d, cfg.dtype, split=args.split, kernel=args.kernel, auto_compress=True,
+                  unordered=args.unordered)
     rows = args.rows if args.rows is not None else (cfg.B - 1 if args.compress else cfg.B - cfg.m // 2)
     if args.chunk:
         rows = args.rows if args.rows is not None else cfg.B - args.chunk
@@ -47,9 +51,14 @@ def main():
         kv.view(torch.float32).normal_()
     else:
         kv.view(torch.float16 if cfg.dtype == "f16" else torch.bfloat16).normal_()
-    sh.lib.sh_restore(h._h, rows, 4 * cfg.B)
     g = torch.Generator(device="cuda")
     g.manual_seed(1)
+    if args.unordered:
+        xp = torch.randn(3, rows, U, d, generator=g, device="cuda").to(cfg.torch_dtype)
+        h.prefill(xp[0], xp[1], xp[2])
+        del xp
+    else:
+        sh.lib.sh_restore(h._h, rows, 4 * cfg.B)
     x = torch.randn(3, args.steps, U, d, generator=g, device="cuda").to(cfg.torch_dtype)
     out = torch.empty(U, d, device="cuda")
     torch.cuda.synchronize()
