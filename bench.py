@@ -199,7 +199,7 @@ def cuda_arm(args, cfg, rank, world):
     streams = [wl.Stream(cfg, device=dev, layer=l + 1000 * rank) for l in range(Ly)]
     handles = [sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, U, d, cfg.dtype, device=dev, auto_compress=False,
                          split=args.split, kernel=args.kernel,
-                         prefill_chunk=False if args.no_prefill_chunk else None,
+                         prefill_chunk=0 if args.no_prefill_chunk else args.prefill_chunk_kernel,
                          recompute_record=args.recompute_record, unordered=args.unordered_compaction)
                for _ in range(Ly)]
 
@@ -380,6 +380,8 @@ def main():
                     help="SH_OPT_COMPACTION = 0 (the library's default): stable left-compaction, slots stay sorted by "
                          "position.  The benchmark runs SH_OPT_COMPACTION = 1 (holes filled from the tail, at most m "
                          "rows move per compression; same kept sets)")
+    ap.add_argument("--prefill-chunk-kernel", type=int, default=None, choices=[1, 2, 3],
+                    help="SH_OPT_PREFILL_CHUNK for the untimed prompt phase: 1 library's choice, 2 warp-level MMA kernel, 3 tcgen05 kernel")
     ap.add_argument("--no-prefill-chunk", action="store_true", help="stream the prompt one decode step per token")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (tuning runs)")
     args = ap.parse_args()

@@ -67,7 +67,8 @@ typedef enum {
                                  token per step; 1: it is recomputed at every compression from the queries of
                                  the last w steps (the library keeps them: heads*w*head_dim extra elements)
                                  scored against the cache as it is then (Algorithm 2 as stated; Section 4.1,
-                                 "Overhead Tradeoff").  fp16/bf16, head_dim 128 only.  Set before sh_bind:
+                                 "Overhead Tradeoff").  fp16/bf16, head_dim 128, budgets up to about 700
+                                 (else SH_EINVAL).  Set before sh_bind:
                                  it changes sh_workspace_bytes. */
     SH_OPT_COMPACTION = 6,    /* 0 (default): stable left-compaction, slots stay sorted by stream position;
                                  1: every hole left by a dropped token below n-m is filled with a kept row from
@@ -75,7 +76,9 @@ typedef enum {
                                  particular order: sh_state's pos tells which token sits where.  The kept set is
                                  the same either way. */
     SH_OPT_PREFILL_CHUNK = 4, /* 1 (default): sh_prefill hands the tokens between two compressions to the chunk
-                                 kernel where the shape allows it; 0: one decode step per token */
+                                 kernel where the shape allows it (fp16/bf16, head_dim 128: the tcgen05 kernel,
+                                 any budget); 0: one decode step per token; 2: the warp-level MMA chunk kernel
+                                 (budgets up to about 700); 3: same as 1 */
     SH_OPT_DECODE_KERNEL = 3  /* 0 (default): chosen from the shape; 1: one CTA (or cluster) per unit with
                                  direct loads; 2: persistent CTAs fed by bulk asynchronous copies
                                  (stored rows of 256 bytes or more: fp32, and fp16/bf16 with head_dim 128; SH_OPT_SPLIT

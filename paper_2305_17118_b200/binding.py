@@ -133,7 +133,7 @@ class Handle:
         if unordered:
             self.set_option(SH_OPT_COMPACTION, 1.0)
         if prefill_chunk is not None:
-            self.set_option(SH_OPT_PREFILL_CHUNK, 1.0 if prefill_chunk else 0.0)
+            self.set_option(SH_OPT_PREFILL_CHUNK, float(int(prefill_chunk)))
         self.set_option(SH_OPT_AUTO_COMPRESS, 1.0 if auto_compress else 0.0)
         self.workspace_bytes = int(lib.sh_workspace_bytes(h))
         with torch.cuda.device(self.device):
@@ -145,7 +145,7 @@ class Handle:
 
     def __del__(self):
         h, self._h = getattr(self, "_h", None), None
-        if h:
+        if h and lib is not None:      # at interpreter shutdown the module globals may already be gone
             lib.sh_destroy(h)
 
     def _check(self, rc: int):

@@ -272,7 +272,7 @@ int sh_set_option(sh_handle h, int key, double value) {
             const int mode = (int)value;
             if (mode != 0 && mode != 1) return SH_EINVAL;
             if (h->slab) return SH_ESTATE;                       // changes the workspace layout
-            if (mode == 1 && sh_prefill_chunk_capacity(h) == 0) return SH_EINVAL;   // needs the tensor-core kernel's shapes
+            if (mode == 1 && !sh_recount_supported(h)) return SH_EINVAL;   // needs the recount kernel's shapes
             h->record_mode = mode;
             make_layout(h);
             return SH_OK;
@@ -283,9 +283,12 @@ int sh_set_option(sh_handle h, int key, double value) {
             h->unordered = mode;
             return SH_OK;
         }
-        case SH_OPT_PREFILL_CHUNK:
-            h->prefill_chunk = value != 0.0;
+        case SH_OPT_PREFILL_CHUNK: {
+            const int mode = (int)value;
+            if (mode < 0 || mode > 3) return SH_EINVAL;
+            h->prefill_chunk = mode;
             return SH_OK;
+        }
         case SH_OPT_DECODE_KERNEL: {
             const int k = (int)value;
             if (k < 0 || k > 2) return SH_EINVAL;

@@ -1,0 +1,431 @@
+// Chunked prompt step on the 5th-generation tensor cores (tcgen05.mma, accumulators in tensor memory).
+//
+// Same computation as the warp-level kernel of sh_prefill_chunk.cu: up to 64 consecutive steps of one
+// unit in one CTA; step i attends with q_i over the n0 cached rows plus the chunk's tokens 0..i and
+// writes its comparison bits into its own bit-plane row.  What differs is where the work runs:
+//
+//   * S = Q.K^T is issued by one thread as tcgen05.mma (M = 128, N = 128 keys per tile, K = 16 per
+//     instruction), operands in shared memory in the canonical no-swizzle core-matrix order, the
+//     fp32 result in tensor memory.  The 64 queries occupy rows 0..63 and again rows 64..127, so
+//     that all 128 lanes of tensor memory carry data: thread i and thread i + 64 own the same
+//     query and split the columns (keys) of every tile between them.
+//   * The row statistics need every logit against the final row sum, and a whole row of logits
+//     (B up to 32768) fits neither in tensor memory nor in shared memory.  So the logits are
+//     computed twice - tensor-core time is cheap here: a first sweep over the key tiles keeps a
+//     running maximum and sum per row (one thread per row: no shuffles), a second sweep recomputes
+//     S tile by tile, forms e = 2^(s - M), packs the record bits of 32 keys into a word by plain
+//     register arithmetic, and hands P (high and low 16-bit parts) to the second contraction.
+//     No limit on B follows from this structure.
+//   * O^T = V^T.P^T accumulates in tensor memory as [128 columns of d][64 queries]: V tiles are
+//     the MN-major A operand exactly as they lie in the cache (rows of d), P the K-major B operand.
+//
+// Every mbarrier wait is bounded; tensor memory is released on every path.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "sh_async.cuh"
+#include "sh_internal.h"
+
+namespace {
+
+using namespace shasync;
+
+constexpr int D = 128;            // head_dim served by this kernel
+constexpr int TN = 64;            // keys per tile
+constexpr int CQ = 64;            // queries per CTA
+constexpr int NT = 256;           // threads per CTA: two per lane of tensor memory (warps w and w + 4 share a lane quadrant)
+constexpr int GROUP = 2048;       // bytes of 8 rows of 256 B in core-matrix order: [16 chunks][8 rows][16 B]
+constexpr int TILE = (TN / 8) * GROUP;          // 32 KB
+constexpr int Q_BYTES = (2 * CQ / 8) * GROUP;   // 128 rows
+constexpr int PG = (TN / 8) * 128;              // bytes of 8 rows of P (TN keys each) in core-matrix order
+constexpr int P_BYTES = (CQ / 8) * PG;          // 64 rows x TN keys x 2 B
+constexpr int HC = TN / 4;                      // columns of a tile per thread (four threads share a query row)
+static_assert(HC == 16, "a thread reads its 16 columns with one tcgen05.ld and owns half a record word");
+constexpr int TMEM_COLS = 256;    // power of two covering two S tiles and O^T; two CTAs fit in the 512 columns of an SM
+constexpr int S_COL = 0;          // two S tiles: columns [0, TN) and [TN, 2 TN)
+constexpr int O_COL = 2 * TN;     // O^T: CQ columns
+
+constexpr int OFF_Q = 0;
+constexpr int OFF_K = OFF_Q + Q_BYTES;
+constexpr int OFF_V = OFF_K + 2 * TILE;
+constexpr int OFF_PH = OFF_V + 2 * TILE;
+constexpr int OFF_PL = OFF_PH + P_BYTES;
+constexpr int OFF_STAT = OFF_PL + P_BYTES;      // M[64], L[64] floats (the per-thread m[128], l[128] of the first sweep
+                                                // meet in the P buffer, which is idle between the sweeps)
+constexpr int OFF_BAR = OFF_STAT + 4 * (64 + 64);
+constexpr int SMEM_BYTES = OFF_BAR + 64;
+static_assert(P_BYTES >= 4 * 2 * NT, "the first sweep's statistics alias the P buffer");
+static_assert(2 * (SMEM_BYTES + 1024) <= 228 * 1024, "two CTAs per SM");
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, no swizzle: start address, leading and stride byte offsets in
+// units of 16 bytes, descriptor version 1 (bits 46..47).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46);
+}
+// Instruction descriptor of kind::f16: fp32 accumulator, 16-bit A and B of format fmt (0 f16, 1 bf16).
+__device__ __forceinline__ uint32_t instr_desc(int fmt, int a_mn_major, int M, int N) {
+    return (1u << 4) | ((uint32_t)fmt << 7) | ((uint32_t)fmt << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)(N >> 3) << 17) |
+           ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// The mbarrier gets one arrival when every tcgen05.mma issued so far by this thread has finished.
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 16 consecutive columns of this thread's lane (lane = 32 * (warp % 4) + lane id).
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// 32 consecutive columns of this thread's lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+template <int DT> struct Split;
+template <> struct Split<SH_F16> {
+    static constexpr int FMT = 0;
+    // p0, p1 in [0, 1] -> packed high parts and packed low parts (p = hi + lo up to ~2^-22)
+    static __device__ __forceinline__ void run(float p0, float p1, uint32_t &hi, uint32_t &lo) {
+        const __half2 h = __floats2half2_rn(p0, p1);
+        const float2 hf = __half22float2(h);
+        const __half2 l = __floats2half2_rn(p0 - hf.x, p1 - hf.y);
+        hi = *reinterpret_cast<const uint32_t *>(&h);
+        lo = *reinterpret_cast<const uint32_t *>(&l);
+    }
+};
+template <> struct Split<SH_BF16> {
+    static constexpr int FMT = 1;
+    static __device__ __forceinline__ void run(float p0, float p1, uint32_t &hi, uint32_t &lo) {
+        const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+        const float2 hf = __bfloat1622float2(h);
+        const __nv_bfloat162 l = __floats2bfloat162_rn(p0 - hf.x, p1 - hf.y);
+        hi = *reinterpret_cast<const uint32_t *>(&h);
+        lo = *reinterpret_cast<const uint32_t *>(&l);
+    }
+};
+
+// Start filling a tile buffer with rows [j0, j0 + TN) of the unit's K or V as seen by the chunk
+// (cached rows, then the chunk's own tokens, zeros beyond), 16-byte piece (row, ch) going to
+// [row / 8][ch][row % 8]: the canonical no-swizzle order, K-major for K, MN-major for V.
+__device__ __forceinline__ void load_tile(char *tile, const char *cache_u, const char *chunk, int j0, int n0, int n_tot,
+                                          size_t chunk_stride) {
+    // consecutive threads take the 8 rows of a core matrix, then the next 16-byte column: a warp writes 512
+    // contiguous bytes of shared memory and reads 8 x 64 contiguous bytes of global memory
+    for (int idx = threadIdx.x; idx < TN * 16; idx += NT) {
+        const int row = ((idx >> 7) << 3) | (idx & 7), ch = (idx >> 3) & 15;
+        const int j = j0 + row;
+        char *dst = tile + (row >> 3) * GROUP + ch * 128 + (row & 7) * 16;
+        if (j < n0) cp_async16(dst, cache_u + (size_t)j * (D * 2) + ch * 16);
+        else if (j < n_tot) cp_async16(dst, chunk + (size_t)(j - n0) * chunk_stride + ch * 16);
+        else *reinterpret_cast<uint4 *>(dst) = make_uint4(0, 0, 0, 0);
+    }
+}
+
+
+template <int DT>
+__global__ void __launch_bounds__(NT, 2) sh_chunk_umma_kernel(const ChunkParams p) {
+    using SP = Split<DT>;
+    extern __shared__ __align__(128) unsigned char sm[];
+    char *Qs = reinterpret_cast<char *>(sm) + OFF_Q;
+    char *Kt = reinterpret_cast<char *>(sm) + OFF_K;
+    char *Vt = reinterpret_cast<char *>(sm) + OFF_V;
+    char *Ph = reinterpret_cast<char *>(sm) + OFF_PH;
+    char *Pl = reinterpret_cast<char *>(sm) + OFF_PL;
+    float *m_sh = reinterpret_cast<float *>(sm + OFF_PH);
+    float *l_sh = m_sh + NT;
+    float *Mfin = reinterpret_cast<float *>(sm + OFF_STAT), *Lfin = Mfin + 64;
+    uint64_t *bar_s = reinterpret_cast<uint64_t *>(sm + OFF_BAR);
+    uint64_t *bar_pv = bar_s + 2;        // bar_s[0], bar_s[1]: one per S buffer
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bar_s + 3);
+
+    const int u = blockIdx.x, tid = threadIdx.x, warp = tid >> 5;
+    // this thread's query and its quarter of every tile's columns: warps w and w + 4 read the same 32 lanes
+    const int i = tid & 63, quarter = ((tid >> 6) & 1) * 2 + (tid >> 7);
+    const int n0 = p.n0, c = p.c, n_tot = n0 + c;
+    const int ntiles = (n_tot + TN - 1) / TN;
+    const int step0 = p.t0 + 1;
+    const size_t tstride = (size_t)p.Utot * D * 2;       // bytes between consecutive tokens of one unit
+    const char *Kc = p.K + (size_t)u * p.B * D * 2;
+    const char *Vc = p.V + (size_t)u * p.B * D * 2;
+    const char *kchunk = p.k + (size_t)u * D * 2, *vchunk = p.v + (size_t)u * D * 2;
+
+    // ---- tensor memory, barriers
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+        mbar_init(bar_s, 1);
+        mbar_init(bar_s + 1, 1);
+        mbar_init(bar_pv, 1);
+        fence_barrier_init();
+    }
+    // ---- queries (rows beyond c are zero), twice: rows 0..63 and 64..127
+    for (int idx = tid; idx < CQ * 16; idx += NT) {
+        const int row = idx >> 4, ch = idx & 15;
+        uint4 val = make_uint4(0, 0, 0, 0);
+        if (row < c) {
+            val = *reinterpret_cast<const uint4 *>(p.q + (size_t)row * tstride + (size_t)u * D * 2 + ch * 16);
+            if (p.qring)      // remembered for a later recount
+                *reinterpret_cast<uint4 *>(p.qring + ((size_t)u * p.w + (step0 + row) % p.w) * (D * 2) + ch * 16) = val;
+        }
+        char *dst = Qs + (row >> 3) * GROUP + ch * 128 + (row & 7) * 16;
+        *reinterpret_cast<uint4 *>(dst) = val;
+        *reinterpret_cast<uint4 *>(dst + (CQ / 8) * GROUP) = val;
+    }
+    // ---- append the chunk's keys, values and positions to the cache (nothing in this launch reads them back from there)
+    if (tid < c) p.pos[(size_t)u * p.B + n0 + tid] = step0 + tid;
+    for (int idx = tid; idx < c * 16; idx += NT) {
+        const int row = idx >> 4, ch = idx & 15;
+        const size_t src = (size_t)row * tstride + (size_t)u * D * 2 + ch * 16;
+        const size_t dst = ((size_t)u * p.B + n0 + row) * (D * 2) + ch * 16;
+        *reinterpret_cast<uint4 *>(p.K + dst) = *reinterpret_cast<const uint4 *>(p.k + src);
+        *reinterpret_cast<uint4 *>(p.V + dst) = *reinterpret_cast<const uint4 *>(p.v + src);
+    }
+    load_tile(Kt, Kc, kchunk, 0, n0, n_tot, tstride);
+    if (ntiles > 1) load_tile(Kt + TILE, Kc, kchunk, TN, n0, n_tot, tstride);
+    cp_async_commit();
+    cp_async_wait_all();
+    fence_async_shared();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tbase = *tmem_slot;
+    const uint32_t lane_addr = tbase + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t q_addr = smem_u32(Qs), k_addr = smem_u32(Kt), v_addr = smem_u32(Vt), ph_addr = smem_u32(Ph), pl_addr = smem_u32(Pl);
+    const uint32_t idesc_s = instr_desc(SP::FMT, 0, 128, TN);
+    const uint32_t idesc_pv = instr_desc(SP::FMT, 1, 128, CQ);
+    auto issue_s = [&](int kt) {       // S tile kt = Q . K_tile^T into S buffer kt & 1 (one thread)
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks)
+            umma_f16(tbase + S_COL + (kt & 1) * TN, smem_desc(q_addr + ks * 256, 128, GROUP),
+                     smem_desc(k_addr + (kt & 1) * TILE + ks * 256, 128, GROUP), idesc_s, ks > 0);
+        umma_commit(bar_s + (kt & 1));
+    };
+
+    // Both sweeps run one tile ahead on the tensor core: S(kt + 1) is issued before the threads turn to
+    // S(kt), and the K tile kt + 2 is fetched as soon as S(kt) has been computed from the buffer it reuses.
+    uint32_t par_s = 0, par_pv = 0;      // bit b of par_s: parity the next wait on bar_s[b] expects
+    bool ok = true;
+    const int nv = n0 + i + 1;           // keys visible to this thread's query
+    const bool live_row = i < c;
+
+    // ---- sweep 1: running maximum and sum of every row
+    float m_run = -INFINITY, l_run = 0.f;
+    if (tid == 0) issue_s(0);
+    for (int kt = 0; kt < ntiles; ++kt) {
+        cp_async_wait_all();
+        fence_async_shared();
+        tc_fence_before();
+        if (!__syncthreads_and(ok)) { ok = false; break; }
+        if (tid == 0 && kt + 1 < ntiles) issue_s(kt + 1);
+        ok = mbar_wait(bar_s + (kt & 1), (par_s >> (kt & 1)) & 1, p.err, 0x501) && ok;
+        par_s ^= 1u << (kt & 1);
+        tc_fence_after();
+        if (kt + 2 < ntiles) load_tile(Kt + (kt & 1) * TILE, Kc, kchunk, (kt + 2) * TN, n0, n_tot, tstride);
+        cp_async_commit();
+        {
+            float sv[HC];
+            tmem_ld16(lane_addr + S_COL + (kt & 1) * TN + quarter * HC, sv);
+            const int lim = live_row ? nv - (kt * TN + quarter * HC) : 0;     // columns of this batch the query sees
+            if (lim > 0) {
+                float bmax = -INFINITY;
+#pragma unroll
+                for (int jj = 0; jj < HC; ++jj) {
+                    sv[jj] = (jj < lim) ? sv[jj] * p.scale_log2e : -INFINITY;
+                    bmax = fmaxf(bmax, sv[jj]);
+                }
+                const float m_new = fmaxf(m_run, bmax);
+                float acc = 0.f;
+#pragma unroll
+                for (int jj = 0; jj < HC; ++jj) acc += ex2_approx(sv[jj] - m_new);
+                l_run = l_run * ex2_approx(m_run - m_new) + acc;
+                m_run = m_new;
+            }
+        }
+    }
+    // ---- the four parts of a row meet (in the P buffer, idle until the second sweep)
+    m_sh[tid] = m_run;
+    l_sh[tid] = l_run;
+    cp_async_wait_all();
+    tc_fence_before();
+    ok = __syncthreads_and(ok) != 0;
+    if (tid < CQ) {
+        float M = -INFINITY, L = 0.f;
+#pragma unroll
+        for (int part = 0; part < NT / CQ; ++part) M = fmaxf(M, m_sh[tid + part * CQ]);
+#pragma unroll
+        for (int part = 0; part < NT / CQ; ++part) {
+            const float mp = m_sh[tid + part * CQ];
+            if (mp > -INFINITY) L += l_sh[tid + part * CQ] * ex2_approx(mp - M);
+        }
+        Mfin[tid] = M;
+        Lfin[tid] = L;
+    }
+    if (ok) {
+        load_tile(Kt, Kc, kchunk, 0, n0, n_tot, tstride);
+        if (ntiles > 1) load_tile(Kt + TILE, Kc, kchunk, TN, n0, n_tot, tstride);
+        if (p.out) load_tile(Vt, Vc, vchunk, 0, n0, n_tot, tstride);
+    }
+    cp_async_commit();
+    cp_async_wait_all();
+    fence_async_shared();
+    __syncthreads();
+
+    // ---- sweep 2: probabilities, record bits, O^T += V^T . P^T
+    const float Mi = Mfin[i], Li = Lfin[i];
+    const float tf = (float)(step0 + i);
+    uint32_t *hrow = p.hist + ((size_t)u * p.w + (step0 + i) % p.w) * p.Bw;
+    if (ok) {
+        if (tid == 0) issue_s(0);
+        for (int kt = 0; kt < ntiles; ++kt) {
+            cp_async_wait_all();       // K(kt + 1) and V(kt) have landed
+            fence_async_shared();
+            tc_fence_before();
+            if (!__syncthreads_and(ok)) { ok = false; break; }
+            if (tid == 0 && kt + 1 < ntiles) issue_s(kt + 1);
+            ok = mbar_wait(bar_s + (kt & 1), (par_s >> (kt & 1)) & 1, p.err, 0x503) && ok;
+            par_s ^= 1u << (kt & 1);
+            if (kt > 0 && p.out) {     // the previous tile's P.V has finished: P and the V buffer it read are free
+                ok = mbar_wait(bar_pv, par_pv, p.err, 0x502) && ok;
+                par_pv ^= 1;
+            }
+            tc_fence_after();
+            if (kt + 2 < ntiles) load_tile(Kt + (kt & 1) * TILE, Kc, kchunk, (kt + 2) * TN, n0, n_tot, tstride);
+            if (kt + 1 < ntiles && p.out) load_tile(Vt + ((kt + 1) & 1) * TILE, Vc, vchunk, (kt + 1) * TN, n0, n_tot, tstride);
+            cp_async_commit();
+            {
+                float sv[HC];
+                tmem_ld16(lane_addr + S_COL + (kt & 1) * TN + quarter * HC, sv);
+                const int j0 = kt * TN + quarter * HC;
+                const int lim = live_row ? nv - j0 : 0;
+                uint32_t word = 0, hi[HC / 2], lo[HC / 2];
+#pragma unroll
+                for (int jj = 0; jj < HC; jj += 2) {
+                    const float e0 = (jj < lim) ? ex2_approx(sv[jj] * p.scale_log2e - Mi) : 0.f;
+                    const float e1 = (jj + 1 < lim) ? ex2_approx(sv[jj + 1] * p.scale_log2e - Mi) : 0.f;
+                    // step t: low_j = [alpha_j < 1/t] = [e_j * t < L]
+                    word |= (uint32_t)(jj < lim && e0 * tf < Li) << jj;
+                    word |= (uint32_t)(jj + 1 < lim && e1 * tf < Li) << (jj + 1);
+                    SP::run(e0, e1, hi[jj >> 1], lo[jj >> 1]);
+                }
+                // 16 slots: half a record word
+                if (live_row && (j0 >> 5) < p.Bw) reinterpret_cast<uint16_t *>(hrow)[j0 >> 4] = (uint16_t)word;
+                if (p.out) {
+#pragma unroll
+                    for (int cc = 0; cc < HC / 8; ++cc) {
+                        const int off = (i >> 3) * PG + (quarter * (HC / 8) + cc) * 128 + (i & 7) * 16;
+                        *reinterpret_cast<uint4 *>(Ph + off) = make_uint4(hi[4 * cc], hi[4 * cc + 1], hi[4 * cc + 2], hi[4 * cc + 3]);
+                        *reinterpret_cast<uint4 *>(Pl + off) = make_uint4(lo[4 * cc], lo[4 * cc + 1], lo[4 * cc + 2], lo[4 * cc + 3]);
+                    }
+                }
+            }
+            if (p.out) {
+                fence_async_shared();
+                tc_fence_before();
+                __syncthreads();
+                if (tid == 0) {
+                    tc_fence_after();
+#pragma unroll
+                    for (int ks = 0; ks < TN / 16; ++ks) {
+                        const uint64_t a = smem_desc(v_addr + (kt & 1) * TILE + ks * 2 * GROUP, GROUP, 128);
+                        umma_f16(tbase + O_COL, a, smem_desc(ph_addr + ks * 256, 128, PG), idesc_pv, (kt > 0 || ks > 0));
+                        umma_f16(tbase + O_COL, a, smem_desc(pl_addr + ks * 256, 128, PG), idesc_pv, 1);
+                    }
+                    umma_commit(bar_pv);
+                }
+            }
+        }
+        // bit-plane words beyond the last tile hold no live slot
+        if (live_row && quarter == 0)
+            for (int wd = ntiles * (TN / 32); wd < p.Bw; ++wd) hrow[wd] = 0;
+        if (p.out && ok) {
+            ok = mbar_wait(bar_pv, par_pv, p.err, 0x504) && ok;
+            tc_fence_after();
+        }
+    }
+    // ---- O^T: lane = output column, tensor-memory column = query
+    if (p.out) {
+        const int dcol = tid & 127, b = tid >> 7;      // output column (lane of tensor memory), half of the queries
+        float ov[32];
+        tmem_ld32(lane_addr + O_COL + b * 32, ov);
+        if (ok) {
+#pragma unroll
+            for (int qq = 0; qq < 32; ++qq) {
+                const int qi = b * 32 + qq;
+                if (qi < c) p.out[((size_t)qi * p.Utot + u) * D + dcol] = ov[qq] / Lfin[qi];
+            }
+        }
+    }
+    cp_async_wait_all();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tbase), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+template <int DT>
+cudaError_t launch(const ChunkParams &p, cudaStream_t s) {
+    auto kern = sh_chunk_umma_kernel<DT>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    kern<<<p.U, NT, SMEM_BYTES, s>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+int sh_chunk_umma_capacity() { return CQ; }
+
+cudaError_t sh_launch_chunk_umma(const ChunkParams &p, int dtype, cudaStream_t s) {
+    if (p.c < 1 || p.c > CQ) return cudaErrorInvalidValue;
+    return dtype == SH_F16 ? launch<SH_F16>(p, s) : launch<SH_BF16>(p, s);
+}

@@ -136,6 +136,32 @@ struct SelectParams {
 };
 
 
+// Chunked prompt step / recount (sh_prefill_chunk.cu, sh_chunk_umma.cu).
+struct ChunkParams {
+    const char *q, *k, *v;   // [c][U][D] time-major, 16-bit elements
+    float *out;              // [c][U][D] fp32 or NULL
+    char *K, *V;             // caches [U][B][D]
+    uint32_t *hist;
+    int32_t *pos;
+    int U, B, Bw, w;
+    int Utot;                // units of the whole handle: tokens of q/k/v/out are Utot rows apart
+    int n0;                  // live rows before the chunk
+    int c;                   // tokens in the chunk (<= CQ, <= w, n0 + c <= B)
+    int t0;                  // tokens streamed before the chunk
+    int SS;                  // row stride of S in floats
+    float scale_log2e;
+    char *qring;             // [U][w][D] queries of the last w steps (row = step mod w), or NULL
+    // recount mode (the record recomputed at compression time): queries come from the ring,
+    // steps first_step .. first_step + nsteps - 1, blockIdx.y selects CQ of them; keys are the
+    // n0 cached rows, visible to a query when their position does not exceed its step
+    int first_step, nsteps;
+    int *err;                // device error word (a bounded wait gave up)
+};
+
+// tcgen05 version of the chunked prompt step (fp16/bf16, head_dim 128, any budget): tokens per launch, launcher.
+int sh_chunk_umma_capacity();
+cudaError_t sh_launch_chunk_umma(const ChunkParams &p, int dtype, cudaStream_t s);
+
 // Launchers (each returns the cudaError_t of its launch and adds to *launches).
 cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches);
 // Scores of a query over the present caches (analysis; p.n = live rows, nothing appended).
@@ -145,6 +171,7 @@ bool sh_decode_tma_supported(const sh_context *c);
 cudaError_t sh_launch_decode_tma(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches);
 // Chunked prompt kernel: tokens one launch can take for this handle (0 = unsupported), and its launcher.
 int sh_prefill_chunk_capacity(const sh_context *c);
+bool sh_recount_supported(const sh_context *c);
 cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const void *k, const void *v, float *out,
                                     int count, cudaStream_t s, long long *launches);
 // Host bookkeeping shared by the compression entry points: is a compression due (some cache full),

@@ -76,25 +76,6 @@ template <> struct Mma<SH_BF16> {
     }
 };
 
-struct ChunkParams {
-    const char *q, *k, *v;   // [c][U][D] time-major, 16-bit elements
-    float *out;              // [c][U][D] fp32 or NULL
-    char *K, *V;             // caches [U][B][D]
-    uint32_t *hist;
-    int32_t *pos;
-    int U, B, Bw, w;
-    int Utot;                // units of the whole handle: tokens of q/k/v/out are Utot rows apart
-    int n0;                  // live rows before the chunk
-    int c;                   // tokens in the chunk (<= CQ, <= w, n0 + c <= B)
-    int t0;                  // tokens streamed before the chunk
-    int SS;                  // row stride of S in floats
-    float scale_log2e;
-    char *qring;             // [U][w][D] queries of the last w steps (row = step mod w), or NULL
-    // recount mode (the record recomputed at compression time): queries come from the ring,
-    // steps first_step .. first_step + nsteps - 1, blockIdx.y selects CQ of them; keys are the
-    // n0 cached rows, visible to a query when their position does not exceed its step
-    int first_step, nsteps;
-};
 
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(smem_dst)), "l"(gsrc) : "memory");
@@ -351,9 +332,16 @@ size_t smem_need(int CQ, int B) {
 int sh_prefill_chunk_capacity(const sh_context *c) {
     if ((c->dtype != SH_F16 && c->dtype != SH_BF16) || c->D != 128) return 0;
     int cq = 0;
-    if (smem_need(32, c->B) <= 200 * 1024) cq = 64;      // one or two CTAs of 32 queries, or one of 64
+    if (c->prefill_chunk != 2) cq = sh_chunk_umma_capacity();     // tcgen05 kernel: any budget
+    else if (smem_need(32, c->B) <= 200 * 1024) cq = 64;          // warp-level kernel: one or two CTAs of 32 queries, or one of 64
     if (cq > c->w) cq = c->w;     // every step of a chunk needs its own bit-plane row
     return cq;
+}
+
+// The recount (record recomputed at compression time) runs on the warp-level kernel, which keeps a
+// whole row of logits in shared memory: budgets up to about 700.
+bool sh_recount_supported(const sh_context *c) {
+    return (c->dtype == SH_F16 || c->dtype == SH_BF16) && c->D == 128 && smem_need(32, c->B) <= 200 * 1024;
 }
 
 // Steps t0+1 .. t0+count (count <= capacity, n0 + count <= B) in one launch.
@@ -370,8 +358,14 @@ cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const vo
     p.SS = s_stride(c->B);
     p.scale_log2e = (float)((double)c->scale * 1.4426950408889634);
     p.qring = sh_pqring(c);
+    p.err = reinterpret_cast<int *>(c->slab + c->L.err);
     cudaError_t e = cudaErrorInvalidValue;
     if (count < 1 || count > sh_prefill_chunk_capacity(c)) return e;
+    if (c->prefill_chunk != 2) {
+        e = sh_launch_chunk_umma(p, c->dtype, s);
+        if (e == cudaSuccess) *launches += 1;
+        return e;
+    }
     // 32 queries per CTA when two such CTAs fit on an SM (the second half of a longer chunk goes to a
     // sibling CTA that re-reads the keys): more warps in flight hide the latencies of this kernel better
     // than sharing the K/V tiles between 64 queries does

@@ -31,6 +31,7 @@ def main():
                     help="SH_OPT_COMPACTION = 1; the cache is then filled by streaming a random prompt through sh_prefill "
                          "(the selection needs real positions), a few launches before the ones of interest")
     ap.add_argument("--chunk", type=int, default=0, help="instead of decode steps, run one prompt chunk of this many tokens")
+    ap.add_argument("--chunk-kernel", type=int, default=None, help="SH_OPT_PREFILL_CHUNK value: 2 warp-level MMA, 3 tcgen05")
     ap.add_argument("--split", type=int, default=None)
     ap.add_argument("--kernel", type=int, default=None, help="1 direct loads, 2 pipelined bulk copies")
     args = ap.parse_args()
@@ -38,7 +39,7 @@ def main():
     U, d = args.units, cfg.head_dim
     torch.cuda.set_device(0)
     h = sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, U, d, cfg.dtype, split=args.split, kernel=args.kernel, auto_compress=True,
-                  unordered=args.unordered)
+                  unordered=args.unordered, prefill_chunk=args.chunk_kernel)
     rows = args.rows if args.rows is not None else (cfg.B - 1 if args.compress else cfg.B - cfg.m // 2)
     if args.chunk:
         rows = args.rows if args.rows is not None else cfg.B - args.chunk

@@ -66,12 +66,13 @@ def test_lockstep_pipelined_kernel(sh, dtype, d, U, B, r, w, m):
 @pytest.mark.parametrize("U,B,r,w,m,sizes", [(5, 150, 9, 37, 41, [64, 7, 33, 1, 50]), (3, 410, 64, 128, 64, [64]),
                                              (2, 700, 5, 64, 300, [32, 17]), (4, 40, 3, 9, 20, [5, 9, 2]),
                                              (130, 96, 8, 70, 30, [64, 31])])
-def test_lockstep_chunked_prompt_kernel(sh, dtype, U, B, r, w, m, sizes):
+@pytest.mark.parametrize("chunk_kernel", [1, 2])
+def test_lockstep_chunked_prompt_kernel(sh, dtype, U, B, r, w, m, sizes, chunk_kernel):
     """sh_prefill_chunk against the oracle replaying the same steps one by one: outputs of
     every step, its record bits, positions, counters and kept sets."""
     d, T = 128, 2 * B + 2 * m + 11
     q, k, v = wl.random_stream(U, d, T, seed=17 + U, dtype=dtype, peaked=3.0, device="cuda")
-    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, prefill_chunk=chunk_kernel)   # 1: tcgen05, 2: warp-level MMA
     blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
     res, orc = run_lockstep_chunked(h, dtype, blk, T, torch.arange(U), TOL[dtype], chunk_sizes=sizes)
     assert res.steps == T and res.compressions >= 3
@@ -79,6 +80,21 @@ def test_lockstep_chunked_prompt_kernel(sh, dtype, U, B, r, w, m, sizes):
     # and the decode step carries on from the state the chunks left
     q2, k2, v2 = wl.random_stream(U, d, 40, seed=99, dtype=dtype, peaked=3.0, device="cuda")
     run_lockstep(h, dtype, lambda t: (q2[t - T - 1], k2[t - T - 1], v2[t - T - 1]), 40, torch.arange(U), TOL[dtype], orc=orc)
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("U,B,r,w,m,sizes", [(2, 2100, 10, 400, 1050, [64, 64, 13]), (150, 33, 2, 70, 11, [64, 3]),
+                                             (1, 129, 1, 64, 64, [64]), (3, 1000, 10, 5, 500, [5, 2])])
+def test_lockstep_chunked_tcgen05_kernel_shapes(sh, dtype, U, B, r, w, m, sizes):
+    """The tcgen05 chunk kernel on shapes the warp-level one cannot take (budgets beyond ~700), with more
+    units than CTA slots, a single key tile, a tile boundary at n0 + 1, and a window shorter than a chunk."""
+    d, T = 128, min(2 * B + 2 * m + 11, B + m + 150)
+    q, k, v = wl.random_stream(U, d, T, seed=27 + U, dtype=dtype, peaked=3.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
+    res, orc = run_lockstep_chunked(h, dtype, blk, T, torch.arange(U), TOL[dtype], chunk_sizes=sizes)
+    assert res.steps == T and res.compressions >= 1
+    assert res.adoptions <= 1e-4 * res.slot_steps + 2
 
 
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
