@@ -166,7 +166,11 @@ __device__ __forceinline__ void load_tile(char *tile, const char *cache_u, const
 }
 
 
-template <int DT>
+// RECOUNT: the record recomputed at compression time.  Queries come from the ring of the last w queries
+// (steps first_step .. first_step + nsteps - 1, blockIdx.y selects 64 of them), keys are the n0 cached rows, a
+// key is visible to a query when its position does not exceed the query's step (slots need not be sorted);
+// nothing is appended and no output is formed: only the bit-plane rows of those steps are rewritten.
+template <int DT, bool RECOUNT>
 __global__ void __launch_bounds__(NT, 2) sh_chunk_umma_kernel(const ChunkParams p) {
     using SP = Split<DT>;
     extern __shared__ __align__(128) unsigned char sm[];
@@ -185,13 +189,23 @@ __global__ void __launch_bounds__(NT, 2) sh_chunk_umma_kernel(const ChunkParams 
     const int u = blockIdx.x, tid = threadIdx.x, warp = tid >> 5;
     // this thread's query and its quarter of every tile's columns: warps w and w + 4 read the same 32 lanes
     const int i = tid & 63, quarter = ((tid >> 6) & 1) * 2 + (tid >> 7);
-    const int n0 = p.n0, c = p.c, n_tot = n0 + c;
+    const int qoff = RECOUNT ? (int)blockIdx.y * CQ : 0;
+    const int n0 = p.n0, c = RECOUNT ? min(CQ, p.nsteps - qoff) : p.c, n_tot = RECOUNT ? n0 : n0 + c;
     const int ntiles = (n_tot + TN - 1) / TN;
-    const int step0 = p.t0 + 1;
+    const int step0 = RECOUNT ? p.first_step + qoff : p.t0 + 1;     // step of this CTA's first query
+    int *pos_sh = reinterpret_cast<int *>(sm + OFF_PL);             // [3][TN] positions of the key tiles (recount only: P is idle)
     const size_t tstride = (size_t)p.Utot * D * 2;       // bytes between consecutive tokens of one unit
     const char *Kc = p.K + (size_t)u * p.B * D * 2;
     const char *Vc = p.V + (size_t)u * p.B * D * 2;
-    const char *kchunk = p.k + (size_t)u * D * 2, *vchunk = p.v + (size_t)u * D * 2;
+    const char *kchunk = RECOUNT ? nullptr : p.k + (size_t)u * D * 2, *vchunk = RECOUNT ? nullptr : p.v + (size_t)u * D * 2;
+    const int32_t *pos_u = p.pos + (size_t)u * p.B;
+    // positions of key tile kt into pos_sh[buf] (slots beyond the cache: never visible)
+    auto load_pos = [&](int buf, int kt) {
+        if (RECOUNT && tid < TN) {
+            const int j = kt * TN + tid;
+            pos_sh[buf * TN + tid] = j < n0 ? pos_u[j] : 0x7fffffff;
+        }
+    };
 
     // ---- tensor memory, barriers
     if (warp == 0) {
@@ -210,25 +224,36 @@ __global__ void __launch_bounds__(NT, 2) sh_chunk_umma_kernel(const ChunkParams 
         const int row = idx >> 4, ch = idx & 15;
         uint4 val = make_uint4(0, 0, 0, 0);
         if (row < c) {
-            val = *reinterpret_cast<const uint4 *>(p.q + (size_t)row * tstride + (size_t)u * D * 2 + ch * 16);
-            if (p.qring)      // remembered for a later recount
-                *reinterpret_cast<uint4 *>(p.qring + ((size_t)u * p.w + (step0 + row) % p.w) * (D * 2) + ch * 16) = val;
+            char *ring_row = p.qring ? p.qring + ((size_t)u * p.w + (step0 + row) % p.w) * (D * 2) + ch * 16 : nullptr;
+            if (RECOUNT) {
+                val = *reinterpret_cast<const uint4 *>(ring_row);
+            } else {
+                val = *reinterpret_cast<const uint4 *>(p.q + (size_t)row * tstride + (size_t)u * D * 2 + ch * 16);
+                if (ring_row) *reinterpret_cast<uint4 *>(ring_row) = val;      // remembered for a later recount
+            }
         }
         char *dst = Qs + (row >> 3) * GROUP + ch * 128 + (row & 7) * 16;
         *reinterpret_cast<uint4 *>(dst) = val;
         *reinterpret_cast<uint4 *>(dst + (CQ / 8) * GROUP) = val;
     }
     // ---- append the chunk's keys, values and positions to the cache (nothing in this launch reads them back from there)
-    if (tid < c) p.pos[(size_t)u * p.B + n0 + tid] = step0 + tid;
-    for (int idx = tid; idx < c * 16; idx += NT) {
+    if (!RECOUNT && tid < c) p.pos[(size_t)u * p.B + n0 + tid] = step0 + tid;
+    for (int idx = tid; idx < (RECOUNT ? 0 : c * 16); idx += NT) {
         const int row = idx >> 4, ch = idx & 15;
         const size_t src = (size_t)row * tstride + (size_t)u * D * 2 + ch * 16;
         const size_t dst = ((size_t)u * p.B + n0 + row) * (D * 2) + ch * 16;
         *reinterpret_cast<uint4 *>(p.K + dst) = *reinterpret_cast<const uint4 *>(p.k + src);
         *reinterpret_cast<uint4 *>(p.V + dst) = *reinterpret_cast<const uint4 *>(p.v + src);
     }
+    // The two sweeps form one sequence of G = 2 ntiles S tiles; tile g covers the keys of tile g mod ntiles.
+    // S buffer, K buffer and mbarrier of tile g: g & 1.  V tile kt (second sweep only) sits in buffer kt & 1.
+    const int G = 2 * ntiles;
+    auto key_tile = [&](int g) { return g < ntiles ? g : g - ntiles; };
     load_tile(Kt, Kc, kchunk, 0, n0, n_tot, tstride);
-    if (ntiles > 1) load_tile(Kt + TILE, Kc, kchunk, TN, n0, n_tot, tstride);
+    load_tile(Kt + TILE, Kc, kchunk, key_tile(1) * TN, n0, n_tot, tstride);
+    load_pos(0, 0);          // positions of tile g sit in buffer g mod 3: written two iterations ahead of their use
+    load_pos(1, key_tile(1));
+    if (p.out) load_tile(Vt, Vc, vchunk, 0, n0, n_tot, tstride);     // idle until the second sweep: fetched early
     cp_async_commit();
     cp_async_wait_all();
     fence_async_shared();
@@ -240,45 +265,69 @@ __global__ void __launch_bounds__(NT, 2) sh_chunk_umma_kernel(const ChunkParams 
     const uint32_t q_addr = smem_u32(Qs), k_addr = smem_u32(Kt), v_addr = smem_u32(Vt), ph_addr = smem_u32(Ph), pl_addr = smem_u32(Pl);
     const uint32_t idesc_s = instr_desc(SP::FMT, 0, 128, TN);
     const uint32_t idesc_pv = instr_desc(SP::FMT, 1, 128, CQ);
-    auto issue_s = [&](int kt) {       // S tile kt = Q . K_tile^T into S buffer kt & 1 (one thread)
+    auto issue_s = [&](int g) {        // S tile g = Q . K_tile^T into S buffer g & 1 (one thread)
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks)
-            umma_f16(tbase + S_COL + (kt & 1) * TN, smem_desc(q_addr + ks * 256, 128, GROUP),
-                     smem_desc(k_addr + (kt & 1) * TILE + ks * 256, 128, GROUP), idesc_s, ks > 0);
-        umma_commit(bar_s + (kt & 1));
+            umma_f16(tbase + S_COL + (g & 1) * TN, smem_desc(q_addr + ks * 256, 128, GROUP),
+                     smem_desc(k_addr + (g & 1) * TILE + ks * 256, 128, GROUP), idesc_s, ks > 0);
+        umma_commit(bar_s + (g & 1));
     };
 
-    // Both sweeps run one tile ahead on the tensor core: S(kt + 1) is issued before the threads turn to
-    // S(kt), and the K tile kt + 2 is fetched as soon as S(kt) has been computed from the buffer it reuses.
+    // The tensor core runs one tile ahead: S(g + 1) is issued before the threads turn to S(g), and the K
+    // tile of g + 2 is fetched as soon as S(g) has been computed from the buffer it reuses.
     uint32_t par_s = 0, par_pv = 0;      // bit b of par_s: parity the next wait on bar_s[b] expects
     bool ok = true;
     const int nv = n0 + i + 1;           // keys visible to this thread's query
     const bool live_row = i < c;
-
-    // ---- sweep 1: running maximum and sum of every row
     float m_run = -INFINITY, l_run = 0.f;
+    float Mi = 0.f, Li = 1.f;
+    const float tf = (float)(step0 + i);
+    uint32_t *hrow = p.hist + ((size_t)u * p.w + (step0 + i) % p.w) * p.Bw;
     if (tid == 0) issue_s(0);
-    for (int kt = 0; kt < ntiles; ++kt) {
-        cp_async_wait_all();
+    for (int g = 0; g < G; ++g) {
+        const int kt = key_tile(g);
+        const bool second = g >= ntiles;
+        cp_async_wait_all();           // K(g + 1) and, in the second sweep, V(kt) have landed
         fence_async_shared();
         tc_fence_before();
         if (!__syncthreads_and(ok)) { ok = false; break; }
-        if (tid == 0 && kt + 1 < ntiles) issue_s(kt + 1);
-        ok = mbar_wait(bar_s + (kt & 1), (par_s >> (kt & 1)) & 1, p.err, 0x501) && ok;
-        par_s ^= 1u << (kt & 1);
+        if (tid == 0 && g + 1 < G) issue_s(g + 1);
+        ok = mbar_wait(bar_s + (g & 1), (par_s >> (g & 1)) & 1, p.err, 0x501) && ok;
+        par_s ^= 1u << (g & 1);
+        if (second && kt > 0 && p.out) {     // the previous tile's P.V has finished: P and the V buffer it read are free
+            ok = mbar_wait(bar_pv, par_pv, p.err, 0x502) && ok;
+            par_pv ^= 1;
+        }
         tc_fence_after();
-        if (kt + 2 < ntiles) load_tile(Kt + (kt & 1) * TILE, Kc, kchunk, (kt + 2) * TN, n0, n_tot, tstride);
+        if (g + 2 < G) {
+            load_tile(Kt + (g & 1) * TILE, Kc, kchunk, key_tile(g + 2) * TN, n0, n_tot, tstride);
+            load_pos((g + 2) % 3, key_tile(g + 2));
+        }
+        if (p.out && second && kt + 1 < ntiles) load_tile(Vt + ((kt + 1) & 1) * TILE, Vc, vchunk, (kt + 1) * TN, n0, n_tot, tstride);
         cp_async_commit();
-        {
-            float sv[HC];
-            tmem_ld16(lane_addr + S_COL + (kt & 1) * TN + quarter * HC, sv);
-            const int lim = live_row ? nv - (kt * TN + quarter * HC) : 0;     // columns of this batch the query sees
-            if (lim > 0) {
+        float sv[HC];
+        tmem_ld16(lane_addr + S_COL + (g & 1) * TN + quarter * HC, sv);
+        const int j0 = kt * TN + quarter * HC;
+        // bit jj of vm: column jj of this batch is visible to the query (causal prefix, or by position in a recount)
+        uint32_t vm;
+        if (RECOUNT) {
+            vm = 0;
+            const int *pt = pos_sh + (g % 3) * TN + quarter * HC;
+#pragma unroll
+            for (int jj = 0; jj < HC; ++jj) vm |= (uint32_t)(pt[jj] <= step0 + i) << jj;
+            if (!live_row) vm = 0;
+        } else {
+            const int lim = live_row ? nv - j0 : 0;
+            vm = lim <= 0 ? 0u : (lim >= HC ? 0xffffu : (1u << lim) - 1u);
+        }
+        if (!second) {
+            // ---- first sweep: running maximum and sum of the row
+            if (vm) {
                 float bmax = -INFINITY;
 #pragma unroll
                 for (int jj = 0; jj < HC; ++jj) {
-                    sv[jj] = (jj < lim) ? sv[jj] * p.scale_log2e : -INFINITY;
+                    sv[jj] = ((vm >> jj) & 1u) ? sv[jj] * p.scale_log2e : -INFINITY;
                     bmax = fmaxf(bmax, sv[jj]);
                 }
                 const float m_new = fmaxf(m_run, bmax);
@@ -288,104 +337,70 @@ __global__ void __launch_bounds__(NT, 2) sh_chunk_umma_kernel(const ChunkParams 
                 l_run = l_run * ex2_approx(m_run - m_new) + acc;
                 m_run = m_new;
             }
-        }
-    }
-    // ---- the four parts of a row meet (in the P buffer, idle until the second sweep)
-    m_sh[tid] = m_run;
-    l_sh[tid] = l_run;
-    cp_async_wait_all();
-    tc_fence_before();
-    ok = __syncthreads_and(ok) != 0;
-    if (tid < CQ) {
-        float M = -INFINITY, L = 0.f;
+            if (g == ntiles - 1) {
+                // the four parts of a row meet (in the P buffer, idle until the second sweep)
+                m_sh[tid] = m_run;
+                l_sh[tid] = l_run;
+                __syncthreads();
+                if (tid < CQ) {
+                    float M = -INFINITY, L = 0.f;
 #pragma unroll
-        for (int part = 0; part < NT / CQ; ++part) M = fmaxf(M, m_sh[tid + part * CQ]);
+                    for (int part = 0; part < NT / CQ; ++part) M = fmaxf(M, m_sh[tid + part * CQ]);
 #pragma unroll
-        for (int part = 0; part < NT / CQ; ++part) {
-            const float mp = m_sh[tid + part * CQ];
-            if (mp > -INFINITY) L += l_sh[tid + part * CQ] * ex2_approx(mp - M);
+                    for (int part = 0; part < NT / CQ; ++part) {
+                        const float mp = m_sh[tid + part * CQ];
+                        if (mp > -INFINITY) L += l_sh[tid + part * CQ] * ex2_approx(mp - M);
+                    }
+                    Mfin[tid] = M;
+                    Lfin[tid] = L;
+                }
+                __syncthreads();
+                Mi = Mfin[i];
+                Li = Lfin[i];
+            }
+            continue;
         }
-        Mfin[tid] = M;
-        Lfin[tid] = L;
-    }
-    if (ok) {
-        load_tile(Kt, Kc, kchunk, 0, n0, n_tot, tstride);
-        if (ntiles > 1) load_tile(Kt + TILE, Kc, kchunk, TN, n0, n_tot, tstride);
-        if (p.out) load_tile(Vt, Vc, vchunk, 0, n0, n_tot, tstride);
-    }
-    cp_async_commit();
-    cp_async_wait_all();
-    fence_async_shared();
-    __syncthreads();
-
-    // ---- sweep 2: probabilities, record bits, O^T += V^T . P^T
-    const float Mi = Mfin[i], Li = Lfin[i];
-    const float tf = (float)(step0 + i);
-    uint32_t *hrow = p.hist + ((size_t)u * p.w + (step0 + i) % p.w) * p.Bw;
-    if (ok) {
-        if (tid == 0) issue_s(0);
-        for (int kt = 0; kt < ntiles; ++kt) {
-            cp_async_wait_all();       // K(kt + 1) and V(kt) have landed
+        // ---- second sweep: probabilities, record bits, O^T += V^T . P^T
+        uint32_t word = 0, hi[HC / 2], lo[HC / 2];
+#pragma unroll
+        for (int jj = 0; jj < HC; jj += 2) {
+            const bool v0 = (vm >> jj) & 1u, v1 = (vm >> (jj + 1)) & 1u;
+            const float e0 = v0 ? ex2_approx(sv[jj] * p.scale_log2e - Mi) : 0.f;
+            const float e1 = v1 ? ex2_approx(sv[jj + 1] * p.scale_log2e - Mi) : 0.f;
+            // step t: low_j = [alpha_j < 1/t] = [e_j * t < L]
+            word |= (uint32_t)(v0 && e0 * tf < Li) << jj;
+            word |= (uint32_t)(v1 && e1 * tf < Li) << (jj + 1);
+            SP::run(e0, e1, hi[jj >> 1], lo[jj >> 1]);
+        }
+        // 16 slots: half a record word
+        if (live_row && (j0 >> 5) < p.Bw) reinterpret_cast<uint16_t *>(hrow)[j0 >> 4] = (uint16_t)word;
+        if (p.out) {
+#pragma unroll
+            for (int cc = 0; cc < HC / 8; ++cc) {
+                const int off = (i >> 3) * PG + (quarter * (HC / 8) + cc) * 128 + (i & 7) * 16;
+                *reinterpret_cast<uint4 *>(Ph + off) = make_uint4(hi[4 * cc], hi[4 * cc + 1], hi[4 * cc + 2], hi[4 * cc + 3]);
+                *reinterpret_cast<uint4 *>(Pl + off) = make_uint4(lo[4 * cc], lo[4 * cc + 1], lo[4 * cc + 2], lo[4 * cc + 3]);
+            }
             fence_async_shared();
             tc_fence_before();
-            if (!__syncthreads_and(ok)) { ok = false; break; }
-            if (tid == 0 && kt + 1 < ntiles) issue_s(kt + 1);
-            ok = mbar_wait(bar_s + (kt & 1), (par_s >> (kt & 1)) & 1, p.err, 0x503) && ok;
-            par_s ^= 1u << (kt & 1);
-            if (kt > 0 && p.out) {     // the previous tile's P.V has finished: P and the V buffer it read are free
-                ok = mbar_wait(bar_pv, par_pv, p.err, 0x502) && ok;
-                par_pv ^= 1;
-            }
-            tc_fence_after();
-            if (kt + 2 < ntiles) load_tile(Kt + (kt & 1) * TILE, Kc, kchunk, (kt + 2) * TN, n0, n_tot, tstride);
-            if (kt + 1 < ntiles && p.out) load_tile(Vt + ((kt + 1) & 1) * TILE, Vc, vchunk, (kt + 1) * TN, n0, n_tot, tstride);
-            cp_async_commit();
-            {
-                float sv[HC];
-                tmem_ld16(lane_addr + S_COL + (kt & 1) * TN + quarter * HC, sv);
-                const int j0 = kt * TN + quarter * HC;
-                const int lim = live_row ? nv - j0 : 0;
-                uint32_t word = 0, hi[HC / 2], lo[HC / 2];
+            __syncthreads();
+            if (tid == 0) {
+                tc_fence_after();
 #pragma unroll
-                for (int jj = 0; jj < HC; jj += 2) {
-                    const float e0 = (jj < lim) ? ex2_approx(sv[jj] * p.scale_log2e - Mi) : 0.f;
-                    const float e1 = (jj + 1 < lim) ? ex2_approx(sv[jj + 1] * p.scale_log2e - Mi) : 0.f;
-                    // step t: low_j = [alpha_j < 1/t] = [e_j * t < L]
-                    word |= (uint32_t)(jj < lim && e0 * tf < Li) << jj;
-                    word |= (uint32_t)(jj + 1 < lim && e1 * tf < Li) << (jj + 1);
-                    SP::run(e0, e1, hi[jj >> 1], lo[jj >> 1]);
+                for (int ks = 0; ks < TN / 16; ++ks) {
+                    const uint64_t a = smem_desc(v_addr + (kt & 1) * TILE + ks * 2 * GROUP, GROUP, 128);
+                    umma_f16(tbase + O_COL, a, smem_desc(ph_addr + ks * 256, 128, PG), idesc_pv, (kt > 0 || ks > 0));
+                    umma_f16(tbase + O_COL, a, smem_desc(pl_addr + ks * 256, 128, PG), idesc_pv, 1);
                 }
-                // 16 slots: half a record word
-                if (live_row && (j0 >> 5) < p.Bw) reinterpret_cast<uint16_t *>(hrow)[j0 >> 4] = (uint16_t)word;
-                if (p.out) {
-#pragma unroll
-                    for (int cc = 0; cc < HC / 8; ++cc) {
-                        const int off = (i >> 3) * PG + (quarter * (HC / 8) + cc) * 128 + (i & 7) * 16;
-                        *reinterpret_cast<uint4 *>(Ph + off) = make_uint4(hi[4 * cc], hi[4 * cc + 1], hi[4 * cc + 2], hi[4 * cc + 3]);
-                        *reinterpret_cast<uint4 *>(Pl + off) = make_uint4(lo[4 * cc], lo[4 * cc + 1], lo[4 * cc + 2], lo[4 * cc + 3]);
-                    }
-                }
-            }
-            if (p.out) {
-                fence_async_shared();
-                tc_fence_before();
-                __syncthreads();
-                if (tid == 0) {
-                    tc_fence_after();
-#pragma unroll
-                    for (int ks = 0; ks < TN / 16; ++ks) {
-                        const uint64_t a = smem_desc(v_addr + (kt & 1) * TILE + ks * 2 * GROUP, GROUP, 128);
-                        umma_f16(tbase + O_COL, a, smem_desc(ph_addr + ks * 256, 128, PG), idesc_pv, (kt > 0 || ks > 0));
-                        umma_f16(tbase + O_COL, a, smem_desc(pl_addr + ks * 256, 128, PG), idesc_pv, 1);
-                    }
-                    umma_commit(bar_pv);
-                }
+                umma_commit(bar_pv);
             }
         }
+    }
+    if (ok) {
         // bit-plane words beyond the last tile hold no live slot
         if (live_row && quarter == 0)
             for (int wd = ntiles * (TN / 32); wd < p.Bw; ++wd) hrow[wd] = 0;
-        if (p.out && ok) {
+        if (p.out) {
             ok = mbar_wait(bar_pv, par_pv, p.err, 0x504) && ok;
             tc_fence_after();
         }
@@ -412,12 +427,13 @@ __global__ void __launch_bounds__(NT, 2) sh_chunk_umma_kernel(const ChunkParams 
     }
 }
 
-template <int DT>
+template <int DT, bool RECOUNT>
 cudaError_t launch(const ChunkParams &p, cudaStream_t s) {
-    auto kern = sh_chunk_umma_kernel<DT>;
+    auto kern = sh_chunk_umma_kernel<DT, RECOUNT>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    kern<<<p.U, NT, SMEM_BYTES, s>>>(p);
+    const unsigned gy = RECOUNT ? (unsigned)((p.nsteps + CQ - 1) / CQ) : 1u;
+    kern<<<dim3(p.U, gy, 1), NT, SMEM_BYTES, s>>>(p);
     return cudaGetLastError();
 }
 
@@ -427,5 +443,10 @@ int sh_chunk_umma_capacity() { return CQ; }
 
 cudaError_t sh_launch_chunk_umma(const ChunkParams &p, int dtype, cudaStream_t s) {
     if (p.c < 1 || p.c > CQ) return cudaErrorInvalidValue;
-    return dtype == SH_F16 ? launch<SH_F16>(p, s) : launch<SH_BF16>(p, s);
+    return dtype == SH_F16 ? launch<SH_F16, false>(p, s) : launch<SH_BF16, false>(p, s);
+}
+
+cudaError_t sh_launch_recount_umma(const ChunkParams &p, int dtype, cudaStream_t s) {
+    if (p.nsteps < 1 || p.out) return cudaErrorInvalidValue;
+    return dtype == SH_F16 ? launch<SH_F16, true>(p, s) : launch<SH_BF16, true>(p, s);
 }

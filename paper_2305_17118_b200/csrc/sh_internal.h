@@ -161,6 +161,7 @@ struct ChunkParams {
 // tcgen05 version of the chunked prompt step (fp16/bf16, head_dim 128, any budget): tokens per launch, launcher.
 int sh_chunk_umma_capacity();
 cudaError_t sh_launch_chunk_umma(const ChunkParams &p, int dtype, cudaStream_t s);
+cudaError_t sh_launch_recount_umma(const ChunkParams &p, int dtype, cudaStream_t s);
 
 // Launchers (each returns the cudaError_t of its launch and adds to *launches).
 cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches);

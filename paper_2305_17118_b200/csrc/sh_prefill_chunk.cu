@@ -338,10 +338,11 @@ int sh_prefill_chunk_capacity(const sh_context *c) {
     return cq;
 }
 
-// The recount (record recomputed at compression time) runs on the warp-level kernel, which keeps a
-// whole row of logits in shared memory: budgets up to about 700.
+// The recount (record recomputed at compression time): any budget on the tcgen05 kernel; the warp-level
+// kernel keeps a whole row of logits in shared memory (budgets up to about 700).
 bool sh_recount_supported(const sh_context *c) {
-    return (c->dtype == SH_F16 || c->dtype == SH_BF16) && c->D == 128 && smem_need(32, c->B) <= 200 * 1024;
+    if ((c->dtype != SH_F16 && c->dtype != SH_BF16) || c->D != 128) return false;
+    return c->prefill_chunk != 2 || smem_need(32, c->B) <= 200 * 1024;
 }
 
 // Steps t0+1 .. t0+count (count <= capacity, n0 + count <= B) in one launch.
@@ -392,7 +393,13 @@ cudaError_t sh_launch_recount(const sh_context *c, cudaStream_t s, long long *la
     p.nsteps = c->t < c->w ? (int)c->t : c->w;
     p.first_step = (int)c->t - p.nsteps + 1;
     if (p.nsteps < 1) return cudaSuccess;
+    p.err = reinterpret_cast<int *>(c->slab + c->L.err);
     cudaError_t e;
+    if (c->prefill_chunk != 2) {
+        e = sh_launch_recount_umma(p, c->dtype, s);
+        if (e == cudaSuccess) *launches += 1;
+        return e;
+    }
     if (smem_need(64, c->B) <= 200 * 1024) e = c->dtype == SH_F16 ? launch_chunk<SH_F16, 64, true>(p, s) : launch_chunk<SH_BF16, 64, true>(p, s);
     else e = c->dtype == SH_F16 ? launch_chunk<SH_F16, 32, true>(p, s) : launch_chunk<SH_BF16, 32, true>(p, s);
     if (e == cudaSuccess) *launches += 1;

@@ -98,15 +98,17 @@ def test_lockstep_chunked_tcgen05_kernel_shapes(sh, dtype, U, B, r, w, m, sizes)
 
 
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
-@pytest.mark.parametrize("U,B,r,w,m", [(5, 150, 9, 37, 41), (3, 410, 64, 128, 64), (140, 96, 8, 70, 30), (2, 40, 3, 9, 20)])
-def test_lockstep_record_recomputed_at_compression(sh, dtype, U, B, r, w, m):
+@pytest.mark.parametrize("U,B,r,w,m,chunk_kernel", [(5, 150, 9, 37, 41, 1), (3, 410, 64, 128, 64, 1), (140, 96, 8, 70, 30, 1),
+                                                    (2, 40, 3, 9, 20, 1), (2, 1300, 10, 200, 650, 1), (5, 150, 9, 37, 41, 2),
+                                                    (3, 410, 64, 128, 64, 2), (140, 96, 8, 70, 30, 2)])
+def test_lockstep_record_recomputed_at_compression(sh, dtype, U, B, r, w, m, chunk_kernel):
     """SH_OPT_RECORD_MODE = 1: Algorithm 2 as stated, the record rebuilt at each compression from
     the stored queries of the last w steps against the present cache."""
-    d, T = 128, 2 * B + 3 * m + 5
+    d, T = 128, min(2 * B + 3 * m + 5, B + 2 * m + 30)
     q, k, v = wl.random_stream(U, d, T, seed=23 + U, dtype=dtype, peaked=3.0, device="cuda")
-    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, recompute_record=True)
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, recompute_record=True, prefill_chunk=chunk_kernel)
     res, orc = run_lockstep_recompute(h, dtype, _stream_fn(q, k, v), T, torch.arange(U), TOL[dtype])
-    assert res.compressions >= 4
+    assert res.compressions >= 3
     assert res.adoptions <= 1e-4 * res.slot_steps + 2
 
 
