@@ -154,14 +154,22 @@ template <> struct Split<SH_BF16> {
 __device__ __forceinline__ void load_tile(char *tile, const char *cache_u, const char *chunk, int j0, int n0, int n_tot,
                                           size_t chunk_stride) {
     // consecutive threads take the 8 rows of a core matrix, then the next 16-byte column: a warp writes 512
-    // contiguous bytes of shared memory and reads 8 x 64 contiguous bytes of global memory
-    for (int idx = threadIdx.x; idx < TN * 16; idx += NT) {
-        const int row = ((idx >> 7) << 3) | (idx & 7), ch = (idx >> 3) & 15;
-        const int j = j0 + row;
-        char *dst = tile + (row >> 3) * GROUP + ch * 128 + (row & 7) * 16;
-        if (j < n0) cp_async16(dst, cache_u + (size_t)j * (D * 2) + ch * 16);
-        else if (j < n_tot) cp_async16(dst, chunk + (size_t)(j - n0) * chunk_stride + ch * 16);
+    // contiguous bytes of shared memory and reads 8 x 64 contiguous bytes of global memory.  With 256
+    // threads a thread keeps its column and walks rows row0, row0 + 16, ...: two row groups further each time.
+    static_assert(NT == 256, "piece idx = tid + 256 k lies 16 rows below piece tid");
+    const int row0 = ((threadIdx.x >> 7) << 3) | (threadIdx.x & 7), ch = (threadIdx.x >> 3) & 15;
+    char *dst = tile + (row0 >> 3) * GROUP + ch * 128 + (row0 & 7) * 16;
+    const char *src_cache = cache_u + (size_t)(j0 + row0) * (D * 2) + ch * 16;
+    const char *src_chunk = chunk + (ptrdiff_t)(j0 + row0 - n0) * (ptrdiff_t)chunk_stride + ch * 16;
+#pragma unroll
+    for (int k = 0; k < TN / 16; ++k) {
+        const int j = j0 + row0 + 16 * k;
+        if (j < n0) cp_async16(dst, src_cache);
+        else if (j < n_tot) cp_async16(dst, src_chunk);
         else *reinterpret_cast<uint4 *>(dst) = make_uint4(0, 0, 0, 0);
+        dst += 2 * GROUP;
+        src_cache += 16 * (D * 2);
+        src_chunk += 16 * (ptrdiff_t)chunk_stride;
     }
 }
 
@@ -219,32 +227,6 @@ __global__ void __launch_bounds__(NT, 2) sh_chunk_umma_kernel(const ChunkParams 
         mbar_init(bar_pv, 1);
         fence_barrier_init();
     }
-    // ---- queries (rows beyond c are zero), twice: rows 0..63 and 64..127
-    for (int idx = tid; idx < CQ * 16; idx += NT) {
-        const int row = idx >> 4, ch = idx & 15;
-        uint4 val = make_uint4(0, 0, 0, 0);
-        if (row < c) {
-            char *ring_row = p.qring ? p.qring + ((size_t)u * p.w + (step0 + row) % p.w) * (D * 2) + ch * 16 : nullptr;
-            if (RECOUNT) {
-                val = *reinterpret_cast<const uint4 *>(ring_row);
-            } else {
-                val = *reinterpret_cast<const uint4 *>(p.q + (size_t)row * tstride + (size_t)u * D * 2 + ch * 16);
-                if (ring_row) *reinterpret_cast<uint4 *>(ring_row) = val;      // remembered for a later recount
-            }
-        }
-        char *dst = Qs + (row >> 3) * GROUP + ch * 128 + (row & 7) * 16;
-        *reinterpret_cast<uint4 *>(dst) = val;
-        *reinterpret_cast<uint4 *>(dst + (CQ / 8) * GROUP) = val;
-    }
-    // ---- append the chunk's keys, values and positions to the cache (nothing in this launch reads them back from there)
-    if (!RECOUNT && tid < c) p.pos[(size_t)u * p.B + n0 + tid] = step0 + tid;
-    for (int idx = tid; idx < (RECOUNT ? 0 : c * 16); idx += NT) {
-        const int row = idx >> 4, ch = idx & 15;
-        const size_t src = (size_t)row * tstride + (size_t)u * D * 2 + ch * 16;
-        const size_t dst = ((size_t)u * p.B + n0 + row) * (D * 2) + ch * 16;
-        *reinterpret_cast<uint4 *>(p.K + dst) = *reinterpret_cast<const uint4 *>(p.k + src);
-        *reinterpret_cast<uint4 *>(p.V + dst) = *reinterpret_cast<const uint4 *>(p.v + src);
-    }
     // The two sweeps form one sequence of G = 2 ntiles S tiles; tile g covers the keys of tile g mod ntiles.
     // S buffer, K buffer and mbarrier of tile g: g & 1.  V tile kt (second sweep only) sits in buffer kt & 1.
     const int G = 2 * ntiles;
@@ -254,6 +236,34 @@ __global__ void __launch_bounds__(NT, 2) sh_chunk_umma_kernel(const ChunkParams 
     load_pos(0, 0);          // positions of tile g sit in buffer g mod 3: written two iterations ahead of their use
     load_pos(1, key_tile(1));
     if (p.out) load_tile(Vt, Vc, vchunk, 0, n0, n_tot, tstride);     // idle until the second sweep: fetched early
+    // ---- queries (rows beyond c are zero), twice: rows 0..63 and 64..127; asynchronous like the first tiles
+    for (int idx = tid; idx < CQ * 16; idx += NT) {
+        const int row = idx >> 4, ch = idx & 15;
+        char *dst = Qs + (row >> 3) * GROUP + ch * 128 + (row & 7) * 16;
+        if (row < c) {
+            const char *src = RECOUNT ? p.qring + ((size_t)u * p.w + (step0 + row) % p.w) * (D * 2) + ch * 16
+                                      : p.q + (size_t)row * tstride + (size_t)u * D * 2 + ch * 16;
+            cp_async16(dst, src);
+            cp_async16(dst + (CQ / 8) * GROUP, src);
+        } else {
+            *reinterpret_cast<uint4 *>(dst) = make_uint4(0, 0, 0, 0);
+            *reinterpret_cast<uint4 *>(dst + (CQ / 8) * GROUP) = make_uint4(0, 0, 0, 0);
+        }
+    }
+    // ---- while those copies fly: append the chunk's keys, values and positions to the cache (nothing in this
+    // launch reads them back from there) and remember the queries for a later recount
+    if (!RECOUNT && tid < c) p.pos[(size_t)u * p.B + n0 + tid] = step0 + tid;
+    for (int idx = tid; idx < (RECOUNT ? 0 : c * 16); idx += NT) {
+        const int row = idx >> 4, ch = idx & 15;
+        const size_t src = (size_t)row * tstride + (size_t)u * D * 2 + ch * 16;
+        const size_t dst = ((size_t)u * p.B + n0 + row) * (D * 2) + ch * 16;
+        const uint4 kk = *reinterpret_cast<const uint4 *>(p.k + src), vv = *reinterpret_cast<const uint4 *>(p.v + src);
+        uint4 qq = make_uint4(0, 0, 0, 0);
+        if (p.qring) qq = *reinterpret_cast<const uint4 *>(p.q + src);
+        *reinterpret_cast<uint4 *>(p.K + dst) = kk;
+        *reinterpret_cast<uint4 *>(p.V + dst) = vv;
+        if (p.qring) *reinterpret_cast<uint4 *>(p.qring + ((size_t)u * p.w + (step0 + row) % p.w) * (D * 2) + ch * 16) = qq;
+    }
     cp_async_commit();
     cp_async_wait_all();
     fence_async_shared();
@@ -368,10 +378,11 @@ __global__ void __launch_bounds__(NT, 2) sh_chunk_umma_kernel(const ChunkParams 
             const float e0 = v0 ? ex2_approx(sv[jj] * p.scale_log2e - Mi) : 0.f;
             const float e1 = v1 ? ex2_approx(sv[jj + 1] * p.scale_log2e - Mi) : 0.f;
             // step t: low_j = [alpha_j < 1/t] = [e_j * t < L]
-            word |= (uint32_t)(v0 && e0 * tf < Li) << jj;
-            word |= (uint32_t)(v1 && e1 * tf < Li) << (jj + 1);
+            word |= (uint32_t)(e0 * tf < Li) << jj;
+            word |= (uint32_t)(e1 * tf < Li) << (jj + 1);
             SP::run(e0, e1, hi[jj >> 1], lo[jj >> 1]);
         }
+        word &= vm;     // a slot the query does not see has no bit
         // 16 slots: half a record word
         if (live_row && (j0 >> 5) < p.Bw) reinterpret_cast<uint16_t *>(hrow)[j0 >> 4] = (uint16_t)word;
         if (p.out) {
