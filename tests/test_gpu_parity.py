@@ -519,6 +519,48 @@ def test_scores_entry_point_matches_oracle_scores(sh, dtype, d, unordered):
         assert not orc.full
 
 
+def test_scores_on_ragged_sequences_and_after_restore(sh):
+    """sh_scores reads each unit's own row count (ragged handle), and a snapshot of an unordered handle
+    replays identically after sh_restore."""
+    dtype, d = "f16", 128
+    lengths = [5, 40, 17]
+    ups, B, r, w, m = 2, 48, 4, 12, 16
+    U, p_max = len(lengths) * ups, max(lengths)
+    q, k, v = wl.random_stream(U, d, p_max + 1, seed=91, dtype=dtype, peaked=3.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, unordered=True)
+    h.prefill_ragged(q[:p_max].contiguous(), k[:p_max].contiguous(), v[:p_max].contiguous(), lengths)
+    n_seq, _ = h.sequence_state()
+    got = h.scores(q[p_max]).cpu().numpy().astype(np.float64)
+    for sq, L in enumerate(lengths):
+        o = oracle.Oracle(ups, B, r, w, m, d)
+        idx = torch.arange(sq * ups, (sq + 1) * ups, device="cuda")
+        for t in range(L):
+            o.step(to_oracle(q[t], idx), to_oracle(k[t], idx), to_oracle(v[t], idx))
+        assert n_seq[sq] == o.n
+        qf = to_oracle(q[p_max], idx)
+        for j, u in enumerate(range(sq * ups, (sq + 1) * ups)):
+            K, _ = o.cache(j)
+            z = K @ qf[j] / math.sqrt(d)
+            e = np.exp(z - z.max())
+            want = np.sort(e / e.sum())
+            assert np.abs(np.sort(got[u, : o.n]) - want).max() <= 1e-4 * want.max() + 1e-9     # same multiset of scores
+            assert (got[u, o.n:] == 0).all()
+    # snapshot / restore on a uniform unordered handle
+    U2 = 4
+    q2, k2, v2 = wl.random_stream(U2, d, 150, seed=92, dtype=dtype, peaked=2.0, device="cuda")
+    g = sh.Handle(B, r, w, m, U2, d, dtype, unordered=True)
+    for t in range(70):
+        g.decode_step(q2[t], k2[t], v2[t])
+    snap = g.snapshot()
+    first = [g.decode_step(q2[t], k2[t], v2[t]).clone() for t in range(70, 150)]
+    s1 = g.state()
+    g.restore(snap)
+    second = [g.decode_step(q2[t], k2[t], v2[t]).clone() for t in range(70, 150)]
+    s2 = g.state()
+    assert all(torch.equal(x, y) for x, y in zip(first, second))
+    assert s1[0] == s2[0] and s1[1] == s2[1] and all((x == y).all() for x, y in zip(s1[2:], s2[2:]))
+
+
 def test_score_change_ratio_diagnostic(sh):
     """(alpha_s - alpha_o) / alpha_o of the last step's query, budgeted cache against full cache, from
     the library; the same from two oracles' caches with the softmax written out here.  Units whose
