@@ -211,6 +211,23 @@ def test_config_opt66b_full_size_sampled_units(sh, unordered):
     assert res.adoptions <= 1e-4 * res.slot_steps + 2
 
 
+def test_config_opt66b_full_size_chunked_prompt_sampled_units(sh):
+    """The prompt phase of the benchmark's workload at full size (9216 units per launch of the tcgen05
+    chunk kernel, unordered compaction as the benchmark runs it), a sample of units in lockstep with
+    the oracle through several compressions, then decode steps from the state the chunks left."""
+    cfg = wl.CONFIGS["opt66b"]
+    st = wl.Stream(cfg, device="cuda")
+    units = wl.sample_units(cfg, 24)
+    h = SortedView(sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, cfg.units, cfg.head_dim, cfg.dtype, auto_compress=False,
+                             unordered=True), units=units)
+    T = cfg.B + 5 * cfg.m + 20
+    blk = lambda t0, t1: st.block(t0, t1)
+    res, orc = run_lockstep_chunked(h, cfg.dtype, blk, T, units, TOL[cfg.dtype], chunk_sizes=[64])
+    assert res.steps == T and res.compressions == 6
+    assert res.adoptions <= 1e-4 * res.slot_steps + 2
+    run_lockstep(h, cfg.dtype, st.step, 30, units, TOL[cfg.dtype], orc=orc)
+
+
 @pytest.mark.parametrize("layer", [0, 39])
 def test_config_opt13b_layer_sampled_units(sh, layer):
     cfg = wl.CONFIGS["opt13b"]
