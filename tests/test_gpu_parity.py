@@ -611,6 +611,71 @@ def test_score_change_ratio_diagnostic(sh):
     assert checked >= U - 2
 
 
+@pytest.mark.parametrize("B,w,m", [(8192, 48, 4096), (2048, 16384, 1024)])
+def test_large_budget_lockstep(sh, B, w, m):
+    """B = 8192: every kernel's large-size path (many key tiles, 256 record words per bit-plane row,
+    selection from global memory); w = 16384: the longest history window the library takes.  Both in
+    lockstep with the oracle through two compressions."""
+    U, d, r, dtype = 1, 64, 10, "f16"
+    T = B + m + 12
+    q, k, v = wl.random_stream(U, d, T, seed=101, dtype=dtype, peaked=2.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    res, _ = run_lockstep(h, dtype, _stream_fn(q, k, v), T, torch.arange(U), TOL[dtype], state_every=2048)
+    assert res.compressions == 2
+
+
+@pytest.mark.parametrize("unordered", [False, True])
+def test_maximum_budget_properties(sh, unordered):
+    """The largest budget the library takes (B = 32768) with the longest window that fits the test
+    (w = 2048): the prompt goes through the chunk kernel, the cache fills, one compression drops
+    m = 16384 tokens.  The oracle would need minutes here, so the check is by properties that hold at
+    any size, plus one step's attention output and scores against the plain definition (softmax of
+    q.K / sqrt(d), then times V) evaluated in fp64 on the rows the library exports."""
+    U, d, B, r, w, m, dtype = 1, 128, 32768, 100, 2048, 16384, "f16"
+    T = B - 1
+    g = torch.Generator(device="cuda")
+    g.manual_seed(7)
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, unordered=unordered)
+    blk = 4096
+    for t0 in range(0, T, blk):
+        n_tok = min(blk, T - t0)
+        x = (torch.randn(3, n_tok, U, d, generator=g, device="cuda") * 0.7).to(torch.float16)
+        h.prefill(x[0], x[1], x[2])
+    assert h.n == B - 1
+    x = (torch.randn(3, U, d, generator=g, device="cuda") * 0.7).to(torch.float16)
+    out = h.decode_step(x[0], x[1], x[2])
+    n, t, pos, cnt, low = h.state()
+    assert n == B and t == B and (pos[0] == np.arange(1, B + 1)).all()
+    assert cnt.max() <= w and (cnt[0, -1] <= 1)
+    K, V = h.export_unit(0)
+    z = K.astype(np.float64) @ x[0][0].double().cpu().numpy() / math.sqrt(d)
+    e = np.exp(z - z.max())
+    alpha = e / e.sum()
+    assert np.abs(out[0].double().cpu().numpy() - alpha @ V.astype(np.float64)).max() <= TOL[dtype]
+    got_alpha = h.scores(x[0]).cpu().numpy().astype(np.float64)[0]
+    assert np.abs(got_alpha - alpha).max() <= 1e-4 * alpha.max() + 1e-9
+    amb = np.abs(alpha - 1.0 / t) <= 1e-6
+    assert ((low[0] == (alpha < 1.0 / t)) | amb).all()          # this step's record bits
+    # compression: m tokens go, none of the r newest, the survivors keep position, counter and rows
+    assert h.compress() == m
+    n2, _, pos2, cnt2, _ = h.state(low=False)
+    assert n2 == B - m and len(set(pos2[0].tolist())) == n2
+    assert set(range(B - r + 1, B + 1)) <= set(pos2[0].tolist())
+    if not unordered:
+        assert (np.diff(pos2[0]) > 0).all()
+    assert (cnt2[0] == cnt[0][pos2[0] - 1]).all()
+    dropped = np.setdiff1d(np.arange(1, B + 1), pos2[0])
+    cand = np.arange(1, B - r + 1)
+    kept_cand = np.setdiff1d(cand, dropped)
+    assert cnt[0][dropped - 1].min() >= cnt[0][kept_cand - 1].max()      # the m largest counters went
+    tie = cnt[0][dropped - 1].min()
+    tie_kept = kept_cand[cnt[0][kept_cand - 1] == tie]
+    tie_dropped = dropped[cnt[0][dropped - 1] == tie]
+    assert len(tie_kept) == 0 or tie_dropped.max() < tie_kept.min()      # oldest first among equals
+    K2, V2 = h.export_unit(0)
+    assert (K2[:n2] == K[pos2[0] - 1]).all() and (V2[:n2] == V[pos2[0] - 1]).all()
+
+
 def test_error_codes(sh):
     import ctypes as C
     lib = sh.lib
