@@ -45,3 +45,65 @@ def test_host_only_calls_validate_arguments():
     assert lib.sh_create(410, 64, 128, 64, 9216, 128, sh.SH_F16, None) == sh.SH_EINVAL
     assert lib.sh_create(40000, 64, 128, 64, 1, 128, sh.SH_F16, C.byref(h)) == sh.SH_EINVAL
     assert lib.sh_select(None, 1, 10, 0, 1, None, None) == sh.SH_EINVAL
+
+
+def _handle(sh, B, r, w, m, heads, d, dtype):
+    h = C.c_void_p()
+    assert sh.lib.sh_create(B, r, w, m, heads, d, sh.DTYPE_CODE[dtype], C.byref(h)) == sh.SH_OK
+    return h
+
+
+def test_option_values_and_the_shapes_they_need():
+    """Host logic of sh_set_option: which values each option takes, and which shapes the chunk kernels
+    and the recompute mode need (no device call is made)."""
+    from paper_2305_17118_b200 import binding as sh
+    lib = sh.lib
+    h = _handle(sh, 410, 64, 128, 64, 16, 128, "f16")
+    assert lib.sh_prefill_chunk_max(h) == 64
+    for key, good, bad in ((sh.SH_OPT_COMPACTION, (0, 1), (2, -1)), (sh.SH_OPT_PREFILL_CHUNK, (0, 1, 2, 3), (4, -1)),
+                           (sh.SH_OPT_DECODE_KERNEL, (0, 1, 2), (3,)), (sh.SH_OPT_SPLIT, (1, 2, 4, 8), (3, 16))):
+        for v in good:
+            assert lib.sh_set_option(h, key, float(v)) == sh.SH_OK, (key, v)
+        for v in bad:
+            assert lib.sh_set_option(h, key, float(v)) == sh.SH_EINVAL, (key, v)
+    before = lib.sh_workspace_bytes(h)
+    assert lib.sh_set_option(h, sh.SH_OPT_RECORD_MODE, 1.0) == sh.SH_OK
+    assert lib.sh_workspace_bytes(h) >= before + 16 * 128 * 128 * 2          # the ring of the last w queries
+    lib.sh_destroy(h)
+    # a window shorter than a chunk bounds the chunk; int4 and head_dim 64 have no chunk kernel
+    h = _handle(sh, 150, 9, 37, 41, 3, 128, "bf16")
+    assert lib.sh_prefill_chunk_max(h) == 37
+    lib.sh_destroy(h)
+    for dtype, d in (("int4", 128), ("f16", 64), ("f32", 128)):
+        h = _handle(sh, 150, 9, 37, 41, 3, d, dtype)
+        assert lib.sh_prefill_chunk_max(h) == 0
+        assert lib.sh_set_option(h, sh.SH_OPT_RECORD_MODE, 1.0) == sh.SH_EINVAL
+        lib.sh_destroy(h)
+    # the warp-level chunk kernel keeps a row of logits in shared memory: it stops at budgets of about 700,
+    # the tcgen05 kernel does not; the recompute mode follows the kernel that is chosen
+    h = _handle(sh, 4000, 10, 400, 2000, 2, 128, "f16")
+    assert lib.sh_prefill_chunk_max(h) == 64
+    assert lib.sh_set_option(h, sh.SH_OPT_PREFILL_CHUNK, 2.0) == sh.SH_OK
+    assert lib.sh_prefill_chunk_max(h) == 0
+    assert lib.sh_set_option(h, sh.SH_OPT_RECORD_MODE, 1.0) == sh.SH_EINVAL
+    assert lib.sh_set_option(h, sh.SH_OPT_PREFILL_CHUNK, 1.0) == sh.SH_OK
+    assert lib.sh_set_option(h, sh.SH_OPT_RECORD_MODE, 1.0) == sh.SH_OK
+    assert lib.sh_set_option(h, sh.SH_OPT_PREFILL_CHUNK, 2.0) == sh.SH_EINVAL      # would strand the recount
+    lib.sh_destroy(h)
+
+
+def test_create_rejects_shapes_outside_the_documented_range():
+    from paper_2305_17118_b200 import binding as sh
+    lib = sh.lib
+    h = C.c_void_p()
+    ok = (410, 64, 128, 64, 16, 128, sh.SH_F16)
+    assert lib.sh_create(*ok, C.byref(h)) == sh.SH_OK
+    lib.sh_destroy(h)
+    for bad in ((0, 0, 1, 1, 1, 128, sh.SH_F16), (32769, 1, 1, 1, 1, 128, sh.SH_F16), (410, 64, 16385, 64, 1, 128, sh.SH_F16),
+                (410, 64, 0, 64, 1, 128, sh.SH_F16), (410, 64, 128, 0, 1, 128, sh.SH_F16), (410, 64, 128, 347, 1, 128, sh.SH_F16),
+                (410, -1, 128, 64, 1, 128, sh.SH_F16), (410, 64, 128, 64, 0, 128, sh.SH_F16), (410, 64, 128, 64, 1, 96, sh.SH_F16),
+                (410, 64, 128, 64, 1, 128, 17)):
+        assert lib.sh_create(*bad, C.byref(h)) == sh.SH_EINVAL, bad
+    assert lib.sh_create(*ok, None) == sh.SH_EINVAL
+    for code in (sh.SH_OK, sh.SH_EINVAL, sh.SH_ESTATE, sh.SH_EFULL, sh.SH_ECUDA, sh.SH_ETOOBIG):
+        assert len(lib.sh_strerror(code)) >= 2
