@@ -8,7 +8,7 @@
 
 namespace {
 
-constexpr int SEL_THREADS = 256;
+constexpr int SEL_THREADS = 128;
 constexpr int CMP_THREADS = 256;
 constexpr int SEL_TIE_CAP = 1024;     // tie classes up to this size are searched from a shared-memory list
 
@@ -332,8 +332,8 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
                 *reinterpret_cast<uint4 *>(rows + (size_t)hole * c.row_bytes + ch * 16) =
                     *reinterpret_cast<const uint4 *>(rows + (size_t)last * c.row_bytes + ch * 16);
             }
-            if (tid >= 64 && tid < 66 && c.scale_bytes) {
-                char *sc = (tid == 64 ? c.Ks : c.Vs) + (size_t)u * c.Bs * c.scale_bytes;
+            if (tid < 2 && c.scale_bytes) {
+                char *sc = (tid == 0 ? c.Ks : c.Vs) + (size_t)u * c.Bs * c.scale_bytes;
                 for (int b = 0; b < c.scale_bytes; ++b) sc[(size_t)hole * c.scale_bytes + b] = sc[(size_t)last * c.scale_bytes + b];
             }
         }
