@@ -1,4 +1,6 @@
-// Chunked prompt step: c consecutive tokens of the stream handled in one launch.
+// Chunked prompt step: c consecutive tokens of the stream handled in one launch.  This file holds the
+// warp-level (mma.sync) kernel, chosen with SH_OPT_PREFILL_CHUNK = 2, and the dispatch between it and the
+// tcgen05 kernel of sh_chunk_umma.cu, which is the default.
 //
 // Between two compressions the method's steps only append, so c steps can be
 // evaluated together: step i (0 <= i < c) attends with q_i over the n0 cached
