@@ -22,6 +22,13 @@
  *   - Every function returns an sh_status (0 = SH_OK, negative = error) and
  *     never aborts, throws or prints.  On error nothing has been enqueued
  *     unless stated otherwise.
+ *   - A handle is not thread-safe: calls on one handle must not overlap (calls on
+ *     different handles may, from any threads).  All calls that touch one
+ *     handle's workspace should be given the same stream, or streams the
+ *     caller has ordered; the library inserts no cross-stream dependencies.
+ *   - Kernels that wait (on mbarriers) do so for a bounded time; one that gives
+ *     up records a code in the workspace's error word, finishes without touching
+ *     further state, and the next sh_state returns SH_EDEVICE.
  *   - Slots [0, n) of a unit's cache are live.  By default they are sorted by
  *     stream position (compaction is stable, so "the r newest" are slots
  *     [n-r, n)); with SH_OPT_COMPACTION = 1 their order is arbitrary.
