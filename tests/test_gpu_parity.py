@@ -48,6 +48,19 @@ def test_lockstep_edge_parameters(sh, B, r, w, m):
     assert res.compressions >= 1
 
 
+@pytest.mark.parametrize("dtype,d", [("f32", 64), ("f32", 128), ("f16", 64), ("bf16", 64), ("int4", 128), ("int4", 64)])
+def test_lockstep_direct_kernel_many_units(sh, dtype, d):
+    """The direct-load decode kernel in the CTA shape it takes from 592 units on (4 warps, more rows per
+    thread), every storage type it serves there; a sample of units in lockstep."""
+    U, B, r, w, m, T = 601, 77, 6, 21, 30, 150
+    q, k, v = wl.random_stream(U, d, T, seed=13, dtype=dtype, peaked=3.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, kernel=1, auto_compress=False)
+    units = torch.tensor([0, 1, 17, 148, 299, 300, 592, 600])
+    res, _ = run_lockstep(h, dtype, _stream_fn(q, k, v), T, units, TOL[dtype])
+    assert res.compressions >= 3
+    assert res.adoptions <= 1e-4 * res.slot_steps + 2
+
+
 @pytest.mark.parametrize("dtype,d", [("f16", 128), ("bf16", 128), ("f32", 128), ("f32", 64)])
 @pytest.mark.parametrize("U,B,r,w,m", [(5, 150, 9, 37, 41), (301, 130, 16, 33, 50), (3, 700, 5, 64, 300), (2, 40, 3, 9, 20)])
 def test_lockstep_pipelined_kernel(sh, dtype, d, U, B, r, w, m):
