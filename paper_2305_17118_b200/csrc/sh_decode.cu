@@ -293,6 +293,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 // S CTAs per unit (a thread-block cluster when S > 1).
 template <int DT, int D, int NW, int R, int S>
 __global__ void __launch_bounds__(NW * 32) sh_decode_kernel(const DecodeParams p) {
+    static_assert((R & (R - 1)) == 0, "the row-sum transposition halves R at every step");
     using E = Elem<DT>;
     constexpr int EPL = E::EPL;
     constexpr int LPR = D / EPL;     // lanes per row
