@@ -292,7 +292,10 @@ __device__ __forceinline__ float warp_sum(float v) {
 // DT dtype, D head_dim, NW warps per CTA, R rows in flight per lane,
 // S CTAs per unit (a thread-block cluster when S > 1).
 template <int DT, int D, int NW, int R, int S>
-__global__ void __launch_bounds__(NW * 32) sh_decode_kernel(const DecodeParams p) {
+// (CTAs of 4 warps are the many-units shape: capped at 64 registers so that 8 of them share an SM - measured
+// at 9216 units, int4 289 -> 237 us, int4 with head_dim 64 249 -> 173 us, 16-bit rows of 128 bytes unchanged;
+// fp32 rows of 512 bytes would spill and keep the compiler's choice)
+__global__ void __launch_bounds__(NW * 32, NW == 4 ? ((DT == SH_F32 && D == 128) ? 4 : 8) : 0) sh_decode_kernel(const DecodeParams p) {
     static_assert((R & (R - 1)) == 0, "the row-sum transposition halves R at every step");
     using E = Elem<DT>;
     constexpr int EPL = E::EPL;
