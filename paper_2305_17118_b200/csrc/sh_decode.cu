@@ -691,7 +691,7 @@ cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStr
     cudaError_t e = cudaErrorInvalidValue;
     // Two shapes of CTA.  With few units per SM the step is latency-bound and a CTA of 8 warps with 8 row
     // loads in flight per thread finishes a unit soonest.  With many units per SM (no cluster split then)
-    // CTAs of 4 warps, each thread holding more rows, spend less on barriers and on the cross-warp merge:
+    // CTAs of 4 warps (16 row loads in flight per thread; int4, whose loads carry 32 elements each: 2), spend less on barriers and on the cross-warp merge:
     // measured at 9216 units on B200, int4 428 -> 289 us, fp16 with head_dim 64 183 -> 149 us, fp32 with
     // head_dim 64 369 -> 298 us; rows of 256 bytes in 16-bit types stay with 8 warps (283 against 309 us).
     const bool many = p.U >= 4 * 148 && c->split == 1;
@@ -709,8 +709,8 @@ cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStr
             else if (c->D == 128) e = launch_split<SH_BF16, 128, 8, 8>(c, p, s);
             break;
         case SH_INT4_G64_F16:
-            if (c->D == 64) e = many ? launch_one<SH_INT4_G64_F16, 64, 4, 4, 1>(c, p, s) : launch_split<SH_INT4_G64_F16, 64, 8, 4>(c, p, s);
-            else if (c->D == 128) e = many ? launch_one<SH_INT4_G64_F16, 128, 4, 4, 1>(c, p, s) : launch_split<SH_INT4_G64_F16, 128, 8, 4>(c, p, s);
+            if (c->D == 64) e = many ? launch_one<SH_INT4_G64_F16, 64, 4, 2, 1>(c, p, s) : launch_split<SH_INT4_G64_F16, 64, 8, 4>(c, p, s);
+            else if (c->D == 128) e = many ? launch_one<SH_INT4_G64_F16, 128, 4, 2, 1>(c, p, s) : launch_split<SH_INT4_G64_F16, 128, 8, 4>(c, p, s);
             break;
         default: break;
     }
