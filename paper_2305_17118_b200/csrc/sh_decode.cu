@@ -683,18 +683,26 @@ cudaError_t sh_launch_scores(const sh_context *c, const DecodeParams &p, float *
 }
 
 cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches) {
-    // Rows of 256 bytes or more stream through the persistent pipelined kernel unless the caller
-    // asked for this one or for a cluster split, or there are too few units to give most SMs one.
-    if (c->kernel != 1 && sh_decode_tma_supported(c) &&
-        (c->kernel == 2 || (p.U >= 128 && !(c->split_explicit && c->split > 1))))
+    // Shapes of launch (crossovers measured on B200, rows of 256 bytes: equal at 12 units per SM, the direct
+    // kernel 6 % ahead from 16 per SM on, the pipelined one 15 % ahead at 8.6).  With very many units per SM
+    // the direct-load kernel in its many-units shape is the fastest for every storage type: CTAs of 4 warps
+    // capped at 64 registers, eight per SM, hide the load latency by occupancy (9216 units, fp16 rows of 256
+    // bytes: 261 us against 273 us for the pipelined kernel).  Below 16 units per SM, rows of 256 bytes or
+    // more stream through the persistent pipelined kernel from 128 units on; the direct kernel takes the
+    // rest, with 4-warp CTAs from 4 units per SM on and 8-warp CTAs (and a cluster split for very few units)
+    // below.  SH_OPT_DECODE_KERNEL = 1 / 2 forces the direct / pipelined kernel.
+    const bool many = p.U >= 4 * 148 && c->split == 1;
+    const bool pipelined_ok = sh_decode_tma_supported(c);
+    const bool prefer_direct = many && (!pipelined_ok || p.U >= 16 * 148);
+    if (c->kernel != 1 && pipelined_ok &&
+        (c->kernel == 2 || (!prefer_direct && p.U >= 128 && !(c->split_explicit && c->split > 1))))
         return sh_launch_decode_tma(c, p, s, launches);
     cudaError_t e = cudaErrorInvalidValue;
     // Two shapes of CTA.  With few units per SM the step is latency-bound and a CTA of 8 warps with 8 row
     // loads in flight per thread finishes a unit soonest.  With many units per SM (no cluster split then)
     // CTAs of 4 warps (16 row loads in flight per thread; int4, whose loads carry 32 elements each: 2), spend less on barriers and on the cross-warp merge:
     // measured at 9216 units on B200, int4 428 -> 289 us, fp16 with head_dim 64 183 -> 149 us, fp32 with
-    // head_dim 64 369 -> 298 us; rows of 256 bytes in 16-bit types stay with 8 warps (283 against 309 us).
-    const bool many = p.U >= 4 * 148 && c->split == 1;
+    // head_dim 64 369 -> 263 us, 16-bit rows of 256 bytes 283 -> 261 us.
     switch (c->dtype) {
         case SH_F32:
             if (c->D == 64) e = many ? launch_one<SH_F32, 64, 4, 16, 1>(c, p, s) : launch_split<SH_F32, 64, 8, 8>(c, p, s);
@@ -702,11 +710,11 @@ cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStr
             break;
         case SH_F16:
             if (c->D == 64) e = many ? launch_one<SH_F16, 64, 4, 16, 1>(c, p, s) : launch_split<SH_F16, 64, 8, 8>(c, p, s);
-            else if (c->D == 128) e = launch_split<SH_F16, 128, 8, 8>(c, p, s);
+            else if (c->D == 128) e = many ? launch_one<SH_F16, 128, 4, 8, 1>(c, p, s) : launch_split<SH_F16, 128, 8, 8>(c, p, s);
             break;
         case SH_BF16:
             if (c->D == 64) e = many ? launch_one<SH_BF16, 64, 4, 16, 1>(c, p, s) : launch_split<SH_BF16, 64, 8, 8>(c, p, s);
-            else if (c->D == 128) e = launch_split<SH_BF16, 128, 8, 8>(c, p, s);
+            else if (c->D == 128) e = many ? launch_one<SH_BF16, 128, 4, 8, 1>(c, p, s) : launch_split<SH_BF16, 128, 8, 8>(c, p, s);
             break;
         case SH_INT4_G64_F16:
             if (c->D == 64) e = many ? launch_one<SH_INT4_G64_F16, 64, 4, 2, 1>(c, p, s) : launch_split<SH_INT4_G64_F16, 64, 8, 4>(c, p, s);
