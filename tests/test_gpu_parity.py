@@ -493,6 +493,39 @@ def test_ragged_sequences_lockstep(sh, dtype, kernel, unordered):
     assert compressions >= 12                    # the sequences fill at different steps
 
 
+@pytest.mark.parametrize("dtype", ["f16", "int4"])
+def test_ragged_sequences_many_units(sh, dtype):
+    """Ragged sequences on the many-units shape of the direct decode kernel (600 units: per-unit row counts
+    read and advanced on the device by 4-warp CTAs), every unit in lockstep, automatic compression."""
+    d, lengths, ups, B, r, w, m, T_dec = 128, [3, 41], 300, 48, 4, 12, 16, 40
+    U, p_max = len(lengths) * ups, max(lengths)
+    q, k, v = wl.random_stream(U, d, p_max + T_dec, seed=57, dtype=dtype, peaked=3.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, kernel=1)
+    h.prefill_ragged(q[:p_max].contiguous(), k[:p_max].contiguous(), v[:p_max].contiguous(), lengths)
+    orcs = []
+    for sq, L in enumerate(lengths):
+        o = oracle.Oracle(ups, B, r, w, m, d, quant=(dtype == "int4"))
+        idx = torch.arange(sq * ups, (sq + 1) * ups, device="cuda")
+        for t in range(L):
+            o.step(to_oracle(q[t], idx), to_oracle(k[t], idx), to_oracle(v[t], idx))
+        orcs.append(o)
+    worst, agree = 0.0, []
+    for step in range(T_dec):
+        ti = p_max + step
+        out = h.decode_step(q[ti], k[ti], v[ti])
+        for sq, o in enumerate(orcs):
+            idx = torch.arange(sq * ups, (sq + 1) * ups, device="cuda")
+            oo, _ = o.step(to_oracle(q[ti], idx), to_oracle(k[ti], idx), to_oracle(v[ti], idx))
+            err = np.abs(out[idx].double().cpu().numpy() - oo).max(axis=1)
+            pos = h.state_full()[0][sq * ups:(sq + 1) * ups, : o.n]
+            same = (pos == o.positions()).all(axis=1)          # a threshold-ambiguous flip may change a unit's kept set
+            worst = max(worst, float(err[same].max()))
+            agree.append(same.mean())
+    n_seq, t_seq = h.sequence_state()
+    assert n_seq.tolist() == [o.n for o in orcs] and t_seq.tolist() == [L + T_dec for L in lengths]
+    assert worst <= TOL[dtype] and min(agree) >= 0.97
+
+
 def test_persistence_diagnostics_match_oracle_scores(sh):
     """Persistence ratio and pivotal-set size (Section 3.2) from the library's record bits, against
     the same quantities from the oracle's fp64 scores on a full (never compressed) cache."""
