@@ -83,9 +83,9 @@ typedef enum {
                                  particular order: sh_state's pos tells which token sits where.  The kept set is
                                  the same either way. */
     SH_OPT_PREFILL_CHUNK = 4, /* 1 (default): sh_prefill hands the tokens between two compressions to the chunk
-                                 kernel where the shape allows it (fp16/bf16, head_dim 128: the tcgen05 kernel,
-                                 any budget); 0: one decode step per token; 2: the warp-level MMA chunk kernel
-                                 (budgets up to about 700); 3: same as 1 */
+                                 kernel where the shape allows it (fp16/bf16/int4 with head_dim 128: the tcgen05
+                                 kernels, any budget); 0: one decode step per token; 2: the warp-level MMA chunk kernel
+                                 (fp16/bf16, budgets up to about 700); 3: same as 1 */
     SH_OPT_DECODE_KERNEL = 3  /* 0 (default): chosen from the shape; 1: one CTA (or cluster) per unit with
                                  direct loads; 2: persistent CTAs fed by bulk asynchronous copies
                                  (stored rows of 256 bytes or more: fp32, and fp16/bf16 with head_dim 128; SH_OPT_SPLIT

@@ -140,7 +140,9 @@ struct SelectParams {
 struct ChunkParams {
     const char *q, *k, *v;   // [c][U][D] time-major, 16-bit elements
     float *out;              // [c][U][D] fp32 or NULL
-    char *K, *V;             // caches [U][B][D]
+    char *K, *V;             // caches [U][B][D] (int4 store: [U][B][D/2] codes)
+    char *Ks, *Vs;           // int4 store: fp16 group scales [U][Bs][D/64]
+    int Bs;                  // int4 store: scale rows per unit
     uint32_t *hist;
     int32_t *pos;
     int U, B, Bw, w;
@@ -162,6 +164,8 @@ struct ChunkParams {
 int sh_chunk_umma_capacity();
 cudaError_t sh_launch_chunk_umma(const ChunkParams &p, int dtype, cudaStream_t s);
 cudaError_t sh_launch_recount_umma(const ChunkParams &p, int dtype, cudaStream_t s);
+// int4-g64 store: the chunked prompt step with codes unpacked into the tensor-core tiles (sh_chunk_umma_int4.cu).
+cudaError_t sh_launch_chunk_umma_int4(const ChunkParams &p, cudaStream_t s);
 
 // Launchers (each returns the cudaError_t of its launch and adds to *launches).
 cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches);

@@ -332,7 +332,12 @@ size_t smem_need(int CQ, int B) {
 
 // Largest number of tokens one chunk launch can take for this handle (0: not supported).
 int sh_prefill_chunk_capacity(const sh_context *c) {
-    if ((c->dtype != SH_F16 && c->dtype != SH_BF16) || c->D != 128) return 0;
+    if (c->D != 128) return 0;
+    if (c->dtype == SH_INT4_G64_F16) {       // int4 store: the tcgen05 kernel only
+        if (c->prefill_chunk == 2) return 0;
+        return sh_chunk_umma_capacity() < c->w ? sh_chunk_umma_capacity() : c->w;
+    }
+    if (c->dtype != SH_F16 && c->dtype != SH_BF16) return 0;
     int cq = 0;
     if (c->prefill_chunk != 2) cq = sh_chunk_umma_capacity();     // tcgen05 kernel: any budget
     else if (smem_need(32, c->B) <= 200 * 1024) cq = 64;          // warp-level kernel: one or two CTAs of 32 queries, or one of 64
@@ -354,6 +359,7 @@ cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const vo
     p.q = static_cast<const char *>(q); p.k = static_cast<const char *>(k); p.v = static_cast<const char *>(v);
     p.out = out;
     p.K = sh_pK(c); p.V = sh_pV(c);
+    p.Ks = sh_pKs(c); p.Vs = sh_pVs(c); p.Bs = c->Bs;
     p.hist = sh_phist(c);
     p.pos = sh_ppos(c);
     p.U = c->ucount; p.Utot = c->U; p.B = c->B; p.Bw = c->Bw; p.w = c->w;
@@ -364,6 +370,11 @@ cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const vo
     p.err = reinterpret_cast<int *>(c->slab + c->L.err);
     cudaError_t e = cudaErrorInvalidValue;
     if (count < 1 || count > sh_prefill_chunk_capacity(c)) return e;
+    if (c->dtype == SH_INT4_G64_F16) {
+        e = sh_launch_chunk_umma_int4(p, s);
+        if (e == cudaSuccess) *launches += 1;
+        return e;
+    }
     if (c->prefill_chunk != 2) {
         e = sh_launch_chunk_umma(p, c->dtype, s);
         if (e == cudaSuccess) *launches += 1;

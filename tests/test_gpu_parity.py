@@ -95,6 +95,28 @@ def test_lockstep_chunked_prompt_kernel(sh, dtype, U, B, r, w, m, sizes, chunk_k
     run_lockstep(h, dtype, lambda t: (q2[t - T - 1], k2[t - T - 1], v2[t - T - 1]), 40, torch.arange(U), TOL[dtype], orc=orc)
 
 
+@pytest.mark.parametrize("U,B,r,w,m,sizes", [(5, 150, 9, 37, 41, [37, 7, 33, 1]), (3, 410, 64, 128, 64, [64]),
+                                             (150, 96, 8, 70, 30, [64, 31]), (2, 1300, 10, 64, 650, [64, 13])])
+def test_lockstep_chunked_int4_store(sh, U, B, r, w, m, sizes):
+    """The chunk kernel of the int4-g64 store (codes as tensor-core operands, scales applied in fp32):
+    outputs, record bits, positions, counters and kept sets against the oracle's quantised cache; then
+    decode steps from the state the chunks left; and the quantised rows equal the oracle's bit for bit."""
+    dtype, d, T = "int4", 128, min(2 * B + 2 * m + 11, B + 2 * m + 60)
+    q, k, v = wl.random_stream(U, d, T, seed=37 + U, dtype=dtype, peaked=3.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
+    res, orc = run_lockstep_chunked(h, dtype, blk, T, torch.arange(U), TOL[dtype], chunk_sizes=sizes)
+    assert res.steps == T and res.compressions >= 2
+    assert res.adoptions <= 1e-4 * res.slot_steps + 2
+    n = h.n
+    for u in (0, U - 1):
+        K, V = h.export_unit(u)
+        oK, oV = orc.cache(u)
+        assert (K[:n].astype(np.float64) == oK).all() and (V[:n].astype(np.float64) == oV).all()
+    q2, k2, v2 = wl.random_stream(U, d, 30, seed=97, dtype=dtype, peaked=3.0, device="cuda")
+    run_lockstep(h, dtype, lambda t: (q2[t - T - 1], k2[t - T - 1], v2[t - T - 1]), 30, torch.arange(U), TOL[dtype], orc=orc)
+
+
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
 @pytest.mark.parametrize("U,B,r,w,m,sizes", [(2, 2100, 10, 400, 1050, [64, 64, 13]), (150, 33, 2, 70, 11, [64, 3]),
                                              (1, 129, 1, 64, 64, [64]), (3, 1000, 10, 5, 500, [5, 2])])
