@@ -413,9 +413,11 @@ def test_prefill_equals_token_by_token_steps(sh):
     assert torch.equal(a.slab[a._slab_off:a._slab_off + 2 * U * B * d * 2], b.slab[b._slab_off:b._slab_off + 2 * U * B * d * 2])
 
 
-@pytest.mark.parametrize("pinned", [True, False])
-def test_host_buffer_step_matches_device_step(sh, pinned):
-    U, d, B, r, w, m, T, dtype = 7, 128, 64, 4, 16, 20, 100, "bf16"
+@pytest.mark.parametrize("pinned,U", [(True, 7), (False, 7), (True, 2400)])
+def test_host_buffer_step_matches_device_step(sh, pinned, U):
+    """sh_decode_step_host against sh_decode_step, bit for bit; 2400 units run the many-units shape of the
+    decode kernel on host-resident inputs."""
+    d, B, r, w, m, T, dtype = 128, 64, 4, 16, 20, 100, "bf16"
     q, k, v = wl.random_stream(U, d, T, seed=6, dtype=dtype, peaked=2.0, device="cuda")
     a = sh.Handle(B, r, w, m, U, d, dtype)
     b = sh.Handle(B, r, w, m, U, d, dtype)
