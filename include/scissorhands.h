@@ -152,8 +152,8 @@ int sh_decode_step_host(sh_handle h, const void *q_host, const void *k_new_host,
  * sh_decode_step (each followed by a compression when the cache fills),
  * whatever SH_OPT_AUTO_COMPRESS says.  q_dev, k_dev, v_dev: time-major
  * [p][heads][head_dim].  out_dev: [p][heads][head_dim] fp32 or NULL to discard.
- * Between two compressions the steps only append, so for fp16/bf16 stores with
- * head_dim 128 they are evaluated up to 64 at a time by a tensor-core kernel
+ * Between two compressions the steps only append, so for fp16, bf16 and int4 stores
+ * with head_dim 128 they are evaluated up to 64 at a time by a tensor-core kernel
  * (causal attention of the chunk over the cache and itself, one record
  * bit-plane row per step); the results equal the per-token path up to fp32
  * summation order.  SH_OPT_PREFILL_CHUNK = 0 forces the per-token path.
