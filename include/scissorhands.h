@@ -74,8 +74,8 @@ typedef enum {
                                  token per step; 1: it is recomputed at every compression from the queries of
                                  the last w steps (the library keeps them: heads*w*head_dim extra elements)
                                  scored against the cache as it is then (Algorithm 2 as stated; Section 4.1,
-                                 "Overhead Tradeoff").  fp16/bf16, head_dim 128 (with SH_OPT_PREFILL_CHUNK = 2
-                                 also: budgets up to about 700); else SH_EINVAL.  Set before sh_bind:
+                                 "Overhead Tradeoff").  fp16/bf16/int4, head_dim 128 (with SH_OPT_PREFILL_CHUNK = 2:
+                                 fp16/bf16 and budgets up to about 700 only); else SH_EINVAL.  Set before sh_bind:
                                  it changes sh_workspace_bytes. */
     SH_OPT_COMPACTION = 6,    /* 0 (default): stable left-compaction, slots stay sorted by stream position;
                                  1: every hole left by a dropped token below n-m is filled with a kept row from

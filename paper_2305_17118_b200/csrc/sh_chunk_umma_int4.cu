@@ -147,6 +147,10 @@ __device__ __forceinline__ void quantise_group(const char *src, char *dst, __hal
 }
 
 
+// RECOUNT: the record recomputed at compression time - queries from the ring of the last w queries (blockIdx.y
+// selects 64 of them), keys the n0 cached rows, a key visible to a query when its position does not exceed the
+// query's step; nothing is appended, no output: only the bit-plane rows of those steps are rewritten.
+template <bool RECOUNT>
 __global__ void __launch_bounds__(NT, 1) sh_chunk_umma_int4_kernel(const ChunkParams p) {
     using SP = Split<SH_F16>;
     extern __shared__ __align__(128) unsigned char sm[];
@@ -165,9 +169,18 @@ __global__ void __launch_bounds__(NT, 1) sh_chunk_umma_int4_kernel(const ChunkPa
 
     const int u = blockIdx.x, tid = threadIdx.x, warp = tid >> 5;
     const int i = tid & 63, quarter = ((tid >> 6) & 1) * 2 + (tid >> 7);
-    const int n0 = p.n0, c = p.c, n_tot = n0 + c;
+    const int qoff = RECOUNT ? (int)blockIdx.y * CQ : 0;
+    const int n0 = p.n0, c = RECOUNT ? min(CQ, p.nsteps - qoff) : p.c, n_tot = RECOUNT ? n0 : n0 + c;
     const int ntiles = (n_tot + TN - 1) / TN;
-    const int step0 = p.t0 + 1;
+    const int step0 = RECOUNT ? p.first_step + qoff : p.t0 + 1;     // step of this CTA's first query
+    int *pos_sh = reinterpret_cast<int *>(sm + OFF_P + 4096);       // [3][TN] positions of the key tiles (recount: P is idle)
+    const int32_t *pos_u = p.pos + (size_t)u * p.B;
+    auto load_pos = [&](int buf, int kt) {
+        if (RECOUNT && tid < TN) {
+            const int j = kt * TN + tid;
+            pos_sh[buf * TN + tid] = j < n0 ? pos_u[j] : 0x7fffffff;
+        }
+    };
     const size_t tstride = (size_t)p.Utot * D * 2;       // bytes between consecutive tokens of one unit (fp16 inputs)
     char *Kc = p.K + (size_t)u * p.B * ROWB;
     char *Vc = p.V + (size_t)u * p.B * ROWB;
@@ -186,7 +199,7 @@ __global__ void __launch_bounds__(NT, 1) sh_chunk_umma_int4_kernel(const ChunkPa
         fence_barrier_init();
     }
     // ---- the chunk's tokens: quantise keys and values into the cache (thread = (row, group, K or V)), positions
-    {
+    if (!RECOUNT) {
         const int row = tid >> 2, g = (tid >> 1) & 1, isv = tid & 1;
         if (row < c) {
             const char *src = (isv ? p.v : p.k) + (size_t)row * tstride + (size_t)u * D * 2 + g * 128;
@@ -195,11 +208,19 @@ __global__ void __launch_bounds__(NT, 1) sh_chunk_umma_int4_kernel(const ChunkPa
         }
         if (tid < c) p.pos[(size_t)u * p.B + n0 + tid] = step0 + tid;
     }
-    // ---- queries (rows beyond c are zero), twice: rows 0..63 and 64..127
+    // ---- queries (rows beyond c are zero), twice: rows 0..63 and 64..127; remembered for a later recount
     for (int idx = tid; idx < CQ * 16; idx += NT) {
         const int row = idx >> 4, ch = idx & 15;
         uint4 val = make_uint4(0, 0, 0, 0);
-        if (row < c) val = *reinterpret_cast<const uint4 *>(p.q + (size_t)row * tstride + (size_t)u * D * 2 + ch * 16);
+        if (row < c) {
+            char *ring_row = p.qring ? p.qring + ((size_t)u * p.w + (step0 + row) % p.w) * (D * 2) + ch * 16 : nullptr;
+            if (RECOUNT) {
+                val = *reinterpret_cast<const uint4 *>(ring_row);
+            } else {
+                val = *reinterpret_cast<const uint4 *>(p.q + (size_t)row * tstride + (size_t)u * D * 2 + ch * 16);
+                if (ring_row) *reinterpret_cast<uint4 *>(ring_row) = val;
+            }
+        }
         char *dst = Qs + (row >> 3) * GROUP + ch * 128 + (row & 7) * 16;
         *reinterpret_cast<uint4 *>(dst) = val;
         *reinterpret_cast<uint4 *>(dst + (CQ / 8) * GROUP) = val;
@@ -212,6 +233,8 @@ __global__ void __launch_bounds__(NT, 1) sh_chunk_umma_int4_kernel(const ChunkPa
     auto key_tile = [&](int g) { return g < ntiles ? g : g - ntiles; };
     store_piece(load_piece(Kc, Ksc, 0, n_tot), Kt, ks_sh);
     store_piece(load_piece(Kc, Ksc, key_tile(1) * TN, n_tot), Kt + TILE, ks_sh + TN * 2);
+    load_pos(0, 0);          // positions of tile g sit in buffer g mod 3
+    load_pos(1, key_tile(1));
     if (p.out) store_piece(load_piece(Vc, Vsc, 0, n_tot), Vt, vs_sh);
     fence_async_shared();
     tc_fence_before();
@@ -264,8 +287,17 @@ __global__ void __launch_bounds__(NT, 1) sh_chunk_umma_int4_kernel(const ChunkPa
         tmem_ld16(lane_addr + S_COL + ((g & 1) * 2 + 1) * TN + quarter * HC, s1);
         const float *ksc = ks_sh + (g % 3) * TN * 2 + quarter * HC * 2;
         const int j0 = kt * TN + quarter * HC;
-        const int lim = live_row ? nv - j0 : 0;
-        const uint32_t vm = lim <= 0 ? 0u : (lim >= HC ? 0xffffu : (1u << lim) - 1u);
+        uint32_t vm;
+        if (RECOUNT) {
+            vm = 0;
+            const int *pt = pos_sh + (g % 3) * TN + quarter * HC;
+#pragma unroll
+            for (int jj = 0; jj < HC; ++jj) vm |= (uint32_t)(pt[jj] <= step0 + i) << jj;
+            if (!live_row) vm = 0;
+        } else {
+            const int lim = live_row ? nv - j0 : 0;
+            vm = lim <= 0 ? 0u : (lim >= HC ? 0xffffu : (1u << lim) - 1u);
+        }
         float sv[HC];
 #pragma unroll
         for (int jj = 0; jj < HC; ++jj) sv[jj] = (s0[jj] * ksc[2 * jj] + s1[jj] * ksc[2 * jj + 1]) * p.scale_log2e;
@@ -349,7 +381,10 @@ __global__ void __launch_bounds__(NT, 1) sh_chunk_umma_int4_kernel(const ChunkPa
             }
         }
         // ---- the next tiles go into the buffers that S(g) and the previous P.V have released
-        if (want_k) store_piece(pk, Kt + (g & 1) * TILE, ks_sh + ((g + 2) % 3) * TN * 2);
+        if (want_k) {
+            store_piece(pk, Kt + (g & 1) * TILE, ks_sh + ((g + 2) % 3) * TN * 2);
+            load_pos((g + 2) % 3, key_tile(g + 2));
+        }
         if (want_v) store_piece(pv, Vt + ((kt + 1) & 1) * TILE, vs_sh + ((kt + 1) & 1) * TN * 2);
     }
     if (ok) {
@@ -385,8 +420,16 @@ __global__ void __launch_bounds__(NT, 1) sh_chunk_umma_int4_kernel(const ChunkPa
 
 cudaError_t sh_launch_chunk_umma_int4(const ChunkParams &p, cudaStream_t s) {
     if (p.c < 1 || p.c > CQ) return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(sh_chunk_umma_int4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(sh_chunk_umma_int4_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    sh_chunk_umma_int4_kernel<<<p.U, NT, SMEM_BYTES, s>>>(p);
+    sh_chunk_umma_int4_kernel<false><<<p.U, NT, SMEM_BYTES, s>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t sh_launch_recount_umma_int4(const ChunkParams &p, cudaStream_t s) {
+    if (p.nsteps < 1 || p.out) return cudaErrorInvalidValue;
+    cudaError_t e = cudaFuncSetAttribute(sh_chunk_umma_int4_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    sh_chunk_umma_int4_kernel<true><<<dim3(p.U, (unsigned)((p.nsteps + CQ - 1) / CQ), 1), NT, SMEM_BYTES, s>>>(p);
     return cudaGetLastError();
 }

@@ -351,9 +351,13 @@ __global__ void __launch_bounds__(NW * 32, NW == 4 ? ((DT == SH_F32 && D == 128)
     // ---- q chunk of this lane, fp32
     typename E::Q qv;
     E::load_q(reinterpret_cast<const char *>(p.q) + (size_t)u * INB, c, qv);
-    if (!Q4 && p.qring && warp == 0 && sub == 0 && cr == 0)     // remembered for a recount at compression time
-        st_plain(p.qring + ((size_t)u * p.w + hist_row) * INB + c * 16,
-                 ld_plain(reinterpret_cast<const char *>(p.q) + (size_t)u * INB + c * 16));
+    if (p.qring && warp == 0 && sub == 0 && cr == 0) {           // remembered for a recount at compression time
+        constexpr int QCH = Q4 ? 4 : 1;                          // 16-byte pieces of q per lane (int4: a lane covers 32 elements)
+#pragma unroll
+        for (int k = 0; k < QCH; ++k)
+            st_plain(p.qring + ((size_t)u * p.w + hist_row) * INB + (c * QCH + k) * 16,
+                     ld_plain(reinterpret_cast<const char *>(p.q) + (size_t)u * INB + (c * QCH + k) * 16));
+    }
 
     const char *Kb = p.K + (size_t)u * B * ROWB;
     const char *Vb = p.V + (size_t)u * B * ROWB;

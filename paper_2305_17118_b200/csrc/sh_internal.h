@@ -166,6 +166,7 @@ cudaError_t sh_launch_chunk_umma(const ChunkParams &p, int dtype, cudaStream_t s
 cudaError_t sh_launch_recount_umma(const ChunkParams &p, int dtype, cudaStream_t s);
 // int4-g64 store: the chunked prompt step with codes unpacked into the tensor-core tiles (sh_chunk_umma_int4.cu).
 cudaError_t sh_launch_chunk_umma_int4(const ChunkParams &p, cudaStream_t s);
+cudaError_t sh_launch_recount_umma_int4(const ChunkParams &p, cudaStream_t s);
 
 // Launchers (each returns the cudaError_t of its launch and adds to *launches).
 cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches);

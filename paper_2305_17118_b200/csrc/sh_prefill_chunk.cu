@@ -348,7 +348,9 @@ int sh_prefill_chunk_capacity(const sh_context *c) {
 // The recount (record recomputed at compression time): any budget on the tcgen05 kernel; the warp-level
 // kernel keeps a whole row of logits in shared memory (budgets up to about 700).
 bool sh_recount_supported(const sh_context *c) {
-    if ((c->dtype != SH_F16 && c->dtype != SH_BF16) || c->D != 128) return false;
+    if (c->D != 128) return false;
+    if (c->dtype == SH_INT4_G64_F16) return c->prefill_chunk != 2;      // int4 store: the tcgen05 kernel only
+    if (c->dtype != SH_F16 && c->dtype != SH_BF16) return false;
     return c->prefill_chunk != 2 || smem_need(32, c->B) <= 200 * 1024;
 }
 
@@ -407,7 +409,13 @@ cudaError_t sh_launch_recount(const sh_context *c, cudaStream_t s, long long *la
     p.first_step = (int)c->t - p.nsteps + 1;
     if (p.nsteps < 1) return cudaSuccess;
     p.err = reinterpret_cast<int *>(c->slab + c->L.err);
+    p.Ks = sh_pKs(c); p.Vs = sh_pVs(c); p.Bs = c->Bs;
     cudaError_t e;
+    if (c->dtype == SH_INT4_G64_F16) {
+        e = sh_launch_recount_umma_int4(p, s);
+        if (e == cudaSuccess) *launches += 1;
+        return e;
+    }
     if (c->prefill_chunk != 2) {
         e = sh_launch_recount_umma(p, c->dtype, s);
         if (e == cudaSuccess) *launches += 1;

@@ -214,7 +214,7 @@ def run_lockstep_recompute(handle, cfg_dtype: str, inputs, steps: int, units, to
     units = torch.as_tensor(units, dtype=torch.long)
     un = units.numpy()
     if orc is None:
-        orc = oracle_mod.Oracle(len(un), handle.B, handle.r, handle.w, handle.m, handle.D)
+        orc = oracle_mod.Oracle(len(un), handle.B, handle.r, handle.w, handle.m, handle.D, quant=(cfg_dtype == "int4"))
     res = res or LockstepResult()
     dev_units = units.to(handle.device)
     w = handle.w

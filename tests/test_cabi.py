@@ -79,12 +79,14 @@ def test_option_values_and_the_shapes_they_need():
         assert lib.sh_prefill_chunk_max(h) == 0
         assert lib.sh_set_option(h, sh.SH_OPT_RECORD_MODE, 1.0) == sh.SH_EINVAL
         lib.sh_destroy(h)
-    # the int4 store with head_dim 128 has a chunk kernel (tcgen05 only) but no recompute mode
+    # the int4 store with head_dim 128 has a chunk kernel and a recompute mode, on the tcgen05 kernel only
     h = _handle(sh, 150, 9, 37, 41, 3, 128, "int4")
     assert lib.sh_prefill_chunk_max(h) == 37
-    assert lib.sh_set_option(h, sh.SH_OPT_RECORD_MODE, 1.0) == sh.SH_EINVAL
     assert lib.sh_set_option(h, sh.SH_OPT_PREFILL_CHUNK, 2.0) == sh.SH_OK
     assert lib.sh_prefill_chunk_max(h) == 0
+    assert lib.sh_set_option(h, sh.SH_OPT_RECORD_MODE, 1.0) == sh.SH_EINVAL
+    assert lib.sh_set_option(h, sh.SH_OPT_PREFILL_CHUNK, 1.0) == sh.SH_OK
+    assert lib.sh_set_option(h, sh.SH_OPT_RECORD_MODE, 1.0) == sh.SH_OK
     lib.sh_destroy(h)
     # the warp-level chunk kernel keeps a row of logits in shared memory: it stops at budgets of about 700,
     # the tcgen05 kernel does not; the recompute mode follows the kernel that is chosen

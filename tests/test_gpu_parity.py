@@ -147,6 +147,20 @@ def test_lockstep_record_recomputed_at_compression(sh, dtype, U, B, r, w, m, chu
     assert res.adoptions <= 1e-4 * res.slot_steps + 2
 
 
+@pytest.mark.parametrize("U,B,r,w,m", [(5, 150, 9, 37, 41), (3, 410, 64, 128, 64), (140, 96, 8, 70, 30)])
+@pytest.mark.parametrize("unordered", [False, True])
+def test_lockstep_record_recomputed_int4_store(sh, U, B, r, w, m, unordered):
+    """SH_OPT_RECORD_MODE = 1 on the int4 store: the decode kernel keeps the ring of queries, the int4 chunk
+    kernel recounts against the quantised cache (w beyond 64: two CTAs per unit)."""
+    dtype, d, T = "int4", 128, min(2 * B + 3 * m + 5, B + 2 * m + 30)
+    q, k, v = wl.random_stream(U, d, T, seed=43 + U, dtype=dtype, peaked=3.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, recompute_record=True, unordered=unordered)
+    h = SortedView(h) if unordered else h
+    res, orc = run_lockstep_recompute(h, dtype, _stream_fn(q, k, v), T, torch.arange(U), TOL[dtype])
+    assert res.compressions >= 3
+    assert res.adoptions <= 1e-4 * res.slot_steps + 2
+
+
 def test_recompute_mode_through_prefill_and_automatic_compression(sh):
     """Same mode driven the way an application would: chunked sh_prefill, then decode steps with
     automatic compression; compared with the oracle running the same variant on its own."""
