@@ -92,11 +92,11 @@ def to_oracle(x: torch.Tensor, units) -> np.ndarray:
 
 
 def run_lockstep(handle, cfg_dtype: str, inputs, steps: int, units, tol: float, state_every: int = 1,
-                 res: LockstepResult = None, orc=None):
+                 res: LockstepResult = None, orc=None, outs=None):
     """``inputs(t)`` -> (q, k, v) CUDA tensors [U, d] for 1-based step t.
     ``units``: LongTensor of unit indices checked against the oracle.
-    The handle must have been created with auto_compress=False.
-    Returns (LockstepResult, oracle)."""
+    The handle must have been created with auto_compress=False.  ``outs``: a list that receives every
+    step's output tensor [U, d].  Returns (LockstepResult, oracle)."""
     units = torch.as_tensor(units, dtype=torch.long)
     un = units.numpy()
     if orc is None:
@@ -108,6 +108,8 @@ def run_lockstep(handle, cfg_dtype: str, inputs, steps: int, units, tol: float, 
         t = orc.t + 1
         q, k, v = inputs(t)
         out = handle.decode_step(q, k, v)
+        if outs is not None:
+            outs.append(out)
         want_state = (t % state_every == 0) or (orc.n + 1 == handle.B)
         n, tt, pos, cnt, low = handle.state(pos=want_state, counters=want_state, low=True)
         o_out, alpha, o_low, amb = orc.attend(to_oracle(q, dev_units), to_oracle(k, dev_units),
@@ -142,14 +144,21 @@ def run_lockstep(handle, cfg_dtype: str, inputs, steps: int, units, tol: float, 
 
 
 def run_lockstep_chunked(handle, cfg_dtype: str, inputs_block, steps: int, units, tol: float, chunk_sizes=None,
-                         res: LockstepResult = None, orc=None):
+                         res: LockstepResult = None, orc=None, recompute: bool = False, outs=None,
+                         single_via_step: bool = False):
     """Same protocol as run_lockstep, driving the library through sh_prefill_chunk.
 
     ``inputs_block(t0, t1)`` -> (q, k, v) CUDA tensors [t1-t0, U, d] for stream positions t0 .. t1-1
     (1-based).  The library evaluates a whole chunk in one launch; the oracle then replays the chunk
     step by step, and each step's record bits are read back from the unit's bit-planes (no
     compression happens inside a chunk, so nothing has moved them).  ``chunk_sizes`` cycles through
-    requested chunk lengths (clipped to what the library and the remaining budget allow)."""
+    requested chunk lengths (clipped to what the library and the remaining budget allow).  With
+    ``single_via_step`` a chunk of one token goes through sh_decode_step, as sh_prefill does it: with the
+    default sizes the sequence of launches is then exactly sh_prefill's, so a second handle fed through
+    sh_prefill must end bit-identical to this one.
+    ``recompute``: the handle runs SH_OPT_RECORD_MODE = 1; at each compression the library's recomputed
+    bit-planes are compared with the oracle's recount (adoption inside the window) before both compress.
+    ``outs``: a list that receives each chunk's output tensor [cnt, U, d]."""
     units = torch.as_tensor(units, dtype=torch.long)
     un = units.numpy()
     if orc is None:
@@ -167,7 +176,12 @@ def run_lockstep_chunked(handle, cfg_dtype: str, inputs_block, steps: int, units
         t0 = orc.t + 1
         q, k, v = inputs_block(t0, t0 + cnt)
         out = torch.empty(cnt, handle.U, handle.D, device=handle.device)
-        handle.prefill_chunk(q, k, v, out)
+        if cnt == 1 and single_via_step:
+            handle.decode_step(q[0], k[0], v[0], out[0])
+        else:
+            handle.prefill_chunk(q, k, v, out)
+        if outs is not None:
+            outs.append(out)
         n, tt, pos, cnt_rec, _ = handle.state(low=False)
         planes = [handle.export_record(int(u)) for u in un]      # [w, B] bool per sampled unit
         for i in range(cnt):
@@ -193,6 +207,8 @@ def run_lockstep_chunked(handle, cfg_dtype: str, inputs_block, steps: int, units
         assert (pos[un] == orc.positions()).all(), f"after step {orc.t}: positions differ"
         assert (cnt_rec[un].astype(np.int32) == orc.counters()).all(), f"after step {orc.t}: records differ"
         if orc.full:
+            if recompute:
+                _adopt_recount(handle, orc, un, res)
             orc.compress()
             assert handle.compress() == handle.m
             n2, _, pos2, cnt2, _ = handle.state(low=False)
@@ -202,6 +218,28 @@ def run_lockstep_chunked(handle, cfg_dtype: str, inputs_block, steps: int, units
             res.compressions += 1
         done += cnt
     return res, orc
+
+
+def _adopt_recount(handle, orc, un, res):
+    """SH_OPT_RECORD_MODE = 1 at a full cache: the library recomputes its bit-planes, the oracle recounts
+    from its own stored queries; bits may differ only inside the 1e-6 window, where the oracle takes the
+    library's; the counters must then be identical."""
+    t = orc.t
+    handle.recompute_record()
+    nn = orc.n
+    g = np.stack([handle.export_record(int(u))[:, :nn] for u in un])          # [units, w, n]
+    _a, o_low, amb, steps_in = orc.recount()
+    live_rows = steps_in > 0
+    assert not g[:, ~live_rows].any(), "bits in rows of steps outside the window"
+    diff = g != o_low
+    bad = diff & ~amb
+    assert not bad.any(), (f"step {t}: {int(bad.sum())} recomputed bits differ outside the 1e-6 window; "
+                           f"first at (unit, row, slot) {np.argwhere(bad)[0].tolist()}")
+    res.adoptions += int(diff.sum())
+    res.slot_steps += int(live_rows.sum()) * nn * len(un)
+    orc.set_record(g, steps_in)
+    _n1, _, _pos1, cnt1, _ = handle.state(low=False)
+    assert (cnt1[un].astype(np.int32) == orc.counters()).all(), f"step {t}: recomputed records differ"
 
 
 def run_lockstep_recompute(handle, cfg_dtype: str, inputs, steps: int, units, tol: float, res: LockstepResult = None,
@@ -228,21 +266,7 @@ def run_lockstep_recompute(handle, cfg_dtype: str, inputs, steps: int, units, to
         res.max_abs_err = max(res.max_abs_err, err)
         assert err <= tol, f"step {t}: attention output off by {err:.3e} > {tol}"
         if orc.full:
-            handle.recompute_record()
-            nn = orc.n
-            g = np.stack([handle.export_record(int(u))[:, :nn] for u in un])          # [units, w, n]
-            _a, o_low, amb, steps_in = orc.recount()
-            live_rows = steps_in > 0
-            assert not g[:, ~live_rows].any(), "bits in rows of steps outside the window"
-            diff = g != o_low
-            bad = diff & ~amb
-            assert not bad.any(), (f"step {t}: {int(bad.sum())} recomputed bits differ outside the 1e-6 window; "
-                                   f"first at (unit, row, slot) {np.argwhere(bad)[0].tolist()}")
-            res.adoptions += int(diff.sum())
-            res.slot_steps += int(live_rows.sum()) * nn * len(un)
-            orc.set_record(g, steps_in)
-            n1, _, pos1, cnt1, _ = handle.state(low=False)
-            assert (cnt1[un].astype(np.int32) == orc.counters()).all(), f"step {t}: recomputed records differ"
+            _adopt_recount(handle, orc, un, res)
             orc.compress()
             assert handle.compress() == handle.m
             n2, _, pos2, cnt2, _ = handle.state(low=False)
@@ -251,3 +275,18 @@ def run_lockstep_recompute(handle, cfg_dtype: str, inputs, steps: int, units, to
             res.compressions += 1
         res.steps += 1
     return res, orc
+
+
+
+
+def assert_same_state(a, b, rows: bool = True):
+    """Two handles of the library hold bit-identical state: counters, positions, record, this step's
+    bits and (``rows``) every byte of the workspace's K and V regions."""
+    sa, sb = a.state(), b.state()
+    assert sa[0] == sb[0] and sa[1] == sb[1], "n or t differ"
+    for name, x, y in zip(("positions", "counters", "last bits"), sa[2:], sb[2:]):
+        assert (x == y).all(), f"{name} differ"
+    if rows:
+        row_bytes = {0: 4 * a.D, 1: 2 * a.D, 2: 2 * a.D, 3: a.D // 2}[a.dtype]
+        kv = 2 * ((a.U * a.B * row_bytes + 255) // 256 * 256)            # the K region, then the V region
+        assert torch.equal(a.slab[a._slab_off:a._slab_off + kv], b.slab[b._slab_off:b._slab_off + kv]), "K/V rows differ"

@@ -6,7 +6,8 @@ import pytest
 import torch
 
 import oracle
-from lockstep import SortedView, run_lockstep, run_lockstep_chunked, run_lockstep_recompute, to_oracle
+from lockstep import (SortedView, assert_same_state, run_lockstep, run_lockstep_chunked, run_lockstep_recompute,
+                      to_oracle)
 from paper_2305_17118_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -48,10 +49,12 @@ def test_lockstep_edge_parameters(sh, B, r, w, m):
     assert res.compressions >= 1
 
 
-@pytest.mark.parametrize("dtype,d", [("f32", 64), ("f32", 128), ("f16", 64), ("bf16", 64), ("int4", 128), ("int4", 64)])
+@pytest.mark.parametrize("dtype,d", [("f32", 64), ("f32", 128), ("f16", 64), ("bf16", 64), ("f16", 128), ("bf16", 128),
+                                      ("int4", 128), ("int4", 64)])
 def test_lockstep_direct_kernel_many_units(sh, dtype, d):
     """The direct-load decode kernel in the CTA shape it takes from 592 units on (4 warps, more rows per
-    thread), every storage type it serves there; a sample of units in lockstep."""
+    thread), every storage type and head size, i.e. every instance the launcher can pick; a sample of
+    units in lockstep."""
     U, B, r, w, m, T = 601, 77, 6, 21, 30, 150
     q, k, v = wl.random_stream(U, d, T, seed=13, dtype=dtype, peaked=3.0, device="cuda")
     h = sh.Handle(B, r, w, m, U, d, dtype, kernel=1, auto_compress=False)
@@ -163,25 +166,26 @@ def test_lockstep_record_recomputed_int4_store(sh, U, B, r, w, m, unordered):
 
 def test_recompute_mode_through_prefill_and_automatic_compression(sh):
     """Same mode driven the way an application would: chunked sh_prefill, then decode steps with
-    automatic compression; compared with the oracle running the same variant on its own."""
+    automatic compression.  The library decides on its own here, so its per-step bits cannot be handed
+    to the oracle; instead a twin handle is driven through the same launches by hand (chunks, then
+    steps, explicit recount and compression) in lockstep with the oracle, and the free-running handle
+    must end bit-identical to the twin, outputs included."""
     U, d, B, r, w, m, P, T, dtype = 12, 128, 120, 8, 50, 40, 300, 420, "f16"
     q, k, v = wl.random_stream(U, d, T, seed=31, dtype=dtype, peaked=3.0, device="cuda")
     h = sh.Handle(B, r, w, m, U, d, dtype, recompute_record=True)
-    orc = oracle.Oracle(U, B, r, w, m, d)
-    idx = torch.arange(U, device="cuda")
     outs = torch.empty(T, U, d, device="cuda")
     h.prefill(q[:P].contiguous(), k[:P].contiguous(), v[:P].contiguous(), outs[:P])
     for t in range(P, T):
         h.decode_step(q[t], k[t], v[t], outs[t])
-    worst = 0.0
-    for t in range(T):
-        o, _ = orc.step_recompute(to_oracle(q[t], idx), to_oracle(k[t], idx), to_oracle(v[t], idx))
-        worst = max(worst, float(np.abs(outs[t].double().cpu().numpy() - o).max()))
-    n, tt, pos, cnt, _ = h.state(low=False)
-    assert n == orc.n and tt == orc.t
-    same = (pos == orc.positions()).all(axis=1)
-    assert same.mean() >= 0.75          # units without a threshold-ambiguous flip agree exactly
-    assert worst <= TOL[dtype] or same.mean() < 1.0
+    twin = sh.Handle(B, r, w, m, U, d, dtype, recompute_record=True, auto_compress=False)
+    blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
+    t_outs = []
+    res, orc = run_lockstep_chunked(twin, dtype, blk, P, torch.arange(U), TOL[dtype], recompute=True, outs=t_outs,
+                                    single_via_step=True)
+    res2, _ = run_lockstep_recompute(twin, dtype, _stream_fn(q, k, v), T - P, torch.arange(U), TOL[dtype], orc=orc)
+    assert res.compressions + res2.compressions >= 7
+    assert torch.equal(outs[:P], torch.cat(t_outs))
+    assert_same_state(h, twin)
 
 
 def test_paper_hyperparameters_chunked_prompt_then_decode(sh):
@@ -199,27 +203,26 @@ def test_paper_hyperparameters_chunked_prompt_then_decode(sh):
 
 
 def test_prefill_uses_chunks_and_matches_oracle(sh):
-    """sh_prefill with its automatic chunking on the OPT-6.7B-shaped stream, then decode steps in lockstep."""
+    """sh_prefill with its automatic chunking and compression on the OPT-6.7B-shaped stream.  A twin handle
+    is driven through the same sequence of launches by hand, in lockstep with the oracle (every output,
+    record bit, counter and kept set, with adoption inside the 1e-6 window); the handle that went
+    through sh_prefill must be bit-identical to the twin.  Then decode steps in lockstep."""
     cfg = wl.CONFIGS["opt6b"].scaled(units=24, prompt=700)
     st = wl.Stream(cfg, device="cuda")
     h = sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, cfg.units, cfg.head_dim, cfg.dtype, auto_compress=False)
-    orc = oracle.Oracle(cfg.units, cfg.B, cfg.r, cfg.w, cfg.m, cfg.head_dim)
     q, k, v = st.block(1, cfg.prompt + 1)
     out = torch.empty(cfg.prompt, cfg.units, cfg.head_dim, device="cuda")
     before = h.launch_count
     h.prefill(q, k, v, out)
     assert h.launch_count - before < cfg.prompt // 8        # chunks, not one launch per token
-    idx = torch.arange(cfg.units, device="cuda")
-    worst = 0.0
-    for t in range(cfg.prompt):
-        o, _ = orc.step(to_oracle(q[t], idx), to_oracle(k[t], idx), to_oracle(v[t], idx))
-        worst = max(worst, float(np.abs(out[t].double().cpu().numpy() - o).max()))
-    assert worst <= TOL[cfg.dtype]
-    n, t, pos, cnt, _ = h.state(low=False)
-    assert n == orc.n and t == orc.t
-    same = (pos == orc.positions()).all(axis=1)
-    assert same.mean() >= 0.9      # units without a threshold-ambiguous flip must agree exactly
-    assert (cnt[same].astype(np.int32) == orc.counters()[same]).all()
+    twin = sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, cfg.units, cfg.head_dim, cfg.dtype, auto_compress=False)
+    t_outs = []
+    res, orc = run_lockstep_chunked(twin, cfg.dtype, lambda t0, t1: (q[t0 - 1:t1 - 1], k[t0 - 1:t1 - 1], v[t0 - 1:t1 - 1]),
+                                    cfg.prompt, torch.arange(cfg.units), TOL[cfg.dtype], outs=t_outs, single_via_step=True)
+    assert res.compressions == 5
+    assert torch.equal(out, torch.cat(t_outs))
+    assert_same_state(h, twin)
+    run_lockstep(h, cfg.dtype, st.step, 70, torch.arange(cfg.units), TOL[cfg.dtype], orc=orc)
 
 
 # ---- the benchmark's own configurations ----------------------------------------------------
@@ -277,8 +280,11 @@ def test_config_opt66b_full_size_chunked_prompt_sampled_units(sh):
     run_lockstep(h, cfg.dtype, st.step, 30, units, TOL[cfg.dtype], orc=orc)
 
 
-@pytest.mark.parametrize("layer", [0, 39])
+@pytest.mark.parametrize("layer", [0, 13, 26, 39])
 def test_config_opt13b_layer_sampled_units(sh, layer):
+    """One layer's handle of the 40-layer workload at full size (1280 units per launch, the launch the
+    benchmark times), 16 sampled units in lockstep through prompt and decode.  Layers differ only in the
+    seed of their input stream and each has a handle of its own, so four of them sample the forty."""
     cfg = wl.CONFIGS["opt13b"]
     st = wl.Stream(cfg, device="cuda", layer=layer)
     units = wl.sample_units(cfg, 16)
@@ -317,25 +323,24 @@ def test_select_kernel_bit_exact_on_oracle_records(sh, n, r, m):
 
 @pytest.mark.parametrize("dtype", ["f32", "f16", "bf16", "int4"])
 def test_compaction_moves_rows_bit_identically(sh, dtype):
+    """Stored key and value rows after several compressions equal the oracle's bit for bit, on a handle in
+    lockstep with the oracle; and a second handle that compresses by itself (SH_OPT_AUTO_COMPRESS, the
+    default) ends bit-identical to the first, outputs included."""
     U, d, B, r, w, m, T = 4, 128, 96, 8, 20, 40, 200
     q, k, v = wl.random_stream(U, d, T, seed=3, dtype=dtype, peaked=3.0, device="cuda")
-    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=True)
-    orc = oracle.Oracle(U, B, r, w, m, d, quant=(dtype == "int4"))
-    idx = torch.arange(U, device="cuda")
-    for t in range(T):
-        h.decode_step(q[t], k[t], v[t])
-        out, alpha, low, amb = orc.attend(to_oracle(q[t], idx), to_oracle(k[t], idx), to_oracle(v[t], idx))
-        n, _, pos, cnt, glow = h.state()
-        # bits may have been compacted already by the automatic compression: compare through positions
-        orc.record(low)
-        orc.compress()
-        if (pos != orc.positions()).any():
-            pytest.skip("a threshold-ambiguous bit changed the kept set; covered by the lockstep tests")
+    auto = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=True)
+    outs = torch.stack([auto.decode_step(q[t], k[t], v[t]) for t in range(T)])
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    twin_outs = []
+    res, orc = run_lockstep(h, dtype, _stream_fn(q, k, v), T, torch.arange(U), TOL[dtype], outs=twin_outs)
+    assert res.compressions >= 3
     n = h.n
     for u in range(U):
         K, V = h.export_unit(u)
         oK, oV = orc.cache(u)
         assert (K[:n].astype(np.float64) == oK).all() and (V[:n].astype(np.float64) == oV).all()
+    assert torch.equal(outs, torch.stack(twin_outs))
+    assert_same_state(auto, h)
 
 
 # ---- SH_OPT_COMPACTION = 1: holes filled from the tail, slots in no particular order -------------
@@ -462,44 +467,61 @@ def test_snapshot_restore_replays_identically(sh):
     assert s1[0] == s2[0] and s1[1] == s2[1] and all((x == y).all() for x, y in zip(s1[2:], s2[2:]))
 
 
-@pytest.mark.parametrize("dtype,kernel,unordered", [("f16", None, False), ("bf16", 2, False), ("f16", 1, False),
-                                                    ("f32", None, False), ("f16", None, True), ("bf16", 2, True)])
-def test_ragged_sequences_lockstep(sh, dtype, kernel, unordered):
+def _ragged_lockstep(sh, dtype, d, lengths, ups, B, r, w, m, T_dec, kernel, unordered, split, seed):
     """Sequences of different prompt lengths in one handle (sh_prefill_ragged), then decode steps in
-    lockstep: one oracle per sequence, each with its own n, t and compression schedule."""
-    d = 128 if dtype != "f32" else 64
-    lengths = [0, 37, 150, 96, 211, 95]            # empty, short, several compressions, exactly full, long, one short of full
-    nseq, ups, B, r, w, m, T_dec = len(lengths), 3, 96, 8, 40, 30, 170
+    lockstep: one oracle per sequence, each with its own n, t and compression schedule.  Returns the
+    number of steps at which some sequence compressed."""
+    nseq = len(lengths)
     U, p_max = nseq * ups, max(lengths)
-    q, k, v = wl.random_stream(U, d, p_max + T_dec, seed=51, dtype=dtype, peaked=3.0, device="cuda")
-    h = SortedView(sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, kernel=kernel, unordered=unordered))
+    q, k, v = wl.random_stream(U, d, p_max + T_dec, seed=seed, dtype=dtype, peaked=3.0, device="cuda")
+    kw = dict(auto_compress=False, kernel=kernel, unordered=unordered, split=split)
+    raw = sh.Handle(B, r, w, m, U, d, dtype, **kw)
+    h = SortedView(raw)
     out_p = torch.zeros(p_max, U, d, device="cuda")
     h.prefill_ragged(q[:p_max].contiguous(), k[:p_max].contiguous(), v[:p_max].contiguous(), lengths, out_p)
-    orcs, ok = [], []
+    # The prompt of each sequence once more, on a handle of its own that is driven through the same launches
+    # by hand in lockstep with an oracle (adoption inside the 1e-6 window); the ragged handle's units of that
+    # sequence must then hold bit-identical state, which ties every one of them to the oracle.
+    orcs = []
+    pos_r, cnt_r, low_r = raw.state_full()
+    quant = dtype == "int4"
     for sq in range(nseq):
-        o = oracle.Oracle(ups, B, r, w, m, d)
-        idx = torch.arange(sq * ups, (sq + 1) * ups, device="cuda")
-        for t in range(lengths[sq]):
-            oo, _ = o.step(to_oracle(q[t], idx), to_oracle(k[t], idx), to_oracle(v[t], idx))
-            assert np.abs(out_p[t][idx].double().cpu().numpy() - oo).max() <= TOL[dtype]
+        sl = slice(sq * ups, (sq + 1) * ups)
+        twin_raw = sh.Handle(B, r, w, m, ups, d, dtype, **kw)
+        twin = SortedView(twin_raw)
+        qs, ks, vs = (x[:, sl].contiguous() for x in (q, k, v))
+        t_outs = []
+        if lengths[sq] == 0:
+            o = oracle.Oracle(ups, B, r, w, m, d, quant=quant)
+        elif twin_raw.prefill_chunk_max >= 2:
+            blk = lambda t0, t1: (qs[t0 - 1:t1 - 1].contiguous(), ks[t0 - 1:t1 - 1].contiguous(), vs[t0 - 1:t1 - 1].contiguous())
+            _, o = run_lockstep_chunked(twin, dtype, blk, lengths[sq], torch.arange(ups), TOL[dtype], outs=t_outs,
+                                        single_via_step=True)
+        else:
+            _, o = run_lockstep(twin, dtype, _stream_fn(qs, ks, vs), lengths[sq], torch.arange(ups), TOL[dtype], outs=t_outs)
+            t_outs = [x[None] for x in t_outs]
+        if lengths[sq]:
+            assert torch.equal(out_p[: lengths[sq], sl], torch.cat(t_outs))
+        pos_t, cnt_t, low_t = twin_raw.state_full()
+        assert (pos_r[sl] == pos_t).all() and (cnt_r[sl] == cnt_t).all() and (low_r[sl] == low_t).all()
+        for j in sorted(set(range(0, ups, 37)) | {ups - 1}):
+            Kr, Vr = raw.export_unit(sq * ups + j)
+            Kt, Vt = twin_raw.export_unit(j)
+            assert (Kr[: o.n] == Kt[: o.n]).all() and (Vr[: o.n] == Vt[: o.n]).all()
         orcs.append(o)
     n_seq, t_seq = h.sequence_state()
-    assert n_seq.tolist() == [o.n for o in orcs] and t_seq.tolist() == lengths
+    assert n_seq.tolist() == [o.n for o in orcs] and t_seq.tolist() == list(lengths)
     pos, cnt, _ = h.state_full()
     for sq, o in enumerate(orcs):
         sl = slice(sq * ups, (sq + 1) * ups)
-        same = (pos[sl, : o.n] == o.positions()).all() and (cnt[sl, : o.n].astype(np.int32) == o.counters()).all()
-        ok.append(bool(same))                     # a threshold-ambiguous flip in the prompt may change a kept set
+        assert (pos[sl, : o.n] == o.positions()).all() and (cnt[sl, : o.n].astype(np.int32) == o.counters()).all()
         assert (pos[sl, o.n:] == 0).all()
-    assert sum(ok) >= nseq - 1
     compressions = 0
     for step in range(T_dec):
         ti = p_max + step
         out = h.decode_step(q[ti], k[ti], v[ti])
         pos, cnt, low = h.state_full()
         for sq, o in enumerate(orcs):
-            if not ok[sq]:
-                continue
             idx = torch.arange(sq * ups, (sq + 1) * ups, device="cuda")
             sl = slice(sq * ups, (sq + 1) * ups)
             oo, alpha, o_low, amb = o.attend(to_oracle(q[ti], idx), to_oracle(k[ti], idx), to_oracle(v[ti], idx))
@@ -517,8 +539,6 @@ def test_ragged_sequences_lockstep(sh, dtype, kernel, unordered):
             compressions += 1
             pos, cnt, _ = h.state_full()
             for sq in due:
-                if not ok[sq]:
-                    continue
                 o = orcs[sq]
                 assert o.full
                 o.compress()
@@ -526,42 +546,28 @@ def test_ragged_sequences_lockstep(sh, dtype, kernel, unordered):
                 assert (pos[sl, : o.n] == o.positions()).all() and (pos[sl, o.n:] == 0).all()
                 assert (cnt[sl, : o.n].astype(np.int32) == o.counters()).all()
         n_seq, t_seq = h.sequence_state()
-        assert all(n_seq[sq] == orcs[sq].n for sq in range(nseq) if ok[sq])
+        assert all(n_seq[sq] == orcs[sq].n for sq in range(nseq))
         assert t_seq.tolist() == [lengths[sq] + step + 1 for sq in range(nseq)]
+    return compressions
+
+
+@pytest.mark.parametrize("dtype,kernel,unordered", [("f16", None, False), ("bf16", 2, False), ("f16", 1, False),
+                                                    ("f32", None, False), ("f16", None, True), ("bf16", 2, True)])
+def test_ragged_sequences_lockstep(sh, dtype, kernel, unordered):
+    d = 128 if dtype != "f32" else 64
+    lengths = [0, 37, 150, 96, 211, 95]            # empty, short, several compressions, exactly full, long, one short of full
+    compressions = _ragged_lockstep(sh, dtype, d, lengths, ups=3, B=96, r=8, w=40, m=30, T_dec=170, kernel=kernel,
+                                    unordered=unordered, split=2, seed=51)
     assert compressions >= 12                    # the sequences fill at different steps
 
 
 @pytest.mark.parametrize("dtype", ["f16", "int4"])
 def test_ragged_sequences_many_units(sh, dtype):
     """Ragged sequences on the many-units shape of the direct decode kernel (600 units: per-unit row counts
-    read and advanced on the device by 4-warp CTAs), every unit in lockstep, automatic compression."""
-    d, lengths, ups, B, r, w, m, T_dec = 128, [3, 41], 300, 48, 4, 12, 16, 40
-    U, p_max = len(lengths) * ups, max(lengths)
-    q, k, v = wl.random_stream(U, d, p_max + T_dec, seed=57, dtype=dtype, peaked=3.0, device="cuda")
-    h = sh.Handle(B, r, w, m, U, d, dtype, kernel=1)
-    h.prefill_ragged(q[:p_max].contiguous(), k[:p_max].contiguous(), v[:p_max].contiguous(), lengths)
-    orcs = []
-    for sq, L in enumerate(lengths):
-        o = oracle.Oracle(ups, B, r, w, m, d, quant=(dtype == "int4"))
-        idx = torch.arange(sq * ups, (sq + 1) * ups, device="cuda")
-        for t in range(L):
-            o.step(to_oracle(q[t], idx), to_oracle(k[t], idx), to_oracle(v[t], idx))
-        orcs.append(o)
-    worst, agree = 0.0, []
-    for step in range(T_dec):
-        ti = p_max + step
-        out = h.decode_step(q[ti], k[ti], v[ti])
-        for sq, o in enumerate(orcs):
-            idx = torch.arange(sq * ups, (sq + 1) * ups, device="cuda")
-            oo, _ = o.step(to_oracle(q[ti], idx), to_oracle(k[ti], idx), to_oracle(v[ti], idx))
-            err = np.abs(out[idx].double().cpu().numpy() - oo).max(axis=1)
-            pos = h.state_full()[0][sq * ups:(sq + 1) * ups, : o.n]
-            same = (pos == o.positions()).all(axis=1)          # a threshold-ambiguous flip may change a unit's kept set
-            worst = max(worst, float(err[same].max()))
-            agree.append(same.mean())
-    n_seq, t_seq = h.sequence_state()
-    assert n_seq.tolist() == [o.n for o in orcs] and t_seq.tolist() == [L + T_dec for L in lengths]
-    assert worst <= TOL[dtype] and min(agree) >= 0.97
+    read and advanced on the device by 4-warp CTAs), every unit in lockstep."""
+    compressions = _ragged_lockstep(sh, dtype, 128, [3, 41], ups=300, B=48, r=4, w=12, m=16, T_dec=40, kernel=1,
+                                    unordered=False, split=None, seed=57)
+    assert compressions >= 3
 
 
 def test_persistence_diagnostics_match_oracle_scores(sh):
@@ -664,19 +670,21 @@ def test_scores_on_ragged_sequences_and_after_restore(sh):
 
 def test_score_change_ratio_diagnostic(sh):
     """(alpha_s - alpha_o) / alpha_o of the last step's query, budgeted cache against full cache, from
-    the library; the same from two oracles' caches with the softmax written out here.  Units whose
-    kept set differs from the oracle's (a threshold-ambiguous flip on the way) are left out."""
+    the library; the same from two oracles' caches with the softmax written out here.  The budgeted
+    oracle is brought along in lockstep with a twin handle fed through the same launches as the
+    diagnostic's own (adoption inside the 1e-6 window), so every unit is compared."""
     from paper_2305_17118_b200 import diagnostics
     U, d, B, r, w, m, t, dtype = 8, 128, 64, 6, 24, 20, 173, "f16"
     q, k, v = wl.random_stream(U, d, t, seed=87, dtype=dtype, peaked=3.0, device="cuda")
     got = diagnostics.score_change_ratio(q, k, v, dtype, B, r, w, m)
-    o_s, o_o = oracle.Oracle(U, B, r, w, m, d), oracle.Oracle(U, t + 1, 0, 1, 1, d)
+    twin = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
+    _, o_s = run_lockstep_chunked(twin, dtype, blk, t, torch.arange(U), TOL[dtype], single_via_step=True)
+    o_o = oracle.Oracle(U, t + 1, 0, 1, 1, d)
     idx = torch.arange(U, device="cuda")
     for s in range(t):
-        for o in (o_s, o_o):
-            o.step(to_oracle(q[s], idx), to_oracle(k[s], idx), to_oracle(v[s], idx))
+        o_o.step(to_oracle(q[s], idx), to_oracle(k[s], idx), to_oracle(v[s], idx))
     qf = to_oracle(q[t - 1], idx)
-    checked = 0
     for u in range(U):
         def scores(o):
             K, _ = o.cache(u)
@@ -684,15 +692,12 @@ def test_score_change_ratio_diagnostic(sh):
             e = np.exp(z - z.max())
             return e / e.sum()
         pos_s = o_s.positions()[u]
-        if got.kept[u].sum() != len(pos_s) or not got.kept[u][pos_s - 1].all():
-            continue
+        assert got.kept[u].sum() == len(pos_s) and got.kept[u][pos_s - 1].all()
         want = np.full(t, -1.0)
         a_o = scores(o_o)
         want[pos_s - 1] = (scores(o_s) - a_o[pos_s - 1]) / a_o[pos_s - 1]
         assert np.abs(got.ratio[u] - want).max() <= 2e-4
         assert (got.ratio[u][~got.kept[u]] == -1).all() and (got.ratio[u][got.kept[u]] >= -1e-4).all()
-        checked += 1
-    assert checked >= U - 2
 
 
 @pytest.mark.parametrize("B,w,m", [(8192, 48, 4096), (2048, 16384, 1024)])

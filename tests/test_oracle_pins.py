@@ -345,6 +345,56 @@ def test_ambiguity_flag_marks_scores_near_the_threshold():
     assert not low.any() and amb.all()
 
 
+def _stream_with_scores(p):
+    """A stream of t = len(p) tokens whose last query sees exactly the scores p (sum 1): key j is
+    log(p_j) times the j-th unit vector, the last query is all ones, scale 1.  Returns (q, k, v)
+    as [t, 1, t] arrays."""
+    t = len(p)
+    k = np.zeros((t, 1, t))
+    k[np.arange(t), 0, np.arange(t)] = np.log(p)
+    q = np.zeros((t, 1, t))
+    q[t - 1] = 1.0
+    return q, k, np.zeros((t, 1, t))
+
+
+@pytest.mark.parametrize("t", [2, 5, 37])
+@pytest.mark.parametrize("delta,flagged", [(0.0, True), (5e-7, True), (-5e-7, True), (0.99e-6, True), (-0.99e-6, True),
+                                           (1.01e-6, False), (-1.01e-6, False), (2e-6, False), (-2e-6, False),
+                                           (1e-3, False)])
+def test_ambiguity_window_is_one_millionth_wide(t, delta, flagged):
+    # The benchmark definition lets an fp32 implementation disagree with the fp64 comparison
+    # alpha < 1/t only where alpha lies within 1e-6 of 1/t.  Scores are planted exactly: slot 0 gets
+    # 1/t + delta, slot 1 gets 1/t + 3e-3 (well outside), the rest share what is left.
+    assert oracle._load().sho_amb_window() == 1e-6 == oracle.AMB_WINDOW
+    p = np.full(t, 0.0)
+    p[0] = 1.0 / t + delta
+    if t > 2:
+        p[1] = 1.0 / t + 3e-3
+        p[2:] = (1.0 - p[0] - p[1]) / (t - 2)
+    else:
+        p[1] = 1.0 - p[0]
+    q, k, v = _stream_with_scores(p)
+    o = oracle.Oracle(1, t + 1, 0, 4, 1, t, scale=1.0)
+    for s in range(t):
+        out, alpha, low, amb = o.attend(q[s], k[s], v[s])
+        o.record(low)
+    np.testing.assert_allclose(alpha[0], p, rtol=0, atol=1e-15)
+    assert bool(amb[0, 0]) == flagged
+    if delta != 0.0:
+        assert bool(low[0, 0]) == (delta < 0)                  # strict comparison, in fp64
+    if t > 2:
+        assert not amb[0, 1] and not low[0, 1]
+        assert bool(amb[0, 2]) == (abs(p[2] - 1.0 / t) <= 1e-6)
+    # the same query scored again by the recompute-at-compression variant carries the same flag
+    a2, low2, amb2, steps = o.recount()
+    row = t % 4
+    assert steps[row] == t
+    np.testing.assert_allclose(a2[0, row], p, rtol=0, atol=1e-15)
+    assert bool(amb2[0, row, 0]) == flagged and (delta == 0.0 or bool(low2[0, row, 0]) == (delta < 0))
+    if t > 2:
+        assert not amb2[0, row, 1]
+
+
 # --- the record recomputed at compression time -------------------------------------------
 def test_recount_matches_causal_attention_of_stored_queries_over_the_kept_set():
     # From the definition: each of the last w queries against the tokens still cached that
