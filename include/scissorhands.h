@@ -29,9 +29,10 @@
  *   - Kernels that wait (on mbarriers) do so for a bounded time; one that gives
  *     up records a code in the workspace's error word, finishes without touching
  *     further state, and the next sh_state returns SH_EDEVICE.
- *   - Slots [0, n) of a unit's cache are live.  By default they are sorted by
- *     stream position (compaction is stable, so "the r newest" are slots
- *     [n-r, n)); with SH_OPT_COMPACTION = 1 their order is arbitrary.
+ *   - Slots [0, n) of a unit's cache are live, in no particular order (a
+ *     compression fills the holes it makes from the tail); sh_state's positions
+ *     tell which token sits where.  With SH_OPT_COMPACTION = 0 compaction is
+ *     stable and the slots stay sorted by stream position.
  */
 #ifndef SCISSORHANDS_H_
 #define SCISSORHANDS_H_
@@ -77,19 +78,26 @@ typedef enum {
                                  "Overhead Tradeoff").  fp16/bf16/int4, head_dim 128 (with SH_OPT_PREFILL_CHUNK = 2:
                                  fp16/bf16 and budgets up to about 700 only); else SH_EINVAL.  Set before sh_bind:
                                  it changes sh_workspace_bytes. */
-    SH_OPT_COMPACTION = 6,    /* 0 (default): stable left-compaction, slots stay sorted by stream position;
-                                 1: every hole left by a dropped token below n-m is filled with a kept row from
-                                 the tail (at most m rows move instead of nearly all); slots are then in no
-                                 particular order: sh_state's pos tells which token sits where.  The kept set is
-                                 the same either way. */
+    SH_OPT_COMPACTION = 6,    /* 1 (default): every hole left by a dropped token below n-m is filled with a kept
+                                 row from the tail, so at most m rows move per compression; slots are then in no
+                                 particular order: sh_state's pos tells which token sits where.
+                                 0: stable left-compaction, slots stay sorted by stream position (nearly every
+                                 surviving row moves: about three times the time per compression at B = 410,
+                                 m = 64).  The kept set is the same either way: nothing in Algorithm 2 depends
+                                 on where a token is stored. */
     SH_OPT_PREFILL_CHUNK = 4, /* 1 (default): sh_prefill hands the tokens between two compressions to the chunk
                                  kernel where the shape allows it (fp16/bf16/int4 with head_dim 128: the tcgen05
                                  kernels, any budget); 0: one decode step per token; 2: the warp-level MMA chunk kernel
                                  (fp16/bf16, budgets up to about 700); 3: same as 1 */
-    SH_OPT_DECODE_KERNEL = 3  /* 0 (default): chosen from the shape; 1: one CTA (or cluster) per unit with
+    SH_OPT_DECODE_KERNEL = 3, /* 0 (default): chosen from the shape; 1: one CTA (or cluster) per unit with
                                  direct loads; 2: persistent CTAs fed by bulk asynchronous copies
                                  (stored rows of 256 bytes or more: fp32, and fp16/bf16 with head_dim 128; SH_OPT_SPLIT
                                  ignored; other shapes use 1) */
+    SH_OPT_SELFTEST_SKIP_TILE = 7 /* -1 (default): off.  k >= 0: self-test of the give-up path of the bounded waits.
+                                 In the kernel of SH_OPT_DECODE_KERNEL = 2 the first CTA never requests the k-th
+                                 tile of rows it was due to stream, so the wait for that tile runs out after
+                                 about a second, the CTA finishes without touching further cache state, and the
+                                 next sh_state returns SH_EDEVICE.  Outputs of such a step are meaningless. */
 } sh_option;
 
 /*
@@ -131,8 +139,10 @@ int sh_set_option(sh_handle h, int key, double value);
  * "Overhead Tradeoff" paragraph describes).  With SH_OPT_AUTO_COMPRESS the
  * compression of Algorithm 2 follows when n == B.
  * q_dev, k_new_dev, v_new_dev: [heads][head_dim] in the handle's dtype (fp16
- * for the int4 store), 16-byte aligned.  attn_out_dev: [heads][head_dim] fp32.
- * Errors: SH_EFULL when n == B on entry, SH_EINVAL, SH_ESTATE, SH_ECUDA.
+ * for the int4 store), 16-byte aligned.  attn_out_dev: [heads][head_dim] fp32,
+ * 4-byte aligned.
+ * Errors: SH_EFULL when n == B on entry, SH_EINVAL (NULL or misaligned pointer, more than
+ * 2^24 - 1 tokens streamed), SH_ESTATE, SH_ECUDA.
  */
 int sh_decode_step(sh_handle h, const void *q_dev, const void *k_new_dev, const void *v_new_dev,
                    float *attn_out_dev, void *stream);
@@ -198,8 +208,9 @@ int sh_prefill_chunk_max(sh_handle h);
  * Algorithm 2 for every unit, if the cache is full (n == B): importance
  * record I_j = number of the last w steps at which token j was below the
  * threshold; the r newest tokens are not candidates; the m candidates with
- * the largest I are dropped, the oldest first among equal I; survivors keep
- * their order (K, V, record and positions are compacted in place); n <- n-m.
+ * the largest I are dropped, the oldest first among equal I; K, V, record and
+ * positions of the survivors are compacted in place into slots [0, n-m) (see
+ * SH_OPT_COMPACTION for their order); n <- n-m.
  * A no-op when n < B.  *evicted_per_unit (may be NULL) receives m or 0.
  */
 int sh_compress(sh_handle h, void *stream, int *evicted_per_unit);
@@ -212,17 +223,25 @@ int sh_compress(sh_handle h, void *stream, int *evicted_per_unit);
  * serving engine that gives all of HBM to its own KV-block pool has nothing
  * left to ask for, and code inside a latency-critical decode loop must avoid
  * the device-wide synchronisation an allocation implies.  For them this entry
- * point keeps the selection scratch (one int32 per unit and slot, written by
- * the select-m kernel and read by the compaction kernel) in a static device
- * array inside the library instead of the workspace's scratch region, and
- * calls no allocator of any kind.
+ * point keeps the selection's result list (one int32 per unit and slot: the
+ * source slot of every surviving row, or the list of moves, written by the
+ * select-m kernel and read by the compaction kernel) in a static device array
+ * inside the library instead of the workspace's region for it, and calls no
+ * allocator of any kind.  Only that list is static: the record, the positions
+ * and a per-unit move count stay in the handle's workspace, as for sh_compress.
+ * Where one kernel does selection and compaction together (SH_OPT_COMPACTION = 1
+ * with bit-planes that fit in shared memory) no list leaves the kernel and the
+ * array is not touched.
  *
  * Limit: heads * B <= SH_STATIC_SCRATCH_MAX_ENTRIES (4 MiB of device memory,
  * held by every GPU that loads the library until the process exits); beyond it
  * the call returns SH_ETOOBIG and does nothing.  Inputs and outputs are the
  * handle's bound workspace, exactly as for sh_compress.
  * The first call on each device looks up the array's device address (with that
- * device current); make that first call before any stream capture.
+ * device current).  Make that first call at start-up: before any stream
+ * capture, and before the rest of device memory is handed to a pool, since the
+ * CUDA runtime may load the library's device code, and with it reserve the
+ * array, only then.
  * All calls on a device share the one array and it keeps the previous call's
  * contents.  Nothing in it needs to start at zero: the selection writes every
  * entry the compaction reads.  Two calls whose kernels overlap on the GPU
@@ -236,8 +255,10 @@ int sh_compress_static(sh_handle h, void *stream, int *evicted_per_unit);
  * selection kernel on its own: counters_dev [units][n] uint16 (tokens in
  * position order); evicted_dev [units][m] int32 receives the indices of the
  * dropped tokens in ascending order.  Needs 0 <= r, 1 <= m <= n - r,
- * n <= 65535, every counter <= 16384.  Uses no handle and no workspace.
+ * n <= SH_SELECT_MAX_N (counters and histogram share the CTA's shared memory),
+ * every counter <= 16384; SH_EINVAL otherwise.  Uses no handle and no workspace.
  */
+#define SH_SELECT_MAX_N 40000
 int sh_select(const uint16_t *counters_dev, int units, int n, int r, int m, int32_t *evicted_dev,
               void *stream);
 
@@ -285,7 +306,11 @@ int sh_export_unit(sh_handle h, int unit, float *K_host, float *V_host, void *st
 
 /*
  * Resume from a workspace image: after the caller has copied back a saved
- * copy of the whole workspace, set the host counters that went with it.
+ * copy of the whole workspace, set the host counters that went with it
+ * (0 <= n <= B, n <= t < 2^24; with n == B the next call must be sh_compress).
+ * Not available once sh_prefill_ragged has run (SH_ESTATE): the per-sequence
+ * counters then live in the workspace image itself and one (n, t) pair cannot
+ * describe them.  Errors: SH_EINVAL, SH_ESTATE.
  */
 int sh_restore(sh_handle h, int n, long long t);
 

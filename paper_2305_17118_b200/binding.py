@@ -21,6 +21,8 @@ SH_STATIC_SCRATCH_MAX_ENTRIES = 1 << 20
 SH_F32, SH_F16, SH_BF16, SH_INT4_G64_F16 = 0, 1, 2, 3
 SH_OPT_SOFTMAX_SCALE, SH_OPT_SPLIT, SH_OPT_AUTO_COMPRESS, SH_OPT_DECODE_KERNEL, SH_OPT_PREFILL_CHUNK, SH_OPT_RECORD_MODE = 0, 1, 2, 3, 4, 5
 SH_OPT_COMPACTION = 6
+SH_OPT_SELFTEST_SKIP_TILE = 7
+SH_SELECT_MAX_N = 40000
 
 DTYPE_CODE = {"f32": SH_F32, "f16": SH_F16, "bf16": SH_BF16, "int4": SH_INT4_G64_F16}
 INPUT_TORCH_DTYPE = {SH_F32: torch.float32, SH_F16: torch.float16, SH_BF16: torch.bfloat16,
@@ -35,12 +37,7 @@ EXPORTS = ["sh_create", "sh_destroy", "sh_workspace_bytes", "sh_bind", "sh_set_o
 
 def _load() -> C.CDLL:
     path = _build.LIB
-    override = os.environ.get("SH_LIBRARY")      # an alternative build of the same library
-    if override:
-        if not os.path.exists(override):
-            raise ImportError(f"SH_LIBRARY={override} does not exist")
-        path = override
-    elif _build.stale():
+    if _build.stale():
         try:
             path = _build.build()
         except Exception as e:  # no nvcc here: use what was shipped, if anything
@@ -111,7 +108,7 @@ class Handle:
     def __init__(self, B: int, r: int, w: int, m: int, heads: int, head_dim: int, dtype, device="cuda:0",
                  split: Optional[int] = None, scale: Optional[float] = None, auto_compress: bool = True,
                  kernel: Optional[int] = None, prefill_chunk: Optional[bool] = None, recompute_record: bool = False,
-                 unordered: bool = False):
+                 unordered: Optional[bool] = None):
         self.dtype = DTYPE_CODE[dtype] if isinstance(dtype, str) else int(dtype)
         self.B, self.r, self.w, self.m, self.U, self.D = B, r, w, m, heads, head_dim
         self.Bw = (B + 31) // 32
@@ -130,8 +127,8 @@ class Handle:
             self.set_option(SH_OPT_DECODE_KERNEL, kernel)
         if recompute_record:
             self.set_option(SH_OPT_RECORD_MODE, 1.0)
-        if unordered:
-            self.set_option(SH_OPT_COMPACTION, 1.0)
+        if unordered is not None:
+            self.set_option(SH_OPT_COMPACTION, 1.0 if unordered else 0.0)
         if prefill_chunk is not None:
             self.set_option(SH_OPT_PREFILL_CHUNK, float(int(prefill_chunk)))
         self.set_option(SH_OPT_AUTO_COMPRESS, 1.0 if auto_compress else 0.0)

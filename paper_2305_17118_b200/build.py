@@ -36,23 +36,42 @@ def stale() -> bool:
 
 
 def build(force: bool = False, verbose: bool = False, out: str = LIB) -> str:
-    """Compile every .cu under csrc/ into one shared library.  Returns its path."""
+    """Compile every .cu under csrc/ (one nvcc process per file, in parallel) and link them into one shared
+    library.  Returns its path."""
     if out == LIB and not force and not stale():
         return LIB
     os.makedirs(os.path.dirname(out), exist_ok=True)
-    tmp = out + f".{os.getpid()}.tmp"
-    cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-shared", "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC, "-o", tmp]
+    obj_dir = os.path.join(os.path.dirname(out), f"obj.{os.getpid()}")
+    os.makedirs(obj_dir, exist_ok=True)
+    nvcc = _nvcc()
+    flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
+             "-I", INCLUDE, "-I", CSRC]
     if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += os.environ.get("SH_NVCC_FLAGS", "").split()
-    cmd += sources()
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if res.returncode != 0:
-        raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
-    if verbose:
-        print(res.stderr)
-    os.replace(tmp, out)
+        flags += ["-Xptxas", "-v"]
+    try:
+        jobs = []
+        for src in sources():
+            obj = os.path.join(obj_dir, os.path.basename(src) + ".o")
+            jobs.append((src, obj, subprocess.Popen([nvcc, *flags, "-c", src, "-o", obj], stdout=subprocess.PIPE,
+                                                    stderr=subprocess.STDOUT, text=True)))
+        log = []
+        for src, obj, proc in jobs:
+            text, _ = proc.communicate()
+            log.append(text)
+            if proc.returncode != 0:
+                for _s, _o, other in jobs:
+                    if other.poll() is None:
+                        other.kill()
+                raise RuntimeError(f"nvcc failed on {os.path.basename(src)}:\n{text}")
+        tmp = out + f".{os.getpid()}.tmp"
+        res = subprocess.run([nvcc, "-shared", "-o", tmp, *[obj for _s, obj, _p in jobs]], capture_output=True, text=True)
+        if res.returncode != 0:
+            raise RuntimeError("link failed:\n" + res.stdout + res.stderr)
+        if verbose:
+            print("".join(log))
+        os.replace(tmp, out)
+    finally:
+        shutil.rmtree(obj_dir, ignore_errors=True)
     return out
 
 

@@ -171,6 +171,7 @@ int do_step(sh_context *c, const void *q, const void *k, const void *v, float *o
     p.t = (int)(c->t + 1);
     p.hist_row = (int)((c->t + 1) % c->w);
     p.scale_log2e = (float)((double)c->scale * LOG2E);
+    p.selftest_skip_tile = c->selftest_skip_tile;
     cudaError_t e = sh_launch_decode(c, p, s, &c->launches);
     if (e != cudaSuccess) return cuda_fail(c, e);
     c->started = true;
@@ -215,8 +216,9 @@ int sh_create(int B, int r, int w, int m, int heads, int head_dim, int dtype, sh
     c->kernel = 0;
     c->prefill_chunk = 1;
     c->record_mode = 0;
-    c->unordered = 0;
+    c->unordered = 1;
     c->record_fresh_t = -1;
+    c->selftest_skip_tile = -1;
     c->started = false;
     c->slab = nullptr; c->slab_bytes = 0;
     c->launches = 0;
@@ -300,6 +302,11 @@ int sh_set_option(sh_handle h, int key, double value) {
             h->kernel = k;
             return SH_OK;
         }
+        case SH_OPT_SELFTEST_SKIP_TILE: {
+            if (!(value >= -1.0 && value < 1e9)) return SH_EINVAL;
+            h->selftest_skip_tile = (int)value;
+            return SH_OK;
+        }
         default: return SH_EINVAL;
     }
 }
@@ -308,6 +315,7 @@ int sh_decode_step(sh_handle h, const void *q_dev, const void *k_new_dev, const 
                    float *attn_out_dev, void *stream) {
     if (!h || !q_dev || !k_new_dev || !v_new_dev || !attn_out_dev) return SH_EINVAL;
     if (misaligned(q_dev) || misaligned(k_new_dev) || misaligned(v_new_dev)) return SH_EINVAL;
+    if (reinterpret_cast<uintptr_t>(attn_out_dev) & 3u) return SH_EINVAL;
     if (!h->slab) return SH_ESTATE;
     if (cache_full(h)) return SH_EFULL;
     if (h->t + 1 >= (1 << 24)) return SH_EINVAL;   // the threshold test multiplies by t in fp32
@@ -331,6 +339,7 @@ static void *pinned_alias(const void *host_ptr) {
 int sh_decode_step_host(sh_handle h, const void *q_host, const void *k_new_host, const void *v_new_host,
                         float *attn_out_host, void *stream) {
     if (!h || !q_host || !k_new_host || !v_new_host || !attn_out_host) return SH_EINVAL;
+    if (reinterpret_cast<uintptr_t>(attn_out_host) & 3u) return SH_EINVAL;
     if (!h->slab) return SH_ESTATE;
     if (cache_full(h)) return SH_EFULL;
     if (h->t + 1 >= (1 << 24)) return SH_EINVAL;
@@ -537,7 +546,7 @@ int sh_compress(sh_handle h, void *stream, int *evicted_per_unit) {
 }
 
 int sh_select(const uint16_t *counters_dev, int units, int n, int r, int m, int32_t *evicted_dev, void *stream) {
-    if (!counters_dev || !evicted_dev || units < 1 || n < 1 || n > 65535 || r < 0 || m < 1 || m > n - r)
+    if (!counters_dev || !evicted_dev || units < 1 || n < 1 || n > SH_SELECT_MAX_N || r < 0 || m < 1 || m > n - r)
         return SH_EINVAL;
     SelectParams sp = {};
     sp.hist = nullptr;
@@ -613,14 +622,13 @@ int sh_export_unit(sh_handle h, int unit, float *K_host, float *V_host, void *st
 }
 
 int sh_restore(sh_handle h, int n, long long t) {
-    if (!h || n < 0 || n >= h->B || t < n) return SH_EINVAL;
+    if (!h || n < 0 || n > h->B || t < n || t >= (1 << 24)) return SH_EINVAL;
     if (!h->slab) return SH_ESTATE;
+    if (h->ragged) return SH_ESTATE;      // per-sequence counters live on the device: one (n, t) cannot describe them
     h->n = n;
     h->t = t;
     h->started = true;
     h->record_fresh_t = -1;
-    h->ragged = false;
-    h->n_seq.clear(); h->t_seq.clear();
     return SH_OK;
 }
 

@@ -9,14 +9,10 @@
 #pragma once
 #include <stdint.h>
 
-#ifndef SH_WAIT_LIMIT
-#define SH_WAIT_LIMIT (1u << 26)
-#endif
-#ifndef SH_WAIT_NS
-#define SH_WAIT_NS 1000000000ull
-#endif
-
 namespace shasync {
+
+constexpr uint32_t WAIT_POLLS = 1u << 26;              // polls before a wait gives up, and
+constexpr unsigned long long WAIT_NS = 1000000000ull;  // nanoseconds on the global timer, whichever comes first
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -56,9 +52,9 @@ __device__ __forceinline__ unsigned long long global_ns() {
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *err, int code) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
-    for (uint32_t i = 1; i < SH_WAIT_LIMIT; ++i) {
+    for (uint32_t i = 1; i < WAIT_POLLS; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 255u) == 0 && global_ns() - t0 > SH_WAIT_NS) break;
+        if ((i & 255u) == 0 && global_ns() - t0 > WAIT_NS) break;
     }
     if (err) atomicCAS(err, 0, code);
     return false;

@@ -41,6 +41,7 @@ struct sh_context {
     long long record_fresh_t;   // record_mode 1: step for which the bit-planes were last recomputed (-1: never)
     int prefill_chunk;  // SH_OPT_PREFILL_CHUNK: 1 = sh_prefill may batch tokens between compressions
     int kernel;      // SH_OPT_DECODE_KERNEL: 0 automatic, 1 direct loads, 2 pipelined bulk copies
+    int selftest_skip_tile;   // SH_OPT_SELFTEST_SKIP_TILE: -1, or the tile CTA 0's producer leaves out
     bool started;    // a step has run: options are frozen
     char *slab;
     size_t slab_bytes;
@@ -90,6 +91,7 @@ struct DecodeParams {
     int hist_row;   // t mod w
     int t;          // 1-based stream position of this step's token
     float scale_log2e;
+    int selftest_skip_tile;   // pipelined kernel only: -1, or the tile (counted per CTA) that CTA 0's producer leaves out
 };
 
 struct CompactParams {

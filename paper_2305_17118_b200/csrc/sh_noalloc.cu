@@ -1,13 +1,14 @@
-// sh_compress_static: the compression step with its selection scratch held in
-// a static device array instead of the caller's workspace.
+// sh_compress_static: the compression step with the selection's result list held
+// in a static device array instead of the caller's workspace.
 //
 // Who needs this: an inference server that hands all of HBM to its own KV-block
 // pool at start-up has nothing left for cudaMalloc afterwards, and a caller
 // inside a latency-critical decode loop cannot afford cudaMalloc's implicit
-// device synchronisation.  Such a caller may have carved the handle's workspace
-// out of memory it already owned; this entry point lets the compression run
-// without touching any allocator, and without depending on the workspace's
-// scratch region.
+// device synchronisation.  This entry point runs the compression without
+// touching any allocator.  Only the int32 list that the selection kernel hands
+// to the compaction kernel (source slot per surviving row, or the hole/filler
+// moves) lives in the static array; the per-unit move count, like the record and
+// the positions, stays in the handle's workspace.
 #include <mutex>
 
 #include "sh_internal.h"

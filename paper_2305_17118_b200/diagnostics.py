@@ -74,7 +74,7 @@ class ScoreChange:
 
 
 def score_change_ratio(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, dtype: str, B: int, r: int, w: int, m: int,
-                       device="cuda:0", unordered: bool = False) -> ScoreChange:
+                       device="cuda:0", unordered=None) -> ScoreChange:
     """Change ratio of the attention scores (the paper's ablation on attention score error):
     the t tokens of ``q, k, v`` ([t, units, head_dim], storage dtype, CUDA) are streamed through a
     handle with budget ``B`` (compressing as it goes) and through one that keeps everything; the

@@ -99,6 +99,8 @@ def run_lockstep(handle, cfg_dtype: str, inputs, steps: int, units, tol: float, 
     step's output tensor [U, d].  Returns (LockstepResult, oracle)."""
     units = torch.as_tensor(units, dtype=torch.long)
     un = units.numpy()
+    if not isinstance(handle, SortedView):          # slots are compared in position order, whatever the compaction mode
+        handle = SortedView(handle, units=un)
     if orc is None:
         orc = oracle_mod.Oracle(len(un), handle.B, handle.r, handle.w, handle.m, handle.D,
                                 quant=(cfg_dtype == "int4"))
@@ -161,6 +163,8 @@ def run_lockstep_chunked(handle, cfg_dtype: str, inputs_block, steps: int, units
     ``outs``: a list that receives each chunk's output tensor [cnt, U, d]."""
     units = torch.as_tensor(units, dtype=torch.long)
     un = units.numpy()
+    if not isinstance(handle, SortedView):          # slots are compared in position order, whatever the compaction mode
+        handle = SortedView(handle, units=un)
     if orc is None:
         orc = oracle_mod.Oracle(len(un), handle.B, handle.r, handle.w, handle.m, handle.D,
                                 quant=(cfg_dtype == "int4"))
@@ -251,6 +255,8 @@ def run_lockstep_recompute(handle, cfg_dtype: str, inputs, steps: int, units, to
     positions and kept sets must be identical."""
     units = torch.as_tensor(units, dtype=torch.long)
     un = units.numpy()
+    if not isinstance(handle, SortedView):          # slots are compared in position order, whatever the compaction mode
+        handle = SortedView(handle, units=un)
     if orc is None:
         orc = oracle_mod.Oracle(len(un), handle.B, handle.r, handle.w, handle.m, handle.D, quant=(cfg_dtype == "int4"))
     res = res or LockstepResult()

@@ -45,6 +45,14 @@ def test_host_only_calls_validate_arguments():
     assert lib.sh_create(410, 64, 128, 64, 9216, 128, sh.SH_F16, None) == sh.SH_EINVAL
     assert lib.sh_create(40000, 64, 128, 64, 1, 128, sh.SH_F16, C.byref(h)) == sh.SH_EINVAL
     assert lib.sh_select(None, 1, 10, 0, 1, None, None) == sh.SH_EINVAL
+    one = C.c_void_p(16)          # never dereferenced: the size check comes first
+    assert lib.sh_select(one, 1, sh.SH_SELECT_MAX_N + 1, 0, 1, one, None) == sh.SH_EINVAL
+    h2 = C.c_void_p()
+    assert lib.sh_create(16, 2, 8, 6, 4, 64, sh.SH_F16, C.byref(h2)) == sh.SH_OK
+    assert lib.sh_restore(h2, 3, 3) == sh.SH_ESTATE                 # nothing bound
+    assert lib.sh_set_option(h2, sh.SH_OPT_SELFTEST_SKIP_TILE, -2.0) == sh.SH_EINVAL
+    assert lib.sh_set_option(h2, sh.SH_OPT_SELFTEST_SKIP_TILE, 3.0) == sh.SH_OK
+    lib.sh_destroy(h2)
 
 
 def _handle(sh, B, r, w, m, heads, d, dtype):

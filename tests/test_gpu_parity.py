@@ -29,10 +29,13 @@ def _stream_fn(q, k, v):
 @pytest.mark.parametrize("dtype,d", [("f32", 64), ("f32", 128), ("f16", 128), ("f16", 64), ("bf16", 128),
                                       ("bf16", 64), ("int4", 128), ("int4", 64)])
 @pytest.mark.parametrize("split", [1, 2, 4, 8])
-def test_lockstep_small(sh, dtype, d, split):
+@pytest.mark.parametrize("stable", [False, True])
+def test_lockstep_small(sh, dtype, d, split, stable):
+    """Every storage type and head size, every cluster split, both compaction modes (the default, which
+    fills holes from the tail, and the stable one)."""
     U, B, r, w, m, T = 5, 150, 9, 37, 41, 420      # ragged: B, w not multiples of 32; several tiles
     q, k, v = wl.random_stream(U, d, T, seed=7 + split, dtype=dtype, peaked=3.0, device="cuda")
-    h = sh.Handle(B, r, w, m, U, d, dtype, split=split, auto_compress=False)
+    h = sh.Handle(B, r, w, m, U, d, dtype, split=split, auto_compress=False, unordered=not stable)
     res, _ = run_lockstep(h, dtype, _stream_fn(q, k, v), T, torch.arange(U), TOL[dtype])
     assert res.compressions >= 6
     assert res.adoptions <= 1e-4 * res.slot_steps + 2
@@ -40,11 +43,12 @@ def test_lockstep_small(sh, dtype, d, split):
 
 @pytest.mark.parametrize("B,r,w,m", [(33, 0, 1, 33), (64, 63, 5, 1), (32, 4, 100, 7), (1000, 10, 400, 500),
                                      (2, 1, 3, 1), (97, 5, 64, 92), (3000, 10, 400, 1500)])
-def test_lockstep_edge_parameters(sh, B, r, w, m):
+@pytest.mark.parametrize("stable", [False, True])
+def test_lockstep_edge_parameters(sh, B, r, w, m, stable):
     U, d, dtype = 3, 64, "f16"
     T = min(3 * B + 50, 1300) if B <= 1000 else B + 100
     q, k, v = wl.random_stream(U, d, T, seed=B, dtype=dtype, peaked=2.0, device="cuda")
-    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, unordered=not stable)
     res, _ = run_lockstep(h, dtype, _stream_fn(q, k, v), T, torch.arange(U), TOL[dtype])
     assert res.compressions >= 1
 
@@ -106,7 +110,7 @@ def test_lockstep_chunked_int4_store(sh, U, B, r, w, m, sizes):
     decode steps from the state the chunks left; and the quantised rows equal the oracle's bit for bit."""
     dtype, d, T = "int4", 128, min(2 * B + 2 * m + 11, B + 2 * m + 60)
     q, k, v = wl.random_stream(U, d, T, seed=37 + U, dtype=dtype, peaked=3.0, device="cuda")
-    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    h = SortedView(sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False))
     blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
     res, orc = run_lockstep_chunked(h, dtype, blk, T, torch.arange(U), TOL[dtype], chunk_sizes=sizes)
     assert res.steps == T and res.compressions >= 2
@@ -238,11 +242,12 @@ def test_config_tiny_every_step(sh):
 
 
 @pytest.mark.parametrize("name", ["opt6b", "opt6b_int4"])
-def test_config_opt6b_shapes(sh, name):
+@pytest.mark.parametrize("stable", [False, True])
+def test_config_opt6b_shapes(sh, name, stable):
     cfg = wl.CONFIGS[name]
     st = wl.Stream(cfg, device="cuda")
     units = wl.sample_units(cfg, 48)
-    h = sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, cfg.units, cfg.head_dim, cfg.dtype, auto_compress=False)
+    h = sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, cfg.units, cfg.head_dim, cfg.dtype, auto_compress=False, unordered=not stable)
     res, _ = run_lockstep(h, cfg.dtype, st.step, cfg.total_steps, units, TOL[cfg.dtype], state_every=16)
     assert res.compressions == 26
     assert res.adoptions <= 1e-4 * res.slot_steps + 2
@@ -322,21 +327,22 @@ def test_select_kernel_bit_exact_on_oracle_records(sh, n, r, m):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "f16", "bf16", "int4"])
-def test_compaction_moves_rows_bit_identically(sh, dtype):
+@pytest.mark.parametrize("stable", [False, True])
+def test_compaction_moves_rows_bit_identically(sh, dtype, stable):
     """Stored key and value rows after several compressions equal the oracle's bit for bit, on a handle in
     lockstep with the oracle; and a second handle that compresses by itself (SH_OPT_AUTO_COMPRESS, the
     default) ends bit-identical to the first, outputs included."""
     U, d, B, r, w, m, T = 4, 128, 96, 8, 20, 40, 200
     q, k, v = wl.random_stream(U, d, T, seed=3, dtype=dtype, peaked=3.0, device="cuda")
-    auto = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=True)
+    auto = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=True, unordered=not stable)
     outs = torch.stack([auto.decode_step(q[t], k[t], v[t]) for t in range(T)])
-    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, unordered=not stable)
     twin_outs = []
     res, orc = run_lockstep(h, dtype, _stream_fn(q, k, v), T, torch.arange(U), TOL[dtype], outs=twin_outs)
     assert res.compressions >= 3
-    n = h.n
+    n, by_pos = h.n, SortedView(h)
     for u in range(U):
-        K, V = h.export_unit(u)
+        K, V = by_pos.export_unit(u)
         oK, oV = orc.cache(u)
         assert (K[:n].astype(np.float64) == oK).all() and (V[:n].astype(np.float64) == oV).all()
     assert torch.equal(outs, torch.stack(twin_outs))
@@ -789,3 +795,91 @@ def test_error_codes(sh):
         hd.set_option(sh.SH_OPT_SPLIT, 2)    # options are frozen after the first step
     assert lib.sh_decode_step(hd._h, None, buf.data_ptr(), buf.data_ptr(), out.data_ptr(), None) == sh.SH_EINVAL
     assert lib.sh_decode_step(hd._h, buf.data_ptr() + 2, buf.data_ptr(), buf.data_ptr(), out.data_ptr(), None) == sh.SH_EINVAL
+
+
+def test_bounded_wait_gives_up_and_reports_device_error(sh):
+    """The give-up path of the kernels' bounded waits, made to happen without faulting anything: with
+    SH_OPT_SELFTEST_SKIP_TILE the first CTA of the pipelined decode kernel never requests one of its tiles
+    (no copy is in flight for it), so the wait for that tile runs out after about a second.  The kernel
+    must end by itself, sh_state must say SH_EDEVICE from then on, later calls on the handle must return
+    normally, and a fresh handle on the same device must work."""
+    import ctypes as C
+    import time
+    U, d, B, r, w, m, dtype = 5, 128, 300, 4, 16, 100, "f16"
+    q, k, v = wl.random_stream(U, d, 200, seed=77, dtype=dtype, peaked=2.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, kernel=2, auto_compress=False)
+    h.set_option(sh.SH_OPT_SELFTEST_SKIP_TILE, 1)      # the second tile CTA 0 would stream in a launch
+    for t in range(129):                               # up to 128 cached rows a unit is a single tile: nothing is skipped
+        h.decode_step(q[t], k[t], v[t])
+    assert sh.lib.sh_state(h._h, None, None, None, None, None, None) == sh.SH_OK
+    t0 = time.time()
+    h.decode_step(q[129], k[129], v[129])              # 129 cached rows: two tiles, the second never arrives
+    rc = sh.lib.sh_state(h._h, None, None, None, None, None, None)
+    took = time.time() - t0
+    assert rc == sh.SH_EDEVICE and took < 20.0
+    assert b"bounded wait" in sh.lib.sh_strerror(rc)
+    n, t = C.c_int(0), C.c_longlong(0)
+    assert sh.lib.sh_state(h._h, None, C.byref(n), C.byref(t), None, None, None) == sh.SH_EDEVICE     # sticky
+    assert n.value == 130 and t.value == 130
+    out = torch.empty(U, d, device="cuda")
+    assert sh.lib.sh_decode_step(h._h, q[130].data_ptr(), k[130].data_ptr(), v[130].data_ptr(), out.data_ptr(), None) == sh.SH_OK
+    assert sh.lib.sh_state(h._h, None, None, None, None, None, None) == sh.SH_EDEVICE
+    torch.cuda.synchronize()
+    # the device and the library are fine: a fresh handle runs in lockstep with the oracle
+    g = sh.Handle(B, r, w, m, U, d, dtype, kernel=2, auto_compress=False)
+    res, _ = run_lockstep(g, dtype, _stream_fn(q, k, v), 200, torch.arange(U), TOL[dtype])
+    assert res.steps == 200
+
+
+def test_restore_boundaries_and_output_alignment(sh):
+    import ctypes as C
+    U, d, B, r, w, m, dtype = 4, 64, 16, 2, 8, 6, "f16"
+    q, k, v = wl.random_stream(U, d, 40, seed=78, dtype=dtype, device="cuda")
+    # a snapshot taken at a full cache (manual compression) can be resumed: the next call is sh_compress
+    a = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    b = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    for t in range(B):
+        a.decode_step(q[t], k[t], v[t])
+        b.decode_step(q[t], k[t], v[t])
+    snap = a.snapshot()
+    assert snap[1] == B
+    for t in range(B, 30):
+        for h in (a, b):
+            h.compress()
+            h.decode_step(q[t], k[t], v[t])
+    a.restore(snap)
+    out = torch.empty(U, d, device="cuda")
+    with pytest.raises(sh.ShError) as ei:
+        a.decode_step(q[B], k[B], v[B], out)
+    assert ei.value.status == sh.SH_EFULL
+    for t in range(B, 30):
+        a.compress()
+        a.decode_step(q[t], k[t], v[t])
+    assert_same_state(a, b)
+    assert sh.lib.sh_restore(a._h, B + 1, 100) == sh.SH_EINVAL
+    assert sh.lib.sh_restore(a._h, 5, 4) == sh.SH_EINVAL
+    # once sequences differ in length one (n, t) pair cannot describe the handle
+    rg = sh.Handle(B, r, w, m, U, d, dtype)
+    rg.prefill_ragged(q[:9].contiguous(), k[:9].contiguous(), v[:9].contiguous(), [3, 9])
+    assert sh.lib.sh_restore(rg._h, 3, 3) == sh.SH_ESTATE
+    n_seq, t_seq = rg.sequence_state()
+    assert n_seq.tolist() == [3, 9] and t_seq.tolist() == [3, 9]          # untouched
+    rg.decode_step(q[9], k[9], v[9])
+    assert rg.sequence_state()[0].tolist() == [4, 10]
+    # the output pointer is checked like the inputs
+    buf = torch.empty(U * d + 4, device="cuda")
+    assert sh.lib.sh_decode_step(b._h, q[30].data_ptr(), k[30].data_ptr(), v[30].data_ptr(), buf.data_ptr() + 2, None) == sh.SH_EINVAL
+    assert sh.lib.sh_decode_step(b._h, q[30].data_ptr(), k[30].data_ptr(), v[30].data_ptr(), buf.data_ptr() + 4, None) == sh.SH_OK
+
+
+def test_select_at_its_size_limit(sh):
+    n, r, m = sh.SH_SELECT_MAX_N, 1000, 300
+    rng = np.random.default_rng(5)
+    I = rng.integers(0, 16385, size=(2, n)).astype(np.int32)
+    I[1] = rng.integers(0, 3, size=n)
+    got = sh.select(torch.from_numpy(I).cuda(), r, m).cpu().numpy()
+    for i in range(2):
+        assert (got[i] == oracle.select(I[i], r, m)).all()
+    big = torch.zeros(1, n + 1, dtype=torch.int16, device="cuda")
+    out = torch.empty(1, m, dtype=torch.int32, device="cuda")
+    assert sh.lib.sh_select(big.data_ptr(), 1, n + 1, r, m, out.data_ptr(), None) == sh.SH_EINVAL

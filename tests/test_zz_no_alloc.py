@@ -18,10 +18,17 @@ from paper_2305_17118_b200 import workloads as wl
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("dtype,unordered", [("f16", False), ("int4", False), ("f16", True)])
-def test_static_scratch_compress_matches_regular_compress_twice(dtype, unordered):
+@pytest.mark.parametrize("dtype,unordered,shape", [
+    ("f16", False, (37, 128, 100, 8, 24, 30)),        # stable compaction: the static array holds every survivor's source slot
+    ("int4", False, (37, 128, 100, 8, 24, 30)),
+    ("f16", False, (700, 64, 410, 64, 128, 64)),      # 287 000 entries of the array in use
+    ("f16", True, (3, 64, 1000, 10, 700, 400)),       # hole filling with bit-planes too large for the one-kernel path:
+                                                      # the static array carries the list of moves between two kernels
+    ("f16", True, (37, 128, 100, 8, 24, 30)),         # one-kernel path: same entry point, the array stays untouched
+])
+def test_static_scratch_compress_matches_regular_compress_twice(dtype, unordered, shape):
     from paper_2305_17118_b200 import binding as sh
-    U, d, B, r, w, m = 37, 128, 100, 8, 24, 30
+    U, d, B, r, w, m = shape
     T = B + m + 5     # fills once at step B, again at step B + m
     q, k, v = wl.random_stream(U, d, T, seed=21, dtype=dtype, peaked=3.0, device="cuda")
     a = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, unordered=unordered)
