@@ -10,12 +10,19 @@ The default workload is the OPT-66B-shaped one the headline metric is quoted on
 (batch 128 x 72 heads, head_dim 128, fp16 K/V, B=410, prompt 2048); the prompt is
 streamed through the same path, untimed, before the timed decode steps.
 
-Prints ONE JSON line.  `value` = steps/s with inputs resident in HBM; `e2e` =
-the same through sh_decode_step_host with pinned host buffers (copies inside the
-timed region); `roofline` = algorithmic K+V bytes of the fused decode kernel per
-launch / its mean CUDA-event duration, against the measured HBM copy peak;
-`cpu_baseline` = the CPU oracle timed on this machine's host cores on a bounded
-sample.  `--impl reference` times only that oracle.
+The timed window of K steps is run REPEATS times, each time from the restored
+post-prompt state and after W warm-up steps, so every repetition covers the same
+stream positions; `value` is the median repetition (steps/s with inputs resident
+in HBM), `repeats` lists them all.  A window may or may not contain a compression
+(the cache fills every m steps), so the cost of one compression is also measured
+on its own from a restored state with a full cache (`compress`), in the
+compaction mode the run uses and in the other one.
+
+Prints ONE JSON line.  `e2e` = the same metric through sh_decode_step_host with
+pinned host buffers (copies inside the timed region); `roofline` = algorithmic
+K+V bytes of the fused decode kernel per launch / its mean CUDA-event duration,
+against the measured HBM copy peak; `cpu_baseline` = the CPU oracle timed on this
+box's host cores on a bounded sample.  `--impl reference` times only that oracle.
 """
 from __future__ import annotations
 
@@ -38,7 +45,9 @@ METRIC = "compressed_decode_attn_steps_per_s"
 UNIT = "steps/s"
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
+REPEATS = 3
 ES = {"f32": 4.0, "f16": 2.0, "bf16": 2.0, "int4": 0.5 + 2.0 / 64.0}
+INT4_LANE_INSTR_PER_BYTE = 10.0   # int4 decode kernel: warp instructions x 32 / stored bytes read, from its ncu capture
 
 
 def measured_peak():
@@ -54,7 +63,7 @@ class ClockSampler:
     """SM clock and throttle reasons sampled through NVML (read-only) while the
     timed region runs."""
 
-    def __init__(self, index: int, period_s: float = 0.01):
+    def __init__(self, index: int, period_s: float = 0.001):
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
         self._thr = None
@@ -89,6 +98,7 @@ class ClockSampler:
 
     def __enter__(self):
         if self.nv:
+            self._stop.clear()
             self._thr = threading.Thread(target=self._run, daemon=True)
             self._thr.start()
         return self
@@ -97,6 +107,7 @@ class ClockSampler:
         self._stop.set()
         if self._thr:
             self._thr.join()
+            self._thr = None
 
     def summary(self):
         if not self.samples:
@@ -129,6 +140,18 @@ def live_rows_schedule(cfg, first_step: int, count: int):
         if n == cfg.B:
             n -= cfg.m
     return out
+
+
+def config_record(cfg, args, world: int):
+    """The `config` object of the JSON line: the same keys and values in both arms."""
+    kv_bytes = 2 * cfg.layers * cfg.units * cfg.B * cfg.head_dim * ES[cfg.dtype]
+    return {"workload": cfg.name, "batch": cfg.batch, "heads": cfg.heads, "layers": cfg.layers,
+            "units": cfg.units * cfg.layers, "head_dim": cfg.head_dim, "kv_dtype": cfg.dtype, "B": cfg.B, "r": cfg.r,
+            "w": cfg.w, "m": cfg.m, "prompt": cfg.prompt,
+            "record": "recomputed at compression" if args.recompute_record else "online",
+            "compaction": "stable" if args.stable_compaction else "hole filling (library default)",
+            "l2": "flushed between steps" if kv_bytes < 2 * L2_BYTES else "inputs larger than L2",
+            "kv_bytes": kv_bytes, "parallelism": f"units replicated x{world}" if world > 1 else "1 GPU"}
 
 
 # --------------------------------------------------------------------------- CPU oracle arm
@@ -175,8 +198,7 @@ def reference_arm(args, cfg, rank):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / value if value else None,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": cfg.name, "units": cfg.units, "layers": cfg.layers, "head_dim": cfg.head_dim,
-                   "kv_dtype": cfg.dtype, "B": cfg.B, "r": cfg.r, "w": cfg.w, "m": cfg.m},
+        "config": config_record(cfg, args, int(os.environ.get("WORLD_SIZE", "1"))),
         "cpu_baseline": info,
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -185,6 +207,55 @@ def reference_arm(args, cfg, rank):
 
 
 # --------------------------------------------------------------------------- CUDA arm
+def make_handles(sh, cfg, args, dev, stable: bool, layers: int):
+    return [sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, cfg.units, cfg.head_dim, cfg.dtype, device=dev, auto_compress=False,
+                      split=args.split, kernel=args.kernel,
+                      prefill_chunk=0 if args.no_prefill_chunk else args.prefill_chunk_kernel,
+                      recompute_record=args.recompute_record, unordered=False if stable else None)
+            for _ in range(layers)]
+
+
+def stream_prompt(cfg, handles, streams):
+    """The prompt through sh_prefill, untimed part of the benchmark.  Returns (device ms, block size)."""
+    blk = max(1, min(256, (1 << 31) // (cfg.units * cfg.head_dim * 2 * 3)))
+    ms = 0.0
+    for h, st in zip(handles, streams):
+        for t0 in range(1, cfg.prompt + 1, blk):
+            q, k, v = st.block(t0, min(t0 + blk, cfg.prompt + 1))
+            pa, pb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            pa.record()
+            h.prefill(q, k, v)
+            pb.record()
+            torch.cuda.synchronize()
+            ms += pa.elapsed_time(pb)
+    return ms, blk
+
+
+def time_compression(cfg, h, snap, dec_l, out, reps: int = REPEATS):
+    """CUDA-event time of one sh_compress of handle `h` (all its units), `reps` times, each from the
+    restored post-prompt state advanced until the cache is full.  dec_l: that layer's decode inputs."""
+    times, launches = [], 0
+    for _ in range(reps):
+        h.restore(snap)
+        n, i = snap[1], 0
+        while n < cfg.B:
+            h.decode_step(dec_l[0][i % len(dec_l[0])], dec_l[1][i % len(dec_l[0])], dec_l[2][i % len(dec_l[0])], out)
+            n += 1
+            i += 1
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = h.launch_count
+        torch.cuda.synchronize()
+        a.record()
+        assert h.compress() == cfg.m
+        b.record()
+        torch.cuda.synchronize()
+        launches = h.launch_count - l0
+        times.append(a.elapsed_time(b))
+    return {"ms_best": min(times), "ms_median": statistics.median(times), "ms_all": times, "kernel_launches": launches,
+            "units": cfg.units, "steps_between_compressions": cfg.m,
+            "ms_per_step_amortised": statistics.median(times) / cfg.m}
+
+
 def cuda_arm(args, cfg, rank, world):
     from paper_2305_17118_b200 import binding as sh
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -197,24 +268,10 @@ def cuda_arm(args, cfg, rank, world):
     K, W = args.steps, args.warmup
     U, d, Ly = cfg.units, cfg.head_dim, cfg.layers
     streams = [wl.Stream(cfg, device=dev, layer=l + 1000 * rank) for l in range(Ly)]
-    handles = [sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, U, d, cfg.dtype, device=dev, auto_compress=False,
-                         split=args.split, kernel=args.kernel,
-                         prefill_chunk=0 if args.no_prefill_chunk else args.prefill_chunk_kernel,
-                         recompute_record=args.recompute_record, unordered=args.unordered_compaction)
-               for _ in range(Ly)]
+    handles = make_handles(sh, cfg, args, dev, args.stable_compaction, Ly)
 
     # ---- prompt: streamed through the same path, untimed
-    blk = max(1, min(256, (1 << 31) // (U * d * 2 * 3)))
-    prompt_ms = 0.0
-    for l, (h, st) in enumerate(zip(handles, streams)):
-        for t0 in range(1, cfg.prompt + 1, blk):
-            q, k, v = st.block(t0, min(t0 + blk, cfg.prompt + 1))
-            pa, pb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            pa.record()
-            h.prefill(q, k, v)
-            pb.record()
-            torch.cuda.synchronize()
-            prompt_ms += pa.elapsed_time(pb)
+    prompt_ms, blk = stream_prompt(cfg, handles, streams)
     # ---- decode inputs resident in HBM; cycle if the run is longer than the buffer
     n_in = min(W + K, max(1, int(6e9 // (Ly * U * d * 2 * 3))))
     dec = [st.block(cfg.prompt + 1, cfg.prompt + 1 + n_in) for st in streams]
@@ -226,6 +283,7 @@ def cuda_arm(args, cfg, rank, world):
     out = torch.empty(U, d, device=dev)
 
     def one_step(i, timed_pairs=None):
+        done = 0
         for l, h in enumerate(handles):
             q, k, v = dec[l][0][i % n_in], dec[l][1][i % n_in], dec[l][2][i % n_in]
             if timed_pairs is not None:
@@ -236,7 +294,8 @@ def cuda_arm(args, cfg, rank, world):
                 timed_pairs.append((a, b))
             else:
                 h.decode_step(q, k, v, out)
-            h.compress()           # no-op unless the cache just filled
+            done += h.compress() != 0          # no-op unless the cache just filled
+        return done
 
     def barrier():
         torch.cuda.synchronize()
@@ -244,35 +303,40 @@ def cuda_arm(args, cfg, rank, world):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident timing
-    for i in range(W):
-        one_step(i)
-    launches0 = sum(h.launch_count for h in handles)
-    pairs, step_pairs = [], []
+    # ---- device-resident timing: REPEATS windows of K steps over the same stream positions
     sampler = ClockSampler(local)
-    barrier()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with sampler:
-        ev0.record()
-        for i in range(W, W + K):
-            if flush:
-                flush_buf.fill_(i & 0xFF)
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record()
-                one_step(i, pairs)
-                b.record()
-                step_pairs.append((a, b))
-            else:
-                one_step(i, pairs)
-        ev1.record()
+    rep_ms, rep_value, kern_ms, launches, compressions = [], [], [], 0, 0
+    for rep in range(REPEATS):
+        for h, s in zip(handles, snaps):
+            h.restore(s)
+        for i in range(W):
+            one_step(i)
+        launches0 = sum(h.launch_count for h in handles)
+        pairs, step_pairs, compressions = [], [], 0
         barrier()
-    launches = sum(h.launch_count for h in handles) - launches0
-    if flush:
-        total_ms = sum(a.elapsed_time(b) for a, b in step_pairs)
-    else:
-        total_ms = ev0.elapsed_time(ev1)
-    kern_ms = [a.elapsed_time(b) for a, b in pairs]
-    ms_per_step, value = job_throughput(total_ms, K, world, dist, dev)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with sampler:
+            ev0.record()
+            for i in range(W, W + K):
+                if flush:
+                    flush_buf.fill_(i & 0xFF)
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record()
+                    compressions += one_step(i, pairs)
+                    b.record()
+                    step_pairs.append((a, b))
+                else:
+                    compressions += one_step(i, pairs)
+            ev1.record()
+            barrier()
+        launches = sum(h.launch_count for h in handles) - launches0
+        total_ms = sum(a.elapsed_time(b) for a, b in step_pairs) if flush else ev0.elapsed_time(ev1)
+        kern_ms += [a.elapsed_time(b) for a, b in pairs]
+        ms_step, val = job_throughput(total_ms, K, world, dist, dev)
+        rep_ms.append(ms_step)
+        rep_value.append(val)
+    ms_per_step = statistics.median(rep_ms)
+    value = statistics.median(rep_value)
 
     # ---- roofline of the fused decode kernel (one launch = one layer's units)
     n_sched = live_rows_schedule(cfg, cfg.prompt + W + 1, K)
@@ -288,11 +352,37 @@ def cuda_arm(args, cfg, rank, world):
                 traffic = tr["dram_bytes_per_unit_row"] * statistics.fmean(n_sched) * U
     except Exception:
         pass
-    roofline = {"bound": "hbm", "kernel": "sh_decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+    roofline = {"bound": "hbm", "kernel": handles[0].decode_kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
                 "frac_of_8TBs_nominal": achieved / 8000.0, "alg_bytes_per_launch": alg_bytes_launch,
                 "avg_launch_us": kern_avg_ms * 1e3, "launches_timed": len(kern_ms),
                 "decode_kernel_share_of_step": kern_avg_ms * Ly / ms_per_step}
+    if flush:
+        roofline["note"] = ("working set below 2x L2 (flushed between steps) and fewer than two units per SM: the step is "
+                            "bound by launch and load latency, not by HBM; the fraction is reported for completeness")
+    if cfg.dtype == "int4":
+        # CUDA-core unpacking of 4-bit codes is bound by instruction issue before HBM: peak derived from
+        # the kernel's instructions per stored byte and the SMs' issue rate at the sampled clock.
+        mhz = sampler.summary()["sm_mhz"] or 1965.0
+        issue_peak = 148 * 4 * mhz * 1e6 * 32 / INT4_LANE_INSTR_PER_BYTE / 1e9
+        roofline.update({"bound": "alu", "peak": issue_peak, "frac": achieved / issue_peak,
+                         "peak_source": (f"derived: 148 SMs x 4 schedulers x 1 warp instruction per clock x 32 lanes at {mhz:.0f} MHz "
+                                         f"/ {INT4_LANE_INSTR_PER_BYTE} lane-instructions per stored byte (profiles/)"),
+                         "frac_of_measured_hbm": achieved / peak})
+
+    # ---- the compression on its own (steps c1-c4), in the mode of this run and in the other one
+    compress = None
+    if rank == 0 and not args.no_compress_timing:
+        mode = "stable" if args.stable_compaction else "hole filling"
+        compress = {mode: time_compression(cfg, handles[0], snaps[0], dec[0], out)}
+        other = make_handles(sh, cfg, args, dev, not args.stable_compaction, 1)
+        stream_prompt(cfg, other, streams[:1])
+        torch.cuda.synchronize()
+        compress["hole filling" if args.stable_compaction else "stable"] = time_compression(
+            cfg, other[0], other[0].snapshot(), dec[0], out)
+        del other
+        compress["note"] = ("one sh_compress over one layer's units from a restored state with a full cache; "
+                            "it recurs every m steps, ms_per_step_amortised = median / m")
 
     # ---- end to end: host buffers through sh_decode_step_host
     e2e = None
@@ -344,12 +434,11 @@ def cuda_arm(args, cfg, rank, world):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": {"f32": "f32", "f16": "f16", "bf16": "bf16", "int4": "int4"}[cfg.dtype] + " KV, f32 accumulate",
         "data": "synthetic",
-        "config": {"workload": cfg.name, "batch": cfg.batch, "heads": cfg.heads, "layers": Ly, "units": U * Ly,
-                   "head_dim": d, "kv_dtype": cfg.dtype, "B": cfg.B, "r": cfg.r, "w": cfg.w, "m": cfg.m,
-                   "prompt": cfg.prompt, "record": "recomputed at compression" if args.recompute_record else "online",
-                   "compaction": "unordered" if args.unordered_compaction else "stable",
-                   "l2": "flushed between steps" if flush else "inputs larger than L2",
-                   "kv_bytes": kv_bytes, "parallelism": f"units replicated x{world}" if world > 1 else "1 GPU"},
+        "config": config_record(cfg, args, world),
+        "repeats": {"n": REPEATS, "value_best": max(rep_value), "value_median": value, "values": rep_value,
+                    "ms_per_step": rep_ms, "from": "post-prompt snapshot restored before every repetition, then warm-up"},
+        "n_range": [min(n_sched), max(n_sched)], "n_mean": statistics.fmean(n_sched),
+        "compressions_timed": compressions, "compress": compress,
         "attn_GBps": statistics.fmean(n_sched) * U * Ly * d * ES[cfg.dtype] * 2 / (ms_per_step * 1e-3) / 1e9,
         "prompt": {"tokens": cfg.prompt, "ms": prompt_ms, "tokens_per_s": cfg.prompt * 1e3 / prompt_ms if prompt_ms else None,
                    "chunked": bool(handles[0].prefill_chunk_max) and not args.no_prefill_chunk,
@@ -376,20 +465,26 @@ def main():
                     help="variant: rebuild the importance record at each compression from stored queries")
     ap.add_argument("--kv-dtype", default=None, choices=["f32", "f16", "bf16", "int4"], help="override the workload's K/V dtype")
     ap.add_argument("--head-dim", type=int, default=None, choices=[64, 128], help="override the workload's head_dim")
-    ap.add_argument("--stable-compaction", dest="unordered_compaction", action="store_false",
-                    help="SH_OPT_COMPACTION = 0 (the library's default): stable left-compaction, slots stay sorted by "
-                         "position.  The benchmark runs SH_OPT_COMPACTION = 1 (holes filled from the tail, at most m "
-                         "rows move per compression; same kept sets)")
+    ap.add_argument("--stable-compaction", action="store_true",
+                    help="SH_OPT_COMPACTION = 0: stable left-compaction, slots stay sorted by position.  The default "
+                         "is the library's: holes filled from the tail, at most m rows move per compression; same kept sets")
+    ap.add_argument("--no-compress-timing", action="store_true", help="skip the separate timing of sh_compress (tuning runs)")
     ap.add_argument("--prefill-chunk-kernel", type=int, default=None, choices=[1, 2, 3],
                     help="SH_OPT_PREFILL_CHUNK for the untimed prompt phase: 1 library's choice, 2 warp-level MMA kernel, 3 tcgen05 kernel")
     ap.add_argument("--no-prefill-chunk", action="store_true", help="stream the prompt one decode step per token")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (tuning runs)")
+    ap.add_argument("--units", type=int, default=None,
+                    help="override the workload's units per launch (a smaller case of the same kernels, for profiler captures)")
+    ap.add_argument("--prompt", type=int, default=None, help="override the workload's prompt length (same purpose)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     cfg = wl.CONFIGS[args.config]
-    if args.kv_dtype or args.head_dim:      # shape variants of a named workload (not the benchmark's own lines)
-        cfg = cfg.scaled(name=f"{cfg.name}[{args.kv_dtype or cfg.dtype},d{args.head_dim or cfg.head_dim}]",
-                         dtype=args.kv_dtype or cfg.dtype, head_dim=args.head_dim or cfg.head_dim)
+    if args.kv_dtype or args.head_dim or args.units or args.prompt:      # shape variants of a named workload (not the benchmark's own lines)
+        tag = ",".join(x for x in (args.kv_dtype, f"d{args.head_dim}" if args.head_dim else None,
+                                   f"units{args.units}" if args.units else None,
+                                   f"prompt{args.prompt}" if args.prompt else None) if x)
+        cfg = cfg.scaled(name=f"{cfg.name}[{tag}]", dtype=args.kv_dtype or cfg.dtype, head_dim=args.head_dim or cfg.head_dim,
+                         units=args.units or cfg.units, prompt=args.prompt or cfg.prompt)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":

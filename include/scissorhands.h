@@ -317,6 +317,11 @@ int sh_restore(sh_handle h, int n, long long t);
 /* Number of kernels this handle has launched since creation. */
 long long sh_launch_count(sh_handle h);
 
+/* Which fused decode kernel sh_decode_step launches for this handle's shape and options
+ * (see SH_OPT_DECODE_KERNEL): 1 = one CTA or cluster per unit with direct loads, 2 = persistent
+ * CTAs fed by bulk asynchronous copies.  For reports and profiles. */
+int sh_decode_kernel_choice(sh_handle h);
+
 /* Text for a status code; never NULL. */
 const char *sh_strerror(int status);
 

@@ -32,7 +32,7 @@ EXPORTS = ["sh_create", "sh_destroy", "sh_workspace_bytes", "sh_bind", "sh_set_o
            "sh_decode_step_host", "sh_prefill", "sh_prefill_chunk", "sh_prefill_chunk_max", "sh_export_record", "sh_recompute_record", "sh_prefill_ragged",
            "sh_sequence_state",
            "sh_compress", "sh_compress_static", "sh_scores", "sh_select", "sh_state", "sh_export_unit",
-           "sh_restore", "sh_launch_count", "sh_strerror", "sh_last_cuda_error"]
+           "sh_restore", "sh_launch_count", "sh_decode_kernel_choice", "sh_strerror", "sh_last_cuda_error"]
 
 
 def _load() -> C.CDLL:
@@ -70,6 +70,7 @@ def _load() -> C.CDLL:
     lib.sh_restore.argtypes = [vp, C.c_int, C.c_longlong]
     lib.sh_launch_count.argtypes = [vp]
     lib.sh_launch_count.restype = C.c_longlong
+    lib.sh_decode_kernel_choice.argtypes = [vp]
     lib.sh_strerror.argtypes = [C.c_int]
     lib.sh_strerror.restype = C.c_char_p
     lib.sh_last_cuda_error.argtypes = [vp]
@@ -318,6 +319,11 @@ class Handle:
     @property
     def launch_count(self) -> int:
         return int(lib.sh_launch_count(self._h))
+
+    @property
+    def decode_kernel(self) -> str:
+        """Name of the fused decode kernel sh_decode_step launches for this handle."""
+        return {1: "sh_decode_kernel", 2: "sh_decode_tma_kernel"}[int(lib.sh_decode_kernel_choice(self._h))]
 
 
 def select(counters: torch.Tensor, r: int, m: int, stream=None) -> torch.Tensor:

@@ -634,6 +634,8 @@ int sh_restore(sh_handle h, int n, long long t) {
 
 long long sh_launch_count(sh_handle h) { return h ? h->launches : 0; }
 
+int sh_decode_kernel_choice(sh_handle h) { return h ? sh_decode_kernel_for(h, h->U) : SH_EINVAL; }
+
 const char *sh_strerror(int status) {
     switch (status) {
         case SH_OK: return "ok";

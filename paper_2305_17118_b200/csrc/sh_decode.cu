@@ -686,7 +686,8 @@ cudaError_t sh_launch_scores(const sh_context *c, const DecodeParams &p, float *
     return e;
 }
 
-cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches) {
+// Which decode kernel serves `units` units of this handle: 2 = pipelined (sh_decode_tma.cu), 1 = direct loads.
+int sh_decode_kernel_for(const sh_context *c, int units) {
     // Shapes of launch (crossovers measured on B200, rows of 256 bytes: equal at 12 units per SM, the direct
     // kernel 6 % ahead from 16 per SM on, the pipelined one 15 % ahead at 8.6).  With very many units per SM
     // the direct-load kernel in its many-units shape is the fastest for every storage type: CTAs of 4 warps
@@ -695,12 +696,18 @@ cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStr
     // more stream through the persistent pipelined kernel from 128 units on; the direct kernel takes the
     // rest, with 4-warp CTAs from 4 units per SM on and 8-warp CTAs (and a cluster split for very few units)
     // below.  SH_OPT_DECODE_KERNEL = 1 / 2 forces the direct / pipelined kernel.
-    const bool many = p.U >= 4 * 148 && c->split == 1;
+    const bool many = units >= 4 * 148 && c->split == 1;
     const bool pipelined_ok = sh_decode_tma_supported(c);
-    const bool prefer_direct = many && (!pipelined_ok || p.U >= 16 * 148);
+    const bool prefer_direct = many && (!pipelined_ok || units >= 16 * 148);
     if (c->kernel != 1 && pipelined_ok &&
-        (c->kernel == 2 || (!prefer_direct && p.U >= 128 && !(c->split_explicit && c->split > 1))))
-        return sh_launch_decode_tma(c, p, s, launches);
+        (c->kernel == 2 || (!prefer_direct && units >= 128 && !(c->split_explicit && c->split > 1))))
+        return 2;
+    return 1;
+}
+
+cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches) {
+    const bool many = p.U >= 4 * 148 && c->split == 1;
+    if (sh_decode_kernel_for(c, p.U) == 2) return sh_launch_decode_tma(c, p, s, launches);
     cudaError_t e = cudaErrorInvalidValue;
     // Two shapes of CTA.  With few units per SM the step is latency-bound and a CTA of 8 warps with 8 row
     // loads in flight per thread finishes a unit soonest.  With many units per SM (no cluster split then)

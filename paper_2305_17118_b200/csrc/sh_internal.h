@@ -174,6 +174,7 @@ cudaError_t sh_launch_recount_umma_int4(const ChunkParams &p, cudaStream_t s);
 cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches);
 // Scores of a query over the present caches (analysis; p.n = live rows, nothing appended).
 cudaError_t sh_launch_scores(const sh_context *c, const DecodeParams &p, float *alpha_out, cudaStream_t s, long long *launches);
+int sh_decode_kernel_for(const sh_context *c, int units);
 // Pipelined (bulk-copy ring) variant of the decode kernel and its applicability test.
 bool sh_decode_tma_supported(const sh_context *c);
 cudaError_t sh_launch_decode_tma(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches);
