@@ -95,3 +95,33 @@ def score_change_ratio(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, dtype:
     alpha_s[rows, pos - 1] = a_s[:, :n]
     kept[rows, pos - 1] = True
     return ScoreChange((alpha_s - a_o) / a_o, kept, alpha_s, a_o, t)
+
+
+@dataclasses.dataclass
+class RecordModeOverlap:
+    overlap: np.ndarray      # [units] |kept_online n kept_recomputed| / n
+    overlap_old: np.ndarray  # [units] the same over the tokens outside the recent window only (those the record decided)
+    n: int                   # tokens kept per unit
+    t: int
+
+
+def record_mode_overlap(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, dtype: str, B: int, r: int, w: int, m: int,
+                        device="cuda:0") -> RecordModeOverlap:
+    """Kept sets under the two ways of obtaining the importance record (Section 4.1, "Overhead Tradeoff"):
+    kept online during generation (one comparison per cached token per step, against the cache as it was
+    at that step) or recomputed at each compression from the last w queries against the cache as it is
+    then (Algorithm 2 as stated).  The same ``q, k, v`` ([t, units, head_dim], storage dtype, CUDA) are
+    streamed through one handle of each kind; returned is, per unit, the fraction of kept tokens the two
+    have in common.  Everything but the set intersection runs in the CUDA kernels."""
+    t, U, d = q.shape
+    a = sh.Handle(B, r, w, m, U, d, dtype, device=device)
+    b = sh.Handle(B, r, w, m, U, d, dtype, device=device, recompute_record=True)
+    a.prefill(q, k, v)
+    b.prefill(q, k, v)
+    n, _, pos_a, _, _ = a.state(counters=False, low=False)
+    n_b, _, pos_b, _, _ = b.state(counters=False, low=False)
+    assert n == n_b
+    both = np.array([len(np.intersect1d(pos_a[u], pos_b[u])) for u in range(U)])
+    old = t - r
+    both_old = np.array([len(np.intersect1d(pos_a[u][pos_a[u] <= old], pos_b[u][pos_b[u] <= old])) for u in range(U)])
+    return RecordModeOverlap(both / n, both_old / max(n - min(r, n), 1), n, t)

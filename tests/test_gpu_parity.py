@@ -883,3 +883,22 @@ def test_select_at_its_size_limit(sh):
     big = torch.zeros(1, n + 1, dtype=torch.int16, device="cuda")
     out = torch.empty(1, m, dtype=torch.int32, device="cuda")
     assert sh.lib.sh_select(big.data_ptr(), 1, n + 1, r, m, out.data_ptr(), None) == sh.SH_EINVAL
+
+
+def test_record_mode_overlap_diagnostic(sh):
+    """Kept sets with the record kept online against the record recomputed at compression: both handles keep the
+    recent window, so the overlap is at least r/n; each side's kept set is checked against an oracle running the
+    same variant in lockstep with a twin handle, which makes the reported overlap the oracle's as well."""
+    from paper_2305_17118_b200 import diagnostics
+    U, d, B, r, w, m, t, dtype = 6, 128, 64, 6, 24, 20, 173, "f16"
+    q, k, v = wl.random_stream(U, d, t, seed=88, dtype=dtype, peaked=3.0, device="cuda")
+    got = diagnostics.record_mode_overlap(q, k, v, dtype, B, r, w, m)
+    blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
+    _, o_a = run_lockstep_chunked(sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False), dtype, blk, t, torch.arange(U),
+                                  TOL[dtype], single_via_step=True)
+    _, o_b = run_lockstep_chunked(sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, recompute_record=True), dtype, blk,
+                                  t, torch.arange(U), TOL[dtype], single_via_step=True, recompute=True)
+    pa, pb = o_a.positions(), o_b.positions()
+    want = np.array([len(np.intersect1d(pa[u], pb[u])) for u in range(U)]) / o_a.n
+    assert got.n == o_a.n == o_b.n and np.abs(got.overlap - want).max() < 1e-12
+    assert (got.overlap >= r / got.n - 1e-12).all() and (got.overlap <= 1).all()
