@@ -48,6 +48,12 @@ def _load():
     ip = c.POINTER(c.c_int)
     lib.sho_create.restype = c.c_void_p
     lib.sho_create.argtypes = [c.c_int] * 6 + [c.c_double, c.c_int]
+    lib.sho_create_reading.restype = c.c_void_p
+    lib.sho_create_reading.argtypes = [c.c_int] * 6 + [c.c_double] + [c.c_int] * 5
+    lib.sho_cap.argtypes = [c.c_void_p]
+    lib.sho_import_compressed.argtypes = [c.c_void_p, c.c_void_p]
+    lib.sho_select_newest_first.argtypes = [ip, c.c_int, c.c_int, c.c_int, ip]
+    lib.sho_select_newest_first.restype = None
     lib.sho_destroy.argtypes = [c.c_void_p]
     lib.sho_destroy.restype = None
     lib.sho_threads.restype = c.c_int
@@ -109,16 +115,30 @@ class Oracle:
     amount of Algorithms 1 and 2.  ``scale`` multiplies the logits (default
     1/sqrt(head_dim)).  ``quant`` selects the int4 group-64 store.  Inputs must
     already be rounded to the storage dtype of the implementation under test.
+
+    Alternative readings of the paper (all off by default; the CUDA library
+    implements the defaults only): ``threshold`` 0 = 1/t of each step, 1 = 1/t of
+    the compression step for the whole window (Algorithm 2 literally), 2 = 1/n;
+    ``window_plus1`` = the w+1 steps of Algorithm 2's range [t-w, t];
+    ``tie_newest`` = among equal counters drop the newest first (a stable
+    ascending argsort cut at [:-m]); ``trigger_literal`` = Algorithm 1's
+    "if n > B": the cache holds up to B+1 tokens for one step.
     """
 
     def __init__(self, units: int, B: int, r: int, w: int, m: int, head_dim: int,
-                 scale: Optional[float] = None, quant: bool = False):
+                 scale: Optional[float] = None, quant: bool = False, threshold: int = 0,
+                 window_plus1: bool = False, tie_newest: bool = False, trigger_literal: bool = False):
         self._lib = _load()
         if scale is None:
             scale = 1.0 / np.sqrt(head_dim)
-        self.U, self.B, self.r, self.w, self.m, self.d = units, B, r, w, m, head_dim
+        self.U, self.r, self.w, self.m, self.d = units, r, w, m, head_dim
+        self.budget = B
         self.scale, self.quant = float(scale), bool(quant)
-        self._h = self._lib.sho_create(units, B, r, w, m, head_dim, float(scale), int(quant))
+        self._h = self._lib.sho_create_reading(units, B, r, w, m, head_dim, float(scale), int(quant), int(threshold),
+                                               int(window_plus1), int(tie_newest), int(trigger_literal))
+        # rows of storage per unit (the stride of every [U, .] array below): the budget, or one more
+        # under the literal trigger reading
+        self.B = int(self._lib.sho_cap(self._h)) if self._h else B
         if not self._h:
             raise ValueError("invalid oracle parameters (need 1 <= m <= B - r, w >= 1, "
                              "head_dim % 64 == 0 for the int4 store)")
@@ -192,6 +212,16 @@ class Oracle:
         got = self._lib.sho_compress(self._h, _ip(ev))
         return ev if got else None
 
+    def import_compressed(self, src: "Oracle") -> int:
+        """The prompting stage read as a bulk operation: ``src`` streamed the whole prompt under a
+        budget that never made it compress; its cache is brought under this oracle's budget by
+        rounds of Algorithm 2 on the record as it stands, and the survivors become this (fresh)
+        oracle's cache.  Returns the number of rounds."""
+        rounds = int(self._lib.sho_import_compressed(self._h, src._h))
+        if rounds < 0:
+            raise ValueError("oracles do not match, the target is not fresh, or too few candidates")
+        return rounds
+
     # -- the record recomputed at compression time (Algorithm 2 as stated) ----
     def recount(self):
         """Scores of the last w queries against the present cache (causal by
@@ -235,15 +265,17 @@ class Oracle:
         return out, self.compress()
 
 
-def select(I, r: int, m: int) -> np.ndarray:
+def select(I, r: int, m: int, newest_first: bool = False) -> np.ndarray:
     """Selection of Algorithm 2 on given counters (tokens in position order):
-    indices of the ``m`` dropped tokens, ascending."""
+    indices of the ``m`` dropped tokens, ascending.  ``newest_first``: the
+    alternative tie-break (among equal counters the newest go)."""
     I = np.ascontiguousarray(np.asarray(I, dtype=np.int32))
     n = I.shape[0]
     if not (0 <= r and 1 <= m <= n - r):
         raise ValueError("need 1 <= m <= n - r")
     ev = np.zeros(m, dtype=np.int32)
-    _load().sho_select(_ip(I), n, r, m, _ip(ev))
+    lib = _load()
+    (lib.sho_select_newest_first if newest_first else lib.sho_select)(_ip(I), n, r, m, _ip(ev))
     return np.sort(ev)
 
 

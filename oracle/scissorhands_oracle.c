@@ -49,6 +49,19 @@
  * streams, the budget saw-tooth, and an independent scalar int4 quantiser.
  * Which of the alternative readings the authors used is "parity unpinned":
  * the paper prints no numbers that would decide it.
+ *
+ * Alternative readings (sho_create_reading; the CUDA library implements the
+ * defaults only).  Each is what another reader could take from the same lines:
+ *   threshold 1: Algorithm 2 literally compares every step of the window with
+ *                1/t of the compression step, not of the step itself;
+ *   threshold 2: 1/n, the mean of the scores actually normalised over n tokens;
+ *   window    1: Algorithm 2's range [t-w, t] taken literally has w+1 steps;
+ *   tie       1: a stable ascending argsort cut at [:-m] drops, among equal
+ *                counters, the newest tokens instead of the oldest;
+ *   trigger   1: Algorithm 1's "if n > B" literally: the cache may hold B+1
+ *                tokens for one step, and compression leaves B+1-m.
+ *   prompt    1: the prompting stage of Section 2 read as a bulk operation (see
+ *                sho_prefill_bulk) instead of the token stream of Definition 4.1.
  */
 #include <math.h>
 #include <stdint.h>
@@ -62,15 +75,20 @@ typedef struct {
     int n;            /* live tokens */
     double *K, *V;    /* [B][d] stored (already rounded / dequantised) values */
     int *pos;         /* [B] 1-based stream position of each live token, ascending */
-    int *h_cnt;       /* [B] how many (step, low) pairs the token has received */
-    int *h_step;      /* [B][w] the last w pairs: step numbers */
-    uint8_t *h_low;   /* [B][w] the last w pairs: low flags */
+    int *h_cnt;       /* [cap] how many (step, low) pairs the token has received */
+    int *h_step;      /* [cap][hw] the last hw pairs: step numbers */
+    uint8_t *h_low;   /* [cap][hw] the last hw pairs: low flags */
+    double *h_alpha;  /* [cap][hw] the last hw pairs: the score itself (threshold reading 1 needs it) */
+    double *last_alpha; /* [cap] scores of the step just attended, until sho_record files them */
     double *Q;        /* [w][d] queries of the last w steps (slot = step mod w) */
     int *q_step;      /* [w] step of each stored query, 0 = none */
 } unit_t;
 
 typedef struct {
     int U, B, r, w, m, d, quant;
+    int cap;          /* rows of storage per unit: B, or B+1 under trigger reading 1 */
+    int hw;           /* history entries kept per token: w, or w+1 under window reading 1 */
+    int thr_mode, win_plus1, tie_newest, trig_literal;   /* alternative readings, all 0 by default */
     double scale;
     long t;           /* tokens streamed so far */
     unit_t *unit;
@@ -92,36 +110,52 @@ void sho_destroy(sho_t *o) {
         for (int u = 0; u < o->U; ++u) {
             unit_t *x = &o->unit[u];
             free(x->K); free(x->V); free(x->pos); free(x->h_cnt); free(x->h_step); free(x->h_low); free(x->Q); free(x->q_step);
+            free(x->h_alpha); free(x->last_alpha);
         }
         free(o->unit);
     }
     free(o);
 }
 
-sho_t *sho_create(int U, int B, int r, int w, int m, int d, double scale, int quant) {
+sho_t *sho_create_reading(int U, int B, int r, int w, int m, int d, double scale, int quant,
+                          int thr_mode, int win_plus1, int tie_newest, int trig_literal) {
     if (U < 1 || B < 1 || r < 0 || w < 1 || m < 1 || m > B - r || d < 1) return NULL;
     if (quant && d % 64) return NULL;
+    if (thr_mode < 0 || thr_mode > 2) return NULL;
     sho_t *o = calloc(1, sizeof *o);
     if (!o) return NULL;
     o->U = U; o->B = B; o->r = r; o->w = w; o->m = m; o->d = d; o->quant = quant; o->scale = scale;
+    o->thr_mode = thr_mode; o->win_plus1 = !!win_plus1; o->tie_newest = !!tie_newest; o->trig_literal = !!trig_literal;
+    o->cap = B + o->trig_literal;
+    o->hw = w + o->win_plus1;
     o->t = 0;
     o->unit = calloc((size_t)U, sizeof(unit_t));
     if (!o->unit) { free(o); return NULL; }
     for (int u = 0; u < U; ++u) {
         unit_t *x = &o->unit[u];
         x->n = 0;
-        x->K = calloc((size_t)B * d, sizeof(double));
-        x->V = calloc((size_t)B * d, sizeof(double));
-        x->pos = calloc((size_t)B, sizeof(int));
-        x->h_cnt = calloc((size_t)B, sizeof(int));
-        x->h_step = calloc((size_t)B * w, sizeof(int));
-        x->h_low = calloc((size_t)B * w, 1);
+        const size_t cap = (size_t)o->cap, hw = (size_t)o->hw;
+        x->K = calloc(cap * d, sizeof(double));
+        x->V = calloc(cap * d, sizeof(double));
+        x->pos = calloc(cap, sizeof(int));
+        x->h_cnt = calloc(cap, sizeof(int));
+        x->h_step = calloc(cap * hw, sizeof(int));
+        x->h_low = calloc(cap * hw, 1);
+        x->h_alpha = calloc(cap * hw, sizeof(double));
+        x->last_alpha = calloc(cap, sizeof(double));
         x->Q = calloc((size_t)w * d, sizeof(double));
         x->q_step = calloc((size_t)w, sizeof(int));
-        if (!x->K || !x->V || !x->pos || !x->h_cnt || !x->h_step || !x->h_low || !x->Q || !x->q_step) { sho_destroy(o); return NULL; }
+        if (!x->K || !x->V || !x->pos || !x->h_cnt || !x->h_step || !x->h_low || !x->h_alpha || !x->last_alpha || !x->Q ||
+            !x->q_step) { sho_destroy(o); return NULL; }
     }
     return o;
 }
+
+sho_t *sho_create(int U, int B, int r, int w, int m, int d, double scale, int quant) {
+    return sho_create_reading(U, B, r, w, m, d, scale, quant, 0, 0, 0, 0);
+}
+
+int sho_cap(const sho_t *o) { return o->cap; }
 
 /* int4 group-64 round trip of one row, float32 rule stated in the header. */
 static void quant_row(const double *x, int d, double *stored, int8_t *codes, float *scales) {
@@ -156,23 +190,24 @@ void sho_quantize(const double *x, int rows, int d, double *stored, int8_t *code
 
 int sho_n(const sho_t *o) { return o->unit[0].n; }
 long sho_t_now(const sho_t *o) { return o->t; }
-int sho_full(const sho_t *o) { return o->unit[0].n == o->B; }
+/* Is a compression due?  n == B by default (so n < B holds between steps, Definition 4.1);
+ * under trigger reading 1, Algorithm 1's literal n > B, i.e. n == B+1. */
+int sho_full(const sho_t *o) { return o->unit[0].n == o->cap; }
 
 /*
  * Steps 1 and 2 (and the comparison of step 3, not yet recorded).
- * q, k, v: [U][d].  out: [U][d].  alpha: [U][B] (first n entries of each row
- * valid).  low, amb: [U][B] bytes; amb_j = 1 when alpha_j lies within
+ * q, k, v: [U][d].  out: [U][d].  alpha: [U][cap] (first n entries of each row
+ * valid; cap = sho_cap() = B unless trigger reading 1).  low, amb: [U][cap] bytes; amb_j = 1 when alpha_j lies within
  * sho_amb_window() of the threshold, where an fp32 implementation may
  * legitimately decide the comparison the other way.
  * Returns -1 if the cache is already full (the caller forgot to compress).
  */
 int sho_attend(sho_t *o, const double *q, const double *k, const double *v,
                double *out, double *alpha, uint8_t *low, uint8_t *amb) {
-    const int B = o->B, d = o->d;
+    const int B = o->cap, d = o->d;
     if (o->unit[0].n >= B) return -1;
     o->t += 1;
     const long t = o->t;
-    const double thr = 1.0 / (double)t;
 #pragma omp parallel for schedule(static)
     for (int u = 0; u < o->U; ++u) {
         unit_t *x = &o->unit[u];
@@ -210,7 +245,9 @@ int sho_attend(sho_t *o, const double *q, const double *k, const double *v,
         for (int i = 0; i < d; ++i) ou[i] = 0.0;
         for (j = 0; j < n; ++j)
             for (int i = 0; i < d; ++i) ou[i] += a[j] * x->V[(size_t)j * d + i];
-        /* 3. the comparison against 1/t */
+        /* 3. the comparison against 1/t (threshold reading 2: against 1/n, the mean score) */
+        const double thr = o->thr_mode == 2 ? 1.0 / (double)n : 1.0 / (double)t;
+        for (j = 0; j < n; ++j) x->last_alpha[j] = a[j];
         for (j = 0; j < B; ++j) {
             low[(size_t)u * B + j] = (j < n) && (a[j] < thr);
             amb[(size_t)u * B + j] = (j < n) && (fabs(a[j] - thr) <= sho_amb_window());
@@ -221,7 +258,7 @@ int sho_attend(sho_t *o, const double *q, const double *k, const double *v,
 
 /* Step 3: remember this step's low flags, [U][B], for every live token. */
 void sho_record(sho_t *o, const uint8_t *low) {
-    const int B = o->B, w = o->w;
+    const int B = o->cap, w = o->hw;
     const long t = o->t;
 #pragma omp parallel for schedule(static)
     for (int u = 0; u < o->U; ++u) {
@@ -230,42 +267,49 @@ void sho_record(sho_t *o, const uint8_t *low) {
             int slot = x->h_cnt[j] % w;
             x->h_step[(size_t)j * w + slot] = (int)t;
             x->h_low[(size_t)j * w + slot] = low[(size_t)u * B + j] ? 1 : 0;
+            x->h_alpha[(size_t)j * w + slot] = x->last_alpha[j];
             x->h_cnt[j] += 1;
         }
     }
 }
 
-/* I_j of Algorithm 2 at the current t: low flags among steps (t-w, t]. */
+/* I_j of Algorithm 2 at the current t: low flags among steps (t-w, t] (window reading 1: [t-w, t]).
+ * Threshold reading 1 decides every step of the window against 1/t of the present step instead of
+ * using the flag taken at that step. */
 static int counter_of(const sho_t *o, const unit_t *x, int j) {
-    const int w = o->w;
-    int have = x->h_cnt[j] < w ? x->h_cnt[j] : w;
+    const int hw = o->hw;
+    const long first = o->t - o->w + (o->win_plus1 ? 0 : 1);     /* first step of the window */
+    int have = x->h_cnt[j] < hw ? x->h_cnt[j] : hw;
     int c = 0;
-    for (int s = 0; s < have; ++s)
-        if ((long)x->h_step[(size_t)j * w + s] > o->t - w && x->h_low[(size_t)j * w + s]) c += 1;
+    for (int s = 0; s < have; ++s) {
+        if ((long)x->h_step[(size_t)j * hw + s] < first) continue;
+        if (o->thr_mode == 1) c += x->h_alpha[(size_t)j * hw + s] < 1.0 / (double)o->t;
+        else c += x->h_low[(size_t)j * hw + s] ? 1 : 0;
+    }
     return c;
 }
 
-/* Counters of all live tokens, [U][B] (entries past n are 0). */
+/* Counters of all live tokens, [U][cap] (entries past n are 0). */
 void sho_counters(const sho_t *o, int *I) {
     for (int u = 0; u < o->U; ++u) {
         const unit_t *x = &o->unit[u];
-        for (int j = 0; j < o->B; ++j) I[(size_t)u * o->B + j] = j < x->n ? counter_of(o, x, j) : 0;
+        for (int j = 0; j < o->cap; ++j) I[(size_t)u * o->cap + j] = j < x->n ? counter_of(o, x, j) : 0;
     }
 }
 
-/* Positions of all live tokens, [U][B] (entries past n are 0). */
+/* Positions of all live tokens, [U][cap] (entries past n are 0). */
 void sho_positions(const sho_t *o, int *pos) {
     for (int u = 0; u < o->U; ++u) {
         const unit_t *x = &o->unit[u];
-        for (int j = 0; j < o->B; ++j) pos[(size_t)u * o->B + j] = j < x->n ? x->pos[j] : 0;
+        for (int j = 0; j < o->cap; ++j) pos[(size_t)u * o->cap + j] = j < x->n ? x->pos[j] : 0;
     }
 }
 
-/* Stored K and V rows of one unit, [B][d] each (rows past n are 0). */
+/* Stored K and V rows of one unit, [cap][d] each (rows past n are 0). */
 void sho_cache(const sho_t *o, int u, double *K, double *V) {
     const unit_t *x = &o->unit[u];
-    memset(K, 0, sizeof(double) * o->B * o->d);
-    memset(V, 0, sizeof(double) * o->B * o->d);
+    memset(K, 0, sizeof(double) * o->cap * o->d);
+    memset(V, 0, sizeof(double) * o->cap * o->d);
     memcpy(K, x->K, sizeof(double) * x->n * o->d);
     memcpy(V, x->V, sizeof(double) * x->n * o->d);
 }
@@ -276,18 +320,55 @@ void sho_cache(const sho_t *o, int u, double *K, double *V) {
  * candidate with the largest counter is taken, the oldest among equals.
  * evict[] receives the chosen indices in the order chosen.
  */
-void sho_select(const int *I, int n, int r, int m, int *evict) {
+static void select_tie(const int *I, int n, int r, int m, int *evict, int tie_newest) {
     uint8_t *gone = calloc((size_t)n, 1);
     for (int e = 0; e < m; ++e) {
         int best = -1;
         for (int j = 0; j < n - r; ++j) {
             if (gone[j]) continue;
-            if (best < 0 || I[j] > I[best]) best = j;   /* strict >: earlier index wins ties */
+            /* strict >: the earlier index wins ties; tie reading 1 (>=): the later one does */
+            if (best < 0 || I[j] > I[best] || (tie_newest && I[j] == I[best])) best = j;
         }
         evict[e] = best;
         if (best >= 0) gone[best] = 1;
     }
     free(gone);
+}
+
+void sho_select(const int *I, int n, int r, int m, int *evict) { select_tie(I, n, r, m, evict, 0); }
+void sho_select_newest_first(const int *I, int n, int r, int m, int *evict) { select_tie(I, n, r, m, evict, 1); }
+
+/* Algorithm 2 on one unit as it stands: counters at the present t, the r newest protected, the m
+ * candidates first in the order dropped, the rest moved up in order.  evicted_pos: [m] or NULL. */
+static void compress_unit(const sho_t *o, unit_t *x, int m, int r, int *evicted_pos) {
+    const int d = o->d, w = o->hw;
+    const int n = x->n;
+    int *I = malloc(sizeof(int) * n);
+    int *ev = malloc(sizeof(int) * m);
+    uint8_t *drop = calloc((size_t)n, 1);
+    for (int j = 0; j < n; ++j) I[j] = counter_of(o, x, j);
+    select_tie(I, n, r, m, ev, o->tie_newest);
+    for (int e = 0; e < m; ++e) drop[ev[e]] = 1;
+    int keep = 0, ne = 0;
+    for (int j = 0; j < n; ++j) {
+        if (drop[j]) {
+            if (evicted_pos) evicted_pos[ne] = x->pos[j];
+            ne += 1;
+            continue;
+        }
+        if (keep != j) {
+            memcpy(x->K + (size_t)keep * d, x->K + (size_t)j * d, sizeof(double) * d);
+            memcpy(x->V + (size_t)keep * d, x->V + (size_t)j * d, sizeof(double) * d);
+            x->pos[keep] = x->pos[j];
+            x->h_cnt[keep] = x->h_cnt[j];
+            memcpy(x->h_step + (size_t)keep * w, x->h_step + (size_t)j * w, sizeof(int) * w);
+            memcpy(x->h_low + (size_t)keep * w, x->h_low + (size_t)j * w, w);
+            memcpy(x->h_alpha + (size_t)keep * w, x->h_alpha + (size_t)j * w, sizeof(double) * w);
+        }
+        keep += 1;
+    }
+    x->n = keep;
+    free(I); free(ev); free(drop);
 }
 
 /*
@@ -296,39 +377,53 @@ void sho_select(const int *I, int n, int r, int m, int *evict) {
  * Returns the number of tokens dropped per unit (m or 0).
  */
 int sho_compress(sho_t *o, int *evicted_pos) {
-    const int B = o->B, d = o->d, w = o->w, m = o->m, r = o->r;
-    if (o->unit[0].n < B) return 0;
+    if (o->unit[0].n < o->cap) return 0;
 #pragma omp parallel for schedule(static)
-    for (int u = 0; u < o->U; ++u) {
-        unit_t *x = &o->unit[u];
-        const int n = x->n;
-        int *I = malloc(sizeof(int) * n);
-        int *ev = malloc(sizeof(int) * m);
-        uint8_t *drop = calloc((size_t)n, 1);
-        for (int j = 0; j < n; ++j) I[j] = counter_of(o, x, j);
-        sho_select(I, n, r, m, ev);
-        for (int e = 0; e < m; ++e) drop[ev[e]] = 1;
-        int keep = 0, ne = 0;
-        for (int j = 0; j < n; ++j) {
-            if (drop[j]) {
-                if (evicted_pos) evicted_pos[(size_t)u * m + ne] = x->pos[j];
-                ne += 1;
-                continue;
-            }
-            if (keep != j) {
-                memcpy(x->K + (size_t)keep * d, x->K + (size_t)j * d, sizeof(double) * d);
-                memcpy(x->V + (size_t)keep * d, x->V + (size_t)j * d, sizeof(double) * d);
-                x->pos[keep] = x->pos[j];
-                x->h_cnt[keep] = x->h_cnt[j];
-                memcpy(x->h_step + (size_t)keep * w, x->h_step + (size_t)j * w, sizeof(int) * w);
-                memcpy(x->h_low + (size_t)keep * w, x->h_low + (size_t)j * w, w);
-            }
-            keep += 1;
-        }
-        x->n = keep;
-        free(I); free(ev); free(drop);
+    for (int u = 0; u < o->U; ++u)
+        compress_unit(o, &o->unit[u], o->m, o->r, evicted_pos ? evicted_pos + (size_t)u * o->m : NULL);
+    return o->m;
+}
+
+/*
+ * The prompting stage read as a bulk operation (Section 2: the prompt's keys and values are computed
+ * and cached in full before generation starts) instead of Definition 4.1's token stream: `src` has
+ * streamed the whole prompt under a budget that never made it compress, so its outputs are full causal
+ * attention and its record holds the prompt's last w steps.  The prompt's cache is then brought under
+ * dst's budget by Algorithm 2 applied as often as needed - same record, m tokens per round, the r
+ * newest protected, until fewer than B tokens remain (trigger reading 1: no more than B) - and what
+ * survives, with its record, becomes dst's cache; dst continues at t = src's t.
+ * src and dst must agree in U, d, w, quant and readings; dst must be fresh.  Returns the number of
+ * rounds, or -1 on a mismatch.  src is left compressed.
+ */
+int sho_import_compressed(sho_t *dst, sho_t *src) {
+    if (dst->U != src->U || dst->d != src->d || dst->w != src->w || dst->hw != src->hw || dst->quant != src->quant ||
+        dst->thr_mode != src->thr_mode || dst->tie_newest != src->tie_newest || dst->t != 0)
+        return -1;
+    const int stop = dst->cap;            /* compress while n >= stop */
+    int rounds = 0;
+    while (src->unit[0].n >= stop) {
+        if (src->unit[0].n - dst->r < dst->m) return -1;
+#pragma omp parallel for schedule(static)
+        for (int u = 0; u < src->U; ++u) compress_unit(src, &src->unit[u], dst->m, dst->r, NULL);
+        rounds += 1;
     }
-    return m;
+    const int d = dst->d, hw = dst->hw;
+    for (int u = 0; u < src->U; ++u) {
+        unit_t *a = &dst->unit[u];
+        const unit_t *b = &src->unit[u];
+        a->n = b->n;
+        memcpy(a->K, b->K, sizeof(double) * b->n * d);
+        memcpy(a->V, b->V, sizeof(double) * b->n * d);
+        memcpy(a->pos, b->pos, sizeof(int) * b->n);
+        memcpy(a->h_cnt, b->h_cnt, sizeof(int) * b->n);
+        memcpy(a->h_step, b->h_step, sizeof(int) * b->n * hw);
+        memcpy(a->h_low, b->h_low, (size_t)b->n * hw);
+        memcpy(a->h_alpha, b->h_alpha, sizeof(double) * b->n * hw);
+        memcpy(a->Q, b->Q, sizeof(double) * dst->w * d);
+        memcpy(a->q_step, b->q_step, sizeof(int) * dst->w);
+    }
+    dst->t = src->t;
+    return rounds;
 }
 
 /*
@@ -339,10 +434,10 @@ int sho_compress(sho_t *o, int *evicted_pos) {
  * cache as it is now, restricted to the tokens that already existed at that
  * query's step (pos <= step: attention is causal), and compared with 1/step.
  * Tokens evicted since then are gone, so the scores are normalised over the
- * survivors.  alpha, low, amb: [U][w][B], row (step mod w); steps: [w] (0 = no query).
+ * survivors.  alpha, low, amb: [U][w][cap], row (step mod w); steps: [w] (0 = no query).
  */
 void sho_recount(const sho_t *o, double *alpha, uint8_t *low, uint8_t *amb, int *steps) {
-    const int B = o->B, d = o->d, w = o->w;
+    const int B = o->cap, d = o->d, w = o->w;
     for (int s = 0; s < w; ++s) {
         int st = o->unit[0].q_step[s];
         steps[s] = (st > 0 && (long)st > o->t - w && (long)st <= o->t) ? st : 0;
@@ -379,9 +474,9 @@ void sho_recount(const sho_t *o, double *alpha, uint8_t *low, uint8_t *amb, int 
 }
 
 /* Replace every live token's history by the given recomputed flags
- * ([U][w][B], row = step mod w, steps as returned by sho_recount). */
+ * ([U][w][cap], row = step mod w, steps as returned by sho_recount). */
 void sho_set_record(sho_t *o, const uint8_t *low, const int *steps) {
-    const int B = o->B, w = o->w;
+    const int B = o->cap, w = o->w, hw = o->hw;
 #pragma omp parallel for schedule(static)
     for (int u = 0; u < o->U; ++u) {
         unit_t *x = &o->unit[u];
@@ -391,9 +486,10 @@ void sho_set_record(sho_t *o, const uint8_t *low, const int *steps) {
                 if (st < 1) continue;
                 const int s = (int)(st % w);
                 if (steps[s] != (int)st || x->pos[j] > st) continue;
-                const int slot = x->h_cnt[j] % w;
-                x->h_step[(size_t)j * w + slot] = (int)st;
-                x->h_low[(size_t)j * w + slot] = low[((size_t)u * w + s) * B + j] ? 1 : 0;
+                const int slot = x->h_cnt[j] % hw;
+                x->h_step[(size_t)j * hw + slot] = (int)st;
+                x->h_low[(size_t)j * hw + slot] = low[((size_t)u * w + s) * B + j] ? 1 : 0;
+                x->h_alpha[(size_t)j * hw + slot] = low[((size_t)u * w + s) * B + j] ? 0.0 : 1.0;   /* only the flag is known */
                 x->h_cnt[j] += 1;
             }
         }

@@ -255,9 +255,9 @@ def _parse_golden(path):
 
 def test_selection_hand_worked_examples():
     cases = _parse_golden(os.path.join(GOLDEN, "select_micro_example.txt"))
-    assert len(cases) == 2
+    assert len(cases) == 3 and sum("tie" in c for c in cases) == 1
     for c in cases:
-        ev = oracle.select(c["I"], c["r"][0], c["m"][0])
+        ev = oracle.select(c["I"], c["r"][0], c["m"][0], newest_first=bool(c.get("tie", [0])[0]))
         assert (ev + 1).tolist() == c["dropped_positions"]
         kept = [p for p in range(1, len(c["I"]) + 1) if p not in set((ev + 1).tolist())]
         assert kept == c["kept_positions"]
@@ -444,3 +444,78 @@ def test_step_recompute_keeps_the_budget_and_full_attention_when_it_never_fills(
     for t in range(T):
         o2.step_recompute(q[t], k[t], v[t])
         assert o2.n < 10
+
+
+# --- alternative readings of the paper (oracle only) ------------------------------------------------
+@pytest.mark.parametrize("reading", [dict(threshold=1), dict(threshold=2), dict(window_plus1=True), dict(tie_newest=True),
+                                     dict(trigger_literal=True),
+                                     dict(threshold=1, window_plus1=True, tie_newest=True, trigger_literal=True)])
+@pytest.mark.parametrize("B,r,w,m", [(8, 2, 4, 3), (9, 3, 20, 1), (7, 1, 1, 6), (12, 4, 7, 2)])
+def test_alternative_readings_match_bruteforce(reading, B, r, w, m):
+    # Algorithm 2's fixed threshold 1/t of the compression step, the 1/n threshold, the w+1-step window,
+    # newest-first ties and Algorithm 1's literal "n > B" trigger, each against the brute force that
+    # evaluates the same reading from the full table of scores.
+    T, U, d = 45, 2, 4
+    q, k, v = _stream(T, U, d, 300 + B, peaked=3.0)
+    o = oracle.Oracle(U, B, r, w, m, d, **reading)
+    bf = [BruteForceUnit(B, r, w, m, d, 1 / math.sqrt(d), **reading) for _ in range(U)]
+    cap = B + (1 if reading.get("trigger_literal") else 0)
+    n_compress = 0
+    for t in range(T):
+        out, alpha, low, amb = o.attend(q[t], k[t], v[t])
+        o.record(low)
+        pos_before = o.positions()
+        assert o.n <= cap
+        dropped = o.compress()
+        for u in range(U):
+            bout, balpha, bdropped = bf[u].step(q[t, u], k[t, u], v[t, u])
+            np.testing.assert_allclose(out[u], bout, atol=1e-13)
+            np.testing.assert_allclose(alpha[u], [balpha[p] for p in pos_before[u]], atol=1e-14)
+            assert (dropped is None) == (bdropped is None)
+            if bdropped is not None:
+                assert dropped[u].tolist() == bdropped
+            assert o.positions()[u].tolist() == sorted(bf[u].live)
+            bI = bf[u].counters()
+            assert o.counters()[u].tolist() == [bI[p] for p in o.positions()[u]]
+        n_compress += dropped is not None
+        assert o.n < cap
+    assert n_compress >= 5
+
+
+@pytest.mark.parametrize("reading", [dict(), dict(tie_newest=True), dict(trigger_literal=True)])
+@pytest.mark.parametrize("p,B,r,w,m", [(30, 8, 2, 5, 3), (23, 12, 4, 40, 2), (9, 9, 3, 4, 1), (7, 9, 3, 4, 1)])
+def test_bulk_prompt_reading_matches_bruteforce(reading, p, B, r, w, m):
+    # Prompt cached in full (Section 2), record from its last w steps, then Algorithm 2 in rounds until the
+    # cache is under budget; generation continues from there.  Brute force: full attention over the
+    # prompt, one sort for the rounds, then its usual steps.
+    T, U, d = p + 25, 2, 4
+    q, k, v = _stream(T, U, d, 400 + p, peaked=3.0)
+    src = oracle.Oracle(U, p + 1, 0, w, 1, d, **{kk: vv for kk, vv in reading.items() if kk != "trigger_literal"})
+    bf = [BruteForceUnit(10 ** 6, r, w, m, d, 1 / math.sqrt(d), **reading) for _ in range(U)]
+    for t in range(p):
+        out, dropped = src.step(q[t], k[t], v[t])
+        assert dropped is None
+        for u in range(U):
+            bout, _, _ = bf[u].step(q[t, u], k[t, u], v[t, u])
+            np.testing.assert_allclose(out[u], bout, atol=1e-13)       # full causal attention over the prompt
+    dst = oracle.Oracle(U, B, r, w, m, d, **reading)
+    rounds = dst.import_compressed(src)
+    cap = B + (1 if reading.get("trigger_literal") else 0)
+    want_rounds = 0 if p < cap else (p - cap) // m + 1
+    assert rounds == want_rounds and dst.n == p - rounds * m < cap and dst.t == p
+    for u in range(U):
+        brounds, _gone = bf[u].shrink_below(B, m, r)
+        bf[u].B = B
+        assert brounds == rounds
+        assert dst.positions()[u].tolist() == sorted(bf[u].live)
+        bI = bf[u].counters()
+        assert dst.counters()[u].tolist() == [bI[pp] for pp in dst.positions()[u]]
+        if r:
+            assert set(range(p - min(r, dst.n) + 1, p + 1)) <= set(dst.positions()[u].tolist())
+    for t in range(p, T):                                               # generation goes on as usual
+        out, dropped = dst.step(q[t], k[t], v[t])
+        for u in range(U):
+            bout, _, bdropped = bf[u].step(q[t, u], k[t, u], v[t, u])
+            np.testing.assert_allclose(out[u], bout, atol=1e-13)
+            assert (dropped is None) == (bdropped is None)
+            assert dst.positions()[u].tolist() == sorted(bf[u].live)
