@@ -173,6 +173,32 @@ int sh_prefill(sh_handle h, const void *q_dev, const void *k_dev, const void *v_
                float *out_dev, void *stream);
 
 /*
+ * The prompting stage read as a bulk operation (Section 2: the prompt's keys and values are computed
+ * and cached in full before generation starts), as an alternative to the token stream of
+ * Definition 4.1 that sh_prefill implements.  `src` holds a cache that was never compressed (a handle
+ * whose budget exceeds the prompt, fed through sh_prefill: its outputs are full causal attention and
+ * its record holds the prompt's last w steps).  Algorithm 2 is applied to it as often as needed with
+ * dst's r and m - same record, m tokens per round, the r newest protected - until fewer than dst's
+ * B tokens remain; the survivors with their record, positions (and stored queries) become the cache
+ * of `dst`, which continues at t = src's t.  src is left compressed.
+ * dst must be bound and fresh (nothing streamed); both must agree in heads, head_dim, dtype, w and
+ * SH_OPT_RECORD_MODE, and neither may hold ragged sequences.  Asynchronous on `stream`.
+ * Errors: SH_EINVAL (mismatch, or fewer than m candidates outside the recent window), SH_ESTATE, SH_ECUDA.
+ */
+int sh_import_compressed(sh_handle dst, sh_handle src, void *stream);
+
+/*
+ * The same in one call for a fresh handle h: the p prompt tokens (layout as sh_prefill, 1 <= p <= 32767)
+ * are attended in full in a scratch workspace of sh_prefill_bulk_scratch_bytes(h, p) bytes (device
+ * memory, 256-byte aligned, the caller's; it holds the whole prompt's keys and values and may be freed
+ * or reused once `stream` has passed this call), then compressed into h as sh_import_compressed does.
+ * out_dev: [p][heads][head_dim] fp32 or NULL.
+ */
+int sh_prefill_bulk(sh_handle h, const void *q_dev, const void *k_dev, const void *v_dev, int p, float *out_dev,
+                    void *scratch_dev, size_t scratch_bytes, void *stream);
+size_t sh_prefill_bulk_scratch_bytes(sh_handle h, int p);
+
+/*
  * Prompts of different lengths (Section 4.1 treats one head of one sequence; a batch is many such
  * streams, and real batches are ragged).  The handle's units are n_sequences groups of
  * heads / n_sequences consecutive units; sequence i consumes the first lengths_host[i] <= p_max

@@ -32,7 +32,8 @@ EXPORTS = ["sh_create", "sh_destroy", "sh_workspace_bytes", "sh_bind", "sh_set_o
            "sh_decode_step_host", "sh_prefill", "sh_prefill_chunk", "sh_prefill_chunk_max", "sh_export_record", "sh_recompute_record", "sh_prefill_ragged",
            "sh_sequence_state",
            "sh_compress", "sh_compress_static", "sh_scores", "sh_select", "sh_state", "sh_export_unit",
-           "sh_restore", "sh_launch_count", "sh_decode_kernel_choice", "sh_strerror", "sh_last_cuda_error"]
+           "sh_restore", "sh_launch_count", "sh_decode_kernel_choice", "sh_import_compressed", "sh_prefill_bulk",
+           "sh_prefill_bulk_scratch_bytes", "sh_strerror", "sh_last_cuda_error"]
 
 
 def _load() -> C.CDLL:
@@ -71,6 +72,10 @@ def _load() -> C.CDLL:
     lib.sh_launch_count.argtypes = [vp]
     lib.sh_launch_count.restype = C.c_longlong
     lib.sh_decode_kernel_choice.argtypes = [vp]
+    lib.sh_import_compressed.argtypes = [vp, vp, vp]
+    lib.sh_prefill_bulk.argtypes = [vp, vp, vp, vp, C.c_int, vp, vp, C.c_size_t, vp]
+    lib.sh_prefill_bulk_scratch_bytes.argtypes = [vp, C.c_int]
+    lib.sh_prefill_bulk_scratch_bytes.restype = C.c_size_t
     lib.sh_strerror.argtypes = [C.c_int]
     lib.sh_strerror.restype = C.c_char_p
     lib.sh_last_cuda_error.argtypes = [vp]
@@ -192,6 +197,26 @@ class Handle:
         optr = _dev(out, torch.float32, n, "out") if out is not None else None
         self._check(lib.sh_prefill(self._h, _dev(q, self.in_dtype, n, "q"), _dev(k, self.in_dtype, n, "k"),
                                    _dev(v, self.in_dtype, n, "v"), p, optr, _stream_ptr(stream)))
+        return out
+
+    # -- sh_import_compressed / sh_prefill_bulk -------------------------------------
+    def import_compressed(self, src: "Handle", stream=None):
+        self._check(lib.sh_import_compressed(self._h, src._h, _stream_ptr(stream)))
+
+    def prefill_bulk(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: Optional[torch.Tensor] = None,
+                     stream=None):
+        p = q.shape[0]
+        n = p * self.U * self.D
+        need = int(lib.sh_prefill_bulk_scratch_bytes(self._h, p))
+        if not need:
+            raise ShError(SH_EINVAL, "prompt length outside 1..32767")
+        with torch.cuda.device(self.device):
+            scratch = torch.empty(need + 256, dtype=torch.uint8, device=self.device)
+        sptr = scratch.data_ptr() + (-scratch.data_ptr()) % 256
+        optr = _dev(out, torch.float32, n, "out") if out is not None else None
+        self._check(lib.sh_prefill_bulk(self._h, _dev(q, self.in_dtype, n, "q"), _dev(k, self.in_dtype, n, "k"),
+                                        _dev(v, self.in_dtype, n, "v"), p, optr, sptr, need, _stream_ptr(stream)))
+        scratch.record_stream(stream or torch.cuda.current_stream())
         return out
 
     # -- sh_prefill_ragged / sh_sequence_state -----------------------------------

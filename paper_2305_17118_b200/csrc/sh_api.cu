@@ -89,7 +89,10 @@ __global__ void sh_fill_counts_kernel(int *n_arr, int *t_arr, int count, int n, 
     if (i < count) { n_arr[i] = n; t_arr[i] = t; }
 }
 
-int do_compress(sh_context *c, cudaStream_t s) {
+// Algorithm 2 on every unit of the active range holding n live rows each: the r newest are protected, m go.
+// The handle's own compression is (B, r, m) of its creation; a prompt cached in full is brought under
+// another handle's budget with that handle's r and m (sh_import_compressed).
+int do_compress_at(sh_context *c, cudaStream_t s, int n, int r, int m, bool own) {
     int rrc = sh_recount_if_needed(c, s);
     if (rrc != SH_OK) return rrc;
     SelectParams sp = {};
@@ -97,7 +100,7 @@ int do_compress(sh_context *c, cudaStream_t s) {
     sp.counters = nullptr;
     sp.src_idx = sh_psrc(c);
     sp.evicted = nullptr;
-    sp.U = c->ucount; sp.B = c->B; sp.Bw = c->Bw; sp.w = c->w; sp.n = c->B; sp.r = c->r; sp.m = c->m;
+    sp.U = c->ucount; sp.B = c->B; sp.Bw = c->Bw; sp.w = c->w; sp.n = n; sp.r = r; sp.m = m;
     sp.cmax = c->w;
     sp.n_arr = sh_pnarr(c);
     sp.unordered = c->unordered;
@@ -111,7 +114,7 @@ int do_compress(sh_context *c, cudaStream_t s) {
     cp.hist = sh_phist(c);
     cp.pos = sh_ppos(c);
     cp.src_idx = sp.src_idx;
-    cp.U = c->ucount; cp.B = c->B; cp.Bw = c->Bw; cp.w = c->w; cp.n = c->B; cp.m = c->m;
+    cp.U = c->ucount; cp.B = c->B; cp.Bw = c->Bw; cp.w = c->w; cp.n = n; cp.m = m;
     cp.row_bytes = c->row_bytes;
     cp.scale_bytes = c->dtype == SH_INT4_G64_F16 ? (c->D / 64) * 2 : 0;
     cp.Bs = c->Bs;
@@ -127,8 +130,55 @@ int do_compress(sh_context *c, cudaStream_t s) {
         if (e == cudaSuccess) e = sh_launch_compact(cp, s, &c->launches);
     }
     if (e != cudaSuccess) return cuda_fail(c, e);
-    sh_after_compression(c);
+    if (own) sh_after_compression(c);
+    else c->n -= m;
     return SH_OK;
+}
+
+int do_compress(sh_context *c, cudaStream_t s) { return do_compress_at(c, s, c->B, c->r, c->m, true); }
+
+// Rows [0, n) of every unit's K, V, scales, positions, bit-planes and (if kept) query ring, from one
+// workspace layout to another (the budgets, hence the strides, differ).  One CTA per unit.
+struct RepackParams {
+    const char *sK, *sV, *sKs, *sVs, *sq;
+    const uint32_t *shist;
+    const int32_t *spos;
+    char *dK, *dV, *dKs, *dVs, *dq;
+    uint32_t *dhist;
+    int32_t *dpos;
+    int n, w, row_bytes, scale_bytes, in_bytes;
+    int sB, dB, sBw, dBw, sBs, dBs;
+};
+
+__global__ void __launch_bounds__(256) sh_repack_kernel(const RepackParams p) {
+    const size_t u = blockIdx.x;
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int pieces = p.n * (p.row_bytes / 16);
+    const uint4 *sk = reinterpret_cast<const uint4 *>(p.sK + u * p.sB * p.row_bytes);
+    const uint4 *sv = reinterpret_cast<const uint4 *>(p.sV + u * p.sB * p.row_bytes);
+    uint4 *dk = reinterpret_cast<uint4 *>(p.dK + u * p.dB * p.row_bytes);
+    uint4 *dv = reinterpret_cast<uint4 *>(p.dV + u * p.dB * p.row_bytes);
+    for (int i = tid; i < pieces; i += nt) { dk[i] = sk[i]; dv[i] = sv[i]; }
+    if (p.scale_bytes) {
+        const int cnt = p.n * (p.scale_bytes / 2);
+        const uint16_t *a = reinterpret_cast<const uint16_t *>(p.sKs + u * p.sBs * p.scale_bytes);
+        const uint16_t *b = reinterpret_cast<const uint16_t *>(p.sVs + u * p.sBs * p.scale_bytes);
+        uint16_t *c = reinterpret_cast<uint16_t *>(p.dKs + u * p.dBs * p.scale_bytes);
+        uint16_t *d = reinterpret_cast<uint16_t *>(p.dVs + u * p.dBs * p.scale_bytes);
+        for (int i = tid; i < cnt; i += nt) { c[i] = a[i]; d[i] = b[i]; }
+    }
+    for (int i = tid; i < p.n; i += nt) p.dpos[u * p.dB + i] = p.spos[u * p.sB + i];
+    const int words = p.sBw < p.dBw ? p.sBw : p.dBw;
+    for (int i = tid; i < p.w * words; i += nt) {
+        const int row = i / words, k = i - row * words;
+        p.dhist[(u * p.w + row) * p.dBw + k] = p.shist[(u * p.w + row) * p.sBw + k];
+    }
+    if (p.sq && p.dq) {
+        const int qp = p.w * (p.in_bytes / 16);
+        const uint4 *a = reinterpret_cast<const uint4 *>(p.sq + u * p.w * p.in_bytes);
+        uint4 *b = reinterpret_cast<uint4 *>(p.dq + u * p.w * p.in_bytes);
+        for (int i = tid; i < qp; i += nt) b[i] = a[i];
+    }
 }
 
 }  // namespace
@@ -440,6 +490,80 @@ int sh_prefill(sh_handle h, const void *q_dev, const void *k_dev, const void *v_
     if (h->t + p >= (1 << 24)) return SH_EINVAL;
     return prefill_range(h, static_cast<const char *>(q_dev), static_cast<const char *>(k_dev),
                          static_cast<const char *>(v_dev), p, out_dev, (cudaStream_t)stream);
+}
+
+int sh_import_compressed(sh_handle dst, sh_handle src, void *stream) {
+    if (!dst || !src || dst == src) return SH_EINVAL;
+    if (!dst->slab || !src->slab) return SH_ESTATE;
+    if (dst->started || dst->t != 0 || dst->n != 0 || dst->ragged || src->ragged) return SH_ESTATE;
+    if (dst->U != src->U || dst->D != src->D || dst->dtype != src->dtype || dst->w != src->w ||
+        dst->record_mode != src->record_mode)
+        return SH_EINVAL;
+    cudaStream_t s = (cudaStream_t)stream;
+    // Algorithm 2 on the record as it stands, as often as needed: fewer than dst->B tokens must remain
+    while (src->n >= dst->B) {
+        if (src->n - dst->r < dst->m) return SH_EINVAL;
+        const int rc = do_compress_at(src, s, src->n, dst->r, dst->m, false);
+        if (rc != SH_OK) return rc;
+    }
+    RepackParams rp = {};
+    rp.sK = sh_pK(src); rp.sV = sh_pV(src); rp.sKs = sh_pKs(src); rp.sVs = sh_pVs(src); rp.sq = sh_pqring(src);
+    rp.shist = sh_phist(src); rp.spos = sh_ppos(src);
+    rp.dK = sh_pK(dst); rp.dV = sh_pV(dst); rp.dKs = sh_pKs(dst); rp.dVs = sh_pVs(dst); rp.dq = sh_pqring(dst);
+    rp.dhist = sh_phist(dst); rp.dpos = sh_ppos(dst);
+    rp.n = src->n; rp.w = src->w; rp.row_bytes = src->row_bytes;
+    rp.scale_bytes = src->dtype == SH_INT4_G64_F16 ? (src->D / 64) * 2 : 0;
+    rp.in_bytes = src->in_bytes;
+    rp.sB = src->B; rp.dB = dst->B; rp.sBw = src->Bw; rp.dBw = dst->Bw; rp.sBs = src->Bs; rp.dBs = dst->Bs;
+    if (rp.n > 0) {
+        sh_repack_kernel<<<dst->U, 256, 0, s>>>(rp);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(dst, e);
+        dst->launches += 1;
+    }
+    dst->n = src->n;
+    dst->t = src->t;
+    dst->started = true;
+    dst->record_fresh_t = -1;
+    return SH_OK;
+}
+
+// A context for the whole prompt: budget p + 1 (never fills), the options of h that shape the kernels.
+static sh_context *bulk_context(const sh_context *h, int p) {
+    sh_handle t = nullptr;
+    if (sh_create(p + 1, 0, h->w, 1, h->U, h->D, h->dtype, &t) != SH_OK) return nullptr;
+    t->scale = h->scale;
+    t->kernel = h->kernel;
+    t->prefill_chunk = h->prefill_chunk;
+    t->unordered = h->unordered;
+    if (h->split_explicit) { t->split = h->split; t->split_explicit = true; }
+    if (h->record_mode && sh_set_option(t, SH_OPT_RECORD_MODE, 1.0) != SH_OK) { sh_destroy(t); return nullptr; }
+    return t;
+}
+
+size_t sh_prefill_bulk_scratch_bytes(sh_handle h, int p) {
+    if (!h || p < 1 || p > 32767) return 0;
+    sh_context *t = bulk_context(h, p);
+    if (!t) return 0;
+    const size_t bytes = t->L.total;
+    sh_destroy(t);
+    return bytes;
+}
+
+int sh_prefill_bulk(sh_handle h, const void *q_dev, const void *k_dev, const void *v_dev, int p, float *out_dev,
+                    void *scratch_dev, size_t scratch_bytes, void *stream) {
+    if (!h || !q_dev || !k_dev || !v_dev || !scratch_dev || p < 1 || p > 32767) return SH_EINVAL;
+    if (!h->slab) return SH_ESTATE;
+    if (h->started || h->t != 0 || h->ragged) return SH_ESTATE;
+    sh_context *t = bulk_context(h, p);
+    if (!t) return SH_EINVAL;
+    int rc = sh_bind(t, scratch_dev, scratch_bytes, stream);
+    if (rc == SH_OK) rc = sh_prefill(t, q_dev, k_dev, v_dev, p, out_dev, stream);
+    if (rc == SH_OK) rc = sh_import_compressed(h, t, stream);
+    if (rc == SH_ECUDA) h->last_err = t->last_err != cudaSuccess ? t->last_err : h->last_err;
+    h->launches += t->launches;
+    sh_destroy(t);
+    return rc;
 }
 
 int sh_prefill_ragged(sh_handle h, const void *q_dev, const void *k_dev, const void *v_dev, int p_max,

@@ -902,3 +902,50 @@ def test_record_mode_overlap_diagnostic(sh):
     want = np.array([len(np.intersect1d(pa[u], pb[u])) for u in range(U)]) / o_a.n
     assert got.n == o_a.n == o_b.n and np.abs(got.overlap - want).max() < 1e-12
     assert (got.overlap >= r / got.n - 1e-12).all() and (got.overlap <= 1).all()
+
+
+@pytest.mark.parametrize("dtype,d,stable", [("f16", 128, False), ("bf16", 128, True), ("int4", 128, False), ("f32", 64, False)])
+@pytest.mark.parametrize("p,B,r,w,m", [(300, 96, 8, 40, 30), (150, 150, 9, 37, 41), (90, 120, 4, 16, 20), (700, 130, 10, 200, 1)])
+def test_bulk_prompt_reading_lockstep(sh, dtype, d, stable, p, B, r, w, m):
+    """The prompting stage read as a bulk operation (sh_import_compressed / sh_prefill_bulk): the prompt is
+    attended in full on a handle that never compresses, in lockstep with an oracle of the same budget;
+    both sides then bring that cache under the real budget by rounds of Algorithm 2 on the record as it
+    stands, and must hold the same tokens, records and rows; generation continues in lockstep.  The
+    one-call form must end bit-identical to the composed one."""
+    if m == 1 and dtype != "f16":
+        pytest.skip("570 rounds of one token: one storage type is enough")
+    U, T_dec = 4, 80
+    q, k, v = wl.random_stream(U, d, p + T_dec, seed=111 + p, dtype=dtype, peaked=3.0, device="cuda")
+    kw = dict(auto_compress=False, unordered=not stable)
+    src = sh.Handle(p + 1, 0, w, 1, U, d, dtype, **kw)
+    o_src = oracle.Oracle(U, p + 1, 0, w, 1, d, quant=(dtype == "int4"))
+    blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
+    outs = []
+    if src.prefill_chunk_max >= 2:
+        run_lockstep_chunked(src, dtype, blk, p, torch.arange(U), TOL[dtype], orc=o_src, outs=outs, single_via_step=True)
+    else:
+        run_lockstep(src, dtype, _stream_fn(q, k, v), p, torch.arange(U), TOL[dtype], orc=o_src, outs=outs)
+        outs = [x[None] for x in outs]
+    dst = sh.Handle(B, r, w, m, U, d, dtype, **kw)
+    dst.import_compressed(src)
+    o_dst = oracle.Oracle(U, B, r, w, m, d, quant=(dtype == "int4"))
+    rounds = o_dst.import_compressed(o_src)
+    assert rounds == (0 if p < B else (p - B) // m + 1)
+    view = SortedView(dst)
+    n, t, pos, cnt, _ = view.state(low=False)
+    assert n == o_dst.n == p - rounds * m and t == o_dst.t == p
+    assert (pos == o_dst.positions()).all() and (cnt.astype(np.int32) == o_dst.counters()).all()
+    for u in range(U):
+        K, V = view.export_unit(u)
+        oK, oV = o_dst.cache(u)
+        assert (K[:n].astype(np.float64) == oK).all() and (V[:n].astype(np.float64) == oV).all()
+    one = sh.Handle(B, r, w, m, U, d, dtype, **kw)
+    out1 = torch.empty(p, U, d, device="cuda")
+    one.prefill_bulk(q[:p].contiguous(), k[:p].contiguous(), v[:p].contiguous(), out1)
+    assert torch.equal(out1, torch.cat(outs))
+    sa, sb = one.state(), dst.state()
+    assert sa[0] == sb[0] and sa[1] == sb[1] and all((x == y).all() for x, y in zip(sa[2:], sb[2:]))
+    res, _ = run_lockstep(dst, dtype, lambda tt: (q[tt - 1], k[tt - 1], v[tt - 1]), T_dec, torch.arange(U), TOL[dtype], orc=o_dst)
+    assert res.steps == T_dec
+    with pytest.raises(sh.ShError):
+        dst.import_compressed(src)                     # the target must be fresh
