@@ -75,9 +75,9 @@ typedef enum {
                                  token per step; 1: it is recomputed at every compression from the queries of
                                  the last w steps (the library keeps them: heads*w*head_dim extra elements)
                                  scored against the cache as it is then (Algorithm 2 as stated; Section 4.1,
-                                 "Overhead Tradeoff").  fp16/bf16/int4, head_dim 128 (with SH_OPT_PREFILL_CHUNK = 2:
-                                 fp16/bf16 and budgets up to about 700 only); else SH_EINVAL.  Set before sh_bind:
-                                 it changes sh_workspace_bytes. */
+                                 "Overhead Tradeoff").  Every storage type and head size (with
+                                 SH_OPT_PREFILL_CHUNK = 2: fp16/bf16, head_dim 128 and budgets up to about 700
+                                 only, else SH_EINVAL).  Set before sh_bind: it changes sh_workspace_bytes. */
     SH_OPT_COMPACTION = 6,    /* 1 (default): every hole left by a dropped token below n-m is filled with a kept
                                  row from the tail, so at most m rows move per compression; slots are then in no
                                  particular order: sh_state's pos tells which token sits where.
@@ -85,10 +85,12 @@ typedef enum {
                                  surviving row moves: about three times the time per compression at B = 410,
                                  m = 64).  The kept set is the same either way: nothing in Algorithm 2 depends
                                  on where a token is stored. */
-    SH_OPT_PREFILL_CHUNK = 4, /* 1 (default): sh_prefill hands the tokens between two compressions to the chunk
-                                 kernel where the shape allows it (fp16/bf16/int4 with head_dim 128: the tcgen05
-                                 kernels, any budget); 0: one decode step per token; 2: the warp-level MMA chunk kernel
-                                 (fp16/bf16, budgets up to about 700); 3: same as 1 */
+    SH_OPT_PREFILL_CHUNK = 4, /* 1 (default): sh_prefill hands the tokens between two compressions to a chunk
+                                 kernel: the tcgen05 kernels for fp16/bf16/int4 with head_dim 128 (any budget),
+                                 the CUDA-core kernel for fp32 rows and for head_dim 64; 0: one decode step per
+                                 token; 2: the warp-level MMA chunk kernel where it applies (fp16/bf16, head_dim
+                                 128, budgets up to about 700); 3: same as 1; 4: the CUDA-core kernel for every
+                                 shape */
     SH_OPT_DECODE_KERNEL = 3, /* 0 (default): chosen from the shape; 1: one CTA (or cluster) per unit with
                                  direct loads; 2: persistent CTAs fed by bulk asynchronous copies
                                  (stored rows of 256 bytes or more: fp32, and fp16/bf16 with head_dim 128; SH_OPT_SPLIT
@@ -162,11 +164,12 @@ int sh_decode_step_host(sh_handle h, const void *q_host, const void *k_new_host,
  * sh_decode_step (each followed by a compression when the cache fills),
  * whatever SH_OPT_AUTO_COMPRESS says.  q_dev, k_dev, v_dev: time-major
  * [p][heads][head_dim].  out_dev: [p][heads][head_dim] fp32 or NULL to discard.
- * Between two compressions the steps only append, so for fp16, bf16 and int4 stores
- * with head_dim 128 they are evaluated up to 64 at a time by a tensor-core kernel
- * (causal attention of the chunk over the cache and itself, one record
- * bit-plane row per step); the results equal the per-token path up to fp32
- * summation order.  SH_OPT_PREFILL_CHUNK = 0 forces the per-token path.
+ * Between two compressions the steps only append, so they are evaluated up to
+ * 64 at a time by a chunk kernel (causal attention of the chunk over the cache
+ * and itself, one record bit-plane row per step: on the tensor cores for fp16,
+ * bf16 and int4 stores with head_dim 128, on CUDA cores otherwise); the results
+ * equal the per-token path up to fp32 summation order.  SH_OPT_PREFILL_CHUNK = 0
+ * forces the per-token path.
  * At most 2^24 - 1 tokens may be streamed through a handle.
  */
 int sh_prefill(sh_handle h, const void *q_dev, const void *k_dev, const void *v_dev, int p,
@@ -223,7 +226,7 @@ int sh_sequence_state(sh_handle h, int *n_host, long long *t_host, int capacity)
  * One chunk of the prompt without the compression: steps t+1 .. t+count for
  * every unit in one launch (see sh_prefill).  Needs 1 <= count <=
  * sh_prefill_chunk_max(h) and count <= B - n; returns SH_EINVAL otherwise
- * (sh_prefill_chunk_max is 0 when the handle's dtype or shape is not served).
+ * (sh_prefill_chunk_max is min(64, w), or 0 where SH_OPT_PREFILL_CHUNK = 2 does not apply).
  * Layout as sh_prefill.  The caller compresses when n reaches B.
  */
 int sh_prefill_chunk(sh_handle h, const void *q_dev, const void *k_dev, const void *v_dev, int count,

@@ -170,6 +170,11 @@ cudaError_t sh_launch_recount_umma(const ChunkParams &p, int dtype, cudaStream_t
 cudaError_t sh_launch_chunk_umma_int4(const ChunkParams &p, cudaStream_t s);
 cudaError_t sh_launch_recount_umma_int4(const ChunkParams &p, cudaStream_t s);
 
+// CUDA-core chunk kernel: every storage type and head size (sh_chunk_simt.cu).
+int sh_chunk_simt_capacity();
+cudaError_t sh_launch_chunk_simt(const ChunkParams &p, int dtype, int D, cudaStream_t s);
+cudaError_t sh_launch_recount_simt(const ChunkParams &p, int dtype, int D, cudaStream_t s);
+
 // Launchers (each returns the cudaError_t of its launch and adds to *launches).
 cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches);
 // Scores of a query over the present caches (analysis; p.n = live rows, nothing appended).

@@ -331,8 +331,12 @@ size_t smem_need(int CQ, int B) {
 }  // namespace
 
 // Largest number of tokens one chunk launch can take for this handle (0: not supported).
+// Does the CUDA-core chunk kernel serve this handle?  It takes what the tensor-core kernels do not (fp32 rows,
+// head_dim 64), and everything when SH_OPT_PREFILL_CHUNK = 4 asks for it.
+static bool use_simt(const sh_context *c) { return c->prefill_chunk == 4 || c->D != 128 || c->dtype == SH_F32; }
+
 int sh_prefill_chunk_capacity(const sh_context *c) {
-    if (c->D != 128) return 0;
+    if (use_simt(c)) return sh_chunk_simt_capacity() < c->w ? sh_chunk_simt_capacity() : c->w;
     if (c->dtype == SH_INT4_G64_F16) {       // int4 store: the tcgen05 kernel only
         if (c->prefill_chunk == 2) return 0;
         return sh_chunk_umma_capacity() < c->w ? sh_chunk_umma_capacity() : c->w;
@@ -348,7 +352,7 @@ int sh_prefill_chunk_capacity(const sh_context *c) {
 // The recount (record recomputed at compression time): any budget on the tcgen05 kernel; the warp-level
 // kernel keeps a whole row of logits in shared memory (budgets up to about 700).
 bool sh_recount_supported(const sh_context *c) {
-    if (c->D != 128) return false;
+    if (use_simt(c)) return true;
     if (c->dtype == SH_INT4_G64_F16) return c->prefill_chunk != 2;      // int4 store: the tcgen05 kernel only
     if (c->dtype != SH_F16 && c->dtype != SH_BF16) return false;
     return c->prefill_chunk != 2 || smem_need(32, c->B) <= 200 * 1024;
@@ -372,6 +376,11 @@ cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const vo
     p.err = reinterpret_cast<int *>(c->slab + c->L.err);
     cudaError_t e = cudaErrorInvalidValue;
     if (count < 1 || count > sh_prefill_chunk_capacity(c)) return e;
+    if (use_simt(c)) {
+        e = sh_launch_chunk_simt(p, c->dtype, c->D, s);
+        if (e == cudaSuccess) *launches += 1;
+        return e;
+    }
     if (c->dtype == SH_INT4_G64_F16) {
         e = sh_launch_chunk_umma_int4(p, s);
         if (e == cudaSuccess) *launches += 1;
@@ -411,6 +420,11 @@ cudaError_t sh_launch_recount(const sh_context *c, cudaStream_t s, long long *la
     p.err = reinterpret_cast<int *>(c->slab + c->L.err);
     p.Ks = sh_pKs(c); p.Vs = sh_pVs(c); p.Bs = c->Bs;
     cudaError_t e;
+    if (use_simt(c)) {
+        e = sh_launch_recount_simt(p, c->dtype, c->D, s);
+        if (e == cudaSuccess) *launches += 1;
+        return e;
+    }
     if (c->dtype == SH_INT4_G64_F16) {
         e = sh_launch_recount_umma_int4(p, s);
         if (e == cudaSuccess) *launches += 1;

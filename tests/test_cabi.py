@@ -68,7 +68,7 @@ def test_option_values_and_the_shapes_they_need():
     lib = sh.lib
     h = _handle(sh, 410, 64, 128, 64, 16, 128, "f16")
     assert lib.sh_prefill_chunk_max(h) == 64
-    for key, good, bad in ((sh.SH_OPT_COMPACTION, (0, 1), (2, -1)), (sh.SH_OPT_PREFILL_CHUNK, (0, 1, 2, 3), (4, -1)),
+    for key, good, bad in ((sh.SH_OPT_COMPACTION, (0, 1), (2, -1)), (sh.SH_OPT_PREFILL_CHUNK, (0, 1, 2, 3, 4, 1), (5, -1)),
                            (sh.SH_OPT_DECODE_KERNEL, (0, 1, 2), (3,)), (sh.SH_OPT_SPLIT, (1, 2, 4, 8), (3, 16))):
         for v in good:
             assert lib.sh_set_option(h, key, float(v)) == sh.SH_OK, (key, v)
@@ -78,15 +78,19 @@ def test_option_values_and_the_shapes_they_need():
     assert lib.sh_set_option(h, sh.SH_OPT_RECORD_MODE, 1.0) == sh.SH_OK
     assert lib.sh_workspace_bytes(h) >= before + 16 * 128 * 128 * 2          # the ring of the last w queries
     lib.sh_destroy(h)
-    # a window shorter than a chunk bounds the chunk; int4 and head_dim 64 have no chunk kernel
+    # a window shorter than a chunk bounds the chunk; every storage type and head size has a chunk kernel
+    # and the recompute mode (fp32 rows and head_dim 64 on CUDA cores)
     h = _handle(sh, 150, 9, 37, 41, 3, 128, "bf16")
     assert lib.sh_prefill_chunk_max(h) == 37
     lib.sh_destroy(h)
-    for dtype, d in (("int4", 64), ("f16", 64), ("f32", 128)):
-        h = _handle(sh, 150, 9, 37, 41, 3, d, dtype)
-        assert lib.sh_prefill_chunk_max(h) == 0
-        assert lib.sh_set_option(h, sh.SH_OPT_RECORD_MODE, 1.0) == sh.SH_EINVAL
-        lib.sh_destroy(h)
+    for dtype in ("f32", "f16", "bf16", "int4"):
+        for d in (64, 128):
+            h = _handle(sh, 410, 64, 128, 64, 3, d, dtype)
+            assert lib.sh_prefill_chunk_max(h) == 64, (dtype, d)
+            assert lib.sh_set_option(h, sh.SH_OPT_PREFILL_CHUNK, 4.0) == sh.SH_OK
+            assert lib.sh_prefill_chunk_max(h) == 64
+            assert lib.sh_set_option(h, sh.SH_OPT_RECORD_MODE, 1.0) == sh.SH_OK, (dtype, d)
+            lib.sh_destroy(h)
     # the int4 store with head_dim 128 has a chunk kernel and a recompute mode, on the tcgen05 kernel only
     h = _handle(sh, 150, 9, 37, 41, 3, 128, "int4")
     assert lib.sh_prefill_chunk_max(h) == 37

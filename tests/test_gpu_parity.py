@@ -949,3 +949,61 @@ def test_bulk_prompt_reading_lockstep(sh, dtype, d, stable, p, B, r, w, m):
     assert res.steps == T_dec
     with pytest.raises(sh.ShError):
         dst.import_compressed(src)                     # the target must be fresh
+
+
+_SIMT_SHAPES = [("f32", 64, None), ("f32", 128, None), ("f16", 64, None), ("bf16", 64, None), ("int4", 64, None),
+                ("f16", 128, 4), ("bf16", 128, 4), ("int4", 128, 4)]
+
+
+@pytest.mark.parametrize("dtype,d,mode", _SIMT_SHAPES)
+@pytest.mark.parametrize("U,B,r,w,m,sizes", [(5, 150, 9, 37, 41, [64, 7, 33, 1, 50]), (3, 410, 64, 128, 64, [64]),
+                                             (130, 96, 8, 70, 30, [64, 31]), (2, 1300, 10, 64, 650, [64, 13]),
+                                             (4, 40, 3, 9, 20, [5, 9, 2])])
+def test_lockstep_chunked_cuda_core_kernel(sh, dtype, d, mode, U, B, r, w, m, sizes):
+    """The CUDA-core chunk kernel: the storage types and head sizes the tensor-core kernels do not take
+    (fp32 rows, head_dim 64), and the others when forced (SH_OPT_PREFILL_CHUNK = 4).  Every step's output,
+    record bits, positions, counters and kept sets against the oracle; int4 rows bit-identical; then
+    decode steps from the state the chunks left."""
+    T = min(2 * B + 2 * m + 11, B + 2 * m + 60)
+    q, k, v = wl.random_stream(U, d, T + 30, seed=47 + U, dtype=dtype, peaked=3.0, device="cuda")
+    h = SortedView(sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, prefill_chunk=mode))
+    assert h.prefill_chunk_max == min(64, w)
+    blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
+    res, orc = run_lockstep_chunked(h, dtype, blk, T, torch.arange(U), TOL[dtype], chunk_sizes=sizes)
+    assert res.steps == T and res.compressions >= 2
+    assert res.adoptions <= 1e-4 * res.slot_steps + 2
+    if dtype == "int4":
+        n = h.n
+        for u in (0, U - 1):
+            K, V = h.export_unit(u)
+            oK, oV = orc.cache(u)
+            assert (K[:n].astype(np.float64) == oK).all() and (V[:n].astype(np.float64) == oV).all()
+    run_lockstep(h, dtype, _stream_fn(q, k, v), 30, torch.arange(U), TOL[dtype], orc=orc)
+
+
+@pytest.mark.parametrize("dtype,d,mode", _SIMT_SHAPES)
+@pytest.mark.parametrize("U,B,r,w,m", [(5, 150, 9, 37, 41), (3, 410, 64, 128, 64), (140, 96, 8, 70, 30), (2, 300, 10, 200, 150)])
+@pytest.mark.parametrize("stable", [False, True])
+def test_lockstep_record_recomputed_cuda_core_kernel(sh, dtype, d, mode, U, B, r, w, m, stable):
+    """SH_OPT_RECORD_MODE = 1 (Algorithm 2 as stated) on every storage type and head size: the recount runs
+    on the CUDA-core kernel (w beyond 64: several CTAs per unit), visibility by position in both compaction modes."""
+    T = min(2 * B + 3 * m + 5, B + 2 * m + 30)
+    q, k, v = wl.random_stream(U, d, T, seed=53 + U, dtype=dtype, peaked=3.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, recompute_record=True, prefill_chunk=mode, unordered=not stable)
+    res, orc = run_lockstep_recompute(h, dtype, _stream_fn(q, k, v), T, torch.arange(U), TOL[dtype])
+    assert res.compressions >= 2
+    assert res.adoptions <= 1e-4 * res.slot_steps + 2
+
+
+@pytest.mark.parametrize("recompute", [False, True])
+def test_config_tiny_chunked_prompt_and_both_record_modes(sh, recompute):
+    """The fp32, head_dim 64 workload with its prompt through the chunk kernel, and Algorithm 2 as stated."""
+    cfg = wl.CONFIGS["tiny"]
+    st = wl.Stream(cfg, device="cuda")
+    h = sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, cfg.units, cfg.head_dim, cfg.dtype, auto_compress=False, recompute_record=recompute)
+    res, orc = run_lockstep_chunked(h, cfg.dtype, st.block, cfg.prompt, torch.arange(cfg.units), TOL[cfg.dtype],
+                                    recompute=recompute, single_via_step=True)
+    assert res.steps == cfg.prompt
+    run = run_lockstep_recompute if recompute else run_lockstep
+    res2, _ = run(h, cfg.dtype, st.step, cfg.decode, torch.arange(cfg.units), TOL[cfg.dtype], orc=orc)
+    assert res2.compressions == 13

@@ -26,7 +26,7 @@ def _draw(rng):
     unordered = rng.random() < 0.5
     kernel = rng.choice([None, None, 1, 2])
     mode = rng.choice(["decode", "decode", "chunk", "recompute"])
-    if mode in ("chunk", "recompute") and (d != 128 or dtype == "f32" or w < 2):
+    if mode in ("chunk", "recompute") and w < 2:
         mode = "decode"
     return dtype, d, U, B, r, w, m, unordered, kernel, mode
 
