@@ -255,14 +255,14 @@ __global__ void __launch_bounds__(NT, 2) sh_chunk_simt_kernel(const ChunkParams 
             float mx = fmaxf(fmaxf(s[a][0], s[a][1]), fmaxf(s[a][2], s[a][3]));
 #pragma unroll
             for (int o = 8; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            // (no branch around the shuffles: the two query rows of a warp may differ in what they see)
             const float m_new = fmaxf(m_run[a], mx);
-            if (m_new != -INFINITY) {
-                float sum = ex2a(s[a][0] - m_new) + ex2a(s[a][1] - m_new) + ex2a(s[a][2] - m_new) + ex2a(s[a][3] - m_new);
+            const float ref = m_new == -INFINITY ? 0.f : m_new;      // nothing visible yet: every term below is 2^(-inf) = 0
+            float sum = ex2a(s[a][0] - ref) + ex2a(s[a][1] - ref) + ex2a(s[a][2] - ref) + ex2a(s[a][3] - ref);
 #pragma unroll
-                for (int o = 8; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-                l_run[a] = l_run[a] * ex2a(m_run[a] - m_new) + sum;      // 2^(-inf) = 0 on the first tile
-                m_run[a] = m_new;
-            }
+            for (int o = 8; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            l_run[a] = l_run[a] * ex2a(m_run[a] - ref) + sum;
+            m_run[a] = m_new;
         }
         __syncthreads();      // tile consumed
     }
