@@ -218,15 +218,28 @@ __global__ void __launch_bounds__(NT, 2) sh_chunk_simt_kernel(const ChunkParams 
         for (int a = 0; a < 4; ++a)
 #pragma unroll
             for (int b = 0; b < 4; ++b) s[a][b] = 0.f;
-#pragma unroll 8
-        for (int i = 0; i < D; ++i) {
-            const float4 q4 = *reinterpret_cast<const float4 *>(Qt + i * TS + 4 * ty);
-            const float4 k4 = *reinterpret_cast<const float4 *>(Kt + i * TS + 4 * tx);
-            const float qa[4] = {q4.x, q4.y, q4.z, q4.w}, kb[4] = {k4.x, k4.y, k4.z, k4.w};
+        // blocks of 16 elements are summed on their own and then added up: the rounding error of a long
+        // sequential fp32 sum would otherwise eat the 1e-5 tolerance of fp32 stores at large logits
+        for (int i0 = 0; i0 < D; i0 += 16) {
+            float part[4][4];
 #pragma unroll
             for (int a = 0; a < 4; ++a)
 #pragma unroll
-                for (int b = 0; b < 4; ++b) s[a][b] = fmaf(qa[a], kb[b], s[a][b]);
+                for (int b = 0; b < 4; ++b) part[a][b] = 0.f;
+#pragma unroll
+            for (int i = i0; i < i0 + 16; ++i) {
+                const float4 q4 = *reinterpret_cast<const float4 *>(Qt + i * TS + 4 * ty);
+                const float4 k4 = *reinterpret_cast<const float4 *>(Kt + i * TS + 4 * tx);
+                const float qa[4] = {q4.x, q4.y, q4.z, q4.w}, kb[4] = {k4.x, k4.y, k4.z, k4.w};
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) part[a][b] = fmaf(qa[a], kb[b], part[a][b]);
+            }
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) s[a][b] += part[a][b];
         }
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
