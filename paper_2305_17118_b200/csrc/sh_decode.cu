@@ -315,6 +315,8 @@ __global__ void __launch_bounds__(NW * 32, NW == 4 ? ((DT == SH_F32 && D == 128)
     const int u = blockIdx.x / S;
     const int cr = (S > 1) ? (int)(blockIdx.x % S) : 0;
     const int B = p.B;
+    sh_pdl_launch_dependents();
+    sh_pdl_wait();            // the preceding kernel of the stream is complete: global memory may be touched
     // live rows including this step's token, the step number and its bit-plane row: the same for
     // every unit (kernel arguments) unless the handle serves sequences of different lengths
     int n = p.n, t_step = p.t, hist_row = p.hist_row;
@@ -574,14 +576,17 @@ cudaError_t launch_one(const sh_context *c, const DecodeParams &p, cudaStream_t 
     cfg.blockDim = dim3(NW * 32, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     if (S > 1) {
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = S;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = S;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
     }
     return cudaLaunchKernelEx(&cfg, kern, p);
 }

@@ -143,6 +143,7 @@ __global__ void __launch_bounds__(NWC * 32 + 32, CPS) sh_decode_tma_kernel(const
     auto cached_rows = [&](int u) { return p.n_arr ? p.n_arr[u] : p.n - 1; };
     auto tiles_of = [](int n_old) { return n_old > 0 ? (n_old + SR - 1) / SR : 1; };   // the first tile also carries q and the new token
 
+    sh_pdl_launch_dependents();
     if (tid == 0) {
         for (int s = 0; s < NST; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], NWC); }
         drain = 0;
@@ -150,6 +151,7 @@ __global__ void __launch_bounds__(NWC * 32 + 32, CPS) sh_decode_tma_kernel(const
         fence_barrier_init();
     }
     __syncthreads();
+    sh_pdl_wait();            // the preceding kernel of the stream is complete: global memory may be touched
 
     if (warp == NWC) {
         // ------------------------------------------------------------ producer
@@ -393,8 +395,17 @@ cudaError_t launch_tma(const sh_context *c, const DecodeParams &p, cudaStream_t 
     int dev = 0;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int grid = p.U < sms * CPS ? p.U : sms * CPS;
-    kern<<<grid, NWC * 32 + 32, smem, s>>>(p, reinterpret_cast<int *>(c->slab + c->L.err));
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(NWC * 32 + 32, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, p, reinterpret_cast<int *>(c->slab + c->L.err));
 }
 
 }  // namespace

@@ -59,6 +59,17 @@ struct sh_context {
     std::vector<long long> t_seq;
 };
 
+// Programmatic dependent launch.  The decode kernels are launched with programmatic stream serialisation:
+// the next kernel of the stream may be scheduled while this one still runs, which hides its launch latency
+// and start-up behind this kernel's tail.  sh_pdl_launch_dependents() (first thing in the kernel) says the
+// next kernel may be scheduled once every CTA of this one has got that far; sh_pdl_wait() returns when the
+// preceding kernel of the stream has completed and its writes are visible: nothing that depends on earlier
+// work (any global memory of the workspace or of the caller) is touched before it.
+#ifdef __CUDACC__
+__device__ __forceinline__ void sh_pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void sh_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+
 // Base pointers of the active unit range inside the workspace.
 inline char *sh_pK(const sh_context *c) { return c->slab + c->L.K + (size_t)c->u0 * c->B * c->row_bytes; }
 inline char *sh_pV(const sh_context *c) { return c->slab + c->L.V + (size_t)c->u0 * c->B * c->row_bytes; }
