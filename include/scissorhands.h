@@ -348,7 +348,9 @@ long long sh_launch_count(sh_handle h);
 
 /* Which fused decode kernel sh_decode_step launches for this handle's shape and options
  * (see SH_OPT_DECODE_KERNEL): 1 = one CTA or cluster per unit with direct loads, 2 = persistent
- * CTAs fed by bulk asynchronous copies.  For reports and profiles. */
+ * CTAs fed by bulk asynchronous copies, 3 = the int4 store's kernel for many units (codes unpacked
+ * to fp16, dot products as tensor-core MMAs; chosen automatically from 592 units on with head_dim
+ * 128, SH_OPT_DECODE_KERNEL = 1 keeps the CUDA-core kernel).  For reports and profiles. */
 int sh_decode_kernel_choice(sh_handle h);
 
 /* Text for a status code; never NULL. */

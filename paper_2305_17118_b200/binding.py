@@ -348,7 +348,7 @@ class Handle:
     @property
     def decode_kernel(self) -> str:
         """Name of the fused decode kernel sh_decode_step launches for this handle."""
-        return {1: "sh_decode_kernel", 2: "sh_decode_tma_kernel"}[int(lib.sh_decode_kernel_choice(self._h))]
+        return {1: "sh_decode_kernel", 2: "sh_decode_tma_kernel", 3: "sh_decode_int4_mma_kernel"}[int(lib.sh_decode_kernel_choice(self._h))]
 
 
 def select(counters: torch.Tensor, r: int, m: int, stream=None) -> torch.Tensor:

@@ -561,6 +561,8 @@ __global__ void __launch_bounds__(NW * 32, NW == 4 ? ((DT == SH_F32 && D == 128)
     }
 }
 
+#include "sh_decode_int4_mma.inl"
+
 template <int DT, int D, int NW, int R, int S>
 cudaError_t launch_one(const sh_context *c, const DecodeParams &p, cudaStream_t s) {
     const int B = c->B;
@@ -691,7 +693,8 @@ cudaError_t sh_launch_scores(const sh_context *c, const DecodeParams &p, float *
     return e;
 }
 
-// Which decode kernel serves `units` units of this handle: 2 = pipelined (sh_decode_tma.cu), 1 = direct loads.
+// Which decode kernel serves `units` units of this handle: 2 = pipelined (sh_decode_tma.cu), 3 = int4 rows on the
+// tensor cores (sh_decode_int4_mma.inl), 1 = direct loads.
 int sh_decode_kernel_for(const sh_context *c, int units) {
     // Shapes of launch (crossovers measured on B200, rows of 256 bytes: equal at 12 units per SM, the direct
     // kernel 6 % ahead from 16 per SM on, the pipelined one 15 % ahead at 8.6).  With very many units per SM
@@ -707,12 +710,16 @@ int sh_decode_kernel_for(const sh_context *c, int units) {
     if (c->kernel != 1 && pipelined_ok &&
         (c->kernel == 2 || (!prefer_direct && units >= 128 && !(c->split_explicit && c->split > 1))))
         return 2;
+    // int4 store, many units: codes unpacked to fp16 and multiplied on the tensor cores (9216 units: 158 us against
+    // 223 us on CUDA cores), unless the caller asked for the CUDA-core kernel or the budget outgrows its shared memory
+    if (many && c->kernel != 1 && c->dtype == SH_INT4_G64_F16 && c->D == 128 && int4_mma_smem(c->B) <= 200 * 1024) return 3;
     return 1;
 }
 
 cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStream_t s, long long *launches) {
     const bool many = p.U >= 4 * 148 && c->split == 1;
-    if (sh_decode_kernel_for(c, p.U) == 2) return sh_launch_decode_tma(c, p, s, launches);
+    const int which = sh_decode_kernel_for(c, p.U);
+    if (which == 2) return sh_launch_decode_tma(c, p, s, launches);
     cudaError_t e = cudaErrorInvalidValue;
     // Two shapes of CTA.  With few units per SM the step is latency-bound and a CTA of 8 warps with 8 row
     // loads in flight per thread finishes a unit soonest.  With many units per SM (no cluster split then)
@@ -734,7 +741,12 @@ cudaError_t sh_launch_decode(const sh_context *c, const DecodeParams &p, cudaStr
             break;
         case SH_INT4_G64_F16:
             if (c->D == 64) e = many ? launch_one<SH_INT4_G64_F16, 64, 4, 2, 1>(c, p, s) : launch_split<SH_INT4_G64_F16, 64, 8, 4>(c, p, s);
-            else if (c->D == 128) e = many ? launch_one<SH_INT4_G64_F16, 128, 4, 2, 1>(c, p, s) : launch_split<SH_INT4_G64_F16, 128, 8, 4>(c, p, s);
+            else if (c->D == 128) {
+                // many units: unpacked codes go to the tensor cores (sh_decode_int4_mma.inl) unless the caller
+                // asked for the CUDA-core kernel by name
+                if (many) e = which == 3 ? launch_int4_mma<4, 1, 1, 8>(c, p, s) : launch_one<SH_INT4_G64_F16, 128, 4, 2, 1>(c, p, s);
+                else e = launch_split<SH_INT4_G64_F16, 128, 8, 4>(c, p, s);
+            }
             break;
         default: break;
     }

@@ -1007,3 +1007,32 @@ def test_config_tiny_chunked_prompt_and_both_record_modes(sh, recompute):
     run = run_lockstep_recompute if recompute else run_lockstep
     res2, _ = run(h, cfg.dtype, st.step, cfg.decode, torch.arange(cfg.units), TOL[cfg.dtype], orc=orc)
     assert res2.compressions == 13
+
+
+@pytest.mark.parametrize("U,B,r,w,m", [(601, 77, 6, 21, 30), (600, 410, 64, 128, 64), (592, 33, 0, 1, 33), (700, 150, 9, 37, 1)])
+@pytest.mark.parametrize("recompute", [False, True])
+def test_lockstep_int4_tensor_core_decode_kernel(sh, U, B, r, w, m, recompute):
+    """The decode kernel the library picks for the int4 store from 592 units on (codes unpacked to fp16, dot
+    products as warp-level MMAs): sampled units in lockstep, ragged row counts (n not a multiple of 8 or 16),
+    the step's own token quantised bit-identically, and the query ring kept for the recompute mode."""
+    dtype, d = "int4", 128
+    T = min(B + 2 * m + 40, B + 150)
+    q, k, v = wl.random_stream(U, d, T, seed=59 + B, dtype=dtype, peaked=3.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, recompute_record=recompute)
+    units = torch.tensor([0, 1, 17, 148, 299, 300, 591, U - 1])
+    run = run_lockstep_recompute if recompute else run_lockstep
+    res, orc = run(h, dtype, _stream_fn(q, k, v), T, units, TOL[dtype])
+    assert res.compressions >= 2
+    assert res.adoptions <= 1e-4 * res.slot_steps + 2
+    view = SortedView(h, units=units.numpy())
+    n = h.n
+    for i, u in enumerate(units.tolist()):
+        K, V = view.export_unit(u)
+        oK, oV = orc.cache(i)
+        assert (K[:n].astype(np.float64) == oK).all() and (V[:n].astype(np.float64) == oV).all()
+
+
+def test_ragged_sequences_int4_tensor_core_kernel(sh):
+    compressions = _ragged_lockstep(sh, "int4", 128, [3, 41], ups=300, B=48, r=4, w=12, m=16, T_dec=40, kernel=None,
+                                    unordered=None, split=None, seed=58)
+    assert compressions >= 3
