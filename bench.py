@@ -489,15 +489,17 @@ def main():
     ap.add_argument("--units", type=int, default=None,
                     help="override the workload's units per launch (a smaller case of the same kernels, for profiler captures)")
     ap.add_argument("--prompt", type=int, default=None, help="override the workload's prompt length (same purpose)")
+    ap.add_argument("--layers", type=int, default=None, help="override the workload's number of layers (same purpose)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     cfg = wl.CONFIGS[args.config]
-    if args.kv_dtype or args.head_dim or args.units or args.prompt:      # shape variants of a named workload (not the benchmark's own lines)
+    if args.kv_dtype or args.head_dim or args.units or args.prompt or args.layers:      # shape variants of a named workload (not the benchmark's own lines)
         tag = ",".join(x for x in (args.kv_dtype, f"d{args.head_dim}" if args.head_dim else None,
                                    f"units{args.units}" if args.units else None,
-                                   f"prompt{args.prompt}" if args.prompt else None) if x)
+                                   f"prompt{args.prompt}" if args.prompt else None,
+                                   f"layers{args.layers}" if args.layers else None) if x)
         cfg = cfg.scaled(name=f"{cfg.name}[{tag}]", dtype=args.kv_dtype or cfg.dtype, head_dim=args.head_dim or cfg.head_dim,
-                         units=args.units or cfg.units, prompt=args.prompt or cfg.prompt)
+                         units=args.units or cfg.units, prompt=args.prompt or cfg.prompt, layers=args.layers or cfg.layers)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":

@@ -904,16 +904,19 @@ def test_record_mode_overlap_diagnostic(sh):
     assert (got.overlap >= r / got.n - 1e-12).all() and (got.overlap <= 1).all()
 
 
-@pytest.mark.parametrize("dtype,d,stable", [("f16", 128, False), ("bf16", 128, True), ("int4", 128, False), ("f32", 64, False)])
-@pytest.mark.parametrize("p,B,r,w,m", [(300, 96, 8, 40, 30), (150, 150, 9, 37, 41), (90, 120, 4, 16, 20), (700, 130, 10, 200, 1)])
+_BULK_STORES = [("f16", 128, False), ("bf16", 128, True), ("int4", 128, False), ("f32", 64, False)]
+_BULK_SHAPES = [(300, 96, 8, 40, 30), (150, 150, 9, 37, 41), (90, 120, 4, 16, 20)]
+
+
+# (the last shape drops one token per round, 570 rounds: one storage type is enough for it)
+@pytest.mark.parametrize("dtype,d,stable,p,B,r,w,m", [st + sh_ for sh_ in _BULK_SHAPES for st in _BULK_STORES] +
+                         [("f16", 128, False, 700, 130, 10, 200, 1)])
 def test_bulk_prompt_reading_lockstep(sh, dtype, d, stable, p, B, r, w, m):
     """The prompting stage read as a bulk operation (sh_import_compressed / sh_prefill_bulk): the prompt is
     attended in full on a handle that never compresses, in lockstep with an oracle of the same budget;
     both sides then bring that cache under the real budget by rounds of Algorithm 2 on the record as it
     stands, and must hold the same tokens, records and rows; generation continues in lockstep.  The
     one-call form must end bit-identical to the composed one."""
-    if m == 1 and dtype != "f16":
-        pytest.skip("570 rounds of one token: one storage type is enough")
     U, T_dec = 4, 80
     q, k, v = wl.random_stream(U, d, p + T_dec, seed=111 + p, dtype=dtype, peaked=3.0, device="cuda")
     kw = dict(auto_compress=False, unordered=not stable)
