@@ -47,7 +47,7 @@ L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
 REPEATS = 3
 ES = {"f32": 4.0, "f16": 2.0, "bf16": 2.0, "int4": 0.5 + 2.0 / 64.0}
-INT4_LANE_INSTR_PER_BYTE = 10.0   # int4 decode kernel: warp instructions x 32 / stored bytes read, from its ncu capture
+INT4_LANE_INSTR_PER_BYTE = 7.4    # int4 decode kernel (many units): warp instructions x 32 / stored bytes read, from its ncu capture
 
 
 def measured_peak():
@@ -402,38 +402,43 @@ def cuda_arm(args, cfg, rank, world):
     if rank == 0 or dist:
         for h, s in zip(handles, snaps):
             h.restore(s)
-        Ke = min(K, n_in)
-        host = [[x[:Ke].cpu().pin_memory() for x in dec[l]] for l in range(Ly)]
+        Ke = min(K, n_in - W) if n_in > W else min(K, n_in)
+        first = W if n_in >= W + Ke else 0          # the same stream positions as the device-resident windows
+        host = [[x[:first + Ke].cpu().pin_memory() for x in dec[l]] for l in range(Ly)]
         oh = torch.empty(U, d).pin_memory()
         # raw addresses of every step's pinned rows, looked up once: the timed loop only makes the C call
-        ptrs = [[(host[l][0][i].data_ptr(), host[l][1][i].data_ptr(), host[l][2][i].data_ptr()) for i in range(Ke)]
+        ptrs = [[(host[l][0][i].data_ptr(), host[l][1][i].data_ptr(), host[l][2][i].data_ptr()) for i in range(first + Ke)]
                 for l in range(Ly)]
         oh_ptr, st_ptr = oh.data_ptr(), torch.cuda.current_stream().cuda_stream
-        for i in range(min(W, Ke)):
-            for l, h in enumerate(handles):
-                h.decode_step_host(host[l][0][i], host[l][1][i], host[l][2][i], oh)
-                h.compress()
-        for h, s in zip(handles, snaps):
-            h.restore(s)
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        n_live = snaps[0][1]          # the schedule is data-independent: the caller knows when a compression is due
-        e0.record()
-        for i in range(Ke):
-            n_live += 1
-            for l, h in enumerate(handles):
-                qp, kp, vp = ptrs[l][i]
-                h.decode_step_host_raw(qp, kp, vp, oh_ptr, st_ptr)
-                if n_live == cfg.B:
-                    h.compress()
-            if n_live == cfg.B:
-                n_live -= cfg.m
-        e1.record()
-        barrier()
-        _, e_value = job_throughput(e0.elapsed_time(e1), Ke, world, dist, dev)
+        e_values = []
+        for _rep in range(REPEATS):
+            for h, s in zip(handles, snaps):
+                h.restore(s)
+            n_live = snaps[0][1]          # the schedule is data-independent: the caller knows when a compression is due
+
+            def host_steps(i0, i1):
+                nonlocal n_live
+                for i in range(i0, i1):
+                    n_live += 1
+                    for l, h in enumerate(handles):
+                        qp, kp, vp = ptrs[l][i]
+                        h.decode_step_host_raw(qp, kp, vp, oh_ptr, st_ptr)
+                        if n_live == cfg.B:
+                            h.compress()
+                    if n_live == cfg.B:
+                        n_live -= cfg.m
+            host_steps(0, first)          # warm-up, untimed
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            host_steps(first, first + Ke)
+            e1.record()
+            barrier()
+            e_values.append(job_throughput(e0.elapsed_time(e1), Ke, world, dist, dev)[1])
+        e_value = statistics.median(e_values)
         in_b = Ly * U * d * (4 if cfg.dtype == "f32" else 2) * 3
         e2e = {"value": e_value, "unit": UNIT, "h2d_bytes_per_step": in_b,
-               "d2h_bytes_per_step": Ly * U * d * 4, "steps": Ke}
+               "d2h_bytes_per_step": Ly * U * d * 4, "steps": Ke, "values": e_values}
 
     if rank != 0:
         if dist:
