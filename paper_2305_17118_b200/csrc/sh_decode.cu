@@ -225,30 +225,41 @@ template <int DT> __device__ __forceinline__ void load_input(const void *row, in
     }
 }
 
-// Quantise this lane's 32 elements (half a group of 64; the partner lane c^1
-// holds the other half): a = max|x| over the group, sc = fp16(a / 7),
-// code = clamp(rint(x / sc), -7, 7), all in IEEE fp32.  On return f holds the
-// dequantised values code*sc; the packed codes and the scale are returned.
-__device__ __forceinline__ uint4 quantize32(float *f, float &sc_out) {
-    float a = 0.f;
-#pragma unroll
-    for (int i = 0; i < 32; ++i) a = fmaxf(a, fabsf(f[i]));
-    a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
-    const float sc = __half2float(__float2half_rn(__fdiv_rn(a, 7.0f)));
-    uint32_t w[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        w[k] = 0;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            float code = 0.f;
-            if (sc != 0.f) code = fminf(fmaxf(rintf(__fdiv_rn(f[8 * k + e], sc)), -7.f), 7.f);
-            f[8 * k + e] = code * sc;
-            w[k] |= (uint32_t)((int)code + 8) << (4 * ((e >> 1) + 4 * (e & 1)));
-        }
+// Quantisation of a row of the int4 store, all in IEEE fp32: a = max|x| over a group of 64, sc = fp16(a / 7),
+// code = clamp(rint(x / sc), -7, 7), stored value code * sc.  The row is spread over a whole warp: lane l holds elements EPT*l .. EPT*l + EPT - 1 of a
+// row of D fp16 values (EPT = D / 32; a scale group of 64 is 64 / EPT lanes, an 8-code word 8 / EPT lanes).
+// Writes the row's codes and scales and leaves the dequantised values in x.
+template <int D>
+__device__ __forceinline__ void int4_append_row(const char *src_row, char *dst_row, __half *dst_scales, float (&x)[D / 32], int lane) {
+    constexpr int EPT = D / 32, GL = 64 / EPT, LPW = 8 / EPT;
+    static_assert(EPT == 2 || EPT == 4, "head_dim 64 or 128");
+    if constexpr (EPT == 4) {
+        const uint2 in = *reinterpret_cast<const uint2 *>(src_row + 8 * lane);
+        const float2 a = __half22float2(*reinterpret_cast<const __half2 *>(&in.x)), b = __half22float2(*reinterpret_cast<const __half2 *>(&in.y));
+        x[0] = a.x; x[1] = a.y; x[2] = b.x; x[3] = b.y;
+    } else {
+        const float2 a = __half22float2(*reinterpret_cast<const __half2 *>(src_row + 4 * lane));
+        x[0] = a.x; x[1] = a.y;
     }
-    sc_out = sc;
-    return make_uint4(w[0], w[1], w[2], w[3]);
+    float amax = 0.f;
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) amax = fmaxf(amax, fabsf(x[e]));
+#pragma unroll
+    for (int o = GL / 2; o; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    const float sc = __half2float(__float2half_rn(__fdiv_rn(amax, 7.0f)));
+    uint32_t word = 0;
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) {
+        float code = 0.f;
+        if (sc != 0.f) code = fminf(fmaxf(rintf(__fdiv_rn(x[e], sc)), -7.f), 7.f);
+        x[e] = code * sc;
+        const int ew = EPT * (lane % LPW) + e;              // element within its 8-code word
+        word |= (uint32_t)((int)code + 8) << (4 * ((ew >> 1) + 4 * (ew & 1)));
+    }
+#pragma unroll
+    for (int o = LPW / 2; o; o >>= 1) word |= __shfl_xor_sync(0xffffffffu, word, o);
+    if (lane % LPW == 0) reinterpret_cast<uint32_t *>(dst_row)[lane / LPW] = word;
+    if (lane % GL == 0) dst_scales[lane / GL] = __float2half_rn(sc);
 }
 
 // ---------------------------------------------------------------- reductions
@@ -309,7 +320,7 @@ __global__ void __launch_bounds__(NW * 32, NW == 4 ? ((DT == SH_F32 && D == 128)
     const int INB = (DT == SH_F32) ? D * 4 : D * 2;
 
     extern __shared__ __align__(16) float smem[];
-    // s_sh[cap] | red[NW*D] | wred[NW] | xM[8] | xL[8] | xo[D]
+    // s_sh[cap] | red[NW*D] | wred[NW] | xM[8] | xL[8] | xo[D] | vn[D]
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int sub = lane / LPR, c = lane % LPR;
     const int u = blockIdx.x / S;
@@ -342,6 +353,7 @@ __global__ void __launch_bounds__(NW * 32, NW == 4 ? ((DT == SH_F32 && D == 128)
     float *xM = wred + NW;
     float *xL = xM + 8;
     float *xo = xL + 8;
+    float *vn = xo + D;                 // int4 store: dequantised value row of this step's token
 
     if constexpr (S > 1) cg::this_cluster().sync();   // every CTA of the cluster is running: its shared memory may be written
 
@@ -408,25 +420,38 @@ __global__ void __launch_bounds__(NW * 32, NW == 4 ? ((DT == SH_F32 && D == 128)
     float fv_new[EPL];
 #pragma unroll
     for (int e = 0; e < EPL; ++e) fv_new[e] = 0.f;
-    if (has_new && warp == 0) {
+    if constexpr (Q4) {
+        // warp 0 quantises, appends and scores the key row, warp 1 quantises and appends the value row
+        if (has_new && warp < 2) {
+            constexpr int EPT = D / 32;
+            float x[EPT];
+            const char *src = reinterpret_cast<const char *>(warp == 0 ? p.k_new : p.v_new) + (size_t)u * INB;
+            int4_append_row<D>(src, (warp == 0 ? p.K : p.V) + ((size_t)u * B + n_old) * ROWB,
+                               reinterpret_cast<__half *>(warp == 0 ? p.Ks : p.Vs) + ((size_t)u * p.Bs + n_old) * (D / 64), x, lane);
+            if (warp == 0) {
+                const __half *qh = reinterpret_cast<const __half *>(reinterpret_cast<const char *>(p.q) + (size_t)u * INB) + EPT * lane;
+                float a = 0.f;
+#pragma unroll
+                for (int e = 0; e < EPT; ++e) a = fmaf(__half2float(qh[e]), x[e], a);
+                a = warp_sum(a);
+                const float s = a * p.scale_log2e;
+                if (lane == 0) {
+                    s_sh[n_old - lo] = s;
+                    p.pos[(size_t)u * B + n_old] = t_step;
+                }
+                lmax = fmaxf(lmax, s);
+            } else {
+#pragma unroll
+                for (int e = 0; e < EPT; ++e) vn[EPT * lane + e] = x[e];
+            }
+        }
+    } else if (has_new && warp == 0) {
         float fk[EPL];
         load_input<DT>(reinterpret_cast<const char *>(p.k_new) + (size_t)u * INB, c, fk);
         load_input<DT>(reinterpret_cast<const char *>(p.v_new) + (size_t)u * INB, c, fv_new);
         char *kdst = p.K + ((size_t)u * B + n_old) * ROWB + c * 16;
         char *vdst = p.V + ((size_t)u * B + n_old) * ROWB + c * 16;
-        if constexpr (Q4) {
-            float sck, scv;
-            const uint4 ck = quantize32(fk, sck);
-            const uint4 cv = quantize32(fv_new, scv);
-            if (sub == 0) {
-                st_plain(kdst, ck);
-                st_plain(vdst, cv);
-                if ((c & 1) == 0) {
-                    reinterpret_cast<__half *>(p.Ks)[((size_t)u * p.Bs + n_old) * (D / 64) + (c >> 1)] = __float2half_rn(sck);
-                    reinterpret_cast<__half *>(p.Vs)[((size_t)u * p.Bs + n_old) * (D / 64) + (c >> 1)] = __float2half_rn(scv);
-                }
-            }
-        } else if (sub == 0) {
+        if (sub == 0) {
             st_plain(kdst, ld_plain(reinterpret_cast<const char *>(p.k_new) + (size_t)u * INB + c * 16));
             st_plain(vdst, ld_plain(reinterpret_cast<const char *>(p.v_new) + (size_t)u * INB + c * 16));
         }
@@ -497,7 +522,7 @@ __global__ void __launch_bounds__(NW * 32, NW == 4 ? ((DT == SH_F32 && D == 128)
 #pragma unroll
         for (int i = 0; i < R; ++i) E::axpy(acc, pe[i], raw[i]);
     }
-    if (has_new && warp == 0 && sub == 0) {
+    if (!Q4 && has_new && warp == 0 && sub == 0) {
         const float e_new = s_sh[n_old - lo];
 #pragma unroll
         for (int e = 0; e < EPL; ++e) acc[e] = fmaf(e_new, fv_new[e], acc[e]);
@@ -516,6 +541,7 @@ __global__ void __launch_bounds__(NW * 32, NW == 4 ? ((DT == SH_F32 && D == 128)
     if (tid < D) {
 #pragma unroll
         for (int i = 0; i < NW; ++i) o += red[i * D + tid];
+        if (Q4 && has_new) o = fmaf(s_sh[n_old - lo], vn[tid], o);      // the step's own token (int4 store: see above)
     }
 
     if constexpr (S > 1) {
@@ -567,7 +593,7 @@ template <int DT, int D, int NW, int R, int S>
 cudaError_t launch_one(const sh_context *c, const DecodeParams &p, cudaStream_t s) {
     const int B = c->B;
     const int cap = (S > 1) ? ((((B + S - 1) / S) + 31) & ~31) : ((B + 31) & ~31);
-    const size_t smem = sizeof(float) * ((size_t)cap + (size_t)NW * D + NW + 8 + 8 + D);
+    const size_t smem = sizeof(float) * ((size_t)cap + (size_t)NW * D + NW + 8 + 8 + 2 * D);
     auto kern = sh_decode_kernel<DT, D, NW, R, S>;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

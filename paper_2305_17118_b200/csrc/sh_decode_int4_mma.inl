@@ -21,8 +21,8 @@
 // 2/3: group 1 hi/lo), so the product keeps ~fp32 accuracy; rows of dims below 64 read columns 0+1, the
 // others 2+3.
 //
-// The step's own token is quantised, appended and scored by warp 0 in fp32 exactly as in the CUDA-core
-// kernel; softmax, record bits and the cross-warp merge are the same as there.
+// The step's own token is quantised and appended by warps 0 (key, which it also scores) and 1 (value) in fp32
+// with the arithmetic of the CUDA-core kernel; softmax, record bits and the cross-warp merge are the same as there.
 
 __device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -126,32 +126,12 @@ __global__ void __launch_bounds__(NW * 32, MB) sh_decode_int4_mma_kernel(const D
         }
     }
 
-    // ---- the token of this step: warp 0 quantises and appends its key and scores it, warp 1 does the value row.
-    // Lane l holds elements 4l..4l+3 of the row (a scale group is 16 lanes); same arithmetic as quantize32.
+    // ---- the token of this step: warp 0 quantises and appends its key and scores it, warp 1 does the value row
     if (warp < 2) {
-        const char *src = reinterpret_cast<const char *>(warp == 0 ? p.k_new : p.v_new) + (size_t)u * INB;
-        const uint2 in = *reinterpret_cast<const uint2 *>(src + 8 * lane);
-        const float2 x01 = __half22float2(*reinterpret_cast<const __half2 *>(&in.x));
-        const float2 x23 = __half22float2(*reinterpret_cast<const __half2 *>(&in.y));
-        float x[4] = {x01.x, x01.y, x23.x, x23.y};
-        float a = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
-#pragma unroll
-        for (int o = 8; o; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
-        const float sc = __half2float(__float2half_rn(__fdiv_rn(a, 7.0f)));
-        uint32_t word = 0;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            float code = 0.f;
-            if (sc != 0.f) code = fminf(fmaxf(rintf(__fdiv_rn(x[e], sc)), -7.f), 7.f);
-            x[e] = code * sc;
-            const int ew = 4 * (lane & 1) + e;                  // element within its 8-code word
-            word |= (uint32_t)((int)code + 8) << (4 * ((ew >> 1) + 4 * (ew & 1)));
-        }
-        word |= __shfl_xor_sync(0xffffffffu, word, 1);
-        char *dst = (warp == 0 ? p.K : p.V) + ((size_t)u * B + n_old) * ROWB;
-        if ((lane & 1) == 0) reinterpret_cast<uint32_t *>(dst)[lane >> 1] = word;
-        if ((lane & 15) == 0)
-            reinterpret_cast<__half *>(warp == 0 ? p.Ks : p.Vs)[((size_t)u * p.Bs + n_old) * G + (lane >> 4)] = __float2half_rn(sc);
+        float x[4];
+        int4_append_row<D>(reinterpret_cast<const char *>(warp == 0 ? p.k_new : p.v_new) + (size_t)u * INB,
+                           (warp == 0 ? p.K : p.V) + ((size_t)u * B + n_old) * ROWB,
+                           reinterpret_cast<__half *>(warp == 0 ? p.Ks : p.Vs) + ((size_t)u * p.Bs + n_old) * G, x, lane);
         if (warp == 0) {
             const uint2 qin = *reinterpret_cast<const uint2 *>(qrow + 8 * lane);
             const float2 q01 = __half22float2(*reinterpret_cast<const __half2 *>(&qin.x));
