@@ -47,7 +47,8 @@ L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
 REPEATS = 3
 ES = {"f32": 4.0, "f16": 2.0, "bf16": 2.0, "int4": 0.5 + 2.0 / 64.0}
-INT4_LANE_INSTR_PER_BYTE = 7.4    # int4 decode kernel (many units): warp instructions x 32 / stored bytes read, from its ncu capture
+# int4 decode kernels: warp instructions x 32 / stored bytes read, from their ncu captures (profiles/)
+INT4_LANE_INSTR_PER_BYTE = {"sh_decode_int4_mma_kernel": 7.4, "sh_decode_kernel": 10.0}
 
 
 def measured_peak():
@@ -377,10 +378,11 @@ def cuda_arm(args, cfg, rank, world):
         # CUDA-core unpacking of 4-bit codes is bound by instruction issue before HBM: peak derived from
         # the kernel's instructions per stored byte and the SMs' issue rate at the sampled clock.
         mhz = sampler.summary()["sm_mhz"] or 1965.0
-        issue_peak = 148 * 4 * mhz * 1e6 * 32 / INT4_LANE_INSTR_PER_BYTE / 1e9
+        ipb = INT4_LANE_INSTR_PER_BYTE[handles[0].decode_kernel]
+        issue_peak = 148 * 4 * mhz * 1e6 * 32 / ipb / 1e9
         roofline.update({"bound": "alu", "peak": issue_peak, "frac": achieved / issue_peak,
                          "peak_source": (f"derived: 148 SMs x 4 schedulers x 1 warp instruction per clock x 32 lanes at {mhz:.0f} MHz "
-                                         f"/ {INT4_LANE_INSTR_PER_BYTE} lane-instructions per stored byte (profiles/)"),
+                                         f"/ {ipb} lane-instructions per stored byte (profiles/)"),
                          "frac_of_measured_hbm": achieved / peak})
 
     # ---- the compression on its own (steps c1-c4), in the mode of this run and in the other one
