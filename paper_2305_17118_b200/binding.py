@@ -44,7 +44,11 @@ def _load() -> C.CDLL:
         except Exception as e:  # no nvcc here: use what was shipped, if anything
             if not os.path.exists(_build.LIB):
                 raise ImportError(f"libscissorhands.so is not built and cannot be built: {e}") from e
-    lib = C.CDLL(path)
+    return declare(C.CDLL(path))
+
+
+def declare(lib: C.CDLL) -> C.CDLL:
+    """Argument and result types of every entry point, on a loaded build of the library."""
     vp, ip, llp = C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_longlong)
     lib.sh_create.argtypes = [C.c_int] * 7 + [C.POINTER(vp)]
     lib.sh_destroy.argtypes = [vp]

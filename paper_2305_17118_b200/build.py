@@ -12,6 +12,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB_DIR = os.path.join(PKG, "lib")
 LIB = os.path.join(LIB_DIR, "libscissorhands.so")
+LIB_DEBUG_BOUNDS = os.path.join(LIB_DIR, "libscissorhands_bounds.so")
 INCLUDE = os.path.join(ROOT, "include")
 
 
@@ -26,20 +27,24 @@ def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def stale() -> bool:
-    if not os.path.exists(LIB):
+def stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    mt = os.path.getmtime(LIB)
+    mt = os.path.getmtime(lib)
     deps = sources() + glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(CSRC, "*.inl")) \
         + glob.glob(os.path.join(INCLUDE, "*.h"))
     return any(os.path.getmtime(f) > mt for f in deps)
 
 
-def build(force: bool = False, verbose: bool = False, out: str = LIB) -> str:
+def build(force: bool = False, verbose: bool = False, out: str = LIB, debug_bounds: bool = False) -> str:
     """Compile every .cu under csrc/ (one nvcc process per file, in parallel) and link them into one shared
-    library.  Returns its path."""
-    if out == LIB and not force and not stale():
-        return LIB
+    library.  Returns its path.  ``debug_bounds``: the bounds-checked build (-DSH_DEBUG_BOUNDS: every index a
+    kernel derives from workspace state is range-checked and a violation is reported through the device error
+    word instead of being dereferenced), written to lib/libscissorhands_bounds.so."""
+    if debug_bounds and out == LIB:
+        out = LIB_DEBUG_BOUNDS
+    if not force and os.path.exists(out) and not stale(out):
+        return out
     os.makedirs(os.path.dirname(out), exist_ok=True)
     obj_dir = os.path.join(os.path.dirname(out), f"obj.{os.getpid()}")
     os.makedirs(obj_dir, exist_ok=True)
@@ -48,6 +53,8 @@ def build(force: bool = False, verbose: bool = False, out: str = LIB) -> str:
              "-I", INCLUDE, "-I", CSRC]
     if verbose:
         flags += ["-Xptxas", "-v"]
+    if debug_bounds:
+        flags += ["-DSH_DEBUG_BOUNDS"]
     try:
         jobs = []
         for src in sources():

@@ -102,6 +102,7 @@ int do_compress_at(sh_context *c, cudaStream_t s, int n, int r, int m, bool own)
     sp.evicted = nullptr;
     sp.U = c->ucount; sp.B = c->B; sp.Bw = c->Bw; sp.w = c->w; sp.n = n; sp.r = r; sp.m = m;
     sp.cmax = c->w;
+    sp.err = reinterpret_cast<int *>(c->slab + c->L.err);
     sp.n_arr = sh_pnarr(c);
     sp.unordered = c->unordered;
     sp.pos = sh_ppos(c);
@@ -222,6 +223,7 @@ int do_step(sh_context *c, const void *q, const void *k, const void *v, float *o
     p.hist_row = (int)((c->t + 1) % c->w);
     p.scale_log2e = (float)((double)c->scale * LOG2E);
     p.selftest_skip_tile = c->selftest_skip_tile;
+    p.err = reinterpret_cast<int *>(c->slab + c->L.err);
     cudaError_t e = sh_launch_decode(c, p, s, &c->launches);
     if (e != cudaSuccess) return cuda_fail(c, e);
     c->started = true;
@@ -654,6 +656,7 @@ int sh_scores(sh_handle h, const void *q, float *alpha_out, void *stream) {
     p.U = h->ucount; p.B = h->B; p.Bs = h->Bs;
     p.n = h->n;
     p.scale_log2e = (float)((double)h->scale * LOG2E);
+    p.err = reinterpret_cast<int *>(h->slab + h->L.err);
     cudaError_t e = sh_launch_scores(h, p, alpha_out, (cudaStream_t)stream, &h->launches);
     if (e != cudaSuccess) return cuda_fail(h, e);
     return SH_OK;

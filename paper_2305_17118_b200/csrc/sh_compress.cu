@@ -100,12 +100,14 @@ __device__ __forceinline__ void compress_masks(uint32_t m, uint32_t *mv_out) {
 // before each word.  hmask..fmv: shared arrays of Bw, Bw, Bw, 5 Bw, 5 Bw words.  Ends with a barrier.
 template <class HoleOf, class FillerOf>
 __device__ __forceinline__ void build_fill_masks(HoleOf hole_of, FillerOf filler_of, int h, int Bw, uint32_t *hmask,
-                                                 uint32_t *fmask, uint32_t *hoff, uint32_t *hmv, uint32_t *fmv) {
+                                                 uint32_t *fmask, uint32_t *hoff, uint32_t *hmv, uint32_t *fmv,
+                                                 int n_keep, int n, int *err) {
     const int tid = threadIdx.x, nt = blockDim.x;
     for (int k = tid; k < Bw; k += nt) { hmask[k] = 0; fmask[k] = 0; }
     __syncthreads();
     for (int k = tid; k < h; k += nt) {
         const int d = hole_of(k), sj = filler_of(k);
+        if (!SH_BOUNDS_OK(d >= 0 && d < n_keep && sj >= n_keep && sj < n, err, 0x711)) continue;
         atomicOr(&hmask[d >> 5], 1u << (d & 31));
         atomicOr(&fmask[sj >> 5], 1u << (sj & 31));
     }
@@ -184,6 +186,7 @@ __device__ __forceinline__ void fill_rows(const CompactParams &p, int u, int wha
                 char *rows = idx >= per ? Vr : Kr;
                 const int rem = idx >= per ? idx - per : idx;
                 const int k = rem >> lsh, ch = rem & (lpr - 1);
+                if (!SH_BOUNDS_OK(hole_of(k) >= 0 && hole_of(k) < p.n - p.m && filler_of(k) >= p.n - p.m && filler_of(k) < p.n, p.err, 0x712)) continue;
                 dst[i] = rows + (size_t)hole_of(k) * p.row_bytes + ch * 16;
                 val[i] = *reinterpret_cast<const uint4 *>(rows + (size_t)filler_of(k) * p.row_bytes + ch * 16);
             }
@@ -208,7 +211,9 @@ template <class HoleOf, class FillerOf>
 __device__ __forceinline__ void fill_positions(const CompactParams &p, int u, int h, HoleOf hole_of, FillerOf filler_of) {
     const int tid = threadIdx.x, nt = blockDim.x, n_keep = p.n - p.m;
     int32_t *pos = p.pos + (size_t)u * p.B;
-    for (int k = tid; k < h; k += nt) pos[hole_of(k)] = pos[filler_of(k)];
+    for (int k = tid; k < h; k += nt)
+        if (SH_BOUNDS_OK(hole_of(k) >= 0 && hole_of(k) < n_keep && filler_of(k) >= n_keep && filler_of(k) < p.n, p.err, 0x713))
+            pos[hole_of(k)] = pos[filler_of(k)];
     __syncthreads();                                 // every filler is read before the tail is zeroed
     for (int j = n_keep + tid; j < p.n; j += nt) pos[j] = 0;
     if (p.n_arr && tid == 0) p.n_arr[u] = n_keep;    // the unit is compacted
@@ -234,6 +239,7 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
         return;
     }
 
+    if (!SH_BOUNDS_OK(n >= 1 && n <= p.B && m >= 1 && m <= n - p.r, p.err, 0x717)) return;
     for (int i = tid; i <= p.cmax; i += SEL_THREADS) bins[i] = 0;
     if (FROM_HIST) {
         const uint32_t *hist_u = p.hist + (size_t)u * p.w * p.Bw;
@@ -474,7 +480,7 @@ __global__ void __launch_bounds__(SEL_THREADS) sh_select_kernel(const SelectPara
             const int Bw = p.Bw, w = p.w, pst = Bw | 1;
             uint32_t *hmask = reinterpret_cast<uint32_t *>(sm + p.fuse_off + 2 * m);
             uint32_t *fmask = hmask + Bw, *hoff = fmask + Bw, *hmv = hoff + Bw, *fmv = hmv + 5 * Bw;
-            build_fill_masks(hole_of, filler_of, h, Bw, hmask, fmask, hoff, hmv, fmv);
+            build_fill_masks(hole_of, filler_of, h, Bw, hmask, fmask, hoff, hmv, fmv, n_keep, n, p.mv.err);
             fill_record_rows(planes, pst, w, n, n_keep, Bw, hmask, fmask, hoff, hmv, fmv);   // the rows staged for counting
             __syncthreads();
             uint32_t *hist_w = p.mv.hist + (size_t)u * w * Bw;
@@ -555,7 +561,10 @@ __global__ void __launch_bounds__(ROWS_THREADS) sh_compact_rows_kernel(const Com
             if (d != a && src[d - 1] + 1 == s0) continue;        // inside someone else's run
             int len = 1;
             while (d + len < b && src[d + len] == s0 + len) ++len;
-            shasync::bulk_g2s(buf + (size_t)(d - a) * rb, rows + (size_t)s0 * rb, (uint32_t)len * rb, &bar);
+            // (bounds-checked build: a run out of range is replaced by the rows already at its destination, so the
+            // barrier's byte count still holds and nothing out of range is read)
+            const int s_ok = SH_BOUNDS_OK(s0 >= d && s0 + len <= p.n, p.err, 0x714) ? s0 : d;
+            shasync::bulk_g2s(buf + (size_t)(d - a) * rb, rows + (size_t)s_ok * rb, (uint32_t)len * rb, &bar);
         }
         ok = __syncthreads_and(shasync::mbar_wait(&bar, phase, p.err, 1));   // uniform across the CTA
         phase ^= 1;
@@ -577,7 +586,7 @@ __global__ void __launch_bounds__(ROWS_THREADS) sh_compact_rows_kernel(const Com
             for (int base = 0; base < p.n; base += ROWS_THREADS) {
                 const int d = base + tid;
                 uint32_t val = 0;
-                if (d < n_keep) val = sc[src[d]];
+                if (d < n_keep && SH_BOUNDS_OK(src[d] >= d && src[d] < p.n, p.err, 0x716)) val = sc[src[d]];
                 __syncthreads();
                 if (d < p.n) sc[d] = val;
             }
@@ -586,7 +595,7 @@ __global__ void __launch_bounds__(ROWS_THREADS) sh_compact_rows_kernel(const Com
             for (int base = 0; base < p.n; base += ROWS_THREADS) {
                 const int d = base + tid;
                 uint16_t val = 0;
-                if (d < n_keep) val = sc[src[d]];
+                if (d < n_keep && SH_BOUNDS_OK(src[d] >= d && src[d] < p.n, p.err, 0x716)) val = sc[src[d]];
                 __syncthreads();
                 if (d < p.n) sc[d] = val;
             }
@@ -618,6 +627,7 @@ __global__ void __launch_bounds__(CMP_THREADS) sh_compact_record_kernel(const Co
     __syncthreads();
     for (int d = tid; d < n_keep; d += CMP_THREADS) {
         const int sj = src[d];
+        if (!SH_BOUNDS_OK(sj >= d && sj < p.n, p.err, 0x715)) continue;
         atomicOr(&keep[sj >> 5], 1u << (sj & 31));
     }
     __syncthreads();
@@ -665,7 +675,7 @@ __global__ void __launch_bounds__(CMP_THREADS) sh_compact_record_kernel(const Co
     for (int base = 0; base < p.n; base += CMP_THREADS) {
         const int d = base + threadIdx.x;
         int32_t val = 0;
-        if (d < n_keep) val = pos[src[d]];
+        if (d < n_keep && SH_BOUNDS_OK(src[d] >= d && src[d] < p.n, p.err, 0x715)) val = pos[src[d]];
         __syncthreads();
         if (d < p.n) pos[d] = val;
     }
@@ -707,7 +717,7 @@ __global__ void __launch_bounds__(CMP_THREADS) sh_fill_holes_kernel(const Compac
         for (int i = tid; i < nr * Bw; i += CMP_THREADS) { const int rr = row_of(i); rows_sh[rr * stride + (i - rr * Bw)] = hist_u[(size_t)s0 * Bw + i]; }
     };
     stage_rows(0);                           // does not depend on the move list: in flight while the masks are built
-    build_fill_masks(hole_of, filler_of, h, Bw, hmask, fmask, hoff, hmv, fmv);
+    build_fill_masks(hole_of, filler_of, h, Bw, hmask, fmask, hoff, hmv, fmv, n_keep, p.n, p.err);
     for (int s0 = 0; s0 < w; s0 += p.rec_rows) {
         const int nr = min(p.rec_rows, w - s0);
         if (s0) {

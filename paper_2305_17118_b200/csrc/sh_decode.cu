@@ -336,6 +336,8 @@ __global__ void __launch_bounds__(NW * 32, NW == 4 ? ((DT == SH_F32 && D == 128)
         t_step = p.t_arr[u] + 1;
         hist_row = t_step % p.w;
     }
+    // (the same for every CTA of a cluster: all of them leave before the first cluster barrier)
+    if (!SH_BOUNDS_OK(n >= 1 && n <= B && t_step >= n && hist_row >= 0 && hist_row < p.w, p.err, 0x701)) return;
     const int n_old = n - 1;
 
     int chunk, lo;
@@ -637,6 +639,7 @@ __global__ void __launch_bounds__(256) sh_scores_kernel(const DecodeParams p, fl
     const int sub = lane / LPR, c = lane % LPR;
     const int u = blockIdx.x, B = p.B;
     const int n = p.n_arr ? p.n_arr[u] : p.n;
+    if (!SH_BOUNDS_OK(n >= 0 && n <= B, p.err, 0x702)) return;
     typename E::Q qv;
     E::load_q(reinterpret_cast<const char *>(p.q) + (size_t)u * INB, c, qv);
     const char *Kb = p.K + (size_t)u * B * ROWB;

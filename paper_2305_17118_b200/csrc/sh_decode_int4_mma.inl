@@ -65,6 +65,7 @@ __global__ void __launch_bounds__(NW * 32, MB) sh_decode_int4_mma_kernel(const D
         t_step = p.t_arr[u] + 1;
         hist_row = t_step % p.w;
     }
+    if (!SH_BOUNDS_OK(n >= 1 && n <= B && t_step >= n && hist_row >= 0 && hist_row < p.w, p.err, 0x703)) return;
     const int n_old = n - 1;
     const int cap = (B + 31) & ~31;
     float *s_sh = smem;                 // [cap] scaled logits, then e_j

@@ -163,6 +163,7 @@ __global__ void __launch_bounds__(NWC * 32 + 32, CPS) sh_decode_tma_kernel(const
                 const char *Kb = p.K + (size_t)u * B * ROWB;
                 const char *Vb = p.V + (size_t)u * B * ROWB;
                 const int n_old = cached_rows(u), ntiles = tiles_of(n_old);
+                if (!SH_BOUNDS_OK(n_old >= 0 && n_old < B && (!p.t_arr || p.t_arr[u] >= n_old), err, 0x704)) continue;   // the consumers skip the unit too
                 for (int tl = 0; tl < ntiles; ++tl) {
                     if (it >= NST && !mbar_wait(&empty[s], ph, err, 2)) *(volatile int *)&drain = 1;
                     if (*(volatile int *)&drain) { stop = true; break; }
@@ -198,6 +199,7 @@ __global__ void __launch_bounds__(NWC * 32 + 32, CPS) sh_decode_tma_kernel(const
         for (int u = blockIdx.x; u < p.U; u += gridDim.x, par ^= 1) {
             float *s_sh = s_all + par * capw;
             const int n_old = cached_rows(u), ntiles = tiles_of(n_old), n = n_old + 1;
+            if (!SH_BOUNDS_OK(n_old >= 0 && n_old < B && (!p.t_arr || p.t_arr[u] >= n_old), err, 0x704)) continue;
             const int t_step = p.t_arr ? p.t_arr[u] + 1 : p.t;
             const int hist_row = p.t_arr ? t_step % p.w : p.hist_row;
             const float tf = (float)t_step;

@@ -70,6 +70,17 @@ __device__ __forceinline__ void sh_pdl_launch_dependents() { asm volatile("gridd
 __device__ __forceinline__ void sh_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 #endif
 
+// Bounds-checked build (-DSH_DEBUG_BOUNDS, build.build(debug_bounds=True)): the stand-in for a memory checker.
+// Every index a kernel derives from state it reads back from the workspace (per-unit row counts and step
+// numbers, source slots, move lists) is range-checked before it is used; a violation records a code
+// 0x7xx in the device error word and the unit, or the one access, is skipped, so nothing is read or written
+// out of range and nothing traps.  sh_state then returns SH_EDEVICE.  In the normal build the checks vanish.
+#ifdef SH_DEBUG_BOUNDS
+#define SH_BOUNDS_OK(cond, err, code) ((cond) ? true : ((err) ? (atomicCAS((err), 0, (code)), false) : false))
+#else
+#define SH_BOUNDS_OK(cond, err, code) true
+#endif
+
 // Base pointers of the active unit range inside the workspace.
 inline char *sh_pK(const sh_context *c) { return c->slab + c->L.K + (size_t)c->u0 * c->B * c->row_bytes; }
 inline char *sh_pV(const sh_context *c) { return c->slab + c->L.V + (size_t)c->u0 * c->B * c->row_bytes; }
@@ -102,6 +113,7 @@ struct DecodeParams {
     int hist_row;   // t mod w
     int t;          // 1-based stream position of this step's token
     float scale_log2e;
+    int *err;                 // device error word (bounds-checked build; a bounded wait that gave up)
     int selftest_skip_tile;   // pipelined kernel only: -1, or the tile (counted per CTA) that CTA 0's producer leaves out
 };
 
@@ -131,6 +143,7 @@ struct SelectParams {
     int32_t *evicted;           // [U][m] or NULL
     int U, B, Bw, w, n, r, m;
     int cmax;                   // largest possible counter value
+    int *err;                   // device error word (bounds-checked build), or NULL
     const int *n_arr;           // per-unit live rows, or NULL: units whose cache is not full are skipped
     // unordered mode (holes are filled from the tail, so slots are not sorted by position): the recent
     // window and the tie-break go by the position array; the result is a list of (hole, filler) moves

@@ -65,6 +65,7 @@ extern "C" int sh_compress_static(sh_handle h, void *stream, int *evicted_per_un
     sp.evicted = nullptr;
     sp.U = h->U; sp.B = h->B; sp.Bw = h->Bw; sp.w = h->w; sp.n = h->B; sp.r = h->r; sp.m = h->m;
     sp.cmax = h->w;
+    sp.err = reinterpret_cast<int *>(h->slab + h->L.err);
     sp.n_arr = sh_pnarr(h);
     sp.unordered = h->unordered;
     sp.pos = sh_ppos(h);

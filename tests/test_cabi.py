@@ -22,6 +22,13 @@ def test_library_exports_every_declared_symbol():
         assert hasattr(lib, name), f"{name} is declared in scissorhands.h but not exported"
 
 
+def test_bounds_checked_build_exports_the_same_symbols():
+    from paper_2305_17118_b200 import build
+    lib = C.CDLL(build.build(debug_bounds=True))
+    for name in _declared():
+        assert hasattr(lib, name), name
+
+
 def test_binding_lists_the_same_entry_points():
     from paper_2305_17118_b200 import binding
     assert sorted(binding.EXPORTS) == _declared()
