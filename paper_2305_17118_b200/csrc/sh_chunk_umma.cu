@@ -164,16 +164,31 @@ __global__ void __launch_bounds__(NT, 2) sh_chunk_umma_kernel(const ChunkParams 
     // ---- while those copies fly: append the chunk's keys, values and positions to the cache (nothing in this
     // launch reads them back from there) and remember the queries for a later recount
     if (!RECOUNT && tid < c) p.pos[(size_t)u * p.B + n0 + tid] = step0 + tid;
-    for (int idx = tid; idx < (RECOUNT ? 0 : c * 16); idx += NT) {
-        const int row = idx >> 4, ch = idx & 15;
-        const size_t src = (size_t)row * tstride + (size_t)u * D * 2 + ch * 16;
-        const size_t dst = ((size_t)u * p.B + n0 + row) * (D * 2) + ch * 16;
-        const uint4 kk = *reinterpret_cast<const uint4 *>(p.k + src), vv = *reinterpret_cast<const uint4 *>(p.v + src);
-        uint4 qq = make_uint4(0, 0, 0, 0);
-        if (p.qring) qq = *reinterpret_cast<const uint4 *>(p.q + src);
-        *reinterpret_cast<uint4 *>(p.K + dst) = kk;
-        *reinterpret_cast<uint4 *>(p.V + dst) = vv;
-        if (p.qring) *reinterpret_cast<uint4 *>(p.qring + ((size_t)u * p.w + (step0 + row) % p.w) * (D * 2) + ch * 16) = qq;
+    if constexpr (!RECOUNT) {
+        // up to 64 rows x 16 pieces = 4 pieces per thread: all loads are issued before the first store, so the
+        // thread waits for memory once, not once per piece
+        constexpr int PER = CQ * 16 / NT;
+        uint4 kk[PER], vv[PER], qq[PER];
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const int idx = tid + i * NT, row = idx >> 4, ch = idx & 15;
+            if (row < c) {
+                const size_t src = (size_t)row * tstride + (size_t)u * D * 2 + ch * 16;
+                kk[i] = *reinterpret_cast<const uint4 *>(p.k + src);
+                vv[i] = *reinterpret_cast<const uint4 *>(p.v + src);
+                if (p.qring) qq[i] = *reinterpret_cast<const uint4 *>(p.q + src);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const int idx = tid + i * NT, row = idx >> 4, ch = idx & 15;
+            if (row < c) {
+                const size_t dst = ((size_t)u * p.B + n0 + row) * (D * 2) + ch * 16;
+                *reinterpret_cast<uint4 *>(p.K + dst) = kk[i];
+                *reinterpret_cast<uint4 *>(p.V + dst) = vv[i];
+                if (p.qring) *reinterpret_cast<uint4 *>(p.qring + ((size_t)u * p.w + (step0 + row) % p.w) * (D * 2) + ch * 16) = qq[i];
+            }
+        }
     }
     cp_async_commit();
     cp_async_wait_all();
