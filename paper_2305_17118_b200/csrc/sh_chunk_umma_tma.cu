@@ -1,0 +1,541 @@
+// Chunked prompt step on the 5th-generation tensor cores, persistent CTAs fed by tiled TMA copies.
+//
+// The computation is the one of sh_chunk_umma.cu (up to 64 consecutive steps of one unit: step i attends with
+// q_i over the n0 cached rows plus the chunk's tokens 0..i, writes its comparison bits into its own bit-plane
+// row, and the chunk's keys, values and queries are appended), and so are the two sweeps over the key tiles and
+// the split of P into a high and a low 16-bit part.  What differs is who moves the data and who waits for whom:
+//
+//   * a CTA is persistent: it walks over units blockIdx.x, blockIdx.x + gridDim.x, ...; tensor memory, the
+//     barriers and the tensor maps are set up once, and the tiles of the next unit are requested while the
+//     softmax threads still work on the present one;
+//   * every key, value and query tile is brought in by cp.async.bulk.tensor (one elected thread, CTA-local
+//     destination, no delivery to several CTAs) from 3-D tensor maps over the caches [U][B][128] and over the
+//     chunk's queries [c][U][128]: boxes of 64 rows x 128 bytes in the 128-byte swizzle, which is the K-major
+//     operand layout for Q and K and the MN-major one for V.  Rows past B (and queries past c) are filled with
+//     zeros by the copy engine; rows between n0 + c and the end of the last tile are stale cache rows: their
+//     logits are masked, and the softmax threads zero them in the last value tile before P.V reads it;
+//   * warps 0..7 do the softmax arithmetic; warp 8 issues the MMAs, warp 9 requests query and key tiles, warp 10
+//     value tiles, warp 11 appends the chunk to the cache (plain loads and stores, then a proxy fence: the
+//     tiles that contain the new rows are requested only after the append of their unit is visible).
+//
+// Every wait is bounded; a wait that gives up records its code in the device error word and raises a CTA-wide
+// flag, on which every role leaves; tensor memory is released on every path.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "sh_async.cuh"
+#include "sh_internal.h"
+#include "sh_umma.cuh"
+
+namespace {
+
+using namespace shasync;
+using namespace shumma;
+
+constexpr int D = 128;            // head_dim served by this kernel
+constexpr int TN = 64;            // keys per tile
+constexpr int CQ = 64;            // queries per unit and launch
+constexpr int NT = 256;           // softmax threads: two per lane of tensor memory
+constexpr int NTHREADS = NT + 128;   // + the warps that issue MMAs, request K/Q tiles, request V tiles, append
+constexpr int W_MMA = NT / 32, W_KQ = W_MMA + 1, W_V = W_MMA + 2, W_APPEND = W_MMA + 3;
+constexpr int HALF_K = TN * 128;        // bytes of one box: 64 rows x 64 elements (half of head_dim)
+constexpr int TILE = 2 * HALF_K;        // a key or value tile: [2 halves of d][64 rows][128 B]
+constexpr int HALF_Q = 2 * CQ * 128;    // the queries occupy rows 0..63 and again rows 64..127 (M = 128)
+constexpr int Q_BYTES = 2 * HALF_Q;
+constexpr int KST = 2;                  // key tiles in flight
+constexpr int PG = (TN / 8) * 128;      // bytes of 8 rows of P (TN keys each) in no-swizzle core-matrix order
+constexpr int P_BYTES = (CQ / 8) * PG;
+constexpr int HC = TN / 4;              // columns of a tile per thread (four threads share a query row)
+static_assert(HC == 16, "a thread reads its 16 columns with one tcgen05.ld and owns half a record word");
+constexpr int TMEM_COLS = 256;          // two S tiles and O^T; two CTAs fit in the 512 columns of an SM
+constexpr int S_COL = 0;
+constexpr int O_COL = 2 * TN;
+
+constexpr int OFF_Q = 0;
+constexpr int OFF_K = OFF_Q + Q_BYTES;
+constexpr int OFF_V = OFF_K + KST * TILE;
+constexpr int OFF_PH = OFF_V + 2 * TILE;
+constexpr int OFF_PL = OFF_PH + P_BYTES;
+constexpr int OFF_STAT = OFF_PL + P_BYTES;      // M[64], L[64], 1/L[64]
+constexpr int OFF_BAR = OFF_STAT + 4 * 3 * 64;
+constexpr int SMEM_BYTES = OFF_BAR + 192;
+static_assert(OFF_K % 1024 == 0 && OFF_V % 1024 == 0 && HALF_K % 1024 == 0, "swizzled tiles start on 1024-byte boundaries");
+static_assert(P_BYTES >= 4 * 2 * NT, "the first sweep's statistics alias the P buffer");
+static_assert(2 * (SMEM_BYTES + 1024) <= 228 * 1024, "two CTAs per SM");
+
+// Shared-memory matrix descriptor for the 128-byte swizzle (layout type 2 in bits 61..63).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+    return smem_desc(saddr, lbo, sbo) | (2ull << 61);
+}
+
+// One box of a 3-D tensor map into this CTA's shared memory; completion counted in bytes on `bar`.
+__device__ __forceinline__ void tma_load_3d(void *smem_dst, const CUtensorMap *map, int c0, int c1, int c2, uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
+            smem_u32(smem_dst)),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar))
+        : "memory");
+}
+// Order this thread's earlier plain stores (any state space) before later reads by the copy engine.
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+__device__ __forceinline__ void st_release_shared(int *p, int v) {
+    asm volatile("st.release.cta.shared.u32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+}
+__device__ __forceinline__ int ld_acquire_shared(const int *p) {
+    int v;
+    asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
+    return v;
+}
+// Wait until *ctr >= target; bounded like mbar_wait.
+__device__ __forceinline__ bool counter_wait(const int *ctr, int target, int *err, int code) {
+    if (ld_acquire_shared(ctr) >= target) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t i = 1; i < WAIT_POLLS; ++i) {
+        if (ld_acquire_shared(ctr) >= target) return true;
+        if ((i & 255u) == 0 && global_ns() - t0 > WAIT_NS) break;
+    }
+    if (err) atomicCAS(err, 0, code);
+    return false;
+}
+
+__device__ __forceinline__ void softmax_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory"); }
+
+struct Bars {
+    uint64_t q_full, q_empty;          // the unit's queries landed / its last S has been computed
+    uint64_t k_full[KST], k_empty[KST];
+    uint64_t v_full[2], v_empty[2];
+    uint64_t s_done[2], s_free[2];     // S(g) computed / read out of tensor memory by all softmax threads
+    uint64_t p_ready, pv_done;         // P(kt) written / P.V(kt) computed
+    uint64_t o_free;                   // O^T of the unit read out
+    uint32_t tmem_slot;
+    int abort_flag;                    // a bounded wait gave up somewhere: everybody leaves
+    int appended;                      // units whose chunk rows are in the cache (written by the append warp)
+};
+static_assert(sizeof(Bars) <= 192, "barrier block");
+
+template <int DT>
+__global__ void __launch_bounds__(NTHREADS, 2)
+sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                         const __grid_constant__ CUtensorMap mapV) {
+    using SP = Split<DT>;
+    extern __shared__ __align__(1024) unsigned char sm[];
+    char *Qs = reinterpret_cast<char *>(sm) + OFF_Q;
+    char *Kt = reinterpret_cast<char *>(sm) + OFF_K;
+    char *Vt = reinterpret_cast<char *>(sm) + OFF_V;
+    char *Ph = reinterpret_cast<char *>(sm) + OFF_PH;
+    char *Pl = reinterpret_cast<char *>(sm) + OFF_PL;
+    float *m_sh = reinterpret_cast<float *>(sm + OFF_PH);
+    float *l_sh = m_sh + NT;
+    float *Mfin = reinterpret_cast<float *>(sm + OFF_STAT), *Lfin = Mfin + 64, *Linv = Lfin + 64;
+    Bars *bars = reinterpret_cast<Bars *>(sm + OFF_BAR);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n0 = p.n0, c = p.c, n_tot = n0 + c;
+    const int ntiles = (n_tot + TN - 1) / TN, G = 2 * ntiles;
+    const int step0 = p.t0 + 1;
+    const bool with_out = p.out != nullptr;
+    const int nunits = ((int)p.U - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;     // units of this CTA
+    auto key_tile = [&](int g) { return g < ntiles ? g : g - ntiles; };
+    auto aborted = [&]() { return *(volatile int *)&bars->abort_flag != 0; };
+
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_slot)), "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+        mbar_init(&bars->q_full, 1);
+        mbar_init(&bars->q_empty, 1);
+        for (int s = 0; s < KST; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1); }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1);
+            mbar_init(&bars->s_done[s], 1); mbar_init(&bars->s_free[s], NT);
+        }
+        mbar_init(&bars->p_ready, NT);
+        mbar_init(&bars->pv_done, 1);
+        mbar_init(&bars->o_free, NT);
+        bars->appended = 0;
+        bars->abort_flag = 0;
+        if ((smem_u32(sm) & 1023u) != 0) {      // the swizzled tiles need the 1024-byte alignment the declaration asks for
+            if (p.err) atomicCAS(p.err, 0, 0x520);
+            bars->abort_flag = 1;
+        }
+        fence_barrier_init();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tbase = bars->tmem_slot;
+    const bool start_ok = !aborted();
+
+    if (warp == W_MMA) {
+        // --------------------------------------------------------------------------------------- the issuing thread
+        if (lane == 0 && start_ok) {
+            const uint32_t q_addr = smem_u32(Qs), k_addr = smem_u32(Kt), v_addr = smem_u32(Vt), ph_addr = smem_u32(Ph), pl_addr = smem_u32(Pl);
+            const uint32_t idesc_s = instr_desc(SP::FMT, 0, 128, TN);
+            const uint32_t idesc_pv = instr_desc(SP::FMT, 1, 128, CQ);
+            bool ok = true;
+            auto issue_s = [&](int k, int g) {
+                const int gk = k * G + g, s = gk % KST, b = gk & 1;
+                if (g == 0) ok = ok && mbar_wait(&bars->q_full, k & 1, p.err, 0x521);
+                ok = ok && mbar_wait(&bars->k_full[s], (gk / KST) & 1, p.err, 0x522);
+                if (gk >= 2) ok = ok && mbar_wait(&bars->s_free[b], ((gk >> 1) - 1) & 1, p.err, 0x523);   // S(gk - 2) has been read out
+                if (!ok) return;
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks)
+                    umma_f16(tbase + S_COL + b * TN, smem_desc_sw128(q_addr + (ks >> 2) * HALF_Q + (ks & 3) * 32, 16, 1024),
+                             smem_desc_sw128(k_addr + s * TILE + (ks >> 2) * HALF_K + (ks & 3) * 32, 16, 1024), idesc_s, ks > 0);
+                umma_commit(&bars->k_empty[s]);
+                umma_commit(&bars->s_done[b]);
+                if (g == G - 1) umma_commit(&bars->q_empty);
+            };
+            issue_s(0, 0);
+            for (int k = 0; k < nunits && ok; ++k) {
+                for (int g = 0; g < G && ok; ++g) {
+                    if (g + 1 < G) issue_s(k, g + 1);          // S runs one tile ahead of the softmax threads,
+                    else if (k + 1 < nunits) issue_s(k + 1, 0);   // across the unit boundary too
+                    if (ok && with_out && g >= ntiles) {
+                        const int kt = g - ntiles, gv = k * ntiles + kt, b = gv & 1;
+                        ok = mbar_wait(&bars->p_ready, gv & 1, p.err, 0x524);
+                        ok = ok && mbar_wait(&bars->v_full[b], (gv >> 1) & 1, p.err, 0x525);
+                        if (kt == 0 && k > 0) ok = ok && mbar_wait(&bars->o_free, (k - 1) & 1, p.err, 0x526);   // the previous unit's O^T is in registers
+                        if (!ok) break;
+                        tc_fence_after();
+#pragma unroll
+                        for (int ks = 0; ks < TN / 16; ++ks) {
+                            const uint64_t a = smem_desc_sw128(v_addr + b * TILE + ks * 2048, HALF_K, 1024);
+                            umma_f16(tbase + O_COL, a, smem_desc(ph_addr + ks * 256, 128, PG), idesc_pv, (kt > 0 || ks > 0));
+                            umma_f16(tbase + O_COL, a, smem_desc(pl_addr + ks * 256, 128, PG), idesc_pv, 1);
+                        }
+                        umma_commit(&bars->v_empty[b]);
+                        umma_commit(&bars->pv_done);
+                    }
+                    if (aborted()) ok = false;
+                }
+            }
+            if (!ok) *(volatile int *)&bars->abort_flag = 1;
+        }
+    } else if (warp == W_KQ) {
+        // --------------------------------------------------------------------------------------- query and key tiles
+        if (lane == 0 && start_ok) {
+            bool ok = true;
+            int last = -1, q_last = -1;           // the last key tile (global index) and the last unit's queries requested
+            for (int k = 0; k < nunits && ok; ++k) {
+                const int u = blockIdx.x + k * gridDim.x;
+                if (k > 0) ok = mbar_wait(&bars->q_empty, (k - 1) & 1, p.err, 0x531);
+                if (!ok || aborted()) { ok = false; break; }
+                mbar_arrive_expect_tx(&bars->q_full, Q_BYTES);
+                q_last = k;
+#pragma unroll
+                for (int part = 0; part < 4; ++part)
+                    tma_load_3d(Qs + (part >> 1) * HALF_Q + (part & 1) * CQ * 128, &mapQ, (part >> 1) * 64, u, 0, &bars->q_full);
+                bool appended = false;
+                for (int g = 0; g < G; ++g) {
+                    const int gk = k * G + g, s = gk % KST, kt = key_tile(g);
+                    if (gk >= KST) ok = mbar_wait(&bars->k_empty[s], ((gk / KST) - 1) & 1, p.err, 0x532);
+                    if (ok && !appended && (kt + 1) * TN > n0) {     // this tile holds rows of the chunk
+                        ok = counter_wait(&bars->appended, k + 1, p.err, 0x533);
+                        fence_proxy_async_all();
+                        appended = true;
+                    }
+                    if (!ok || aborted()) { ok = false; break; }
+                    mbar_arrive_expect_tx(&bars->k_full[s], TILE);
+                    tma_load_3d(Kt + s * TILE, &mapK, 0, kt * TN, u, &bars->k_full[s]);
+                    tma_load_3d(Kt + s * TILE + HALF_K, &mapK, 64, kt * TN, u, &bars->k_full[s]);
+                    last = gk;
+                }
+            }
+            if (!ok) {
+                *(volatile int *)&bars->abort_flag = 1;
+                // nobody may be waiting for the copies already requested: let them land before the CTA goes away
+                if (q_last >= 0) mbar_wait(&bars->q_full, q_last & 1, nullptr, 0);     // (a phase that is past reads as complete)
+                for (int gk = last; gk > last - KST && gk >= 0; --gk) mbar_wait(&bars->k_full[gk % KST], (gk / KST) & 1, nullptr, 0);
+            }
+        }
+    } else if (warp == W_V) {
+        // --------------------------------------------------------------------------------------- value tiles
+        if (lane == 0 && start_ok && with_out) {
+            bool ok = true;
+            int last = -1;
+            for (int k = 0; k < nunits && ok; ++k) {
+                const int u = blockIdx.x + k * gridDim.x;
+                bool appended = false;
+                for (int kt = 0; kt < ntiles; ++kt) {
+                    const int gv = k * ntiles + kt, b = gv & 1;
+                    if (gv >= 2) ok = mbar_wait(&bars->v_empty[b], ((gv >> 1) - 1) & 1, p.err, 0x541);
+                    if (ok && !appended && (kt + 1) * TN > n0) {
+                        ok = counter_wait(&bars->appended, k + 1, p.err, 0x542);
+                        fence_proxy_async_all();
+                        appended = true;
+                    }
+                    if (!ok || aborted()) { ok = false; break; }
+                    mbar_arrive_expect_tx(&bars->v_full[b], TILE);
+                    tma_load_3d(Vt + b * TILE, &mapV, 0, kt * TN, u, &bars->v_full[b]);
+                    tma_load_3d(Vt + b * TILE + HALF_K, &mapV, 64, kt * TN, u, &bars->v_full[b]);
+                    last = gv;
+                }
+            }
+            if (!ok) {
+                *(volatile int *)&bars->abort_flag = 1;
+                for (int gv = last; gv > last - 2 && gv >= 0; --gv) mbar_wait(&bars->v_full[gv & 1], (gv >> 1) & 1, nullptr, 0);
+            }
+        }
+    } else if (warp == W_APPEND) {
+        // --------------------------------------------------------------------------------------- the append
+        // keys, values and positions of the chunk into the cache rows n0 .. n0 + c - 1, queries into the ring of the
+        // last w queries; a row of 256 bytes is 16 pieces, the warp moves two rows per instruction
+        if (start_ok) {
+            for (int k = 0; k < nunits; ++k) {
+                if (aborted()) break;
+                const int u = blockIdx.x + k * gridDim.x;
+                const size_t tstride = (size_t)p.Utot * D * 2;
+                for (int base = 0; base < c * 16; base += 4 * 32) {
+                    uint4 kk[4], vv[4], qq[4];
+#pragma unroll
+                    for (int a = 0; a < 4; ++a) {
+                        const int idx = base + a * 32 + lane, row = idx >> 4, ch = idx & 15;
+                        if (row < c) {
+                            const size_t src = (size_t)row * tstride + (size_t)u * D * 2 + ch * 16;
+                            kk[a] = *reinterpret_cast<const uint4 *>(p.k + src);
+                            vv[a] = *reinterpret_cast<const uint4 *>(p.v + src);
+                            if (p.qring) qq[a] = *reinterpret_cast<const uint4 *>(p.q + src);
+                        }
+                    }
+#pragma unroll
+                    for (int a = 0; a < 4; ++a) {
+                        const int idx = base + a * 32 + lane, row = idx >> 4, ch = idx & 15;
+                        if (row < c) {
+                            const size_t dst = ((size_t)u * p.B + n0 + row) * (D * 2) + ch * 16;
+                            *reinterpret_cast<uint4 *>(p.K + dst) = kk[a];
+                            *reinterpret_cast<uint4 *>(p.V + dst) = vv[a];
+                            if (p.qring) *reinterpret_cast<uint4 *>(p.qring + ((size_t)u * p.w + (step0 + row) % p.w) * (D * 2) + ch * 16) = qq[a];
+                        }
+                    }
+                }
+                for (int row = lane; row < c; row += 32) p.pos[(size_t)u * p.B + n0 + row] = step0 + row;
+                fence_proxy_async_all();
+                __syncwarp();
+                if (lane == 0) st_release_shared(&bars->appended, k + 1);
+            }
+        }
+    } else if (start_ok) {
+        // --------------------------------------------------------------------------------------- softmax threads
+        const int i = tid & 63, quarter = ((tid >> 6) & 1) * 2 + (tid >> 7);     // this thread's query and its quarter of every tile's columns
+        const uint32_t lane_addr = tbase + ((uint32_t)((warp & 3) * 32) << 16);
+        uint32_t par_pv = 0;
+        bool ok = true;
+        const int nv = n0 + i + 1;           // keys visible to this thread's query
+        const bool live_row = i < c;
+        const float tf = (float)(step0 + i);
+        for (int k = 0; k < nunits && ok; ++k) {
+            const int u = blockIdx.x + k * gridDim.x;
+            uint32_t *hrow = p.hist + ((size_t)u * p.w + (step0 + i) % p.w) * p.Bw;
+            float m_run = -INFINITY, l_run = 0.f, Mi = 0.f, Li = 1.f;
+            int g_exit = G;                  // the iteration a warp left the loop at, after a wait that gave up
+            for (int g = 0; g < G; ++g) {
+                const int gk = k * G + g, b = gk & 1, kt = key_tile(g);
+                const bool second = g >= ntiles;
+                ok = mbar_wait(&bars->s_done[b], (gk >> 1) & 1, p.err, 0x501) && ok;
+                // (one decision per warp: the tensor-memory loads below are warp-wide)
+                if (__any_sync(0xffffffffu, !ok || aborted())) {
+                    ok = false;
+                    *(volatile int *)&bars->abort_flag = 1;
+                    g_exit = g;
+                    break;
+                }
+                tc_fence_after();
+                float sv[HC];
+                tmem_ld16(lane_addr + S_COL + b * TN + quarter * HC, sv);
+                tc_fence_before();
+                mbar_arrive(&bars->s_free[b]);       // this thread's share of S is in registers
+                const int j0 = kt * TN + quarter * HC;
+                const int lim = live_row ? nv - j0 : 0;
+                const uint32_t vm = lim <= 0 ? 0u : (lim >= HC ? 0xffffu : (1u << lim) - 1u);
+                if (!second) {
+                    if (vm) {
+                        float bmax = -INFINITY;
+#pragma unroll
+                        for (int jj = 0; jj < HC; ++jj) {
+                            sv[jj] = ((vm >> jj) & 1u) ? sv[jj] * p.scale_log2e : -INFINITY;
+                            bmax = fmaxf(bmax, sv[jj]);
+                        }
+                        const float m_new = fmaxf(m_run, bmax);
+                        float acc = 0.f;
+#pragma unroll
+                        for (int jj = 0; jj < HC; ++jj) acc += ex2_approx(sv[jj] - m_new);
+                        l_run = l_run * ex2_approx(m_run - m_new) + acc;
+                        m_run = m_new;
+                    }
+                    if (g == ntiles - 1) {
+                        m_sh[tid] = m_run;
+                        l_sh[tid] = l_run;
+                        softmax_barrier();
+                        if (tid < CQ) {
+                            float M = -INFINITY, L = 0.f;
+#pragma unroll
+                            for (int part = 0; part < NT / CQ; ++part) M = fmaxf(M, m_sh[tid + part * CQ]);
+#pragma unroll
+                            for (int part = 0; part < NT / CQ; ++part) {
+                                const float mp = m_sh[tid + part * CQ];
+                                if (mp > -INFINITY) L += l_sh[tid + part * CQ] * ex2_approx(mp - M);
+                            }
+                            Mfin[tid] = M;
+                            Lfin[tid] = L;
+                            Linv[tid] = 1.f / L;
+                        }
+                        softmax_barrier();
+                        Mi = Mfin[i];
+                        Li = Lfin[i];
+                        softmax_barrier();       // everyone has its row's M and L: the P buffer (m_sh, l_sh) may be written
+                    }
+                    continue;
+                }
+                uint32_t word = 0, hi[HC / 2], lo[HC / 2];
+#pragma unroll
+                for (int jj = 0; jj < HC; jj += 2) {
+                    const bool v0 = (vm >> jj) & 1u, v1 = (vm >> (jj + 1)) & 1u;
+                    const float e0 = v0 ? ex2_approx(sv[jj] * p.scale_log2e - Mi) : 0.f;
+                    const float e1 = v1 ? ex2_approx(sv[jj + 1] * p.scale_log2e - Mi) : 0.f;
+                    word |= (uint32_t)(e0 * tf < Li) << jj;
+                    word |= (uint32_t)(e1 * tf < Li) << (jj + 1);
+                    SP::run(e0, e1, hi[jj >> 1], lo[jj >> 1]);
+                }
+                word &= vm;
+                if (live_row && (j0 >> 5) < p.Bw) reinterpret_cast<uint16_t *>(hrow)[j0 >> 4] = (uint16_t)word;
+                if (with_out) {
+                    const int gv = k * ntiles + kt;
+                    if (kt > 0) {                    // the previous tile's P.V has finished: P is free
+                        ok = mbar_wait(&bars->pv_done, par_pv, p.err, 0x502) && ok;
+                        par_pv ^= 1;
+                    }
+                    const int rz = n_tot - kt * TN;  // rows of this tile that exist
+                    if (rz < TN) ok = mbar_wait(&bars->v_full[gv & 1], (gv >> 1) & 1, p.err, 0x503) && ok;
+                    if (__any_sync(0xffffffffu, !ok)) {
+                        ok = false;
+                        *(volatile int *)&bars->abort_flag = 1;
+                        g_exit = g;
+                        break;
+                    }
+                    if (rz < TN) {                   // (the last tile only) stale cache rows beyond the chunk: zero them for P.V
+                        char *vt = Vt + (gv & 1) * TILE;
+                        for (int idx = tid; idx < (TN - rz) * 16; idx += NT) {
+                            const int row = rz + (idx >> 4), piece = idx & 15;
+                            *reinterpret_cast<uint4 *>(vt + (piece >> 3) * HALF_K + row * 128 + (piece & 7) * 16) = make_uint4(0, 0, 0, 0);
+                        }
+                    }
+#pragma unroll
+                    for (int cc = 0; cc < HC / 8; ++cc) {
+                        const int off = (i >> 3) * PG + (quarter * (HC / 8) + cc) * 128 + (i & 7) * 16;
+                        *reinterpret_cast<uint4 *>(Ph + off) = make_uint4(hi[4 * cc], hi[4 * cc + 1], hi[4 * cc + 2], hi[4 * cc + 3]);
+                        *reinterpret_cast<uint4 *>(Pl + off) = make_uint4(lo[4 * cc], lo[4 * cc + 1], lo[4 * cc + 2], lo[4 * cc + 3]);
+                    }
+                    fence_async_shared();
+                    mbar_arrive(&bars->p_ready);     // this thread's part of P(kt) is in place
+                }
+            }
+            if (g_exit < ntiles) {               // the others may be waiting at the three barriers of the first sweep's end
+                softmax_barrier();
+                softmax_barrier();
+                softmax_barrier();
+            }
+            if (!ok) break;
+            if (live_row && quarter == 0)
+                for (int wd = ntiles * (TN / 32); wd < p.Bw; ++wd) hrow[wd] = 0;
+            if (with_out) {
+                ok = mbar_wait(&bars->pv_done, par_pv, p.err, 0x504) && ok;
+                par_pv ^= 1;
+                if (__any_sync(0xffffffffu, !ok)) {
+                    ok = false;
+                    *(volatile int *)&bars->abort_flag = 1;
+                    break;
+                }
+                tc_fence_after();
+                const int dcol = tid & 127, bq = tid >> 7;
+                float ov[32];
+                tmem_ld32(lane_addr + O_COL + bq * 32, ov);
+                tc_fence_before();
+                mbar_arrive(&bars->o_free);          // O^T may be overwritten by the next unit
+#pragma unroll
+                for (int qq = 0; qq < 32; ++qq) {
+                    const int qi = bq * 32 + qq;
+                    if (qi < c) p.out[((size_t)qi * p.Utot + u) * D + dcol] = ov[qq] * Linv[qi];
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tbase), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+
+typedef CUresult (*EncodeTiled)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up through the runtime (the library does not link against the driver).
+EncodeTiled encoder() {
+    static EncodeTiled fn = [] {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            sym = nullptr;
+        return reinterpret_cast<EncodeTiled>(sym);
+    }();
+    return fn;
+}
+
+// Map over rows of 128 16-bit elements: [dim2][dim1][128], boxes of 64 elements x (box1 x box2) rows, 128-byte swizzle,
+// zeros outside the tensor.
+bool make_map(CUtensorMap *m, const void *base, uint64_t dim1, uint64_t dim2, uint64_t stride1, uint64_t stride2, uint32_t box1,
+              uint32_t box2) {
+    EncodeTiled enc = encoder();
+    if (!enc) return false;
+    const cuuint64_t gdim[3] = {(cuuint64_t)D, dim1, dim2};
+    const cuuint64_t gstride[2] = {stride1, stride2};
+    const cuuint32_t box[3] = {64u, box1, box2};
+    const cuuint32_t estr[3] = {1u, 1u, 1u};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT16, 3, const_cast<void *>(base), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+    static int n = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) v = 0;
+        return v;
+    }();
+    return n;
+}
+
+template <int DT>
+cudaError_t launch_tma(const ChunkParams &p, cudaStream_t s) {
+    CUtensorMap mq, mk, mv;
+    const uint64_t row = (uint64_t)D * 2;
+    if (!make_map(&mq, p.q, (uint64_t)p.Utot, (uint64_t)p.c, row, (uint64_t)p.Utot * row, 1, CQ) ||
+        !make_map(&mk, p.K, (uint64_t)p.B, (uint64_t)p.U, row, (uint64_t)p.B * row, TN, 1) ||
+        !make_map(&mv, p.V, (uint64_t)p.B, (uint64_t)p.U, row, (uint64_t)p.B * row, TN, 1))
+        return cudaErrorNotSupported;
+    auto kern = sh_chunk_umma_tma_kernel<DT>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    const int sms = sm_count();
+    if (sms <= 0) return cudaErrorInvalidDevice;
+    const int grid = p.U < 2 * sms ? p.U : 2 * sms;
+    kern<<<dim3(grid, 1, 1), NTHREADS, SMEM_BYTES, s>>>(p, mq, mk, mv);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t sh_launch_chunk_umma_tma(const ChunkParams &p, int dtype, cudaStream_t s) {
+    if (p.c < 1 || p.c > CQ || p.U < 1) return cudaErrorInvalidValue;
+    return dtype == SH_F16 ? launch_tma<SH_F16>(p, s) : launch_tma<SH_BF16>(p, s);
+}
