@@ -86,11 +86,12 @@ typedef enum {
                                  m = 64).  The kept set is the same either way: nothing in Algorithm 2 depends
                                  on where a token is stored. */
     SH_OPT_PREFILL_CHUNK = 4, /* 1 (default): sh_prefill hands the tokens between two compressions to a chunk
-                                 kernel: the tcgen05 kernels for fp16/bf16/int4 with head_dim 128 (any budget),
-                                 the CUDA-core kernel for fp32 rows and for head_dim 64; 0: one decode step per
-                                 token; 2: the warp-level MMA chunk kernel where it applies (fp16/bf16, head_dim
-                                 128, budgets up to about 700); 3: same as 1; 4: the CUDA-core kernel for every
-                                 shape */
+                                 kernel: the tcgen05 kernels for fp16/bf16/int4 with head_dim 128 (any budget;
+                                 fp16/bf16: persistent CTAs fed by tiled TMA copies), the CUDA-core kernel for
+                                 fp32 rows and for head_dim 64; 0: one decode step per token; 2: the warp-level
+                                 MMA chunk kernel where it applies (fp16/bf16, head_dim 128, budgets up to about
+                                 700); 3: as 1, but fp16/bf16 use the tcgen05 kernel with one CTA per unit and
+                                 per-thread asynchronous copies; 4: the CUDA-core kernel for every shape */
     SH_OPT_DECODE_KERNEL = 3, /* 0 (default): chosen from the shape; 1: one CTA (or cluster) per unit with
                                  direct loads; 2: persistent CTAs fed by bulk asynchronous copies
                                  (stored rows of 256 bytes or more: fp32, and fp16/bf16 with head_dim 128; SH_OPT_SPLIT

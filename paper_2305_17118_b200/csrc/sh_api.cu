@@ -339,7 +339,7 @@ int sh_set_option(sh_handle h, int key, double value) {
         }
         case SH_OPT_PREFILL_CHUNK: {
             const int mode = (int)value;
-            if (mode < 0 || mode > 5) return SH_EINVAL;
+            if (mode < 0 || mode > 4) return SH_EINVAL;
             const int before = h->prefill_chunk;
             h->prefill_chunk = mode;
             if (h->record_mode && !sh_recount_supported(h)) {     // the recount would not fit the chosen kernel

@@ -364,308 +364,6 @@ __global__ void __launch_bounds__(NT, 2) sh_chunk_umma_kernel(const ChunkParams 
     }
 }
 
-// ---------------------------------------------------------------------------------------------------------------
-// The same chunk step with the tensor core driven by a warp of its own.  In the kernel above thread 0 issues the
-// MMAs between two CTA-wide barriers, so 255 threads wait while one builds descriptors, and the tensor core waits
-// while they do arithmetic.  Here warp 8 does nothing but issue: it waits on mbarriers for "key tile landed", "S
-// buffer read out" and "P written", issues S one tile ahead and P.V as soon as its P exists; the 256 softmax threads
-// never meet at a CTA-wide barrier in the loop, they only wait for "S(g) done" and "P.V(kt-1) done".  Chunk mode only
-// (the recount has no second contraction and keeps the kernel above).
-constexpr int NTW = NT + 32;
-constexpr int WS_SMEM_BYTES = SMEM_BYTES + 64;      // five more mbarriers
-static_assert(2 * (WS_SMEM_BYTES + 1024) <= 228 * 1024, "two CTAs per SM");
-
-__device__ __forceinline__ void softmax_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory"); }
-
-template <int DT>
-__global__ void __launch_bounds__(NTW, 2) sh_chunk_umma_ws_kernel(const ChunkParams p) {
-    using SP = Split<DT>;
-    extern __shared__ __align__(128) unsigned char sm[];
-    char *Qs = reinterpret_cast<char *>(sm) + OFF_Q;
-    char *Kt = reinterpret_cast<char *>(sm) + OFF_K;
-    char *Vt = reinterpret_cast<char *>(sm) + OFF_V;
-    char *Ph = reinterpret_cast<char *>(sm) + OFF_PH;
-    char *Pl = reinterpret_cast<char *>(sm) + OFF_PL;
-    float *m_sh = reinterpret_cast<float *>(sm + OFF_PH);
-    float *l_sh = m_sh + NT;
-    float *Mfin = reinterpret_cast<float *>(sm + OFF_STAT), *Lfin = Mfin + 64;
-    uint64_t *bar_s = reinterpret_cast<uint64_t *>(sm + OFF_BAR);     // [2] S(g) computed        (1 arrival: commit)
-    uint64_t *bar_pv = bar_s + 2;                                      //     P.V(kt) computed     (1 arrival: commit)
-    uint64_t *k_ready = bar_s + 3;                                     // [2] key tile in buffer b (NT arrivals)
-    uint64_t *s_free = bar_s + 5;                                      // [2] S buffer b read out  (NT arrivals)
-    uint64_t *p_ready = bar_s + 7;                                     //     P and V tile in place (NT arrivals)
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bar_s + 8);
-    int *abort_flag = reinterpret_cast<int *>(tmem_slot + 1);          // a bounded wait gave up somewhere: everybody leaves
-
-    const int u = blockIdx.x, tid = threadIdx.x, warp = tid >> 5;
-    const int i = tid & 63, quarter = ((tid >> 6) & 1) * 2 + ((tid >> 7) & 1);
-    const int n0 = p.n0, c = p.c, n_tot = n0 + c;
-    const int ntiles = (n_tot + TN - 1) / TN, G = 2 * ntiles;
-    const int step0 = p.t0 + 1;
-    const size_t tstride = (size_t)p.Utot * D * 2;
-    const char *Kc = p.K + (size_t)u * p.B * D * 2;
-    const char *Vc = p.V + (size_t)u * p.B * D * 2;
-    const char *kchunk = p.k + (size_t)u * D * 2, *vchunk = p.v + (size_t)u * D * 2;
-    auto key_tile = [&](int g) { return g < ntiles ? g : g - ntiles; };
-
-    if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    if (tid == 0) {
-        mbar_init(bar_s, 1); mbar_init(bar_s + 1, 1); mbar_init(bar_pv, 1);
-        mbar_init(k_ready, NT); mbar_init(k_ready + 1, NT);
-        mbar_init(s_free, NT); mbar_init(s_free + 1, NT);
-        mbar_init(p_ready, NT);
-        *abort_flag = 0;
-        fence_barrier_init();
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tbase = *tmem_slot;
-
-    if (warp == NT / 32) {
-        // ------------------------------------------------------------------------------------------ the issuing warp
-        if ((tid & 31) == 0) {
-            const uint32_t q_addr = smem_u32(Qs), k_addr = smem_u32(Kt), v_addr = smem_u32(Vt), ph_addr = smem_u32(Ph), pl_addr = smem_u32(Pl);
-            const uint32_t idesc_s = instr_desc(SP::FMT, 0, 128, TN);
-            const uint32_t idesc_pv = instr_desc(SP::FMT, 1, 128, CQ);
-            uint32_t par_k = 0, par_f = 0, par_p = 0;          // bit b: parity the next wait on barrier b expects
-            bool ok = true;
-            auto issue_s = [&](int g) {
-                const int b = g & 1;
-                ok = ok && mbar_wait(k_ready + b, (par_k >> b) & 1, p.err, 0x511);
-                par_k ^= 1u << b;
-                if (g >= 2) {                                   // S(g - 2) has been read out of this buffer
-                    ok = ok && mbar_wait(s_free + b, (par_f >> b) & 1, p.err, 0x512);
-                    par_f ^= 1u << b;
-                }
-                if (!ok) return;
-                tc_fence_after();
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)
-                    umma_f16(tbase + S_COL + b * TN, smem_desc(q_addr + ks * 256, 128, GROUP),
-                             smem_desc(k_addr + b * TILE + ks * 256, 128, GROUP), idesc_s, ks > 0);
-                umma_commit(bar_s + b);
-            };
-            issue_s(0);
-            for (int g = 0; g < G && ok; ++g) {
-                if (g + 1 < G) issue_s(g + 1);
-                if (g >= ntiles && p.out && ok) {
-                    const int kt = g - ntiles;
-                    ok = mbar_wait(p_ready, par_p, p.err, 0x513);
-                    par_p ^= 1;
-                    if (!ok) break;
-                    tc_fence_after();
-#pragma unroll
-                    for (int ks = 0; ks < TN / 16; ++ks) {
-                        const uint64_t a = smem_desc(v_addr + (kt & 1) * TILE + ks * 2 * GROUP, GROUP, 128);
-                        umma_f16(tbase + O_COL, a, smem_desc(ph_addr + ks * 256, 128, PG), idesc_pv, (kt > 0 || ks > 0));
-                        umma_f16(tbase + O_COL, a, smem_desc(pl_addr + ks * 256, 128, PG), idesc_pv, 1);
-                    }
-                    umma_commit(bar_pv);
-                }
-                if (*(volatile int *)abort_flag) ok = false;
-            }
-            if (!ok) *(volatile int *)abort_flag = 1;
-        }
-    } else {
-        // ------------------------------------------------------------------------------------------ softmax threads
-        load_tile(Kt, Kc, kchunk, 0, n0, n_tot, tstride);
-        load_tile(Kt + TILE, Kc, kchunk, key_tile(1) * TN, n0, n_tot, tstride);
-        if (p.out) load_tile(Vt, Vc, vchunk, 0, n0, n_tot, tstride);
-        // queries (rows beyond c are zero), twice: rows 0..63 and 64..127
-        for (int idx = tid; idx < CQ * 16; idx += NT) {
-            const int row = idx >> 4, ch = idx & 15;
-            char *dst = Qs + (row >> 3) * GROUP + ch * 128 + (row & 7) * 16;
-            if (row < c) {
-                const char *src = p.q + (size_t)row * tstride + (size_t)u * D * 2 + ch * 16;
-                cp_async16(dst, src);
-                cp_async16(dst + (CQ / 8) * GROUP, src);
-            } else {
-                *reinterpret_cast<uint4 *>(dst) = make_uint4(0, 0, 0, 0);
-                *reinterpret_cast<uint4 *>(dst + (CQ / 8) * GROUP) = make_uint4(0, 0, 0, 0);
-            }
-        }
-        // while those copies fly: append the chunk's keys, values and positions, remember the queries
-        if (tid < c) p.pos[(size_t)u * p.B + n0 + tid] = step0 + tid;
-        {
-            constexpr int PER = CQ * 16 / NT;
-            uint4 kk[PER], vv[PER], qq[PER];
-#pragma unroll
-            for (int a = 0; a < PER; ++a) {
-                const int idx = tid + a * NT, row = idx >> 4, ch = idx & 15;
-                if (row < c) {
-                    const size_t src = (size_t)row * tstride + (size_t)u * D * 2 + ch * 16;
-                    kk[a] = *reinterpret_cast<const uint4 *>(p.k + src);
-                    vv[a] = *reinterpret_cast<const uint4 *>(p.v + src);
-                    if (p.qring) qq[a] = *reinterpret_cast<const uint4 *>(p.q + src);
-                }
-            }
-#pragma unroll
-            for (int a = 0; a < PER; ++a) {
-                const int idx = tid + a * NT, row = idx >> 4, ch = idx & 15;
-                if (row < c) {
-                    const size_t dst = ((size_t)u * p.B + n0 + row) * (D * 2) + ch * 16;
-                    *reinterpret_cast<uint4 *>(p.K + dst) = kk[a];
-                    *reinterpret_cast<uint4 *>(p.V + dst) = vv[a];
-                    if (p.qring) *reinterpret_cast<uint4 *>(p.qring + ((size_t)u * p.w + (step0 + row) % p.w) * (D * 2) + ch * 16) = qq[a];
-                }
-            }
-        }
-        cp_async_commit();
-        cp_async_wait_all();
-        fence_async_shared();
-        mbar_arrive(k_ready);            // key tiles 0 and 1 (and the queries) are in place
-        mbar_arrive(k_ready + 1);
-
-        const uint32_t lane_addr = tbase + ((uint32_t)((warp & 3) * 32) << 16);
-        uint32_t par_s = 0, par_pv = 0;
-        bool ok = true;
-        int g_exit = G;                      // the iteration a warp left the loop at, after a wait that gave up
-        const int nv = n0 + i + 1;           // keys visible to this thread's query
-        const bool live_row = i < c;
-        float m_run = -INFINITY, l_run = 0.f;
-        float Mi = 0.f, Li = 1.f;
-        const float tf = (float)(step0 + i);
-        uint32_t *hrow = p.hist + ((size_t)u * p.w + (step0 + i) % p.w) * p.Bw;
-        for (int g = 0; g < G; ++g) {
-            const int kt = key_tile(g);
-            const bool second = g >= ntiles;
-            if (g >= 1) {                    // the copies started one iteration ago have landed: key tile g + 1, value tile kt
-                cp_async_wait_all();
-                fence_async_shared();
-                if (g + 1 < G) mbar_arrive(k_ready + ((g + 1) & 1));
-            }
-            ok = mbar_wait(bar_s + (g & 1), (par_s >> (g & 1)) & 1, p.err, 0x501) && ok;
-            par_s ^= 1u << (g & 1);
-            // (one decision per warp: the tensor-memory loads below are warp-wide)
-            if (__any_sync(0xffffffffu, !ok || *(volatile int *)abort_flag != 0)) {
-                ok = false;
-                *(volatile int *)abort_flag = 1;
-                g_exit = g;
-                break;
-            }
-            tc_fence_after();
-            if (g + 2 < G) load_tile(Kt + (g & 1) * TILE, Kc, kchunk, key_tile(g + 2) * TN, n0, n_tot, tstride);
-            cp_async_commit();
-            float sv[HC];
-            tmem_ld16(lane_addr + S_COL + (g & 1) * TN + quarter * HC, sv);
-            tc_fence_before();
-            mbar_arrive(s_free + (g & 1));       // this thread's share of S(g) is in registers
-            const int j0 = kt * TN + quarter * HC;
-            const int lim = live_row ? nv - j0 : 0;
-            const uint32_t vm = lim <= 0 ? 0u : (lim >= HC ? 0xffffu : (1u << lim) - 1u);
-            if (!second) {
-                if (vm) {
-                    float bmax = -INFINITY;
-#pragma unroll
-                    for (int jj = 0; jj < HC; ++jj) {
-                        sv[jj] = ((vm >> jj) & 1u) ? sv[jj] * p.scale_log2e : -INFINITY;
-                        bmax = fmaxf(bmax, sv[jj]);
-                    }
-                    const float m_new = fmaxf(m_run, bmax);
-                    float acc = 0.f;
-#pragma unroll
-                    for (int jj = 0; jj < HC; ++jj) acc += ex2_approx(sv[jj] - m_new);
-                    l_run = l_run * ex2_approx(m_run - m_new) + acc;
-                    m_run = m_new;
-                }
-                if (g == ntiles - 1) {
-                    m_sh[tid] = m_run;
-                    l_sh[tid] = l_run;
-                    softmax_barrier();
-                    if (tid < CQ) {
-                        float M = -INFINITY, L = 0.f;
-#pragma unroll
-                        for (int part = 0; part < NT / CQ; ++part) M = fmaxf(M, m_sh[tid + part * CQ]);
-#pragma unroll
-                        for (int part = 0; part < NT / CQ; ++part) {
-                            const float mp = m_sh[tid + part * CQ];
-                            if (mp > -INFINITY) L += l_sh[tid + part * CQ] * ex2_approx(mp - M);
-                        }
-                        Mfin[tid] = M;
-                        Lfin[tid] = L;
-                    }
-                    softmax_barrier();
-                    Mi = Mfin[i];
-                    Li = Lfin[i];
-                    softmax_barrier();       // everyone has its row's M and L: the P buffer (m_sh, l_sh) may be written
-                }
-                continue;
-            }
-            uint32_t word = 0, hi[HC / 2], lo[HC / 2];
-#pragma unroll
-            for (int jj = 0; jj < HC; jj += 2) {
-                const bool v0 = (vm >> jj) & 1u, v1 = (vm >> (jj + 1)) & 1u;
-                const float e0 = v0 ? ex2_approx(sv[jj] * p.scale_log2e - Mi) : 0.f;
-                const float e1 = v1 ? ex2_approx(sv[jj + 1] * p.scale_log2e - Mi) : 0.f;
-                word |= (uint32_t)(e0 * tf < Li) << jj;
-                word |= (uint32_t)(e1 * tf < Li) << (jj + 1);
-                SP::run(e0, e1, hi[jj >> 1], lo[jj >> 1]);
-            }
-            word &= vm;
-            if (live_row && (j0 >> 5) < p.Bw) reinterpret_cast<uint16_t *>(hrow)[j0 >> 4] = (uint16_t)word;
-            if (p.out) {
-                if (kt > 0) {                    // the previous tile's P.V has finished: P and the V buffer it read are free
-                    ok = mbar_wait(bar_pv, par_pv, p.err, 0x502) && ok;
-                    par_pv ^= 1;
-                    if (__any_sync(0xffffffffu, !ok)) {
-                        ok = false;
-                        *(volatile int *)abort_flag = 1;
-                        g_exit = g;
-                        break;
-                    }
-                }
-                if (kt + 1 < ntiles) load_tile(Vt + ((kt + 1) & 1) * TILE, Vc, vchunk, (kt + 1) * TN, n0, n_tot, tstride);
-                cp_async_commit();
-#pragma unroll
-                for (int cc = 0; cc < HC / 8; ++cc) {
-                    const int off = (i >> 3) * PG + (quarter * (HC / 8) + cc) * 128 + (i & 7) * 16;
-                    *reinterpret_cast<uint4 *>(Ph + off) = make_uint4(hi[4 * cc], hi[4 * cc + 1], hi[4 * cc + 2], hi[4 * cc + 3]);
-                    *reinterpret_cast<uint4 *>(Pl + off) = make_uint4(lo[4 * cc], lo[4 * cc + 1], lo[4 * cc + 2], lo[4 * cc + 3]);
-                }
-                fence_async_shared();
-                mbar_arrive(p_ready);            // this thread's part of P(kt) and of the value tile are in place
-            }
-        }
-        if (g_exit < ntiles) {               // the others may be waiting at the three barriers of the first sweep's end
-            softmax_barrier();
-            softmax_barrier();
-            softmax_barrier();
-        }
-        if (ok) {
-            if (live_row && quarter == 0)
-                for (int wd = ntiles * (TN / 32); wd < p.Bw; ++wd) hrow[wd] = 0;
-            if (p.out) {
-                ok = mbar_wait(bar_pv, par_pv, p.err, 0x504) && ok;
-                tc_fence_after();
-            }
-        }
-        if (p.out) {
-            const int dcol = tid & 127, b = tid >> 7;
-            float ov[32];
-            tmem_ld32(lane_addr + O_COL + b * 32, ov);
-            if (ok) {
-#pragma unroll
-                for (int qq = 0; qq < 32; ++qq) {
-                    const int qi = b * 32 + qq;
-                    if (qi < c) p.out[((size_t)qi * p.Utot + u) * D + dcol] = ov[qq] / Lfin[qi];
-                }
-            }
-        }
-        cp_async_wait_all();
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 0) {
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tbase), "r"(TMEM_COLS) : "memory");
-    }
-}
-
 template <int DT, bool RECOUNT>
 cudaError_t launch(const ChunkParams &p, cudaStream_t s) {
     auto kern = sh_chunk_umma_kernel<DT, RECOUNT>;
@@ -680,21 +378,9 @@ cudaError_t launch(const ChunkParams &p, cudaStream_t s) {
 
 int sh_chunk_umma_capacity() { return CQ; }
 
-namespace {
-template <int DT>
-cudaError_t launch_ws(const ChunkParams &p, cudaStream_t s) {
-    auto kern = sh_chunk_umma_ws_kernel<DT>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, WS_SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    kern<<<dim3(p.U, 1, 1), NTW, WS_SMEM_BYTES, s>>>(p);
-    return cudaGetLastError();
-}
-}  // namespace
-
-cudaError_t sh_launch_chunk_umma(const ChunkParams &p, int dtype, cudaStream_t s, bool issuing_warp) {
+cudaError_t sh_launch_chunk_umma(const ChunkParams &p, int dtype, cudaStream_t s) {
     if (p.c < 1 || p.c > CQ) return cudaErrorInvalidValue;
-    if (!issuing_warp) return dtype == SH_F16 ? launch<SH_F16, false>(p, s) : launch<SH_BF16, false>(p, s);
-    return dtype == SH_F16 ? launch_ws<SH_F16>(p, s) : launch_ws<SH_BF16>(p, s);
+    return dtype == SH_F16 ? launch<SH_F16, false>(p, s) : launch<SH_BF16, false>(p, s);
 }
 
 cudaError_t sh_launch_recount_umma(const ChunkParams &p, int dtype, cudaStream_t s) {

@@ -48,9 +48,10 @@ constexpr int PG = (TN / 8) * 128;      // bytes of 8 rows of P (TN keys each) i
 constexpr int P_BYTES = (CQ / 8) * PG;
 constexpr int HC = TN / 4;              // columns of a tile per thread (four threads share a query row)
 static_assert(HC == 16, "a thread reads its 16 columns with one tcgen05.ld and owns half a record word");
-constexpr int TMEM_COLS = 256;          // two S tiles and O^T; two CTAs fit in the 512 columns of an SM
+constexpr int TMEM_COLS = 256;          // two S tiles and O^T (twice: from P's high and low parts); two CTAs fit in an SM's 512 columns
 constexpr int S_COL = 0;
-constexpr int O_COL = 2 * TN;
+constexpr int O_COL = 2 * TN;           // columns [O_COL, O_COL + CQ): V^T.P_hi^T, the next CQ columns: V^T.P_lo^T
+static_assert(O_COL + 2 * CQ <= TMEM_COLS, "tensor memory columns");
 
 constexpr int OFF_Q = 0;
 constexpr int OFF_K = OFF_Q + Q_BYTES;
@@ -61,6 +62,7 @@ constexpr int OFF_STAT = OFF_PL + P_BYTES;      // M[64], L[64], 1/L[64]
 constexpr int OFF_BAR = OFF_STAT + 4 * 3 * 64;
 constexpr int SMEM_BYTES = OFF_BAR + 192;
 static_assert(OFF_K % 1024 == 0 && OFF_V % 1024 == 0 && HALF_K % 1024 == 0, "swizzled tiles start on 1024-byte boundaries");
+static_assert(OFF_PL == OFF_PH + P_BYTES, "P_hi and P_lo form one B operand of 2 CQ rows");
 static_assert(P_BYTES >= 4 * 2 * NT, "the first sweep's statistics alias the P buffer");
 static_assert(2 * (SMEM_BYTES + 1024) <= 228 * 1024, "two CTAs per SM");
 
@@ -173,22 +175,39 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
     if (warp == W_MMA) {
         // --------------------------------------------------------------------------------------- the issuing thread
         if (lane == 0 && start_ok) {
-            const uint32_t q_addr = smem_u32(Qs), k_addr = smem_u32(Kt), v_addr = smem_u32(Vt), ph_addr = smem_u32(Ph), pl_addr = smem_u32(Pl);
             const uint32_t idesc_s = instr_desc(SP::FMT, 0, 128, TN);
-            const uint32_t idesc_pv = instr_desc(SP::FMT, 1, 128, CQ);
+            const uint32_t idesc_pv = instr_desc(SP::FMT, 1, 128, 2 * CQ);     // N = the queries' high parts, then their low parts
+            // every descriptor this thread will ever use, built once: the loops below only issue
+            uint64_t dq[D / 16], dk[KST][D / 16], dv[2][TN / 16], dp[TN / 16];
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) {
+                dq[ks] = smem_desc_sw128(smem_u32(Qs) + (ks >> 2) * HALF_Q + (ks & 3) * 32, 16, 1024);
+#pragma unroll
+                for (int s = 0; s < KST; ++s) dk[s][ks] = smem_desc_sw128(smem_u32(Kt) + s * TILE + (ks >> 2) * HALF_K + (ks & 3) * 32, 16, 1024);
+            }
+#pragma unroll
+            for (int ks = 0; ks < TN / 16; ++ks) {
+                dv[0][ks] = smem_desc_sw128(smem_u32(Vt) + ks * 2048, HALF_K, 1024);
+                dv[1][ks] = smem_desc_sw128(smem_u32(Vt) + TILE + ks * 2048, HALF_K, 1024);
+                dp[ks] = smem_desc(smem_u32(Ph) + ks * 256, 128, PG);       // 16 row groups: P_hi, then P_lo
+            }
             bool ok = true;
             auto issue_s = [&](int k, int g) {
-                const int gk = k * G + g, s = gk % KST, b = gk & 1;
+                const int gk = k * G + g, b = gk & 1;
+                static_assert(KST == 2, "the key stage of S(gk) is the S buffer's index");
                 if (g == 0) ok = ok && mbar_wait(&bars->q_full, k & 1, p.err, 0x521);
-                ok = ok && mbar_wait(&bars->k_full[s], (gk / KST) & 1, p.err, 0x522);
+                ok = ok && mbar_wait(&bars->k_full[b], (gk / KST) & 1, p.err, 0x522);
                 if (gk >= 2) ok = ok && mbar_wait(&bars->s_free[b], ((gk >> 1) - 1) & 1, p.err, 0x523);   // S(gk - 2) has been read out
                 if (!ok) return;
                 tc_fence_after();
+                if (b == 0) {
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)
-                    umma_f16(tbase + S_COL + b * TN, smem_desc_sw128(q_addr + (ks >> 2) * HALF_Q + (ks & 3) * 32, 16, 1024),
-                             smem_desc_sw128(k_addr + s * TILE + (ks >> 2) * HALF_K + (ks & 3) * 32, 16, 1024), idesc_s, ks > 0);
-                umma_commit(&bars->k_empty[s]);
+                    for (int ks = 0; ks < D / 16; ++ks) umma_f16(tbase + S_COL, dq[ks], dk[0][ks], idesc_s, ks > 0);
+                } else {
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) umma_f16(tbase + S_COL + TN, dq[ks], dk[1][ks], idesc_s, ks > 0);
+                }
+                umma_commit(&bars->k_empty[b]);
                 umma_commit(&bars->s_done[b]);
                 if (g == G - 1) umma_commit(&bars->q_empty);
             };
@@ -205,11 +224,7 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
                         if (!ok) break;
                         tc_fence_after();
 #pragma unroll
-                        for (int ks = 0; ks < TN / 16; ++ks) {
-                            const uint64_t a = smem_desc_sw128(v_addr + b * TILE + ks * 2048, HALF_K, 1024);
-                            umma_f16(tbase + O_COL, a, smem_desc(ph_addr + ks * 256, 128, PG), idesc_pv, (kt > 0 || ks > 0));
-                            umma_f16(tbase + O_COL, a, smem_desc(pl_addr + ks * 256, 128, PG), idesc_pv, 1);
-                        }
+                        for (int ks = 0; ks < TN / 16; ++ks) umma_f16(tbase + O_COL, b ? dv[1][ks] : dv[0][ks], dp[ks], idesc_pv, (kt > 0 || ks > 0));
                         umma_commit(&bars->v_empty[b]);
                         umma_commit(&bars->pv_done);
                     }
@@ -453,15 +468,19 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
                     break;
                 }
                 tc_fence_after();
-                const int dcol = tid & 127, bq = tid >> 7;
-                float ov[32];
-                tmem_ld32(lane_addr + O_COL + bq * 32, ov);
+                const int dcol = tid & 127, bq = tid >> 7;      // this thread's column of d and its half of the queries
+                float oh[2][16], ol[2][16];
+#pragma unroll
+                for (int part = 0; part < 2; ++part) {
+                    tmem_ld16(lane_addr + O_COL + bq * 32 + part * 16, oh[part]);
+                    tmem_ld16(lane_addr + O_COL + CQ + bq * 32 + part * 16, ol[part]);
+                }
                 tc_fence_before();
                 mbar_arrive(&bars->o_free);          // O^T may be overwritten by the next unit
 #pragma unroll
                 for (int qq = 0; qq < 32; ++qq) {
                     const int qi = bq * 32 + qq;
-                    if (qi < c) p.out[((size_t)qi * p.Utot + u) * D + dcol] = ov[qq] * Linv[qi];
+                    if (qi < c) p.out[((size_t)qi * p.Utot + u) * D + dcol] = (oh[qq >> 4][qq & 15] + ol[qq >> 4][qq & 15]) * Linv[qi];
                 }
             }
         }

@@ -188,7 +188,7 @@ struct ChunkParams {
 
 // tcgen05 version of the chunked prompt step (fp16/bf16, head_dim 128, any budget): tokens per launch, launcher.
 int sh_chunk_umma_capacity();
-cudaError_t sh_launch_chunk_umma(const ChunkParams &p, int dtype, cudaStream_t s, bool issuing_warp);
+cudaError_t sh_launch_chunk_umma(const ChunkParams &p, int dtype, cudaStream_t s);
 cudaError_t sh_launch_recount_umma(const ChunkParams &p, int dtype, cudaStream_t s);
 // the same chunk step with persistent CTAs and tiled TMA copies (sh_chunk_umma_tma.cu)
 cudaError_t sh_launch_chunk_umma_tma(const ChunkParams &p, int dtype, cudaStream_t s);

@@ -387,7 +387,7 @@ cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const vo
         return e;
     }
     if (c->prefill_chunk != 2) {
-        e = c->prefill_chunk == 1 ? sh_launch_chunk_umma_tma(p, c->dtype, s) : sh_launch_chunk_umma(p, c->dtype, s, c->prefill_chunk == 5);
+        e = c->prefill_chunk == 1 ? sh_launch_chunk_umma_tma(p, c->dtype, s) : sh_launch_chunk_umma(p, c->dtype, s);
         if (e == cudaSuccess) *launches += 1;
         return e;
     }

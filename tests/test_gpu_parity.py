@@ -86,13 +86,13 @@ def test_lockstep_pipelined_kernel(sh, dtype, d, U, B, r, w, m):
 @pytest.mark.parametrize("U,B,r,w,m,sizes", [(5, 150, 9, 37, 41, [64, 7, 33, 1, 50]), (3, 410, 64, 128, 64, [64]),
                                              (2, 700, 5, 64, 300, [32, 17]), (4, 40, 3, 9, 20, [5, 9, 2]),
                                              (130, 96, 8, 70, 30, [64, 31])])
-@pytest.mark.parametrize("chunk_kernel", [1, 2])
+@pytest.mark.parametrize("chunk_kernel", [1, 2, 3])
 def test_lockstep_chunked_prompt_kernel(sh, dtype, U, B, r, w, m, sizes, chunk_kernel):
     """sh_prefill_chunk against the oracle replaying the same steps one by one: outputs of
     every step, its record bits, positions, counters and kept sets."""
     d, T = 128, 2 * B + 2 * m + 11
     q, k, v = wl.random_stream(U, d, T, seed=17 + U, dtype=dtype, peaked=3.0, device="cuda")
-    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, prefill_chunk=chunk_kernel)   # 1: tcgen05, 2: warp-level MMA
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, prefill_chunk=chunk_kernel)   # 1: tcgen05, persistent CTAs and TMA; 2: warp-level MMA; 3: tcgen05, one CTA per unit
     blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
     res, orc = run_lockstep_chunked(h, dtype, blk, T, torch.arange(U), TOL[dtype], chunk_sizes=sizes)
     assert res.steps == T and res.compressions >= 3
@@ -137,6 +137,40 @@ def test_lockstep_chunked_tcgen05_kernel_shapes(sh, dtype, U, B, r, w, m, sizes)
     res, orc = run_lockstep_chunked(h, dtype, blk, T, torch.arange(U), TOL[dtype], chunk_sizes=sizes)
     assert res.steps == T and res.compressions >= 1
     assert res.adoptions <= 1e-4 * res.slot_steps + 2
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("U,B,r,w,m,sizes", [(700, 150, 9, 64, 41, [64, 7, 33]), (1000, 70, 5, 64, 30, [64]),
+                                             (297, 200, 9, 64, 90, [13, 64])])
+def test_lockstep_chunked_persistent_ctas(sh, dtype, U, B, r, w, m, sizes):
+    """The persistent tcgen05 chunk kernel with more units than CTAs (two per SM): every CTA walks over several
+    units, unevenly many, so its tile rings, the query buffer and the output accumulator are reused across
+    units; chunk lengths that leave stale cache rows in the last value tile, a first tile that already holds
+    rows of the chunk (n0 < 64), and a last unit that is the only second unit of its CTA (U = 297)."""
+    d, T = 128, B + 2 * m + 40
+    q, k, v = wl.random_stream(U, d, T, seed=41 + U, dtype=dtype, peaked=3.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
+    units = torch.cat([torch.arange(0, 6), torch.arange(290, min(U, 310)), torch.arange(U - 5, U)]).unique()
+    res, _ = run_lockstep_chunked(h, dtype, blk, T, units, TOL[dtype], chunk_sizes=sizes)
+    assert res.steps == T and res.compressions >= 2
+    assert res.adoptions <= 1e-4 * res.slot_steps + 2
+
+
+@pytest.mark.parametrize("dtype,U", [("f16", 5), ("bf16", 640)])
+def test_chunked_prompt_without_outputs_leaves_the_same_state(sh, dtype, U):
+    """sh_prefill with no output buffer (the second contraction is skipped altogether) leaves state bit-identical
+    to a twin that asked for the outputs: rows, positions, record, counters."""
+    B, r, w, m, d, T = 150, 9, 64, 41, 128, 400
+    q, k, v = wl.random_stream(U, d, T, seed=5, dtype=dtype, peaked=3.0, device="cuda")
+    a = sh.Handle(B, r, w, m, U, d, dtype)
+    b = sh.Handle(B, r, w, m, U, d, dtype)
+    out = torch.empty(T, U, d, device="cuda")
+    a.prefill(q, k, v, out)
+    b.prefill(q, k, v, None)
+    assert a.state()[1] == T
+    assert_same_state(a, b)
+    assert torch.isfinite(out).all()
 
 
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
