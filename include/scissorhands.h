@@ -100,7 +100,11 @@ typedef enum {
                                  In the kernel of SH_OPT_DECODE_KERNEL = 2 the first CTA never requests the k-th
                                  tile of rows it was due to stream, so the wait for that tile runs out after
                                  about a second, the CTA finishes without touching further cache state, and the
-                                 next sh_state returns SH_EDEVICE.  Outputs of such a step are meaningless. */
+                                 next sh_state returns SH_EDEVICE.  Outputs of such a step are meaningless.
+                                 The persistent tcgen05 chunk kernel (SH_OPT_PREFILL_CHUNK = 1, fp16/bf16,
+                                 head_dim 128) honours it the same way: its first CTA never requests the k-th key
+                                 tile of a launch (tiles counted over both sweeps), every role of that CTA gives up
+                                 within a few seconds and releases its tensor memory. */
 } sh_option;
 
 /*

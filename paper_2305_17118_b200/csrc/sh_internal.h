@@ -184,6 +184,7 @@ struct ChunkParams {
     // n0 cached rows, visible to a query when their position does not exceed its step
     int first_step, nsteps;
     int *err;                // device error word (a bounded wait gave up)
+    int selftest_skip_tile;  // persistent tcgen05 kernel only: -1, or the key tile of its first unit that CTA 0 never requests
 };
 
 // tcgen05 version of the chunked prompt step (fp16/bf16, head_dim 128, any budget): tokens per launch, launcher.

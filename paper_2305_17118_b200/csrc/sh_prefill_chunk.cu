@@ -374,6 +374,7 @@ cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const vo
     p.scale_log2e = (float)((double)c->scale * 1.4426950408889634);
     p.qring = sh_pqring(c);
     p.err = reinterpret_cast<int *>(c->slab + c->L.err);
+    p.selftest_skip_tile = c->selftest_skip_tile;
     cudaError_t e = cudaErrorInvalidValue;
     if (count < 1 || count > sh_prefill_chunk_capacity(c)) return e;
     if (use_simt(c)) {
@@ -406,6 +407,7 @@ cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const vo
 // present cache: rewrites the unit's bit-plane rows of those steps.
 cudaError_t sh_launch_recount(const sh_context *c, cudaStream_t s, long long *launches) {
     ChunkParams p = {};
+    p.selftest_skip_tile = -1;
     p.K = sh_pK(c); p.V = sh_pV(c);
     p.hist = sh_phist(c);
     p.pos = sh_ppos(c);

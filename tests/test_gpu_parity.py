@@ -865,6 +865,32 @@ def test_bounded_wait_gives_up_and_reports_device_error(sh):
     assert res.steps == 200
 
 
+@pytest.mark.parametrize("skip", [0, 1])
+def test_bounded_wait_gives_up_in_the_chunk_kernel(sh, skip):
+    """The same self-test on the persistent tcgen05 chunk kernel: its first CTA never requests one key tile (tile 0:
+    the first sweep's, so the softmax warps leave before the barriers that end the first sweep and have to
+    release one another there; tile 1: the second sweep's).  The MMA-issuing thread, the copy threads and the
+    softmax warps must all give up by themselves within seconds, tensor memory must be released (a fresh handle's
+    chunk kernel allocates it again), and sh_state must report SH_EDEVICE."""
+    import time
+    U, d, B, r, w, m, dtype = 5, 128, 300, 4, 64, 100, "f16"
+    q, k, v = wl.random_stream(U, d, 330, seed=79, dtype=dtype, peaked=2.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    h.set_option(sh.SH_OPT_SELFTEST_SKIP_TILE, skip)
+    out = torch.empty(64, U, d, device="cuda")
+    t0 = time.time()
+    h.prefill_chunk(q[:64].contiguous(), k[:64].contiguous(), v[:64].contiguous(), out)     # one key tile, two sweeps
+    rc = sh.lib.sh_state(h._h, None, None, None, None, None, None)
+    took = time.time() - t0
+    assert rc == sh.SH_EDEVICE and took < 30.0
+    assert b"bounded wait" in sh.lib.sh_strerror(rc)
+    torch.cuda.synchronize()
+    g = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
+    res, _ = run_lockstep_chunked(g, dtype, blk, 330, torch.arange(U), TOL[dtype], chunk_sizes=[64, 20])
+    assert res.steps == 330 and res.compressions >= 1
+
+
 def test_restore_boundaries_and_output_alignment(sh):
     import ctypes as C
     U, d, B, r, w, m, dtype = 4, 64, 16, 2, 8, 6, "f16"
