@@ -494,6 +494,302 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
 }
 
 
+// ---------------------------------------------------------------------------------------------------------------
+// The record recomputed at compression time (Algorithm 2 as stated) on the same structure.  A work item is one
+// unit and up to 128 of its last w steps: the queries come from the ring of stored queries and fill all 128 rows
+// of the MMA (nothing is duplicated), the keys are the n0 cached rows, a key is visible to a query when its
+// position does not exceed the query's step (slots need not be sorted).  Nothing is appended and no output is
+// formed: two sweeps over the key tiles (row maxima and sums, then the comparison bits), and each step's bit-plane
+// row is rewritten.  Warps 0..7: softmax arithmetic, two threads per query row, 32 columns each; warp 8: MMA issue;
+// warp 9: key tiles by TMA and the tiles' positions; warp 10: the queries, gathered from the ring into the
+// swizzled operand layout with plain loads and stores.
+constexpr int RQ = 128;                 // queries per work item
+constexpr int RKST = 2;                 // key tiles in flight
+constexpr int RPD = 4;                  // position tiles in flight (>= RKST + 2: see the producer)
+constexpr int RHC = TN / 2;             // columns of a tile per thread
+constexpr int RTHREADS = NT + 96;
+constexpr int R_TMEM_COLS = 2 * TN;     // two S tiles
+constexpr int ROFF_K = 2 * Q_BYTES;     // two query buffers: the next item's queries are gathered during the present item
+constexpr int ROFF_POS = ROFF_K + RKST * TILE;
+constexpr int ROFF_STAT = ROFF_POS + RPD * TN * 4;        // m[256], l[256], M[128], L[128]
+constexpr int ROFF_BAR = ROFF_STAT + 4 * (2 * NT + 2 * RQ);
+constexpr int R_SMEM_BYTES = ROFF_BAR + 256;
+static_assert(ROFF_K % 1024 == 0, "swizzled tiles start on 1024-byte boundaries");
+static_assert(RPD >= RKST + 2 && (RPD & (RPD - 1)) == 0, "position ring");
+static_assert(2 * (R_SMEM_BYTES + 1024) <= 228 * 1024, "two CTAs per SM");
+
+struct RBars {
+    uint64_t q_full[2], q_empty[2];
+    uint64_t k_full[RKST], k_empty[RKST];
+    uint64_t pos_full[RPD];
+    uint64_t s_done[2], s_free[2];
+    uint32_t tmem_slot;
+    int abort_flag;
+};
+static_assert(sizeof(RBars) <= 256, "barrier block");
+
+template <int DT>
+__global__ void __launch_bounds__(RTHREADS, 2) sh_recount_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap mapK) {
+    using SP = Split<DT>;
+    extern __shared__ __align__(1024) unsigned char sm[];
+    char *Qs = reinterpret_cast<char *>(sm);
+    char *Kt = reinterpret_cast<char *>(sm) + ROFF_K;
+    int *pos_sh = reinterpret_cast<int *>(sm + ROFF_POS);
+    float *m_sh = reinterpret_cast<float *>(sm + ROFF_STAT), *l_sh = m_sh + NT, *Mfin = l_sh + NT, *Lfin = Mfin + RQ;
+    RBars *bars = reinterpret_cast<RBars *>(sm + ROFF_BAR);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n0 = p.n0;
+    const int ntiles = (n0 + TN - 1) / TN, G = 2 * ntiles;
+    const int nblk = (p.nsteps + RQ - 1) / RQ;
+    const int items = p.U * nblk;
+    const int nitems = (items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;     // work items of this CTA
+    auto key_tile = [&](int g) { return g < ntiles ? g : g - ntiles; };
+    auto aborted = [&]() { return *(volatile int *)&bars->abort_flag != 0; };
+
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_slot)), "r"(R_TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+        for (int s = 0; s < 2; ++s) { mbar_init(&bars->q_full[s], 1); mbar_init(&bars->q_empty[s], 1); }
+        for (int s = 0; s < RKST; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1); }
+        for (int s = 0; s < RPD; ++s) mbar_init(&bars->pos_full[s], 1);
+        for (int s = 0; s < 2; ++s) { mbar_init(&bars->s_done[s], 1); mbar_init(&bars->s_free[s], NT); }
+        bars->abort_flag = 0;
+        if ((smem_u32(sm) & 1023u) != 0) {
+            if (p.err) atomicCAS(p.err, 0, 0x560);
+            bars->abort_flag = 1;
+        }
+        fence_barrier_init();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tbase = bars->tmem_slot;
+    const bool start_ok = !aborted() && n0 > 0;
+
+    if (warp == W_MMA) {
+        // --------------------------------------------------------------------------------------- the issuing thread
+        if (lane == 0 && start_ok) {
+            const uint32_t idesc_s = instr_desc(SP::FMT, 0, 128, TN);
+            // descriptors of query buffer 0 and key stage 0; the other buffers lie a fixed number of 16-byte units further
+            uint64_t dq[D / 16], dk[D / 16];
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) {
+                dq[ks] = smem_desc_sw128(smem_u32(Qs) + (ks >> 2) * HALF_Q + (ks & 3) * 32, 16, 1024);
+                dk[ks] = smem_desc_sw128(smem_u32(Kt) + (ks >> 2) * HALF_K + (ks & 3) * 32, 16, 1024);
+            }
+            bool ok = true;
+            for (int k = 0; k < nitems && ok; ++k) {
+                ok = mbar_wait(&bars->q_full[k & 1], (k >> 1) & 1, p.err, 0x561);
+                for (int g = 0; g < G && ok; ++g) {
+                    const int gk = k * G + g, s = gk % RKST, b = gk & 1;
+                    ok = mbar_wait(&bars->k_full[s], (gk / RKST) & 1, p.err, 0x562);
+                    if (gk >= 2) ok = ok && mbar_wait(&bars->s_free[b], ((gk >> 1) - 1) & 1, p.err, 0x563);   // S(gk - 2) has been read out
+                    if (!ok || aborted()) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t qoff = (uint64_t)((k & 1) * (Q_BYTES >> 4)), koff = (uint64_t)(s * (TILE >> 4));
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) umma_f16(tbase + b * TN, dq[ks] + qoff, dk[ks] + koff, idesc_s, ks > 0);
+                    umma_commit(&bars->k_empty[s]);
+                    umma_commit(&bars->s_done[b]);
+                    if (g == G - 1) umma_commit(&bars->q_empty[k & 1]);
+                }
+            }
+            if (!ok) *(volatile int *)&bars->abort_flag = 1;
+        }
+    } else if (warp == W_KQ) {
+        // --------------------------------------------------------------------------------------- key tiles and their positions
+        // the whole warp walks the tiles: lane 0 waits and requests the copy, every lane stores two positions
+        if (start_ok) {
+            bool ok = true;
+            int last = -1;
+            // the positions of a tile are fetched one tile early, so that their latency falls into the wait for the stage
+            auto fetch_pos = [&](int k, int g, int (&pv)[2]) {
+                if (k >= nitems) return;
+                const int u = (blockIdx.x + k * gridDim.x) / nblk, kt = key_tile(g);
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int j = kt * TN + h * 32 + lane;
+                    pv[h] = j < n0 ? p.pos[(size_t)u * p.B + j] : 0x7fffffff;      // slots beyond the cache: never visible
+                }
+            };
+            int pv[2];
+            fetch_pos(0, 0, pv);
+            for (int k = 0; k < nitems && ok; ++k) {
+                const int u = (blockIdx.x + k * gridDim.x) / nblk;
+                for (int g = 0; g < G; ++g) {
+                    const int gk = k * G + g, s = gk % RKST, kt = key_tile(g);
+                    if (lane == 0) {
+                        // S(gk - RKST) has been computed; it was issued after S(gk - RKST - 2) had been read out, and the
+                        // softmax threads read a tile's positions before they release its S buffer: so the positions
+                        // of tile gk - RPD are no longer needed, RPD >= RKST + 2
+                        if (gk >= RKST) ok = mbar_wait(&bars->k_empty[s], ((gk / RKST) - 1) & 1, p.err, 0x571);
+                        if (aborted()) ok = false;
+                    }
+                    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                    if (!ok) break;
+                    if (lane == 0) {
+                        mbar_arrive_expect_tx(&bars->k_full[s], TILE);
+                        tma_load_3d(Kt + s * TILE, &mapK, 0, kt * TN, u, &bars->k_full[s]);
+                        tma_load_3d(Kt + s * TILE + HALF_K, &mapK, 64, kt * TN, u, &bars->k_full[s]);
+                    }
+                    int *pt = pos_sh + (gk % RPD) * TN;
+                    pt[lane] = pv[0];
+                    pt[32 + lane] = pv[1];
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars->pos_full[gk % RPD]);
+                    last = gk;
+                    if (g + 1 < G) fetch_pos(k, g + 1, pv);
+                    else fetch_pos(k + 1, 0, pv);
+                }
+            }
+            if (lane == 0) {
+                if (!ok) *(volatile int *)&bars->abort_flag = 1;
+                for (int gk = last; gk > last - RKST && gk >= 0; --gk) mbar_wait(&bars->k_full[gk % RKST], (gk / RKST) & 1, nullptr, 0);
+            }
+        }
+    } else if (warp == W_V) {
+        // --------------------------------------------------------------------------------------- the queries
+        // rows (step mod w) of the unit's ring, 16 pieces of 16 bytes each, into the K-major 128-byte swizzle:
+        // piece ch of row r goes to half ch / 8, row r, 16-byte column (ch % 8) ^ (r % 8)
+        if (start_ok) {
+            bool ok = true;
+            for (int k = 0; k < nitems && ok; ++k) {
+                const int item = blockIdx.x + k * gridDim.x, u = item / nblk, qb = item % nblk;
+                const int s0 = p.first_step + qb * RQ, c = min(RQ, p.nsteps - qb * RQ);
+                if (lane == 0) {
+                    if (k >= 2) ok = mbar_wait(&bars->q_empty[k & 1], ((k >> 1) - 1) & 1, p.err, 0x581);     // item k - 2 has left this buffer
+                    if (aborted()) ok = false;
+                }
+                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                if (!ok) break;
+                char *Qb = Qs + (k & 1) * Q_BYTES;
+                for (int base = 0; base < RQ * 16; base += 8 * 32) {
+                    uint4 qq[8];
+#pragma unroll
+                    for (int a = 0; a < 8; ++a) {
+                        const int idx = base + a * 32 + lane, row = idx >> 4, ch = idx & 15;
+                        qq[a] = row < c ? *reinterpret_cast<const uint4 *>(p.qring + ((size_t)u * p.w + (s0 + row) % p.w) * (D * 2) + ch * 16)
+                                        : make_uint4(0, 0, 0, 0);
+                    }
+#pragma unroll
+                    for (int a = 0; a < 8; ++a) {
+                        const int idx = base + a * 32 + lane, row = idx >> 4, ch = idx & 15;
+                        *reinterpret_cast<uint4 *>(Qb + (ch >> 3) * HALF_Q + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) = qq[a];
+                    }
+                }
+                fence_async_shared();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars->q_full[k & 1]);
+            }
+            if (lane == 0 && !ok) *(volatile int *)&bars->abort_flag = 1;
+        }
+    } else if (start_ok) {
+        // --------------------------------------------------------------------------------------- softmax threads
+        const int i = tid & 127, half = tid >> 7;        // this thread's query row and its half of every tile's columns
+        const uint32_t lane_addr = tbase + ((uint32_t)((warp & 3) * 32) << 16);
+        bool ok = true;
+        for (int k = 0; k < nitems && ok; ++k) {
+            const int item = blockIdx.x + k * gridDim.x, u = item / nblk, qb = item % nblk;
+            const int s0 = p.first_step + qb * RQ, c = min(RQ, p.nsteps - qb * RQ);
+            const int step = s0 + i;
+            const bool live_row = i < c;
+            const float tf = (float)step;
+            uint32_t *hrow = p.hist + ((size_t)u * p.w + step % p.w) * p.Bw;
+            float m_run = -INFINITY, l_run = 0.f, Mi = 0.f, Li = 1.f;
+            int g_exit = G;
+            for (int g = 0; g < G; ++g) {
+                const int gk = k * G + g, b = gk & 1, kt = key_tile(g);
+                ok = mbar_wait(&bars->s_done[b], (gk >> 1) & 1, p.err, 0x551) && ok;
+                ok = mbar_wait(&bars->pos_full[gk % RPD], (gk / RPD) & 1, p.err, 0x552) && ok;
+                if (__any_sync(0xffffffffu, !ok || aborted())) {
+                    ok = false;
+                    *(volatile int *)&bars->abort_flag = 1;
+                    g_exit = g;
+                    break;
+                }
+                tc_fence_after();
+                float sv[RHC];
+                tmem_ld32(lane_addr + b * TN + half * RHC, sv);
+                tc_fence_before();
+                // bit jj of vm: column jj of this thread's half is visible to its query
+                uint32_t vm = 0;
+                {
+                    const int4 *pt = reinterpret_cast<const int4 *>(pos_sh + (gk % RPD) * TN + half * RHC);
+#pragma unroll
+                    for (int q4 = 0; q4 < RHC / 4; ++q4) {
+                        const int4 pp = pt[q4];
+                        vm |= (uint32_t)(pp.x <= step) << (4 * q4) | (uint32_t)(pp.y <= step) << (4 * q4 + 1) |
+                              (uint32_t)(pp.z <= step) << (4 * q4 + 2) | (uint32_t)(pp.w <= step) << (4 * q4 + 3);
+                    }
+                    if (!live_row) vm = 0;
+                }
+                mbar_arrive(&bars->s_free[b]);       // S is in registers and the tile's positions have been read
+                if (g < ntiles) {
+                    if (vm) {
+                        float bmax = -INFINITY;
+#pragma unroll
+                        for (int jj = 0; jj < RHC; ++jj) {
+                            sv[jj] = ((vm >> jj) & 1u) ? sv[jj] * p.scale_log2e : -INFINITY;
+                            bmax = fmaxf(bmax, sv[jj]);
+                        }
+                        const float m_new = fmaxf(m_run, bmax);
+                        float acc = 0.f;
+#pragma unroll
+                        for (int jj = 0; jj < RHC; ++jj) acc += ex2_approx(sv[jj] - m_new);
+                        l_run = l_run * ex2_approx(m_run - m_new) + acc;
+                        m_run = m_new;
+                    }
+                    if (g == ntiles - 1) {
+                        m_sh[tid] = m_run;
+                        l_sh[tid] = l_run;
+                        softmax_barrier();
+                        if (tid < RQ) {
+                            const float ma = m_sh[tid], mb = m_sh[tid + RQ];
+                            const float M = fmaxf(ma, mb);
+                            float L = 0.f;
+                            if (ma > -INFINITY) L += l_sh[tid] * ex2_approx(ma - M);
+                            if (mb > -INFINITY) L += l_sh[tid + RQ] * ex2_approx(mb - M);
+                            Mfin[tid] = M;
+                            Lfin[tid] = L;
+                        }
+                        softmax_barrier();
+                        Mi = Mfin[i];
+                        Li = Lfin[i];
+                        softmax_barrier();       // everyone has its row's M and L: the next item may overwrite them
+                    }
+                    continue;
+                }
+                uint32_t word = 0;
+#pragma unroll
+                for (int jj = 0; jj < RHC; ++jj) {
+                    const float e = ((vm >> jj) & 1u) ? ex2_approx(sv[jj] * p.scale_log2e - Mi) : 0.f;
+                    word |= (uint32_t)(e * tf < Li) << jj;
+                }
+                word &= vm;
+                if (live_row && kt * 2 + half < p.Bw) hrow[kt * 2 + half] = word;
+            }
+            if (g_exit < ntiles) {               // the others may be waiting at the three barriers of the first sweep's end
+                softmax_barrier();
+                softmax_barrier();
+                softmax_barrier();
+            }
+            if (!ok) break;
+            if (live_row && half == 0)
+                for (int wd = ntiles * (TN / 32); wd < p.Bw; ++wd) hrow[wd] = 0;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tbase), "r"(R_TMEM_COLS) : "memory");
+    }
+}
+
 typedef CUresult (*EncodeTiled)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
                                 const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -552,7 +848,29 @@ cudaError_t launch_tma(const ChunkParams &p, cudaStream_t s) {
     return cudaGetLastError();
 }
 
+template <int DT>
+cudaError_t launch_recount_tma(const ChunkParams &p, cudaStream_t s) {
+    CUtensorMap mk;
+    const uint64_t row = (uint64_t)D * 2;
+    if (!make_map(&mk, p.K, (uint64_t)p.B, (uint64_t)p.U, row, (uint64_t)p.B * row, TN, 1)) return cudaErrorNotSupported;
+    auto kern = sh_recount_umma_tma_kernel<DT>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, R_SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    const int sms = sm_count();
+    if (sms <= 0) return cudaErrorInvalidDevice;
+    const long long items = (long long)p.U * ((p.nsteps + RQ - 1) / RQ);
+    const int grid = items < 2 * sms ? (int)items : 2 * sms;
+    kern<<<dim3(grid, 1, 1), RTHREADS, R_SMEM_BYTES, s>>>(p, mk);
+    return cudaGetLastError();
+}
+
 }  // namespace
+
+cudaError_t sh_launch_recount_umma_tma(const ChunkParams &p, int dtype, cudaStream_t s) {
+    if (p.nsteps < 1 || p.out || p.U < 1) return cudaErrorInvalidValue;
+    if (p.n0 < 1) return cudaSuccess;
+    return dtype == SH_F16 ? launch_recount_tma<SH_F16>(p, s) : launch_recount_tma<SH_BF16>(p, s);
+}
 
 cudaError_t sh_launch_chunk_umma_tma(const ChunkParams &p, int dtype, cudaStream_t s) {
     if (p.c < 1 || p.c > CQ || p.U < 1) return cudaErrorInvalidValue;

@@ -433,7 +433,7 @@ cudaError_t sh_launch_recount(const sh_context *c, cudaStream_t s, long long *la
         return e;
     }
     if (c->prefill_chunk != 2) {
-        e = sh_launch_recount_umma(p, c->dtype, s);
+        e = c->prefill_chunk == 1 ? sh_launch_recount_umma_tma(p, c->dtype, s) : sh_launch_recount_umma(p, c->dtype, s);
         if (e == cudaSuccess) *launches += 1;
         return e;
     }

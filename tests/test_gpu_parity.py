@@ -176,7 +176,9 @@ def test_chunked_prompt_without_outputs_leaves_the_same_state(sh, dtype, U):
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
 @pytest.mark.parametrize("U,B,r,w,m,chunk_kernel", [(5, 150, 9, 37, 41, 1), (3, 410, 64, 128, 64, 1), (140, 96, 8, 70, 30, 1),
                                                     (2, 40, 3, 9, 20, 1), (2, 1300, 10, 200, 650, 1), (5, 150, 9, 37, 41, 2),
-                                                    (3, 410, 64, 128, 64, 2), (140, 96, 8, 70, 30, 2)])
+                                                    (3, 410, 64, 128, 64, 2), (140, 96, 8, 70, 30, 2),
+                                                    (5, 150, 9, 37, 41, 3), (3, 410, 64, 128, 64, 3), (2, 1300, 10, 200, 650, 3),
+                                                    (700, 100, 9, 140, 41, 1), (3, 300, 5, 300, 120, 1)])
 def test_lockstep_record_recomputed_at_compression(sh, dtype, U, B, r, w, m, chunk_kernel):
     """SH_OPT_RECORD_MODE = 1: Algorithm 2 as stated, the record rebuilt at each compression from
     the stored queries of the last w steps against the present cache."""
