@@ -157,6 +157,34 @@ def test_lockstep_chunked_persistent_ctas(sh, dtype, U, B, r, w, m, sizes):
     assert res.adoptions <= 1e-4 * res.slot_steps + 2
 
 
+def _poison_rows(h):
+    """Every byte of the handle's K and V regions becomes 0xFF: NaN in each floating-point storage type."""
+    row_bytes = {0: 4 * h.D, 1: 2 * h.D, 2: 2 * h.D}[h.dtype]
+    kv = 2 * ((h.U * h.B * row_bytes + 255) // 256 * 256)
+    h.slab[h._slab_off:h._slab_off + kv] = 0xFF
+
+
+@pytest.mark.parametrize("dtype,d,chunk_kernel,recompute", [("f16", 128, 1, False), ("bf16", 128, 1, True), ("f16", 128, 3, True),
+                                                            ("f16", 128, 2, False), ("f32", 128, 1, False), ("f16", 64, 1, True),
+                                                            ("f32", 64, 1, False)])
+def test_rows_that_hold_no_token_are_never_used(sh, dtype, d, chunk_kernel, recompute):
+    """A cache whose unused rows hold NaN (a caller's workspace is not cleared by the library): chunks whose last
+    tile reaches past the live rows, the recount, the decode steps and the compressions must neither read such a
+    row into a result nor let it through a masked product (0 x NaN)."""
+    U, B, r, w, m, T = 7, 150, 9, 64, 41, 300
+    q, k, v = wl.random_stream(U, d, T + 40, seed=61, dtype=dtype, peaked=3.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False, prefill_chunk=chunk_kernel, recompute_record=recompute)
+    _poison_rows(h)
+    blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
+    outs = []
+    res, orc = run_lockstep_chunked(h, dtype, blk, T, torch.arange(U), TOL[dtype], chunk_sizes=[64, 7, 33], recompute=recompute,
+                                    outs=outs)
+    assert res.steps == T and res.compressions >= 2
+    assert all(torch.isfinite(o).all() for o in outs)
+    if not recompute:
+        run_lockstep(h, dtype, lambda t: (q[t - 1], k[t - 1], v[t - 1]), 40, torch.arange(U), TOL[dtype], orc=orc)
+
+
 @pytest.mark.parametrize("dtype,U", [("f16", 5), ("bf16", 640)])
 def test_chunked_prompt_without_outputs_leaves_the_same_state(sh, dtype, U):
     """sh_prefill with no output buffer (the second contraction is skipped altogether) leaves state bit-identical
