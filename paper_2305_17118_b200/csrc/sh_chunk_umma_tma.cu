@@ -191,45 +191,61 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
                 dv[1][ks] = smem_desc_sw128(smem_u32(Vt) + TILE + ks * 2048, HALF_K, 1024);
                 dp[ks] = smem_desc(smem_u32(Ph) + ks * 256, 128, PG);       // 16 row groups: P_hi, then P_lo
             }
+            // Two streams of work, each in its own order: S tiles (up to two ahead of the softmax threads, across unit
+            // boundaries too) and P.V tiles.  Whichever has its operands ready is issued next, so neither waits
+            // behind the other's barrier; nothing is ready: poll, with the same bounds as mbar_wait.
             bool ok = true;
-            auto issue_s = [&](int k, int g) {
-                const int gk = k * G + g, b = gk & 1;
-                static_assert(KST == 2, "the key stage of S(gk) is the S buffer's index");
-                if (g == 0) ok = ok && mbar_wait(&bars->q_full, k & 1, p.err, 0x521);
-                ok = ok && mbar_wait(&bars->k_full[b], (gk / KST) & 1, p.err, 0x522);
-                if (gk >= 2) ok = ok && mbar_wait(&bars->s_free[b], ((gk >> 1) - 1) & 1, p.err, 0x523);   // S(gk - 2) has been read out
-                if (!ok) return;
-                tc_fence_after();
-                if (b == 0) {
+            int sk = 0, sg = 0;          // next S: unit index and tile (both sweeps) of this CTA
+            int pk = 0, pt = 0;          // next P.V: unit index and key tile
+            const int pv_units = with_out ? nunits : 0;
+            uint32_t idle = 0;
+            unsigned long long idle_t0 = 0;
+            while (ok && (sk < nunits || pk < pv_units)) {
+                bool did = false;
+                if (sk < nunits) {
+                    const int gk = sk * G + sg, bb = gk & 1;
+                    static_assert(KST == 2, "the key stage of S(gk) is the S buffer's index");
+                    if ((sg != 0 || mbar_try_wait(&bars->q_full, sk & 1)) && mbar_try_wait(&bars->k_full[bb], (gk / KST) & 1) &&
+                        (gk < 2 || mbar_try_wait(&bars->s_free[bb], ((gk >> 1) - 1) & 1))) {      // S(gk - 2) has been read out
+                        tc_fence_after();
+                        if (bb == 0) {
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) umma_f16(tbase + S_COL, dq[ks], dk[0][ks], idesc_s, ks > 0);
-                } else {
+                            for (int ks = 0; ks < D / 16; ++ks) umma_f16(tbase + S_COL, dq[ks], dk[0][ks], idesc_s, ks > 0);
+                        } else {
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) umma_f16(tbase + S_COL + TN, dq[ks], dk[1][ks], idesc_s, ks > 0);
+                            for (int ks = 0; ks < D / 16; ++ks) umma_f16(tbase + S_COL + TN, dq[ks], dk[1][ks], idesc_s, ks > 0);
+                        }
+                        umma_commit(&bars->k_empty[bb]);
+                        umma_commit(&bars->s_done[bb]);
+                        if (sg == G - 1) umma_commit(&bars->q_empty);
+                        if (++sg == G) { sg = 0; ++sk; }
+                        did = true;
+                    }
                 }
-                umma_commit(&bars->k_empty[b]);
-                umma_commit(&bars->s_done[b]);
-                if (g == G - 1) umma_commit(&bars->q_empty);
-            };
-            issue_s(0, 0);
-            for (int k = 0; k < nunits && ok; ++k) {
-                for (int g = 0; g < G && ok; ++g) {
-                    if (g + 1 < G) issue_s(k, g + 1);          // S runs one tile ahead of the softmax threads,
-                    else if (k + 1 < nunits) issue_s(k + 1, 0);   // across the unit boundary too
-                    if (ok && with_out && g >= ntiles) {
-                        const int kt = g - ntiles, gv = k * ntiles + kt, b = gv & 1;
-                        ok = mbar_wait(&bars->p_ready, gv & 1, p.err, 0x524);
-                        ok = ok && mbar_wait(&bars->v_full[b], (gv >> 1) & 1, p.err, 0x525);
-                        if (kt == 0 && k > 0) ok = ok && mbar_wait(&bars->o_free, (k - 1) & 1, p.err, 0x526);   // the previous unit's O^T is in registers
-                        if (!ok) break;
+                if (pk < pv_units) {
+                    const int gv = pk * ntiles + pt, bb = gv & 1;
+                    if (mbar_try_wait(&bars->p_ready, gv & 1) && mbar_try_wait(&bars->v_full[bb], (gv >> 1) & 1) &&
+                        (pt != 0 || pk == 0 || mbar_try_wait(&bars->o_free, (pk - 1) & 1))) {      // the previous unit's O^T is in registers
                         tc_fence_after();
 #pragma unroll
-                        for (int ks = 0; ks < TN / 16; ++ks) umma_f16(tbase + O_COL, b ? dv[1][ks] : dv[0][ks], dp[ks], idesc_pv, (kt > 0 || ks > 0));
-                        umma_commit(&bars->v_empty[b]);
+                        for (int ks = 0; ks < TN / 16; ++ks) umma_f16(tbase + O_COL, bb ? dv[1][ks] : dv[0][ks], dp[ks], idesc_pv, (pt > 0 || ks > 0));
+                        umma_commit(&bars->v_empty[bb]);
                         umma_commit(&bars->pv_done);
+                        if (++pt == ntiles) { pt = 0; ++pk; }
+                        did = true;
                     }
-                    if (aborted()) ok = false;
                 }
+                if (did) {
+                    idle = 0;
+                } else {
+                    if (idle == 0) idle_t0 = global_ns();
+                    ++idle;
+                    if (idle >= WAIT_POLLS || ((idle & 255u) == 0 && global_ns() - idle_t0 > WAIT_NS)) {
+                        if (p.err) atomicCAS(p.err, 0, 0x527);
+                        ok = false;
+                    }
+                }
+                if (aborted()) ok = false;
             }
             if (!ok) *(volatile int *)&bars->abort_flag = 1;
         }
