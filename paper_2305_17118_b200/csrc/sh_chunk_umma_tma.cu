@@ -205,8 +205,8 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
                 if (sk < nunits) {
                     const int gk = sk * G + sg, bb = gk & 1;
                     static_assert(KST == 2, "the key stage of S(gk) is the S buffer's index");
-                    if ((sg != 0 || mbar_try_wait(&bars->q_full, sk & 1)) && mbar_try_wait(&bars->k_full[bb], (gk / KST) & 1) &&
-                        (gk < 2 || mbar_try_wait(&bars->s_free[bb], ((gk >> 1) - 1) & 1))) {      // S(gk - 2) has been read out
+                    if ((sg != 0 || mbar_test(&bars->q_full, sk & 1)) && mbar_test(&bars->k_full[bb], (gk / KST) & 1) &&
+                        (gk < 2 || mbar_test(&bars->s_free[bb], ((gk >> 1) - 1) & 1))) {      // S(gk - 2) has been read out
                         tc_fence_after();
                         if (bb == 0) {
 #pragma unroll
@@ -224,8 +224,8 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
                 }
                 if (pk < pv_units) {
                     const int gv = pk * ntiles + pt, bb = gv & 1;
-                    if (mbar_try_wait(&bars->p_ready, gv & 1) && mbar_try_wait(&bars->v_full[bb], (gv >> 1) & 1) &&
-                        (pt != 0 || pk == 0 || mbar_try_wait(&bars->o_free, (pk - 1) & 1))) {      // the previous unit's O^T is in registers
+                    if (mbar_test(&bars->p_ready, gv & 1) && mbar_test(&bars->v_full[bb], (gv >> 1) & 1) &&
+                        (pt != 0 || pk == 0 || mbar_test(&bars->o_free, (pk - 1) & 1))) {      // the previous unit's O^T is in registers
                         tc_fence_after();
 #pragma unroll
                         for (int ks = 0; ks < TN / 16; ++ks) umma_f16(tbase + O_COL, bb ? dv[1][ks] : dv[0][ks], dp[ks], idesc_pv, (pt > 0 || ks > 0));
