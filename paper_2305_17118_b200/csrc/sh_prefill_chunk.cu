@@ -388,7 +388,11 @@ cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const vo
         return e;
     }
     if (c->prefill_chunk != 2) {
-        e = c->prefill_chunk == 1 ? sh_launch_chunk_umma_tma(p, c->dtype, s) : sh_launch_chunk_umma(p, c->dtype, s);
+        e = c->prefill_chunk == 1 ? sh_launch_chunk_umma_tma(p, c->dtype, s) : cudaErrorNotSupported;
+        if (e == cudaErrorNotSupported) {       // option 3, or a driver without the tensor-map encoder: the per-unit tcgen05 kernel
+            (void)cudaGetLastError();
+            e = sh_launch_chunk_umma(p, c->dtype, s);
+        }
         if (e == cudaSuccess) *launches += 1;
         return e;
     }
@@ -433,7 +437,11 @@ cudaError_t sh_launch_recount(const sh_context *c, cudaStream_t s, long long *la
         return e;
     }
     if (c->prefill_chunk != 2) {
-        e = c->prefill_chunk == 1 ? sh_launch_recount_umma_tma(p, c->dtype, s) : sh_launch_recount_umma(p, c->dtype, s);
+        e = c->prefill_chunk == 1 ? sh_launch_recount_umma_tma(p, c->dtype, s) : cudaErrorNotSupported;
+        if (e == cudaErrorNotSupported) {
+            (void)cudaGetLastError();
+            e = sh_launch_recount_umma(p, c->dtype, s);
+        }
         if (e == cudaSuccess) *launches += 1;
         return e;
     }
