@@ -35,36 +35,44 @@ using namespace shumma;
 
 constexpr int D = 128;            // head_dim served by this kernel
 constexpr int TN = 64;            // keys per tile
-constexpr int CQ = 64;            // queries per unit and launch
-constexpr int NT = 256;           // softmax threads: two per lane of tensor memory
-constexpr int NTHREADS = NT + 128;   // + the warps that issue MMAs, request K/Q tiles, request V tiles, append
-constexpr int W_MMA = NT / 32, W_KQ = W_MMA + 1, W_V = W_MMA + 2, W_APPEND = W_MMA + 3;
+constexpr int NT = 256;           // softmax threads of the narrow chunk kernel and of the recount: two per lane of tensor memory
+constexpr int W_MMA = NT / 32, W_KQ = W_MMA + 1, W_V = W_MMA + 2;      // (recount: warp 10 gathers the queries)
 constexpr int HALF_K = TN * 128;        // bytes of one box: 64 rows x 64 elements (half of head_dim)
 constexpr int TILE = 2 * HALF_K;        // a key or value tile: [2 halves of d][64 rows][128 B]
-constexpr int HALF_Q = 2 * CQ * 128;    // the queries occupy rows 0..63 and again rows 64..127 (M = 128)
+constexpr int HALF_Q = 128 * 128;       // 128 query rows (M = 128) x 64 elements
 constexpr int Q_BYTES = 2 * HALF_Q;
-constexpr int KST = 2;                  // key tiles in flight
 constexpr int PG = (TN / 8) * 128;      // bytes of 8 rows of P (TN keys each) in no-swizzle core-matrix order
-constexpr int P_BYTES = (CQ / 8) * PG;
 constexpr int HC = TN / 4;              // columns of a tile per thread (four threads share a query row)
 static_assert(HC == 16, "a thread reads its 16 columns with one tcgen05.ld and owns half a record word");
-constexpr int TMEM_COLS = 256;          // two S tiles and O^T (twice: from P's high and low parts); two CTAs fit in an SM's 512 columns
 constexpr int S_COL = 0;
-constexpr int O_COL = 2 * TN;           // columns [O_COL, O_COL + CQ): V^T.P_hi^T, the next CQ columns: V^T.P_lo^T
-static_assert(O_COL + 2 * CQ <= TMEM_COLS, "tensor memory columns");
+constexpr int O_COL = 2 * TN;           // columns [O_COL, O_COL + QR): V^T.P_hi^T, the next QR columns: V^T.P_lo^T
 
-constexpr int OFF_Q = 0;
-constexpr int OFF_K = OFF_Q + Q_BYTES;
-constexpr int OFF_V = OFF_K + KST * TILE;
-constexpr int OFF_PH = OFF_V + 2 * TILE;
-constexpr int OFF_PL = OFF_PH + P_BYTES;
-constexpr int OFF_STAT = OFF_PL + P_BYTES;      // M[64], L[64], 1/L[64]
-constexpr int OFF_BAR = OFF_STAT + 4 * 3 * 64;
-constexpr int SMEM_BYTES = OFF_BAR + 192;
-static_assert(OFF_K % 1024 == 0 && OFF_V % 1024 == 0 && HALF_K % 1024 == 0, "swizzled tiles start on 1024-byte boundaries");
-static_assert(OFF_PL == OFF_PH + P_BYTES, "P_hi and P_lo form one B operand of 2 CQ rows");
-static_assert(P_BYTES >= 4 * 2 * NT, "the first sweep's statistics alias the P buffer");
-static_assert(2 * (SMEM_BYTES + 1024) <= 228 * 1024, "two CTAs per SM");
+// Two shapes of the chunk kernel.  Narrow: up to 64 queries, which occupy rows 0..63 and again rows 64..127 of the
+// MMA, 8 softmax warps, two CTAs per SM.  Wide: up to 128 queries, one per row of the MMA (half the S instructions
+// per query), 16 softmax warps, four key tiles in flight, one CTA per SM.
+template <bool WIDE> struct CK {
+    static constexpr int QR = WIDE ? 128 : 64;            // queries per unit and launch
+    static constexpr int NT = 4 * QR;                     // softmax threads: four per query (16 columns of a tile each)
+    static constexpr int NAPP = WIDE ? 4 : 1;             // warps that append (a warp moves the 48 KB of 64 tokens in about 10 us)
+    static constexpr int NTH = NT + 96 + 32 * NAPP;       // + the warps that issue MMAs, request K/Q tiles, request V tiles, append
+    static constexpr int W_MMA = NT / 32, W_KQ = W_MMA + 1, W_V = W_MMA + 2, W_APPEND = W_MMA + 3;
+    static constexpr int CTAS = WIDE ? 1 : 2;             // per SM
+    static constexpr int KST = WIDE ? 4 : 2;              // key tiles in flight
+    static constexpr int P_BYTES = (QR / 8) * PG;         // QR rows x TN keys x 2 B
+    static constexpr int TMEM_COLS = WIDE ? 512 : 256;    // two S tiles, O^T from P_hi and from P_lo (QR columns each), power of two
+    static constexpr int OFF_Q = 0;
+    static constexpr int OFF_K = OFF_Q + Q_BYTES;
+    static constexpr int OFF_V = OFF_K + KST * TILE;
+    static constexpr int OFF_PH = OFF_V + 2 * TILE;
+    static constexpr int OFF_PL = OFF_PH + P_BYTES;       // P_hi and P_lo form one B operand of 2 QR rows
+    static constexpr int OFF_STAT = OFF_PL + P_BYTES;     // M[QR], L[QR], 1/L[QR]
+    static constexpr int OFF_BAR = OFF_STAT + 4 * 3 * QR;
+    static constexpr int SMEM_BYTES = OFF_BAR + 192;
+    static_assert(OFF_K % 1024 == 0 && OFF_V % 1024 == 0 && HALF_K % 1024 == 0, "swizzled tiles start on 1024-byte boundaries");
+    static_assert(P_BYTES >= 4 * 2 * NT, "the first sweep's statistics alias the P buffer");
+    static_assert(CTAS * (SMEM_BYTES + 1024) <= 228 * 1024, "CTAs per SM");
+    static_assert(O_COL + 2 * QR <= TMEM_COLS && CTAS * TMEM_COLS <= 512, "tensor memory columns");
+};
 
 // Shared-memory matrix descriptor for the 128-byte swizzle (layout type 2 in bits 61..63).
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
@@ -102,36 +110,38 @@ __device__ __forceinline__ bool counter_wait(const int *ctr, int target, int *er
     return false;
 }
 
-__device__ __forceinline__ void softmax_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory"); }
+template <int THREADS>
+__device__ __forceinline__ void softmax_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory"); }
 
 struct Bars {
     uint64_t q_full, q_empty;          // the unit's queries landed / its last S has been computed
-    uint64_t k_full[KST], k_empty[KST];
+    uint64_t k_full[4], k_empty[4];
     uint64_t v_full[2], v_empty[2];
     uint64_t s_done[2], s_free[2];     // S(g) computed / read out of tensor memory by all softmax threads
     uint64_t p_ready, pv_done;         // P(kt) written / P.V(kt) computed
     uint64_t o_free;                   // O^T of the unit read out
     uint32_t tmem_slot;
     int abort_flag;                    // a bounded wait gave up somewhere: everybody leaves
-    int appended;                      // units whose chunk rows are in the cache (written by the append warp)
+    int appended[4];                   // per append warp: units whose share of the chunk's rows is in the cache
 };
 static_assert(sizeof(Bars) <= 192, "barrier block");
 
-template <int DT>
-__global__ void __launch_bounds__(NTHREADS, 2)
+template <int DT, bool WIDE>
+__global__ void __launch_bounds__(CK<WIDE>::NTH, CK<WIDE>::CTAS)
 sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                          const __grid_constant__ CUtensorMap mapV) {
     using SP = Split<DT>;
+    using C = CK<WIDE>;
     extern __shared__ __align__(1024) unsigned char sm[];
-    char *Qs = reinterpret_cast<char *>(sm) + OFF_Q;
-    char *Kt = reinterpret_cast<char *>(sm) + OFF_K;
-    char *Vt = reinterpret_cast<char *>(sm) + OFF_V;
-    char *Ph = reinterpret_cast<char *>(sm) + OFF_PH;
-    char *Pl = reinterpret_cast<char *>(sm) + OFF_PL;
-    float *m_sh = reinterpret_cast<float *>(sm + OFF_PH);
-    float *l_sh = m_sh + NT;
-    float *Mfin = reinterpret_cast<float *>(sm + OFF_STAT), *Lfin = Mfin + 64, *Linv = Lfin + 64;
-    Bars *bars = reinterpret_cast<Bars *>(sm + OFF_BAR);
+    char *Qs = reinterpret_cast<char *>(sm) + C::OFF_Q;
+    char *Kt = reinterpret_cast<char *>(sm) + C::OFF_K;
+    char *Vt = reinterpret_cast<char *>(sm) + C::OFF_V;
+    char *Ph = reinterpret_cast<char *>(sm) + C::OFF_PH;
+    char *Pl = reinterpret_cast<char *>(sm) + C::OFF_PL;
+    float *m_sh = reinterpret_cast<float *>(sm + C::OFF_PH);
+    float *l_sh = m_sh + C::NT;
+    float *Mfin = reinterpret_cast<float *>(sm + C::OFF_STAT), *Lfin = Mfin + C::QR, *Linv = Lfin + C::QR;
+    Bars *bars = reinterpret_cast<Bars *>(sm + C::OFF_BAR);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n0 = p.n0, c = p.c, n_tot = n0 + c;
@@ -143,22 +153,22 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
     auto aborted = [&]() { return *(volatile int *)&bars->abort_flag != 0; };
 
     if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_slot)), "r"(TMEM_COLS)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_slot)), "r"(C::TMEM_COLS)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     if (tid == 0) {
         mbar_init(&bars->q_full, 1);
         mbar_init(&bars->q_empty, 1);
-        for (int s = 0; s < KST; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1); }
+        for (int s = 0; s < C::KST; ++s) { mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1); }
         for (int s = 0; s < 2; ++s) {
             mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1);
-            mbar_init(&bars->s_done[s], 1); mbar_init(&bars->s_free[s], NT);
+            mbar_init(&bars->s_done[s], 1); mbar_init(&bars->s_free[s], C::NT);
         }
-        mbar_init(&bars->p_ready, NT);
+        mbar_init(&bars->p_ready, C::NT);
         mbar_init(&bars->pv_done, 1);
-        mbar_init(&bars->o_free, NT);
-        bars->appended = 0;
+        mbar_init(&bars->o_free, C::NT);
+        for (int a = 0; a < 4; ++a) bars->appended[a] = 0;
         bars->abort_flag = 0;
         if ((smem_u32(sm) & 1023u) != 0) {      // the swizzled tiles need the 1024-byte alignment the declaration asks for
             if (p.err) atomicCAS(p.err, 0, 0x520);
@@ -172,24 +182,23 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
     const uint32_t tbase = bars->tmem_slot;
     const bool start_ok = !aborted();
 
-    if (warp == W_MMA) {
+    if (warp == C::W_MMA) {
         // --------------------------------------------------------------------------------------- the issuing thread
         if (lane == 0 && start_ok) {
             const uint32_t idesc_s = instr_desc(SP::FMT, 0, 128, TN);
-            const uint32_t idesc_pv = instr_desc(SP::FMT, 1, 128, 2 * CQ);     // N = the queries' high parts, then their low parts
-            // every descriptor this thread will ever use, built once: the loops below only issue
-            uint64_t dq[D / 16], dk[KST][D / 16], dv[2][TN / 16], dp[TN / 16];
+            const uint32_t idesc_pv = instr_desc(SP::FMT, 1, 128, 2 * C::QR);     // N = the queries' high parts, then their low parts
+            // the descriptors of query buffer, key stage 0, value buffer 0 and P, built once; the other stages and buffers
+            // lie a fixed number of 16-byte units further
+            uint64_t dq[D / 16], dk[D / 16], dv[TN / 16], dp[TN / 16];
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
                 dq[ks] = smem_desc_sw128(smem_u32(Qs) + (ks >> 2) * HALF_Q + (ks & 3) * 32, 16, 1024);
-#pragma unroll
-                for (int s = 0; s < KST; ++s) dk[s][ks] = smem_desc_sw128(smem_u32(Kt) + s * TILE + (ks >> 2) * HALF_K + (ks & 3) * 32, 16, 1024);
+                dk[ks] = smem_desc_sw128(smem_u32(Kt) + (ks >> 2) * HALF_K + (ks & 3) * 32, 16, 1024);
             }
 #pragma unroll
             for (int ks = 0; ks < TN / 16; ++ks) {
-                dv[0][ks] = smem_desc_sw128(smem_u32(Vt) + ks * 2048, HALF_K, 1024);
-                dv[1][ks] = smem_desc_sw128(smem_u32(Vt) + TILE + ks * 2048, HALF_K, 1024);
-                dp[ks] = smem_desc(smem_u32(Ph) + ks * 256, 128, PG);       // 16 row groups: P_hi, then P_lo
+                dv[ks] = smem_desc_sw128(smem_u32(Vt) + ks * 2048, HALF_K, 1024);
+                dp[ks] = smem_desc(smem_u32(Ph) + ks * 256, 128, PG);       // row groups of P_hi, then of P_lo
             }
             // Two streams of work, each in its own order: S tiles (up to two ahead of the softmax threads, across unit
             // boundaries too) and P.V tiles.  Whichever has its operands ready is issued next, so neither waits
@@ -203,19 +212,14 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
             while (ok && (sk < nunits || pk < pv_units)) {
                 bool did = false;
                 if (sk < nunits) {
-                    const int gk = sk * G + sg, bb = gk & 1;
-                    static_assert(KST == 2, "the key stage of S(gk) is the S buffer's index");
-                    if ((sg != 0 || mbar_test(&bars->q_full, sk & 1)) && mbar_test(&bars->k_full[bb], (gk / KST) & 1) &&
+                    const int gk = sk * G + sg, bb = gk & 1, st = gk % C::KST;
+                    if ((sg != 0 || mbar_test(&bars->q_full, sk & 1)) && mbar_test(&bars->k_full[st], (gk / C::KST) & 1) &&
                         (gk < 2 || mbar_test(&bars->s_free[bb], ((gk >> 1) - 1) & 1))) {      // S(gk - 2) has been read out
                         tc_fence_after();
-                        if (bb == 0) {
+                        const uint64_t koff = (uint64_t)(st * (TILE >> 4));
 #pragma unroll
-                            for (int ks = 0; ks < D / 16; ++ks) umma_f16(tbase + S_COL, dq[ks], dk[0][ks], idesc_s, ks > 0);
-                        } else {
-#pragma unroll
-                            for (int ks = 0; ks < D / 16; ++ks) umma_f16(tbase + S_COL + TN, dq[ks], dk[1][ks], idesc_s, ks > 0);
-                        }
-                        umma_commit(&bars->k_empty[bb]);
+                        for (int ks = 0; ks < D / 16; ++ks) umma_f16(tbase + S_COL + bb * TN, dq[ks], dk[ks] + koff, idesc_s, ks > 0);
+                        umma_commit(&bars->k_empty[st]);
                         umma_commit(&bars->s_done[bb]);
                         if (sg == G - 1) umma_commit(&bars->q_empty);
                         if (++sg == G) { sg = 0; ++sk; }
@@ -227,8 +231,9 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
                     if (mbar_test(&bars->p_ready, gv & 1) && mbar_test(&bars->v_full[bb], (gv >> 1) & 1) &&
                         (pt != 0 || pk == 0 || mbar_test(&bars->o_free, (pk - 1) & 1))) {      // the previous unit's O^T is in registers
                         tc_fence_after();
+                        const uint64_t voff = (uint64_t)(bb * (TILE >> 4));
 #pragma unroll
-                        for (int ks = 0; ks < TN / 16; ++ks) umma_f16(tbase + O_COL, bb ? dv[1][ks] : dv[0][ks], dp[ks], idesc_pv, (pt > 0 || ks > 0));
+                        for (int ks = 0; ks < TN / 16; ++ks) umma_f16(tbase + O_COL, dv[ks] + voff, dp[ks], idesc_pv, (pt > 0 || ks > 0));
                         umma_commit(&bars->v_empty[bb]);
                         umma_commit(&bars->pv_done);
                         if (++pt == ntiles) { pt = 0; ++pk; }
@@ -249,7 +254,7 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
             }
             if (!ok) *(volatile int *)&bars->abort_flag = 1;
         }
-    } else if (warp == W_KQ) {
+    } else if (warp == C::W_KQ) {
         // --------------------------------------------------------------------------------------- query and key tiles
         if (lane == 0 && start_ok) {
             bool ok = true;
@@ -262,13 +267,13 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
                 q_last = k;
 #pragma unroll
                 for (int part = 0; part < 4; ++part)
-                    tma_load_3d(Qs + (part >> 1) * HALF_Q + (part & 1) * CQ * 128, &mapQ, (part >> 1) * 64, u, 0, &bars->q_full);
+                    tma_load_3d(Qs + (part >> 1) * HALF_Q + (part & 1) * 64 * 128, &mapQ, (part >> 1) * 64, u, WIDE ? (part & 1) * 64 : 0, &bars->q_full);
                 bool appended = false;
                 for (int g = 0; g < G; ++g) {
-                    const int gk = k * G + g, s = gk % KST, kt = key_tile(g);
-                    if (gk >= KST) ok = mbar_wait(&bars->k_empty[s], ((gk / KST) - 1) & 1, p.err, 0x532);
+                    const int gk = k * G + g, s = gk % C::KST, kt = key_tile(g);
+                    if (gk >= C::KST) ok = mbar_wait(&bars->k_empty[s], ((gk / C::KST) - 1) & 1, p.err, 0x532);
                     if (ok && !appended && (kt + 1) * TN > n0) {     // this tile holds rows of the chunk
-                        ok = counter_wait(&bars->appended, k + 1, p.err, 0x533);
+                        for (int a = 0; a < C::NAPP; ++a) ok = ok && counter_wait(&bars->appended[a], k + 1, p.err, 0x533);
                         fence_proxy_async_all();
                         appended = true;
                     }
@@ -286,9 +291,9 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
             // if the others gave up, nobody waits for the copies requested last: let them land before the CTA goes away
             // (a phase that is past reads as complete, so this costs nothing otherwise)
             if (q_last >= 0) mbar_wait(&bars->q_full, q_last & 1, nullptr, 0);
-            for (int gk = last; gk > last - KST && gk >= 0; --gk) mbar_wait(&bars->k_full[gk % KST], (gk / KST) & 1, nullptr, 0);
+            for (int gk = last; gk > last - C::KST && gk >= 0; --gk) mbar_wait(&bars->k_full[gk % C::KST], (gk / C::KST) & 1, nullptr, 0);
         }
-    } else if (warp == W_V) {
+    } else if (warp == C::W_V) {
         // --------------------------------------------------------------------------------------- value tiles
         if (lane == 0 && start_ok && with_out) {
             bool ok = true;
@@ -300,7 +305,7 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
                     const int gv = k * ntiles + kt, b = gv & 1;
                     if (gv >= 2) ok = mbar_wait(&bars->v_empty[b], ((gv >> 1) - 1) & 1, p.err, 0x541);
                     if (ok && !appended && (kt + 1) * TN > n0) {
-                        ok = counter_wait(&bars->appended, k + 1, p.err, 0x542);
+                        for (int a = 0; a < C::NAPP; ++a) ok = ok && counter_wait(&bars->appended[a], k + 1, p.err, 0x542);
                         fence_proxy_async_all();
                         appended = true;
                     }
@@ -314,7 +319,7 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
             if (!ok) *(volatile int *)&bars->abort_flag = 1;
             for (int gv = last; gv > last - 2 && gv >= 0; --gv) mbar_wait(&bars->v_full[gv & 1], (gv >> 1) & 1, nullptr, 0);
         }
-    } else if (warp == W_APPEND) {
+    } else if (warp >= C::W_APPEND) {
         // --------------------------------------------------------------------------------------- the append
         // keys, values and positions of the chunk into the cache rows n0 .. n0 + c - 1, queries into the ring of the
         // last w queries; a row of 256 bytes is 16 pieces, the warp moves two rows per instruction
@@ -323,7 +328,8 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
                 if (aborted()) break;
                 const int u = blockIdx.x + k * gridDim.x;
                 const size_t tstride = (size_t)p.Utot * D * 2;
-                for (int base = 0; base < c * 16; base += 4 * 32) {
+                const int aw = warp - C::W_APPEND;        // this warp takes every NAPP-th batch of eight rows
+                for (int base = aw * 4 * 32; base < c * 16; base += C::NAPP * 4 * 32) {
                     uint4 kk[4], vv[4], qq[4];
 #pragma unroll
                     for (int a = 0; a < 4; ++a) {
@@ -346,15 +352,17 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
                         }
                     }
                 }
-                for (int row = lane; row < c; row += 32) p.pos[(size_t)u * p.B + n0 + row] = step0 + row;
+                if (aw == 0)
+                    for (int row = lane; row < c; row += 32) p.pos[(size_t)u * p.B + n0 + row] = step0 + row;
                 fence_proxy_async_all();
                 __syncwarp();
-                if (lane == 0) st_release_shared(&bars->appended, k + 1);
+                if (lane == 0) st_release_shared(&bars->appended[aw], k + 1);
             }
         }
     } else if (start_ok) {
         // --------------------------------------------------------------------------------------- softmax threads
-        const int i = tid & 63, quarter = ((tid >> 6) & 1) * 2 + (tid >> 7);     // this thread's query and its quarter of every tile's columns
+        // this thread's query and its quarter of every tile's columns (64 queries: rows 64..127 repeat rows 0..63)
+        const int i = tid & (C::QR - 1), quarter = WIDE ? (tid >> 7) : ((tid >> 6) & 1) * 2 + (tid >> 7);
         const uint32_t lane_addr = tbase + ((uint32_t)((warp & 3) * 32) << 16);
         uint32_t par_pv = 0;
         bool ok = true;
@@ -403,24 +411,24 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
                     if (g == ntiles - 1) {
                         m_sh[tid] = m_run;
                         l_sh[tid] = l_run;
-                        softmax_barrier();
-                        if (tid < CQ) {
+                        softmax_barrier<C::NT>();
+                        if (tid < C::QR) {
                             float M = -INFINITY, L = 0.f;
 #pragma unroll
-                            for (int part = 0; part < NT / CQ; ++part) M = fmaxf(M, m_sh[tid + part * CQ]);
+                            for (int part = 0; part < C::NT / C::QR; ++part) M = fmaxf(M, m_sh[tid + part * C::QR]);
 #pragma unroll
-                            for (int part = 0; part < NT / CQ; ++part) {
-                                const float mp = m_sh[tid + part * CQ];
-                                if (mp > -INFINITY) L += l_sh[tid + part * CQ] * ex2_approx(mp - M);
+                            for (int part = 0; part < C::NT / C::QR; ++part) {
+                                const float mp = m_sh[tid + part * C::QR];
+                                if (mp > -INFINITY) L += l_sh[tid + part * C::QR] * ex2_approx(mp - M);
                             }
                             Mfin[tid] = M;
                             Lfin[tid] = L;
                             Linv[tid] = 1.f / L;
                         }
-                        softmax_barrier();
+                        softmax_barrier<C::NT>();
                         Mi = Mfin[i];
                         Li = Lfin[i];
-                        softmax_barrier();       // everyone has its row's M and L: the P buffer (m_sh, l_sh) may be written
+                        softmax_barrier<C::NT>();       // everyone has its row's M and L: the P buffer (m_sh, l_sh) may be written
                     }
                     continue;
                 }
@@ -452,7 +460,7 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
                     }
                     if (rz < TN) {                   // (the last tile only) stale cache rows beyond the chunk: zero them for P.V
                         char *vt = Vt + (gv & 1) * TILE;
-                        for (int idx = tid; idx < (TN - rz) * 16; idx += NT) {
+                        for (int idx = tid; idx < (TN - rz) * 16; idx += C::NT) {
                             const int row = rz + (idx >> 4), piece = idx & 15;
                             *reinterpret_cast<uint4 *>(vt + (piece >> 3) * HALF_K + row * 128 + (piece & 7) * 16) = make_uint4(0, 0, 0, 0);
                         }
@@ -468,9 +476,9 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
                 }
             }
             if (g_exit < ntiles) {               // the others may be waiting at the three barriers of the first sweep's end
-                softmax_barrier();
-                softmax_barrier();
-                softmax_barrier();
+                softmax_barrier<C::NT>();
+                softmax_barrier<C::NT>();
+                softmax_barrier<C::NT>();
             }
             if (!ok) break;
             if (live_row && quarter == 0)
@@ -484,12 +492,12 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
                     break;
                 }
                 tc_fence_after();
-                const int dcol = tid & 127, bq = tid >> 7;      // this thread's column of d and its half of the queries
+                const int dcol = tid & 127, bq = tid >> 7;      // this thread's column of d and its 32 queries
                 float oh[2][16], ol[2][16];
 #pragma unroll
                 for (int part = 0; part < 2; ++part) {
                     tmem_ld16(lane_addr + O_COL + bq * 32 + part * 16, oh[part]);
-                    tmem_ld16(lane_addr + O_COL + CQ + bq * 32 + part * 16, ol[part]);
+                    tmem_ld16(lane_addr + O_COL + C::QR + bq * 32 + part * 16, ol[part]);
                 }
                 tc_fence_before();
                 mbar_arrive(&bars->o_free);          // O^T may be overwritten by the next unit
@@ -505,7 +513,7 @@ sh_chunk_umma_tma_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
     __syncthreads();
     if (warp == 0) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tbase), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tbase), "r"(C::TMEM_COLS) : "memory");
     }
 }
 
@@ -762,7 +770,7 @@ __global__ void __launch_bounds__(RTHREADS, 2) sh_recount_umma_tma_kernel(const 
                     if (g == ntiles - 1) {
                         m_sh[tid] = m_run;
                         l_sh[tid] = l_run;
-                        softmax_barrier();
+                        softmax_barrier<NT>();
                         if (tid < RQ) {
                             const float ma = m_sh[tid], mb = m_sh[tid + RQ];
                             const float M = fmaxf(ma, mb);
@@ -772,10 +780,10 @@ __global__ void __launch_bounds__(RTHREADS, 2) sh_recount_umma_tma_kernel(const 
                             Mfin[tid] = M;
                             Lfin[tid] = L;
                         }
-                        softmax_barrier();
+                        softmax_barrier<NT>();
                         Mi = Mfin[i];
                         Li = Lfin[i];
-                        softmax_barrier();       // everyone has its row's M and L: the next item may overwrite them
+                        softmax_barrier<NT>();       // everyone has its row's M and L: the next item may overwrite them
                     }
                     continue;
                 }
@@ -789,9 +797,9 @@ __global__ void __launch_bounds__(RTHREADS, 2) sh_recount_umma_tma_kernel(const 
                 if (live_row && kt * 2 + half < p.Bw) hrow[kt * 2 + half] = word;
             }
             if (g_exit < ntiles) {               // the others may be waiting at the three barriers of the first sweep's end
-                softmax_barrier();
-                softmax_barrier();
-                softmax_barrier();
+                softmax_barrier<NT>();
+                softmax_barrier<NT>();
+                softmax_barrier<NT>();
             }
             if (!ok) break;
             if (live_row && half == 0)
@@ -844,21 +852,22 @@ int sm_count() {
     return v;
 }
 
-template <int DT>
+template <int DT, bool WIDE>
 cudaError_t launch_tma(const ChunkParams &p, cudaStream_t s) {
+    using C = CK<WIDE>;
     CUtensorMap mq, mk, mv;
     const uint64_t row = (uint64_t)D * 2;
-    if (!make_map(&mq, p.q, (uint64_t)p.Utot, (uint64_t)p.c, row, (uint64_t)p.Utot * row, 1, CQ) ||
+    if (!make_map(&mq, p.q, (uint64_t)p.Utot, (uint64_t)p.c, row, (uint64_t)p.Utot * row, 1, 64) ||
         !make_map(&mk, p.K, (uint64_t)p.B, (uint64_t)p.U, row, (uint64_t)p.B * row, TN, 1) ||
         !make_map(&mv, p.V, (uint64_t)p.B, (uint64_t)p.U, row, (uint64_t)p.B * row, TN, 1))
         return cudaErrorNotSupported;
-    auto kern = sh_chunk_umma_tma_kernel<DT>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    auto kern = sh_chunk_umma_tma_kernel<DT, WIDE>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     const int sms = sm_count();
     if (sms <= 0) return cudaErrorInvalidDevice;
-    const int grid = p.U < 2 * sms ? p.U : 2 * sms;
-    kern<<<dim3(grid, 1, 1), NTHREADS, SMEM_BYTES, s>>>(p, mq, mk, mv);
+    const int grid = p.U < C::CTAS * sms ? p.U : C::CTAS * sms;
+    kern<<<dim3(grid, 1, 1), C::NTH, C::SMEM_BYTES, s>>>(p, mq, mk, mv);
     return cudaGetLastError();
 }
 
@@ -886,7 +895,10 @@ cudaError_t sh_launch_recount_umma_tma(const ChunkParams &p, int dtype, cudaStre
     return dtype == SH_F16 ? launch_recount_tma<SH_F16>(p, s) : launch_recount_tma<SH_BF16>(p, s);
 }
 
+int sh_chunk_umma_tma_capacity() { return CK<true>::QR; }
+
 cudaError_t sh_launch_chunk_umma_tma(const ChunkParams &p, int dtype, cudaStream_t s) {
-    if (p.c < 1 || p.c > CQ || p.U < 1) return cudaErrorInvalidValue;
-    return dtype == SH_F16 ? launch_tma<SH_F16>(p, s) : launch_tma<SH_BF16>(p, s);
+    if (p.c < 1 || p.c > CK<true>::QR || p.U < 1) return cudaErrorInvalidValue;
+    if (p.c > CK<false>::QR) return dtype == SH_F16 ? launch_tma<SH_F16, true>(p, s) : launch_tma<SH_BF16, true>(p, s);
+    return dtype == SH_F16 ? launch_tma<SH_F16, false>(p, s) : launch_tma<SH_BF16, false>(p, s);
 }

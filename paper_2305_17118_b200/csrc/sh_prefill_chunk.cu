@@ -343,7 +343,8 @@ int sh_prefill_chunk_capacity(const sh_context *c) {
     }
     if (c->dtype != SH_F16 && c->dtype != SH_BF16) return 0;
     int cq = 0;
-    if (c->prefill_chunk != 2) cq = sh_chunk_umma_capacity();     // tcgen05 kernel: any budget
+    if (c->prefill_chunk == 1) cq = sh_chunk_umma_tma_capacity();      // persistent tcgen05 kernel: any budget, up to 128 tokens
+    else if (c->prefill_chunk != 2) cq = sh_chunk_umma_capacity();     // tcgen05 kernel with one CTA per unit: any budget
     else if (smem_need(32, c->B) <= 200 * 1024) cq = 64;          // warp-level kernel: one or two CTAs of 32 queries, or one of 64
     if (cq > c->w) cq = c->w;     // every step of a chunk needs its own bit-plane row
     return cq;
@@ -389,9 +390,20 @@ cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const vo
     }
     if (c->prefill_chunk != 2) {
         e = c->prefill_chunk == 1 ? sh_launch_chunk_umma_tma(p, c->dtype, s) : cudaErrorNotSupported;
-        if (e == cudaErrorNotSupported) {       // option 3, or a driver without the tensor-map encoder: the per-unit tcgen05 kernel
-            (void)cudaGetLastError();
-            e = sh_launch_chunk_umma(p, c->dtype, s);
+        if (e == cudaErrorNotSupported) {       // option 3, or a driver without the tensor-map encoder: the per-unit tcgen05 kernel,
+            (void)cudaGetLastError();           // which takes 64 tokens at a time (the steps of a chunk are consecutive: it splits)
+            const int cap = sh_chunk_umma_capacity();
+            e = cudaSuccess;
+            for (int done = 0; done < count && e == cudaSuccess; done += cap) {
+                ChunkParams part = p;
+                const size_t skip = (size_t)done * c->U * c->D;       // elements of q, k, v and out before token `done`
+                part.q = p.q + skip * 2; part.k = p.k + skip * 2; part.v = p.v + skip * 2;
+                part.out = p.out ? p.out + skip : nullptr;
+                part.n0 = p.n0 + done; part.t0 = p.t0 + done;
+                part.c = count - done < cap ? count - done : cap;
+                e = sh_launch_chunk_umma(part, c->dtype, s);
+                if (e == cudaSuccess && done > 0) *launches += 1;
+            }
         }
         if (e == cudaSuccess) *launches += 1;
         return e;

@@ -74,7 +74,9 @@ def test_option_values_and_the_shapes_they_need():
     from paper_2305_17118_b200 import binding as sh
     lib = sh.lib
     h = _handle(sh, 410, 64, 128, 64, 16, 128, "f16")
-    assert lib.sh_prefill_chunk_max(h) == 64
+    assert lib.sh_prefill_chunk_max(h) == 128          # the persistent tcgen05 kernel: up to 128 tokens, never more than w
+    assert lib.sh_set_option(h, sh.SH_OPT_PREFILL_CHUNK, 3.0) == sh.SH_OK
+    assert lib.sh_prefill_chunk_max(h) == 64           # one CTA per unit: 64
     for key, good, bad in ((sh.SH_OPT_COMPACTION, (0, 1), (2, -1)), (sh.SH_OPT_PREFILL_CHUNK, (0, 1, 2, 3, 4, 1), (5, -1)),
                            (sh.SH_OPT_DECODE_KERNEL, (0, 1, 2), (3,)), (sh.SH_OPT_SPLIT, (1, 2, 4, 8), (3, 16))):
         for v in good:
@@ -93,7 +95,7 @@ def test_option_values_and_the_shapes_they_need():
     for dtype in ("f32", "f16", "bf16", "int4"):
         for d in (64, 128):
             h = _handle(sh, 410, 64, 128, 64, 3, d, dtype)
-            assert lib.sh_prefill_chunk_max(h) == 64, (dtype, d)
+            assert lib.sh_prefill_chunk_max(h) == (128 if d == 128 and dtype in ("f16", "bf16") else 64), (dtype, d)
             assert lib.sh_set_option(h, sh.SH_OPT_PREFILL_CHUNK, 4.0) == sh.SH_OK
             assert lib.sh_prefill_chunk_max(h) == 64
             assert lib.sh_set_option(h, sh.SH_OPT_RECORD_MODE, 1.0) == sh.SH_OK, (dtype, d)
@@ -110,7 +112,7 @@ def test_option_values_and_the_shapes_they_need():
     # the warp-level chunk kernel keeps a row of logits in shared memory: it stops at budgets of about 700,
     # the tcgen05 kernel does not; the recompute mode follows the kernel that is chosen
     h = _handle(sh, 4000, 10, 400, 2000, 2, 128, "f16")
-    assert lib.sh_prefill_chunk_max(h) == 64
+    assert lib.sh_prefill_chunk_max(h) == 128
     assert lib.sh_set_option(h, sh.SH_OPT_PREFILL_CHUNK, 2.0) == sh.SH_OK
     assert lib.sh_prefill_chunk_max(h) == 0
     assert lib.sh_set_option(h, sh.SH_OPT_RECORD_MODE, 1.0) == sh.SH_EINVAL

@@ -185,6 +185,24 @@ def test_rows_that_hold_no_token_are_never_used(sh, dtype, d, chunk_kernel, reco
         run_lockstep(h, dtype, lambda t: (q[t - 1], k[t - 1], v[t - 1]), 40, torch.arange(U), TOL[dtype], orc=orc)
 
 
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("U,B,r,w,m,sizes", [(5, 600, 10, 400, 300, [128, 77, 100, 65]), (330, 300, 9, 128, 150, [128, 90]),
+                                             (3, 200, 3, 128, 128, [128]), (149, 130, 2, 200, 100, [65, 128, 1])])
+def test_lockstep_chunked_wide_kernel(sh, dtype, U, B, r, w, m, sizes):
+    """Chunks of 65 to 128 tokens: the wide shape of the persistent tcgen05 kernel (one query per MMA row, 16
+    softmax warps, one CTA per SM), also with more units than SMs and mixed with chunks of the narrow shape."""
+    d, T = 128, B + 2 * m + 40
+    q, k, v = wl.random_stream(U, d, T + 30, seed=51 + U, dtype=dtype, peaked=3.0, device="cuda")
+    h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
+    assert h.prefill_chunk_max == 128
+    blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
+    units = torch.arange(U) if U <= 8 else torch.cat([torch.arange(0, 4), torch.arange(146, min(U, 152)), torch.arange(U - 3, U)]).unique()
+    res, orc = run_lockstep_chunked(h, dtype, blk, T, units, TOL[dtype], chunk_sizes=sizes)
+    assert res.steps == T and res.compressions >= 2
+    assert res.adoptions <= 1e-4 * res.slot_steps + 2
+    run_lockstep(h, dtype, lambda t: (q[t - 1], k[t - 1], v[t - 1]), 30, units, TOL[dtype], orc=orc)
+
+
 @pytest.mark.parametrize("dtype,U", [("f16", 5), ("bf16", 640)])
 def test_chunked_prompt_without_outputs_leaves_the_same_state(sh, dtype, U):
     """sh_prefill with no output buffer (the second contraction is skipped altogether) leaves state bit-identical
@@ -257,13 +275,13 @@ def test_recompute_mode_through_prefill_and_automatic_compression(sh):
 
 
 def test_paper_hyperparameters_chunked_prompt_then_decode(sh):
-    """The values the paper uses in all its experiments (Section 4.1: r = 10, w = 400, m = 0.5 B), on a
-    budget large enough that the chunk kernel has to fall back to 32 queries per launch."""
+    """The values the paper uses in all its experiments (Section 4.1: r = 10, w = 400, m = 0.5 B): chunks of 128
+    tokens on the wide shape of the persistent kernel."""
     U, d, B, r, w, m, dtype = 3, 128, 600, 10, 400, 300, "bf16"
     T = B + 2 * m + 40
     q, k, v = wl.random_stream(U, d, T + 60, seed=61, dtype=dtype, peaked=3.0, device="cuda")
     h = sh.Handle(B, r, w, m, U, d, dtype, auto_compress=False)
-    assert h.prefill_chunk_max == 64
+    assert h.prefill_chunk_max == 128
     blk = lambda t0, t1: (q[t0 - 1:t1 - 1].contiguous(), k[t0 - 1:t1 - 1].contiguous(), v[t0 - 1:t1 - 1].contiguous())
     res, orc = run_lockstep_chunked(h, dtype, blk, T, torch.arange(U), TOL[dtype])
     assert res.compressions == 3
