@@ -87,7 +87,7 @@ typedef enum {
                                  on where a token is stored. */
     SH_OPT_PREFILL_CHUNK = 4, /* 1 (default): sh_prefill hands the tokens between two compressions to a chunk
                                  kernel: the tcgen05 kernels for fp16/bf16/int4 with head_dim 128 (any budget;
-                                 fp16/bf16: persistent CTAs fed by tiled TMA copies), the CUDA-core kernel for
+                                 fp16/bf16: persistent CTAs fed by tiled TMA copies, up to 128 tokens a launch), the CUDA-core kernel for
                                  fp32 rows and for head_dim 64; 0: one decode step per token; 2: the warp-level
                                  MMA chunk kernel where it applies (fp16/bf16, head_dim 128, budgets up to about
                                  700); 3: as 1, but fp16/bf16 use the tcgen05 kernel with one CTA per unit and
@@ -231,7 +231,8 @@ int sh_sequence_state(sh_handle h, int *n_host, long long *t_host, int capacity)
  * One chunk of the prompt without the compression: steps t+1 .. t+count for
  * every unit in one launch (see sh_prefill).  Needs 1 <= count <=
  * sh_prefill_chunk_max(h) and count <= B - n; returns SH_EINVAL otherwise
- * (sh_prefill_chunk_max is min(64, w), or 0 where SH_OPT_PREFILL_CHUNK = 2 does not apply).
+ * (sh_prefill_chunk_max is min(128, w) on the default kernel of fp16/bf16 stores with head_dim 128,
+ * min(64, w) on every other chunk kernel, or 0 where SH_OPT_PREFILL_CHUNK = 2 does not apply).
  * Layout as sh_prefill.  The caller compresses when n reaches B.
  */
 int sh_prefill_chunk(sh_handle h, const void *q_dev, const void *k_dev, const void *v_dev, int count,
