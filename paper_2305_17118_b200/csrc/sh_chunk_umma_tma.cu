@@ -1,6 +1,6 @@
 // Chunked prompt step on the 5th-generation tensor cores, persistent CTAs fed by tiled TMA copies.
 //
-// The computation is the one of sh_chunk_umma.cu (up to 64 consecutive steps of one unit: step i attends with
+// The computation is the one of sh_chunk_umma.cu (up to 128 consecutive steps of one unit: step i attends with
 // q_i over the n0 cached rows plus the chunk's tokens 0..i, writes its comparison bits into its own bit-plane
 // row, and the chunk's keys, values and queries are appended), and so are the two sweeps over the key tiles and
 // the split of P into a high and a low 16-bit part.  What differs is who moves the data and who waits for whom:
@@ -14,9 +14,10 @@
 //     operand layout for Q and K and the MN-major one for V.  Rows past B (and queries past c) are filled with
 //     zeros by the copy engine; rows between n0 + c and the end of the last tile are stale cache rows: their
 //     logits are masked, and the softmax threads zero them in the last value tile before P.V reads it;
-//   * warps 0..7 do the softmax arithmetic; warp 8 issues the MMAs, warp 9 requests query and key tiles, warp 10
-//     value tiles, warp 11 appends the chunk to the cache (plain loads and stores, then a proxy fence: the
-//     tiles that contain the new rows are requested only after the append of their unit is visible).
+//   * the softmax warps (8 for chunks of up to 64 tokens, 16 for up to 128) do the arithmetic; after them comes one
+//     warp each that issues the MMAs, requests query and key tiles, requests value tiles, and one or four warps
+//     that append the chunk to the cache (plain loads and stores, then a proxy fence: the tiles that contain the
+//     new rows are requested only after the append of their unit is visible).
 //
 // Every wait is bounded; a wait that gives up records its code in the device error word and raises a CTA-wide
 // flag, on which every role leaves; tensor memory is released on every path.
