@@ -232,6 +232,19 @@ def stream_prompt(cfg, handles, streams):
     return ms, blk
 
 
+def prompt_attention_flop(cfg) -> float:
+    """Algorithmic FLOP of the prompt's attention for all units and layers: token t attends over the rows cached
+    when it arrives plus itself (the saw-tooth of Algorithm 1: m rows leave whenever B are reached); two passes
+    over the logits (row statistics, then probabilities and record bits) and one over the values, 2 n d each."""
+    n, rows = 0, 0
+    for _ in range(cfg.prompt):
+        if n == cfg.B:
+            n -= cfg.m
+        n += 1
+        rows += n
+    return 3.0 * 2.0 * rows * cfg.head_dim * cfg.units * cfg.layers
+
+
 def time_compression(cfg, h, snap, dec_l, out, reps: int = REPEATS):
     """CUDA-event time of one sh_compress of handle `h` (all its units), `reps` times, each from the
     restored post-prompt state advanced until the cache is full.  dec_l: that layer's decode inputs."""
@@ -462,6 +475,7 @@ def cuda_arm(args, cfg, rank, world):
         "attn_GBps": statistics.fmean(n_sched) * U * Ly * d * ES[cfg.dtype] * 2 / (ms_per_step * 1e-3) / 1e9,
         "prompt": {"tokens": cfg.prompt, "ms": prompt_ms, "tokens_per_s": cfg.prompt * 1e3 / prompt_ms if prompt_ms else None,
                    "chunked": bool(handles[0].prefill_chunk_max) and not args.no_prefill_chunk,
+                   "attention_tflops_algorithmic": prompt_attention_flop(cfg) / (prompt_ms * 1e-3) / 1e12 if prompt_ms else None,
                    "note": "untimed part of the benchmark; streamed through sh_prefill in blocks of %d tokens" % blk},
         "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": launches,
         "roofline": roofline, "cpu_baseline": cpu,
