@@ -4,7 +4,7 @@
 // unit in one CTA; step i attends with q_i over the n0 cached rows plus the chunk's tokens 0..i and
 // writes its comparison bits into its own bit-plane row.  What differs is where the work runs:
 //
-//   * S = Q.K^T is issued by one thread as tcgen05.mma (M = 128, N = 128 keys per tile, K = 16 per
+//   * S = Q.K^T is issued by one thread as tcgen05.mma (M = 128, N = 64 keys per tile, K = 16 per
 //     instruction), operands in shared memory in the canonical no-swizzle core-matrix order, the
 //     fp32 result in tensor memory.  The 64 queries occupy rows 0..63 and again rows 64..127, so
 //     that all 128 lanes of tensor memory carry data: thread i and thread i + 64 own the same
@@ -37,7 +37,7 @@ constexpr int TN = 64;            // keys per tile
 constexpr int CQ = 64;            // queries per CTA
 constexpr int NT = 256;           // threads per CTA: two per lane of tensor memory (warps w and w + 4 share a lane quadrant)
 constexpr int GROUP = 2048;       // bytes of 8 rows of 256 B in core-matrix order: [16 chunks][8 rows][16 B]
-constexpr int TILE = (TN / 8) * GROUP;          // 32 KB
+constexpr int TILE = (TN / 8) * GROUP;          // 16 KB
 constexpr int Q_BYTES = (2 * CQ / 8) * GROUP;   // 128 rows
 constexpr int PG = (TN / 8) * 128;              // bytes of 8 rows of P (TN keys each) in core-matrix order
 constexpr int P_BYTES = (CQ / 8) * PG;          // 64 rows x TN keys x 2 B
