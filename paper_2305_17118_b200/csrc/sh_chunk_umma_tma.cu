@@ -898,8 +898,33 @@ cudaError_t sh_launch_recount_umma_tma(const ChunkParams &p, int dtype, cudaStre
 
 int sh_chunk_umma_tma_capacity() { return CK<true>::QR; }
 
-cudaError_t sh_launch_chunk_umma_tma(const ChunkParams &p, int dtype, cudaStream_t s) {
+cudaError_t sh_launch_chunk_umma_tma(const ChunkParams &p, int dtype, cudaStream_t s, int *launches) {
+    *launches = 0;
     if (p.c < 1 || p.c > CK<true>::QR || p.U < 1) return cudaErrorInvalidValue;
-    if (p.c > CK<false>::QR) return dtype == SH_F16 ? launch_tma<SH_F16, true>(p, s) : launch_tma<SH_BF16, true>(p, s);
-    return dtype == SH_F16 ? launch_tma<SH_F16, false>(p, s) : launch_tma<SH_BF16, false>(p, s);
+    cudaError_t e;
+    if (p.c <= CK<false>::QR) {
+        e = dtype == SH_F16 ? launch_tma<SH_F16, false>(p, s) : launch_tma<SH_BF16, false>(p, s);
+        if (e == cudaSuccess) *launches = 1;
+        return e;
+    }
+    // More than 64 tokens.  The wide shape runs one CTA per SM: it pays from about four units per SM on (1280 units:
+    // 128 tokens in 0.79 of the time of two narrow launches; 256 units: 1.5 times slower, half the SMs would hold
+    // one unit and wait for the others' second).  With fewer units the chunk goes as two narrow launches.
+    if (p.U >= 4 * sm_count()) {
+        e = dtype == SH_F16 ? launch_tma<SH_F16, true>(p, s) : launch_tma<SH_BF16, true>(p, s);
+        if (e == cudaSuccess) *launches = 1;
+        return e;
+    }
+    for (int done = 0; done < p.c; done += CK<false>::QR) {
+        ChunkParams part = p;
+        const size_t skip = (size_t)done * p.Utot * D;        // elements of q, k, v and out before token `done`
+        part.q = p.q + skip * 2; part.k = p.k + skip * 2; part.v = p.v + skip * 2;
+        part.out = p.out ? p.out + skip : nullptr;
+        part.n0 = p.n0 + done; part.t0 = p.t0 + done;
+        part.c = p.c - done < CK<false>::QR ? p.c - done : CK<false>::QR;
+        e = dtype == SH_F16 ? launch_tma<SH_F16, false>(part, s) : launch_tma<SH_BF16, false>(part, s);
+        if (e != cudaSuccess) return e;
+        *launches += 1;
+    }
+    return cudaSuccess;
 }

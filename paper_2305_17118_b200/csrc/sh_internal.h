@@ -193,7 +193,7 @@ cudaError_t sh_launch_chunk_umma(const ChunkParams &p, int dtype, cudaStream_t s
 cudaError_t sh_launch_recount_umma(const ChunkParams &p, int dtype, cudaStream_t s);
 // the same chunk step with persistent CTAs and tiled TMA copies (sh_chunk_umma_tma.cu)
 int sh_chunk_umma_tma_capacity();
-cudaError_t sh_launch_chunk_umma_tma(const ChunkParams &p, int dtype, cudaStream_t s);
+cudaError_t sh_launch_chunk_umma_tma(const ChunkParams &p, int dtype, cudaStream_t s, int *launches);
 cudaError_t sh_launch_recount_umma_tma(const ChunkParams &p, int dtype, cudaStream_t s);
 // int4-g64 store: the chunked prompt step with codes unpacked into the tensor-core tiles (sh_chunk_umma_int4.cu).
 cudaError_t sh_launch_chunk_umma_int4(const ChunkParams &p, cudaStream_t s);

@@ -389,7 +389,12 @@ cudaError_t sh_launch_prefill_chunk(const sh_context *c, const void *q, const vo
         return e;
     }
     if (c->prefill_chunk != 2) {
-        e = c->prefill_chunk == 1 ? sh_launch_chunk_umma_tma(p, c->dtype, s) : cudaErrorNotSupported;
+        int nl = 0;
+        e = c->prefill_chunk == 1 ? sh_launch_chunk_umma_tma(p, c->dtype, s, &nl) : cudaErrorNotSupported;
+        if (e == cudaSuccess) {
+            *launches += nl;
+            return e;
+        }
         if (e == cudaErrorNotSupported) {       // option 3, or a driver without the tensor-map encoder: the per-unit tcgen05 kernel,
             (void)cudaGetLastError();           // which takes 64 tokens at a time (the steps of a chunk are consecutive: it splits)
             const int cap = sh_chunk_umma_capacity();
