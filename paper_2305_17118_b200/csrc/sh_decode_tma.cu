@@ -450,6 +450,16 @@ cudaError_t launch_dt(const sh_context *c, const DecodeParams &p, cudaStream_t s
         if (c->D == 64)
             return launch_tma<DT, 64, TMA_NWC, Shape<DT, 64>::SR, Shape<DT, 64>::NST, Shape<DT, 64>::LR, TMA_CPS>(c, p, s);
     }
+    if constexpr (DT != SH_F32) {
+        // Between one and two units per SM a single CTA per SM would run two units one after the other on most SMs
+        // and one on the rest; two CTAs per SM with tiles of half the rows take every unit at once.
+        int sms = 148, dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const int capw = (c->B + 31) & ~31;
+        const size_t small = (size_t)TMA_NST * (2 * 64 * 256 + 3 * 256) + sizeof(float) * ((size_t)2 * capw + (size_t)2 * TMA_NWC * 128 + (size_t)2 * TMA_NWC * 2);
+        if (p.U > sms && p.U <= 2 * sms && 2 * (small + 1024) <= 228 * 1024)
+            return launch_tma<DT, 128, TMA_NWC, 64, TMA_NST, TMA_LR, 2>(c, p, s);
+    }
     return launch_tma<DT, 128, TMA_NWC, Shape<DT, 128>::SR, Shape<DT, 128>::NST, Shape<DT, 128>::LR, TMA_CPS>(c, p, s);
 }
 

@@ -69,11 +69,13 @@ def test_lockstep_direct_kernel_many_units(sh, dtype, d):
 
 
 @pytest.mark.parametrize("dtype,d", [("f16", 128), ("bf16", 128), ("f32", 128), ("f32", 64)])
-@pytest.mark.parametrize("U,B,r,w,m", [(5, 150, 9, 37, 41), (301, 130, 16, 33, 50), (3, 700, 5, 64, 300), (2, 40, 3, 9, 20)])
+@pytest.mark.parametrize("U,B,r,w,m", [(5, 150, 9, 37, 41), (301, 130, 16, 33, 50), (3, 700, 5, 64, 300), (2, 40, 3, 9, 20),
+                                       (200, 150, 9, 37, 41), (296, 90, 4, 20, 35)])
 def test_lockstep_pipelined_kernel(sh, dtype, d, U, B, r, w, m):
     """The persistent bulk-copy variant of the decode kernel, forced on shapes that
     cover fewer units than CTAs, more units than SMs, ragged last tiles and tiny caches,
-    for every row size it serves (256 and 512 bytes)."""
+    for every row size it serves (256 and 512 bytes); between one and two units per SM (the last two
+    cases) the 16-bit stores run two CTAs per SM with tiles of 64 rows."""
     T = 2 * B + 2 * m + 7
     q, k, v = wl.random_stream(U, d, T, seed=11 + U, dtype=dtype, peaked=3.0, device="cuda")
     h = sh.Handle(B, r, w, m, U, d, dtype, split=1, kernel=2, auto_compress=False)
