@@ -536,7 +536,8 @@ constexpr int RTHREADS = NT + 96;
 constexpr int R_TMEM_COLS = 2 * TN;     // two S tiles
 constexpr int ROFF_K = 2 * Q_BYTES;     // two query buffers: the next item's queries are gathered during the present item
 constexpr int ROFF_POS = ROFF_K + RKST * TILE;
-constexpr int ROFF_STAT = ROFF_POS + RPD * TN * 4;        // m[256], l[256], M[128], L[128]
+constexpr int ROFF_PMAX = ROFF_POS + RPD * TN * 4;        // per position tile: the largest position in it
+constexpr int ROFF_STAT = ROFF_PMAX + RPD * 4;            // m[256], l[256], M[128], L[128]
 constexpr int ROFF_BAR = ROFF_STAT + 4 * (2 * NT + 2 * RQ);
 constexpr int R_SMEM_BYTES = ROFF_BAR + 256;
 static_assert(ROFF_K % 1024 == 0, "swizzled tiles start on 1024-byte boundaries");
@@ -560,6 +561,7 @@ __global__ void __launch_bounds__(RTHREADS, 2) sh_recount_umma_tma_kernel(const 
     char *Qs = reinterpret_cast<char *>(sm);
     char *Kt = reinterpret_cast<char *>(sm) + ROFF_K;
     int *pos_sh = reinterpret_cast<int *>(sm + ROFF_POS);
+    int *pmax_sh = reinterpret_cast<int *>(sm + ROFF_PMAX);
     float *m_sh = reinterpret_cast<float *>(sm + ROFF_STAT), *l_sh = m_sh + NT, *Mfin = l_sh + NT, *Lfin = Mfin + RQ;
     RBars *bars = reinterpret_cast<RBars *>(sm + ROFF_BAR);
 
@@ -664,6 +666,8 @@ __global__ void __launch_bounds__(RTHREADS, 2) sh_recount_umma_tma_kernel(const 
                     int *pt = pos_sh + (gk % RPD) * TN;
                     pt[lane] = pv[0];
                     pt[32 + lane] = pv[1];
+                    const int tile_max = __reduce_max_sync(0xffffffffu, max(pv[0], pv[1]));
+                    if (lane == 0) pmax_sh[gk % RPD] = tile_max;
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars->pos_full[gk % RPD]);
                     last = gk;
@@ -740,9 +744,11 @@ __global__ void __launch_bounds__(RTHREADS, 2) sh_recount_umma_tma_kernel(const 
                 float sv[RHC];
                 tmem_ld32(lane_addr + b * TN + half * RHC, sv);
                 tc_fence_before();
-                // bit jj of vm: column jj of this thread's half is visible to its query
-                uint32_t vm = 0;
-                {
+                // bit jj of vm: column jj of this thread's half is visible to its query.  Most tiles hold only tokens older
+                // than every query of the item (their largest position says so): nothing to compare
+                uint32_t vm = 0xffffffffu;
+                if (pmax_sh[gk % RPD] > step) {
+                    vm = 0;
                     const int4 *pt = reinterpret_cast<const int4 *>(pos_sh + (gk % RPD) * TN + half * RHC);
 #pragma unroll
                     for (int q4 = 0; q4 < RHC / 4; ++q4) {
@@ -750,8 +756,8 @@ __global__ void __launch_bounds__(RTHREADS, 2) sh_recount_umma_tma_kernel(const 
                         vm |= (uint32_t)(pp.x <= step) << (4 * q4) | (uint32_t)(pp.y <= step) << (4 * q4 + 1) |
                               (uint32_t)(pp.z <= step) << (4 * q4 + 2) | (uint32_t)(pp.w <= step) << (4 * q4 + 3);
                     }
-                    if (!live_row) vm = 0;
                 }
+                if (!live_row) vm = 0;
                 mbar_arrive(&bars->s_free[b]);       // S is in registers and the tile's positions have been read
                 if (g < ntiles) {
                     if (vm) {
