@@ -292,12 +292,14 @@ def test_paper_hyperparameters_chunked_prompt_then_decode(sh):
     run_lockstep(h, dtype, _stream_fn(q, k, v), 60, torch.arange(U), TOL[dtype], orc=orc)
 
 
-def test_prefill_uses_chunks_and_matches_oracle(sh):
-    """sh_prefill with its automatic chunking and compression on the OPT-6.7B-shaped stream.  A twin handle
+@pytest.mark.parametrize("name,units,prompt,compressions", [("opt6b", 24, 700, 5), ("opt13b", 640, 900, 4)])
+def test_prefill_uses_chunks_and_matches_oracle(sh, name, units, prompt, compressions):
+    """sh_prefill with its automatic chunking and compression on the OPT-6.7B-shaped stream (chunks of 64 tokens) and
+    on a layer of the OPT-13B-shaped one with enough units for the wide shape (chunks of 128).  A twin handle
     is driven through the same sequence of launches by hand, in lockstep with the oracle (every output,
     record bit, counter and kept set, with adoption inside the 1e-6 window); the handle that went
     through sh_prefill must be bit-identical to the twin.  Then decode steps in lockstep."""
-    cfg = wl.CONFIGS["opt6b"].scaled(units=24, prompt=700)
+    cfg = wl.CONFIGS[name].scaled(units=units, prompt=prompt)
     st = wl.Stream(cfg, device="cuda")
     h = sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, cfg.units, cfg.head_dim, cfg.dtype, auto_compress=False)
     q, k, v = st.block(1, cfg.prompt + 1)
@@ -306,13 +308,14 @@ def test_prefill_uses_chunks_and_matches_oracle(sh):
     h.prefill(q, k, v, out)
     assert h.launch_count - before < cfg.prompt // 8        # chunks, not one launch per token
     twin = sh.Handle(cfg.B, cfg.r, cfg.w, cfg.m, cfg.units, cfg.head_dim, cfg.dtype, auto_compress=False)
+    sample = torch.arange(cfg.units) if cfg.units <= 32 else torch.tensor([0, 1, 147, 148, 295, 296, cfg.units - 2, cfg.units - 1])
     t_outs = []
     res, orc = run_lockstep_chunked(twin, cfg.dtype, lambda t0, t1: (q[t0 - 1:t1 - 1], k[t0 - 1:t1 - 1], v[t0 - 1:t1 - 1]),
-                                    cfg.prompt, torch.arange(cfg.units), TOL[cfg.dtype], outs=t_outs, single_via_step=True)
-    assert res.compressions == 5
+                                    cfg.prompt, sample, TOL[cfg.dtype], outs=t_outs, single_via_step=True)
+    assert res.compressions == compressions
     assert torch.equal(out, torch.cat(t_outs))
     assert_same_state(h, twin)
-    run_lockstep(h, cfg.dtype, st.step, 70, torch.arange(cfg.units), TOL[cfg.dtype], orc=orc)
+    run_lockstep(h, cfg.dtype, st.step, 70, sample, TOL[cfg.dtype], orc=orc)
 
 
 # ---- the benchmark's own configurations ----------------------------------------------------
